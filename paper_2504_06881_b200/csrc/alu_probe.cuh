@@ -1,0 +1,198 @@
+// Register-only throughput probes of the add + max/min instruction mixes the
+// tropical kernels can be built from.  Each thread keeps a TK x TP block of
+// running extrema and folds taps x[j] + w[i] into them, exactly the inner loop of
+// the forward pass minus its memory traffic.  An empty asm statement that names
+// x and w as read-write operands stops the compiler from hoisting the adds out
+// of the loop without costing an instruction.
+#pragma once
+#include "tconv_common.cuh"
+
+namespace tconv {
+
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float min3f(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// Packed fp32 add: {lo, hi} = {x + wlo, x + whi}, one instruction for two taps.
+__device__ __forceinline__ void add2f(float x, float wlo, float whi, float& lo, float& hi) {
+    unsigned long long xx, ww, tt;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(xx) : "f"(x));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ww) : "f"(wlo), "f"(whi));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(tt) : "l"(xx), "l"(ww));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
+}
+
+enum {
+    PROBE_F32_ADD_MAX2 = 0,      // max-plus / min-plus: add, 2-input max
+    PROBE_F32_ADD_MAX3,          // two adds feed one 3-input max
+    PROBE_F32_ADD2_MAX3,         // packed add of two channels, 3-input max over two taps
+    PROBE_F32_ADD_MINMAX2,       // compound: add, min, max
+    PROBE_F32_ADD_MINMAX3,       // compound: two adds feed a 3-input min and a 3-input max
+    PROBE_F32_ADD2_MINMAX3,      // compound with packed adds
+    PROBE_F32_2ADD_MINMAX2,      // parallel: two adds, min, max
+    PROBE_F32_2ADD_MINMAX3,      // parallel with 3-input min / max
+    PROBE_F32_2ADD2_MINMAX3,     // parallel with packed adds and 3-input min / max
+    PROBE_BF16X2_ADD_MAX,        // bf16 pairs: add, max
+    PROBE_BF16X2_ADD_MINMAX,     // bf16 pairs, compound
+    PROBE_BF16X2_2ADD_MINMAX,    // bf16 pairs, parallel
+    PROBE_F32_ADD_ONLY,          // adds alone (sum-reduced), the FP32 pipe by itself
+    PROBE_F32_MAX2_ONLY,         // 2-input max alone
+    PROBE_F32_MAX3_ONLY,         // 3-input max alone
+    PROBE_COUNT
+};
+
+static const char* const kProbeNames[PROBE_COUNT] = {
+    "f32_add_max2",       "f32_add_max3",      "f32_add2_max3",   "f32_add_minmax2",
+    "f32_add_minmax3",    "f32_add2_minmax3",  "f32_2add_minmax2", "f32_2add_minmax3",
+    "f32_2add2_minmax3",  "bf16x2_add_max",    "bf16x2_add_minmax", "bf16x2_2add_minmax",
+    "f32_add_only",       "f32_max2_only",     "f32_max3_only"};
+
+// Taps folded per thread per loop iteration, by variant (must match the kernel).
+__host__ inline int probe_taps_per_iter(int v) {
+    switch (v) {
+        case PROBE_BF16X2_ADD_MAX:
+        case PROBE_BF16X2_ADD_MINMAX:
+        case PROBE_BF16X2_2ADD_MINMAX: return 4 * 8 * 2 * 2;  // 4 channel pairs x 8 pixels x 2 lanes x 2 taps
+        default: return 8 * 4 * 2;                            // 8 channels x 4 pixels x 2 taps
+    }
+}
+
+#define TCONV_OPAQUE_F(v) asm volatile("" : "+f"(v))
+#define TCONV_OPAQUE_R(v) asm volatile("" : "+r"(v))
+
+template <int V>
+__global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, float* sink) {
+    constexpr int TK = 8, TP = 4;
+    if constexpr (V >= PROBE_BF16X2_ADD_MAX && V <= PROBE_BF16X2_2ADD_MINMAX) {
+        // packed bf16 pairs: a register holds two output channels
+        constexpr int KP = 4, PX = 8;
+        __nv_bfloat162 x[PX + 1], wa[KP], wb[KP], va[KP], vb[KP];
+        __nv_bfloat162 mn[KP][PX], mx[KP][PX];
+        for (int j = 0; j <= PX; ++j) x[j] = __float2bfloat162_rn(seed * (float)(j + threadIdx.x));
+        for (int i = 0; i < KP; ++i) {
+            wa[i] = __float2bfloat162_rn(seed * (float)(i + 3));
+            wb[i] = __float2bfloat162_rn(seed * (float)(i + 5));
+            va[i] = __float2bfloat162_rn(seed * (float)(i + 7));
+            vb[i] = __float2bfloat162_rn(seed * (float)(i + 9));
+            for (int j = 0; j < PX; ++j) { mn[i][j] = x[j]; mx[i][j] = x[j]; }
+        }
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int j = 0; j <= PX; ++j) TCONV_OPAQUE_R(*reinterpret_cast<unsigned*>(&x[j]));
+#pragma unroll
+            for (int i = 0; i < KP; ++i) {
+                TCONV_OPAQUE_R(*reinterpret_cast<unsigned*>(&wa[i]));
+                TCONV_OPAQUE_R(*reinterpret_cast<unsigned*>(&wb[i]));
+                TCONV_OPAQUE_R(*reinterpret_cast<unsigned*>(&va[i]));
+                TCONV_OPAQUE_R(*reinterpret_cast<unsigned*>(&vb[i]));
+            }
+#pragma unroll
+            for (int i = 0; i < KP; ++i)
+#pragma unroll
+                for (int j = 0; j < PX; ++j) {
+                    const __nv_bfloat162 t0 = __hadd2(x[j], wa[i]);
+                    const __nv_bfloat162 t1 = __hadd2(x[j + 1], wb[i]);
+                    if constexpr (V == PROBE_BF16X2_ADD_MAX) {
+                        mx[i][j] = __hmax2(__hmax2(mx[i][j], t0), t1);
+                    } else if constexpr (V == PROBE_BF16X2_ADD_MINMAX) {
+                        mx[i][j] = __hmax2(__hmax2(mx[i][j], t0), t1);
+                        mn[i][j] = __hmin2(__hmin2(mn[i][j], t0), t1);
+                    } else {
+                        const __nv_bfloat162 u0 = __hadd2(x[j], va[i]);
+                        const __nv_bfloat162 u1 = __hadd2(x[j + 1], vb[i]);
+                        mx[i][j] = __hmax2(__hmax2(mx[i][j], u0), u1);
+                        mn[i][j] = __hmin2(__hmin2(mn[i][j], t0), t1);
+                    }
+                }
+        }
+        __nv_bfloat162 r = mx[0][0];
+        for (int i = 0; i < KP; ++i)
+            for (int j = 0; j < PX; ++j) r = __hadd2(r, __hadd2(mx[i][j], mn[i][j]));
+        if (__low2float(r) == 12345.678f) sink[0] = __high2float(r);
+    } else {
+        float x[TP + 1], w0[TK], w1[TK], v0[TK], v1[TK];
+        float mn[TK][TP], mx[TK][TP];
+        for (int j = 0; j <= TP; ++j) x[j] = seed * (float)(j + threadIdx.x);
+        for (int i = 0; i < TK; ++i) {
+            w0[i] = seed * (float)(i + 3);
+            w1[i] = seed * (float)(i + 5);
+            v0[i] = seed * (float)(i + 7);
+            v1[i] = seed * (float)(i + 9);
+            for (int j = 0; j < TP; ++j) { mn[i][j] = x[j]; mx[i][j] = x[j]; }
+        }
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int j = 0; j <= TP; ++j) TCONV_OPAQUE_F(x[j]);
+#pragma unroll
+            for (int i = 0; i < TK; ++i) {
+                TCONV_OPAQUE_F(w0[i]); TCONV_OPAQUE_F(w1[i]);
+                TCONV_OPAQUE_F(v0[i]); TCONV_OPAQUE_F(v1[i]);
+            }
+            constexpr bool packed = (V == PROBE_F32_ADD2_MAX3 || V == PROBE_F32_ADD2_MINMAX3 ||
+                                     V == PROBE_F32_2ADD2_MINMAX3);
+            constexpr bool par = (V == PROBE_F32_2ADD_MINMAX2 || V == PROBE_F32_2ADD_MINMAX3 ||
+                                  V == PROBE_F32_2ADD2_MINMAX3);
+#pragma unroll
+            for (int i = 0; i < TK; i += 2)
+#pragma unroll
+                for (int j = 0; j < TP; ++j) {
+                    // two taps (window positions j, j+1) for the channel pair (i, i+1)
+                    float ta0, tb0, ta1, tb1;      // min-branch sums: tap 0 / 1, channel i / i+1
+                    float ua0, ub0, ua1, ub1;      // max-branch sums (parallel only)
+                    if constexpr (V == PROBE_F32_MAX2_ONLY || V == PROBE_F32_MAX3_ONLY) {
+                        ta0 = x[j]; tb0 = w0[i]; ta1 = x[j + 1]; tb1 = w1[i + 1];
+                    } else if constexpr (packed) {
+                        add2f(x[j], w0[i], w0[i + 1], ta0, tb0);
+                        add2f(x[j + 1], w1[i], w1[i + 1], ta1, tb1);
+                    } else {
+                        ta0 = __fadd_rn(x[j], w0[i]); tb0 = __fadd_rn(x[j], w0[i + 1]);
+                        ta1 = __fadd_rn(x[j + 1], w1[i]); tb1 = __fadd_rn(x[j + 1], w1[i + 1]);
+                    }
+                    if constexpr (par) {
+                        if constexpr (packed) {
+                            add2f(x[j], v0[i], v0[i + 1], ua0, ub0);
+                            add2f(x[j + 1], v1[i], v1[i + 1], ua1, ub1);
+                        } else {
+                            ua0 = __fadd_rn(x[j], v0[i]); ub0 = __fadd_rn(x[j], v0[i + 1]);
+                            ua1 = __fadd_rn(x[j + 1], v1[i]); ub1 = __fadd_rn(x[j + 1], v1[i + 1]);
+                        }
+                    } else {
+                        ua0 = ta0; ub0 = tb0; ua1 = ta1; ub1 = tb1;
+                    }
+                    if constexpr (V == PROBE_F32_ADD_ONLY) {
+                        mx[i][j] += ta0 + ta1;          // 4 adds per 2 taps: an upper bound
+                        mx[i + 1][j] += tb0 + tb1;      // on what the FP32 pipe sustains
+                    } else if constexpr (V == PROBE_F32_ADD_MAX2 || V == PROBE_F32_MAX2_ONLY) {
+                        mx[i][j] = fmaxf(fmaxf(mx[i][j], ta0), ta1);
+                        mx[i + 1][j] = fmaxf(fmaxf(mx[i + 1][j], tb0), tb1);
+                    } else if constexpr (V == PROBE_F32_ADD_MAX3 || V == PROBE_F32_ADD2_MAX3 ||
+                                         V == PROBE_F32_MAX3_ONLY) {
+                        mx[i][j] = max3f(mx[i][j], ta0, ta1);
+                        mx[i + 1][j] = max3f(mx[i + 1][j], tb0, tb1);
+                    } else if constexpr (V == PROBE_F32_ADD_MINMAX2 || V == PROBE_F32_2ADD_MINMAX2) {
+                        mx[i][j] = fmaxf(fmaxf(mx[i][j], ua0), ua1);
+                        mx[i + 1][j] = fmaxf(fmaxf(mx[i + 1][j], ub0), ub1);
+                        mn[i][j] = fminf(fminf(mn[i][j], ta0), ta1);
+                        mn[i + 1][j] = fminf(fminf(mn[i + 1][j], tb0), tb1);
+                    } else {
+                        mx[i][j] = max3f(mx[i][j], ua0, ua1);
+                        mx[i + 1][j] = max3f(mx[i + 1][j], ub0, ub1);
+                        mn[i][j] = min3f(mn[i][j], ta0, ta1);
+                        mn[i + 1][j] = min3f(mn[i + 1][j], tb0, tb1);
+                    }
+                }
+        }
+        float r = 0.0f;
+        for (int i = 0; i < TK; ++i)
+            for (int j = 0; j < TP; ++j) r += mx[i][j] + mn[i][j];
+        if (r == 12345.678f) sink[0] = r;
+    }
+}
+
+}  // namespace tconv

@@ -1,0 +1,279 @@
+// Host side of the C ABI declared in tconv.h: descriptor validation, workspace
+// accounting, kernel selection and launch.  No device memory is allocated here.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+
+#include "alu_probe.cuh"
+#include "tconv_common.cuh"
+#include "tconv_generic.cuh"
+#include "tconv_tiled.cuh"
+
+using namespace tconv;
+
+namespace {
+
+thread_local char g_last_error[256] = "";
+thread_local char g_last_kernel[128] = "";
+
+int cuda_fail(cudaError_t e) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s", cudaGetErrorString(e));
+    return TCONV_ERR_CUDA;
+}
+
+int check_launch() {
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? TCONV_OK : cuda_fail(e);
+}
+
+int out_extent(int in, int pad, int dil, int k, int stride) {
+    const long span = (long)in + 2L * pad - (long)dil * (k - 1) - 1;
+    if (span < 0) return 0;
+    return (int)(span / stride) + 1;
+}
+
+// Validates the descriptor and fills the kernel-side geometry.
+int make_geo(const tconv_desc_t* d, Geo* g) {
+    if (!d) return TCONV_ERR_INVALID_ARG;
+    if (d->N <= 0 || d->C <= 0 || d->H <= 0 || d->W <= 0 || d->K <= 0 || d->R <= 0 || d->S <= 0)
+        return TCONV_ERR_INVALID_ARG;
+    if (d->stride_h <= 0 || d->stride_w <= 0 || d->dil_h <= 0 || d->dil_w <= 0 || d->pad_h < 0 ||
+        d->pad_w < 0)
+        return TCONV_ERR_INVALID_ARG;
+    if (d->mode < TCONV_MAX_PLUS || d->mode > TCONV_PARALLEL) return TCONV_ERR_INVALID_ARG;
+    if (d->chan < TCONV_CHAN_DEFAULT || d->chan > TCONV_CHAN_MIN) return TCONV_ERR_INVALID_ARG;
+    if (d->dtype != TCONV_F32 && d->dtype != TCONV_BF16) return TCONV_ERR_INVALID_ARG;
+    int chan = d->chan;
+    if (chan == TCONV_CHAN_DEFAULT)
+        chan = d->mode == TCONV_MAX_PLUS ? CH_MAX : d->mode == TCONV_MIN_PLUS ? CH_MIN : CH_SUM;
+    if (two_branch(d->mode) && chan != CH_SUM) return TCONV_ERR_UNSUPPORTED;
+    if ((long)d->R * d->S > 256) return TCONV_ERR_UNSUPPORTED;
+    g->N = d->N; g->C = d->C; g->H = d->H; g->W = d->W; g->K = d->K; g->R = d->R; g->S = d->S;
+    g->sh = d->stride_h; g->sw = d->stride_w; g->ph = d->pad_h; g->pw = d->pad_w;
+    g->dh = d->dil_h; g->dw = d->dil_w;
+    g->OH = out_extent(d->H, d->pad_h, d->dil_h, d->R, d->stride_h);
+    g->OW = out_extent(d->W, d->pad_w, d->dil_w, d->S, d->stride_w);
+    g->RS = d->R * d->S;
+    g->mode = d->mode;
+    g->chan = chan;
+    g->wide = g->RS > 16;
+    if (g->OH <= 0 || g->OW <= 0) return TCONV_ERR_INVALID_ARG;
+    // one-dimensional launches index blocks with 31 bits
+    const double outputs = (double)g->N * g->K * g->OH * g->OW;
+    const double inputs = (double)g->N * g->C * g->H * g->W;
+    if (outputs / 256 > 2.0e9 || inputs / 256 > 2.0e9 || (double)g->K * g->C * g->RS > 2.0e9)
+        return TCONV_ERR_TOO_LARGE;
+    return TCONV_OK;
+}
+
+size_t winner_bytes(const Geo& g) {
+    const size_t outs = (size_t)g.N * g.K * g.OH * g.OW;
+    if (g.chan != CH_SUM) return outs * sizeof(int32_t);
+    return outs * g.C * (g.wide ? 2 : 1);
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+bool misaligned(const void* p) { return p && ((uintptr_t)p & 15u) != 0; }
+
+bool force_generic() {
+    static const bool v = [] {
+        const char* e = getenv("TCONV_FORCE_GENERIC");
+        return e && e[0] == '1';
+    }();
+    return v;
+}
+
+template <typename T>
+int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const float* alpha,
+              const float* beta, const float* bias, void* y, void* winners, cudaStream_t st) {
+    if (!force_generic()) {
+        const char* name = nullptr;
+        const int rc = launch_fwd_tiled<T>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta,
+                                           bias, (T*)y, winners, st, &name);
+        if (rc == TCONV_OK) {
+            snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", name);
+            return check_launch();
+        }
+        if (rc != TCONV_ERR_UNSUPPORTED) return rc;
+    }
+    const size_t total = (size_t)g.N * g.K * g.OH * g.OW;
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    fwd_generic_kernel<T><<<blocks, 256, 0, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha,
+                                                  beta, bias, (T*)y, winners);
+    snprintf(g_last_kernel, sizeof(g_last_kernel), "fwd_generic");
+    return check_launch();
+}
+
+template <typename T>
+int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const float* alpha,
+               const float* beta, const void* gy, const void* winners, void* gx, float* gw,
+               float* gw2, float* galpha, float* gbeta, float* gbias, void* ws, size_t ws_bytes,
+               cudaStream_t st) {
+    (void)ws; (void)ws_bytes;
+    const bool twob = two_branch(g.mode);
+    if (gx) {
+        const size_t total = (size_t)g.N * g.C * g.H * g.W;
+        bwd_gx_generic_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+            g, alpha, beta, (const T*)gy, winners, (T*)gx);
+    }
+    if (gw || gw2) {
+        bwd_gw_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C * g.RS), 256, 0, st>>>(
+            g, alpha, beta, (const T*)gy, winners, gw, gw2);
+    }
+    if (twob && (galpha || gbeta)) {
+        bwd_gab_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C), 256, 0, st>>>(
+            g, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, winners, galpha, gbeta);
+    }
+    if (gbias) bwd_bias_kernel<T><<<(unsigned)g.K, 256, 0, st>>>(g, (const T*)gy, gbias);
+    snprintf(g_last_kernel, sizeof(g_last_kernel), "bwd_generic");
+    return check_launch();
+}
+
+}  // namespace
+
+extern "C" {
+
+int tconv_output_shape(const tconv_desc_t* desc, int32_t* OH, int32_t* OW) {
+    Geo g;
+    const int rc = make_geo(desc, &g);
+    if (rc != TCONV_OK) return rc;
+    if (OH) *OH = g.OH;
+    if (OW) *OW = g.OW;
+    return TCONV_OK;
+}
+
+size_t tconv_winner_bytes(const tconv_desc_t* desc) {
+    Geo g;
+    if (make_geo(desc, &g) != TCONV_OK) return 0;
+    return winner_bytes(g);
+}
+
+size_t tconv_workspace_bytes(const tconv_desc_t* desc, int backward) {
+    Geo g;
+    if (make_geo(desc, &g) != TCONV_OK) return 0;
+    if (!backward) return 0;
+    // winners recomputed into the workspace when the caller passes none
+    return align_up(winner_bytes(g), 256);
+}
+
+int tconv_forward(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,
+                  const float* alpha, const float* beta, const float* bias, void* y, void* winners,
+                  void* workspace, size_t workspace_bytes, void* stream) {
+    Geo g;
+    int rc = make_geo(desc, &g);
+    if (rc != TCONV_OK) return rc;
+    if (!x || !w || !y) return TCONV_ERR_INVALID_ARG;
+    if (g.mode == TCONV_PARALLEL && !w2) return TCONV_ERR_INVALID_ARG;
+    if (misaligned(x) || misaligned(w) || misaligned(w2) || misaligned(alpha) || misaligned(beta) ||
+        misaligned(bias) || misaligned(y) || misaligned(winners) || misaligned(workspace))
+        return TCONV_ERR_MISALIGNED;
+    if (workspace_bytes < tconv_workspace_bytes(desc, 0)) return TCONV_ERR_WORKSPACE_TOO_SMALL;
+    if (!two_branch(g.mode)) { alpha = nullptr; beta = nullptr; }
+    cudaStream_t st = (cudaStream_t)stream;
+    g_last_error[0] = 0;
+    if (desc->dtype == TCONV_F32)
+        return forward_t<float>(g, x, w, w2, alpha, beta, bias, y, winners, st);
+    return forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, bias, y, winners, st);
+}
+
+int tconv_backward(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,
+                   const float* alpha, const float* beta, const void* grad_y, const void* winners,
+                   void* grad_x, float* grad_w, float* grad_w2, float* grad_alpha,
+                   float* grad_beta, float* grad_bias, void* workspace, size_t workspace_bytes,
+                   void* stream) {
+    Geo g;
+    int rc = make_geo(desc, &g);
+    if (rc != TCONV_OK) return rc;
+    if (!x || !w || !grad_y) return TCONV_ERR_INVALID_ARG;
+    if (g.mode == TCONV_PARALLEL && !w2) return TCONV_ERR_INVALID_ARG;
+    if (misaligned(x) || misaligned(w) || misaligned(w2) || misaligned(alpha) || misaligned(beta) ||
+        misaligned(grad_y) || misaligned(winners) || misaligned(grad_x) || misaligned(grad_w) ||
+        misaligned(grad_w2) || misaligned(grad_alpha) || misaligned(grad_beta) ||
+        misaligned(grad_bias) || misaligned(workspace))
+        return TCONV_ERR_MISALIGNED;
+    if (!two_branch(g.mode)) { alpha = nullptr; beta = nullptr; grad_alpha = nullptr; grad_beta = nullptr; }
+    if (g.mode != TCONV_PARALLEL) grad_w2 = nullptr;
+    cudaStream_t st = (cudaStream_t)stream;
+    g_last_error[0] = 0;
+    char* ws = (char*)workspace;
+    size_t ws_left = workspace_bytes;
+    if (!winners) {
+        // recompute the winners with a forward pass whose y lands nowhere useful:
+        // the generic and tiled kernels need a y pointer, so the pass is run with
+        // winners only (y == NULL is accepted internally).
+        const size_t wb = align_up(winner_bytes(g), 256);
+        if (!ws || ws_left < wb) return TCONV_ERR_WORKSPACE_TOO_SMALL;
+        void* wbuf = ws;
+        ws += wb;
+        ws_left -= wb;
+        rc = (desc->dtype == TCONV_F32)
+                 ? forward_t<float>(g, x, w, w2, alpha, beta, nullptr, nullptr, wbuf, st)
+                 : forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, nullptr, nullptr, wbuf, st);
+        if (rc != TCONV_OK) return rc;
+        winners = wbuf;
+    }
+    if (desc->dtype == TCONV_F32)
+        return backward_t<float>(g, x, w, w2, alpha, beta, grad_y, winners, grad_x, grad_w, grad_w2,
+                                 grad_alpha, grad_beta, grad_bias, ws, ws_left, st);
+    return backward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, grad_y, winners, grad_x, grad_w,
+                                     grad_w2, grad_alpha, grad_beta, grad_bias, ws, ws_left, st);
+}
+
+double tconv_paper_ops(const tconv_desc_t* desc) {
+    Geo g;
+    if (make_geo(desc, &g) != TCONV_OK) return 0.0;
+    const double P = (double)g.N * g.K * g.OH * g.OW, C = g.C, RS = g.RS;
+    if (g.mode == TCONV_COMPOUND) return ((RS * C + 2 * C - 1) + 2 * (RS - 1) * C + 2 * C) * P;
+    if (g.mode == TCONV_PARALLEL) return ((2 * RS * C + 2 * C - 1) + 2 * (RS - 1) * C + 2 * C) * P;
+    if (g.chan == CH_SUM) return ((C - 1 + RS * C) + (RS - 1) * C) * P;
+    return (RS * C + (RS * C - 1)) * P;
+}
+
+int tconv_alu_probe(int variant, int iters, void* sink, double* taps_per_launch, void* stream) {
+    if (variant < 0 || variant >= PROBE_COUNT || iters <= 0 || !sink) return TCONV_ERR_INVALID_ARG;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const unsigned blocks = (unsigned)sms * 8u;
+    cudaStream_t st = (cudaStream_t)stream;
+    const float seed = 1.0009765625f;
+#define TCONV_PROBE_CASE(V) \
+    case V: alu_probe_kernel<V><<<blocks, 256, 0, st>>>(iters, seed, (float*)sink); break;
+    switch (variant) {
+        TCONV_PROBE_CASE(0) TCONV_PROBE_CASE(1) TCONV_PROBE_CASE(2) TCONV_PROBE_CASE(3)
+        TCONV_PROBE_CASE(4) TCONV_PROBE_CASE(5) TCONV_PROBE_CASE(6) TCONV_PROBE_CASE(7)
+        TCONV_PROBE_CASE(8) TCONV_PROBE_CASE(9) TCONV_PROBE_CASE(10) TCONV_PROBE_CASE(11)
+        TCONV_PROBE_CASE(12) TCONV_PROBE_CASE(13) TCONV_PROBE_CASE(14)
+    }
+#undef TCONV_PROBE_CASE
+    if (taps_per_launch)
+        *taps_per_launch = (double)blocks * 256.0 * iters * probe_taps_per_iter(variant);
+    return check_launch();
+}
+
+const char* tconv_alu_probe_name(int variant) {
+    if (variant < 0 || variant >= PROBE_COUNT) return nullptr;
+    return kProbeNames[variant];
+}
+
+const char* tconv_status_string(int status) {
+    switch (status) {
+        case TCONV_OK: return "ok";
+        case TCONV_ERR_INVALID_ARG: return "invalid argument";
+        case TCONV_ERR_UNSUPPORTED: return "unsupported descriptor";
+        case TCONV_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+        case TCONV_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case TCONV_ERR_CUDA: return "CUDA error";
+        case TCONV_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case TCONV_ERR_TOO_LARGE: return "size too large";
+        default: return "unknown status";
+    }
+}
+
+const char* tconv_last_error(void) { return g_last_error; }
+const char* tconv_last_kernel(void) { return g_last_kernel; }
+
+}  // extern "C"

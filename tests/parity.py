@@ -1,0 +1,127 @@
+"""Helpers of the GPU parity tests: run one layer through the C ABI (via the thin
+binding) and through the CPU oracle on the same seeded inputs, and compare."""
+import numpy as np
+import torch
+
+from oracle import tconv_oracle as ora
+from paper_2504_06881_b200 import inputs, tconv
+
+# tolerances of the contract: forward outputs and winners bit-exact (+0 == -0);
+# gradients within rtol * sum|contribution| elementwise (the summation error bound)
+RTOL_GRAD = {"f32": 1e-5, "bf16": 2e-2}
+
+
+def same_bits(a, b):
+    a = np.asarray(a, np.float32); b = np.asarray(b, np.float32)
+    return (a.view(np.uint32) == b.view(np.uint32)) | ((a == 0) & (b == 0))
+
+
+def to_dev(t, d, dev="cuda"):
+    """numpy layer tensors -> CUDA tensors in the layer's dtypes."""
+    dt = tconv.TORCH_DTYPE[d["dtype"]]
+    out = {}
+    for k, v in t.items():
+        tt = torch.from_numpy(v).to(dev)
+        out[k] = tt.to(dt).contiguous() if k in ("x", "w", "w2", "g") else tt.contiguous()
+    return out
+
+
+def layer_args(d, t):
+    two = d["mode"] in ("compound", "parallel")
+    return dict(w2=t["w2"] if d["mode"] == "parallel" else None,
+                alpha=t["alpha"] if two else None, beta=t["beta"] if two else None)
+
+
+def winners_as_numpy(d, winners):
+    N, C, K = d["N"], d["C"], d["K"]
+    OH, OW = inputs.output_hw(d)
+    chan = ora.resolved_chan(d)
+    raw = winners.cpu().numpy()
+    if chan != "sum":
+        return raw.view(np.int32).reshape(N, K, OH, OW)
+    if d["R"] * d["S"] <= 16:
+        return raw.reshape(N, K, C, OH, OW)
+    return raw.view(np.uint16).reshape(N, K, C, OH, OW)
+
+
+def oracle_wide_codes(d, t, la):
+    """Sum-form winners for windows of more than 16 taps (the oracle emits nibble codes only
+    up to 16 taps): rebuilt per channel from single-channel Max/Min runs of the oracle."""
+    N, C, K = d["N"], d["C"], d["K"]
+    OH, OW = inputs.output_hw(d)
+    codes = np.zeros((N, K, C, OH, OW), np.uint16)
+    for c in range(C):
+        d1 = dict(d, C=1)
+        x1 = np.ascontiguousarray(t["x"][:, c:c + 1])
+        if d["mode"] in ("min_plus", "compound", "parallel"):
+            o = ora.forward(dict(d1, mode="min_plus", chan="min"), x1,
+                            np.ascontiguousarray(t["w"][:, c:c + 1]))
+            codes[:, :, c] |= o["idx"].astype(np.uint16)
+        if d["mode"] in ("max_plus", "compound", "parallel"):
+            wm = t["w2"] if d["mode"] == "parallel" else t["w"]
+            o = ora.forward(dict(d1, mode="max_plus", chan="max"), x1,
+                            np.ascontiguousarray(wm[:, c:c + 1]))
+            codes[:, :, c] |= (o["idx"].astype(np.uint16) << 8)
+    return codes
+
+
+def check_forward(d, t, use_bias=True, check_winners=True):
+    """GPU forward vs oracle: y and winners bit-exact.  Returns (gpu tensors, y, winners)."""
+    la = layer_args(d, t)
+    bias = t["bias"] if use_bias else None
+    ref = ora.forward(d, t["x"], t["w"], la["w2"], la["alpha"], la["beta"], bias)
+    g = to_dev(t, d)
+    ga = layer_args(d, g)
+    y, winners = tconv.forward(d, g["x"], g["w"], ga["w2"], ga["alpha"], ga["beta"],
+                               g["bias"] if use_bias else None, want_winners=check_winners)
+    torch.cuda.synchronize()
+    yg = y.float().cpu().numpy()
+    ok = same_bits(yg, ref["y"])
+    assert ok.all(), (f"{d}: {int((~ok).sum())} of {ok.size} outputs differ; first at "
+                      f"{np.argwhere(~ok)[0]}: gpu {yg[~ok][0]!r} ref {ref['y'][~ok][0]!r} "
+                      f"[{tconv.tconv_last_kernel()}]")
+    if check_winners:
+        wg = winners_as_numpy(d, winners)
+        want = ref["idx"] if ref["idx"] is not None else ref["codes"]
+        if want is None:
+            want = oracle_wide_codes(d, t, la)
+        assert np.array_equal(wg, want), (f"{d}: {int((wg != want).sum())} winners differ "
+                                          f"[{tconv.tconv_last_kernel()}]")
+    return g, y, winners
+
+
+def compare_grads(d, got: dict, ref: dict, rtol=None):
+    rtol = RTOL_GRAD[d["dtype"]] if rtol is None else rtol
+    report = {}
+    for name, (rv, ra) in ref.items():
+        if name not in got:
+            continue
+        gv = got[name].float().cpu().numpy().astype(np.float64)
+        err = np.abs(gv - rv)
+        bound = rtol * ra + 1e-30
+        bad = err > bound
+        scale = max(np.abs(rv).max(), 1e-30)
+        report[name] = float(err.max() / scale)
+        assert not bad.any(), (f"{d} {name}: {int(bad.sum())} of {bad.size} elements off; worst "
+                               f"err {err[bad].max():.3e} vs bound {bound[bad][err[bad].argmax()]:.3e} "
+                               f"[{tconv.tconv_last_kernel()}]")
+    return report
+
+
+def check_layer(d, dists=None, seed=0, use_bias=True, stored_winners=True, recompute=True):
+    """Forward + backward parity of one layer.  Returns the normwise gradient errors."""
+    t = inputs.draw(d, seed, **(dists or {}))
+    g, y, winners = check_forward(d, t, use_bias=use_bias)
+    la = layer_args(d, t)
+    ref = ora.backward(d, t["x"], t["w"], t["g"], la["w2"], la["alpha"], la["beta"])
+    ga = layer_args(d, g)
+    rep = {}
+    if stored_winners:
+        got = tconv.backward(d, g["x"], g["w"], g["g"], ga["w2"], ga["alpha"], ga["beta"], winners)
+        torch.cuda.synchronize()
+        rep = compare_grads(d, got, ref)
+    if recompute:
+        got = tconv.backward(d, g["x"], g["w"], g["g"], ga["w2"], ga["alpha"], ga["beta"], None)
+        torch.cuda.synchronize()
+        rep = compare_grads(d, got, ref)
+    return rep

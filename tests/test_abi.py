@@ -1,0 +1,70 @@
+"""The C-ABI library loads, exports every declared symbol, and its host-side checks work
+(no compute call needs a GPU here)."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+from paper_2504_06881_b200 import inputs, tconv
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+def test_every_declared_symbol_is_exported():
+    header = (ROOT / "include" / "tconv.h").read_text()
+    declared = set(re.findall(r"\b(tconv_[a-z0-9_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    lib = ctypes.CDLL(str(tconv.LIB_PATH))
+    for name in declared:
+        assert hasattr(lib, name), f"{name} declared in tconv.h but not exported"
+    assert declared == set(tconv.SYMBOLS)
+
+
+def test_output_shape_and_sizes():
+    d = inputs.layer(2, 3, 32, 32, 16, 3, 3, stride=1, pad=1, mode="compound")
+    assert tconv.tconv_output_shape(d) == (32, 32)
+    assert tconv.tconv_winner_bytes(d) == 2 * 16 * 3 * 32 * 32
+    assert tconv.tconv_winner_bytes(dict(d, mode="max_plus")) == 4 * 2 * 16 * 32 * 32
+    assert tconv.tconv_winner_bytes(dict(d, R=5, S=5)) == 2 * 2 * 16 * 3 * 30 * 30
+    assert tconv.tconv_workspace_bytes(d, True) >= tconv.tconv_winner_bytes(d)
+    d2 = inputs.layer(1, 1, 56, 56, 1, 3, 3, stride=2, pad=1, dil=1)
+    assert tconv.tconv_output_shape(d2) == (28, 28)
+    d3 = inputs.layer(1, 1, 128, 256, 1, 3, 3, stride=1, pad=2, dil=2)
+    assert tconv.tconv_output_shape(d3) == (128, 256)
+
+
+def test_paper_op_counts_match_section_4_1():
+    N, C, H, W, K, R, S = 2, 5, 9, 8, 3, 3, 3
+    P = N * K * 7 * 6
+    d = inputs.layer(N, C, H, W, K, R, S)
+    assert tconv.tconv_paper_ops(dict(d, mode="max_plus")) == (2 * R * S * C - 1) * P
+    assert tconv.tconv_paper_ops(dict(d, mode="min_plus", chan="sum")) == \
+        ((C - 1 + R * S * C) + (R * S - 1) * C) * P
+    assert tconv.tconv_paper_ops(dict(d, mode="compound")) == \
+        ((R * S * C + 2 * C - 1) + 2 * (R * S - 1) * C + 2 * C) * P
+    assert tconv.tconv_paper_ops(dict(d, mode="parallel")) == \
+        ((2 * R * S * C + 2 * C - 1) + 2 * (R * S - 1) * C + 2 * C) * P
+
+
+def test_host_side_argument_checks():
+    d = inputs.layer(1, 1, 4, 4, 1, 3, 3)
+    with pytest.raises(tconv.TconvError):
+        tconv.tconv_output_shape(dict(d, H=0))
+    with pytest.raises(tconv.TconvError):
+        tconv.tconv_output_shape(dict(d, H=2))          # window larger than the padded input
+    with pytest.raises(tconv.TconvError) as e:
+        tconv.tconv_output_shape(dict(d, mode="compound", chan="max"))
+    assert e.value.status == -2
+    assert tconv.tconv_winner_bytes(dict(d, stride_h=0)) == 0
+    lib = ctypes.CDLL(str(tconv.LIB_PATH))
+    lib.tconv_forward.restype = ctypes.c_int
+    desc = tconv.make_desc(d)
+    vp = ctypes.c_void_p
+    args = [ctypes.byref(desc)] + [vp(0)] * 9 + [ctypes.c_size_t(0), vp(0)]
+    assert lib.tconv_forward(*args) == -1                # NULL tensors
+    args[1] = vp(0x1008); args[2] = vp(0x1000); args[7] = vp(0x1000)
+    assert lib.tconv_forward(*args) == -3                # misaligned x
+    assert tconv.tconv_status_string(-3).startswith("pointer")
+    assert tconv.tconv_alu_probe_name(0) == "f32_add_max2"
+    assert tconv.tconv_alu_probe_name(10_000) is None
