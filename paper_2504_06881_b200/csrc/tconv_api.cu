@@ -86,11 +86,12 @@ bool force_generic() {
 
 template <typename T>
 int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const float* alpha,
-              const float* beta, const float* bias, void* y, void* winners, cudaStream_t st) {
+              const float* beta, const float* bias, void* y, void* winners, void* ws,
+              size_t ws_bytes, cudaStream_t st) {
     if (!force_generic()) {
         const char* name = nullptr;
         const int rc = launch_fwd_tiled<T>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta,
-                                           bias, (T*)y, winners, st, &name);
+                                           bias, (T*)y, winners, ws, ws_bytes, st, &name);
         if (rc == TCONV_OK) {
             snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", name);
             return check_launch();
@@ -152,9 +153,10 @@ size_t tconv_winner_bytes(const tconv_desc_t* desc) {
 size_t tconv_workspace_bytes(const tconv_desc_t* desc, int backward) {
     Geo g;
     if (make_geo(desc, &g) != TCONV_OK) return 0;
-    if (!backward) return 0;
-    // winners recomputed into the workspace when the caller passes none
-    return align_up(winner_bytes(g), 256);
+    const size_t fwd = align_up(tiled_ws_bytes(g), 256);  // repacked weights, alpha, beta
+    if (!backward) return fwd;
+    // winners recomputed (by a forward pass) into the workspace when the caller passes none
+    return align_up(winner_bytes(g), 256) + fwd;
 }
 
 int tconv_forward(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,
@@ -173,8 +175,10 @@ int tconv_forward(const tconv_desc_t* desc, const void* x, const void* w, const 
     cudaStream_t st = (cudaStream_t)stream;
     g_last_error[0] = 0;
     if (desc->dtype == TCONV_F32)
-        return forward_t<float>(g, x, w, w2, alpha, beta, bias, y, winners, st);
-    return forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, bias, y, winners, st);
+        return forward_t<float>(g, x, w, w2, alpha, beta, bias, y, winners, workspace,
+                                workspace_bytes, st);
+    return forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, bias, y, winners, workspace,
+                                    workspace_bytes, st);
 }
 
 int tconv_backward(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,
@@ -199,17 +203,17 @@ int tconv_backward(const tconv_desc_t* desc, const void* x, const void* w, const
     char* ws = (char*)workspace;
     size_t ws_left = workspace_bytes;
     if (!winners) {
-        // recompute the winners with a forward pass whose y lands nowhere useful:
-        // the generic and tiled kernels need a y pointer, so the pass is run with
-        // winners only (y == NULL is accepted internally).
+        // recompute the winners with a forward pass that stores winners only
+        // (the kernels accept y == NULL internally)
         const size_t wb = align_up(winner_bytes(g), 256);
         if (!ws || ws_left < wb) return TCONV_ERR_WORKSPACE_TOO_SMALL;
         void* wbuf = ws;
         ws += wb;
         ws_left -= wb;
         rc = (desc->dtype == TCONV_F32)
-                 ? forward_t<float>(g, x, w, w2, alpha, beta, nullptr, nullptr, wbuf, st)
-                 : forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, nullptr, nullptr, wbuf, st);
+                 ? forward_t<float>(g, x, w, w2, alpha, beta, nullptr, nullptr, wbuf, ws, ws_left, st)
+                 : forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, nullptr, nullptr, wbuf, ws,
+                                            ws_left, st);
         if (rc != TCONV_OK) return rc;
         winners = wbuf;
     }
