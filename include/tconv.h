@@ -71,7 +71,7 @@ typedef enum {
     TCONV_ERR_MISALIGNED = -3,          /* a tensor pointer is not 16-byte aligned                  */
     TCONV_ERR_WORKSPACE_TOO_SMALL = -4, /* workspace_bytes below tconv_workspace_bytes()            */
     TCONV_ERR_CUDA = -5,                /* launch failed; text in tconv_last_error()                */
-    TCONV_ERR_DEVICE_TIMEOUT = -6,      /* a bounded device-side wait gave up                       */
+    TCONV_ERR_DEVICE_TIMEOUT = -6,      /* a bounded device-side wait gave up (tconv_device_status) */
     TCONV_ERR_TOO_LARGE = -7            /* a size exceeds what the entry point supports             */
 } tconv_status_t;
 
@@ -168,6 +168,15 @@ int tconv_alu_probe(int variant, int iters, void *sink, double *taps_per_launch,
 /* Name of probe variant i, NULL past the last one.  Host call. */
 const char *tconv_alu_probe_name(int variant);
 
+/*
+ * Device-side health check.  The kernels wait for their asynchronous copies with a
+ * bounded number of polls; a wait that gives up sets a status word on the device and
+ * the kernel returns early (its outputs are then undefined).  This call synchronises
+ * `stream`, reads the word, clears it, and returns TCONV_OK or
+ * TCONV_ERR_DEVICE_TIMEOUT.
+ */
+int tconv_device_status(void *stream);
+
 /* Text for a status code.  Host call. */
 const char *tconv_status_string(int status);
 
@@ -177,6 +186,10 @@ const char *tconv_last_error(void);
 /* Name of the kernel variant the last tconv_forward / tconv_backward of this
  * thread launched (for benchmark records).  Host call. */
 const char *tconv_last_kernel(void);
+
+/* Number of GPU kernels the calling thread's calls into this library have launched so
+ * far (cumulative).  Host call. */
+long long tconv_launch_count(void);
 
 #ifdef __cplusplus
 }

@@ -11,10 +11,49 @@
 
 using namespace tconv;
 
+namespace tconv {
+// tiled forward launchers, one per (mode, channel combine) translation unit
+int fwd_inst_maxplus_sum(FwdArgs&);
+int fwd_inst_maxplus_max(FwdArgs&);
+int fwd_inst_maxplus_min(FwdArgs&);
+int fwd_inst_minplus_sum(FwdArgs&);
+int fwd_inst_minplus_max(FwdArgs&);
+int fwd_inst_minplus_min(FwdArgs&);
+int fwd_inst_compound(FwdArgs&);
+int fwd_inst_parallel(FwdArgs&);
+}  // namespace tconv
+
+// Set non-zero by a kernel whose bounded wait on a copy gave up.
+__device__ int g_tconv_device_status;
+
 namespace {
+
+int* device_status_ptr() {
+    static int* ptrs[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_tconv_device_status) != cudaSuccess) return nullptr;
+        ptrs[dev] = (int*)p;
+    }
+    return ptrs[dev];
+}
+
+int launch_fwd_tiled(FwdArgs& a) {
+    const Geo& g = a.g;
+    if (g.mode == TCONV_COMPOUND) return fwd_inst_compound(a);
+    if (g.mode == TCONV_PARALLEL) return fwd_inst_parallel(a);
+    if (g.mode == TCONV_MAX_PLUS)
+        return g.chan == CH_MAX ? fwd_inst_maxplus_max(a)
+               : g.chan == CH_MIN ? fwd_inst_maxplus_min(a) : fwd_inst_maxplus_sum(a);
+    return g.chan == CH_MAX ? fwd_inst_minplus_max(a)
+           : g.chan == CH_MIN ? fwd_inst_minplus_min(a) : fwd_inst_minplus_sum(a);
+}
 
 thread_local char g_last_error[256] = "";
 thread_local char g_last_kernel[128] = "";
+thread_local long long g_launches = 0;  // kernels launched by this thread's calls
 
 int cuda_fail(cudaError_t e) {
     snprintf(g_last_error, sizeof(g_last_error), "%s", cudaGetErrorString(e));
@@ -89,11 +128,15 @@ int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const 
               const float* beta, const float* bias, void* y, void* winners, void* ws,
               size_t ws_bytes, cudaStream_t st) {
     if (!force_generic()) {
-        const char* name = nullptr;
-        const int rc = launch_fwd_tiled<T>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta,
-                                           bias, (T*)y, winners, ws, ws_bytes, st, &name);
+        FwdArgs a;
+        a.g = g; a.dtype = sizeof(T) == 4 ? TCONV_F32 : TCONV_BF16;
+        a.x = x; a.w = w; a.w2 = w2; a.alpha = alpha; a.beta = beta; a.bias = bias;
+        a.y = y; a.winners = winners; a.ws = ws; a.ws_bytes = ws_bytes;
+        a.status = device_status_ptr(); a.st = st; a.name = "";
+        const int rc = launch_fwd_tiled(a);
         if (rc == TCONV_OK) {
-            snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", name);
+            snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", a.name);
+            g_launches += 2;  // weight repack + tiled kernel
             return check_launch();
         }
         if (rc != TCONV_ERR_UNSUPPORTED) return rc;
@@ -103,6 +146,7 @@ int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const 
     fwd_generic_kernel<T><<<blocks, 256, 0, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha,
                                                   beta, bias, (T*)y, winners);
     snprintf(g_last_kernel, sizeof(g_last_kernel), "fwd_generic");
+    g_launches += 1;
     return check_launch();
 }
 
@@ -117,16 +161,22 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
         const size_t total = (size_t)g.N * g.C * g.H * g.W;
         bwd_gx_generic_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
             g, alpha, beta, (const T*)gy, winners, (T*)gx);
+        g_launches += 1;
     }
     if (gw || gw2) {
         bwd_gw_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C * g.RS), 256, 0, st>>>(
             g, alpha, beta, (const T*)gy, winners, gw, gw2);
+        g_launches += 1;
     }
     if (twob && (galpha || gbeta)) {
         bwd_gab_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C), 256, 0, st>>>(
             g, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, winners, galpha, gbeta);
+        g_launches += 1;
     }
-    if (gbias) bwd_bias_kernel<T><<<(unsigned)g.K, 256, 0, st>>>(g, (const T*)gy, gbias);
+    if (gbias) {
+        bwd_bias_kernel<T><<<(unsigned)g.K, 256, 0, st>>>(g, (const T*)gy, gbias);
+        g_launches += 1;
+    }
     snprintf(g_last_kernel, sizeof(g_last_kernel), "bwd_generic");
     return check_launch();
 }
@@ -253,6 +303,7 @@ int tconv_alu_probe(int variant, int iters, void* sink, double* taps_per_launch,
         TCONV_PROBE_CASE(12) TCONV_PROBE_CASE(13) TCONV_PROBE_CASE(14)
     }
 #undef TCONV_PROBE_CASE
+    g_launches += 1;
     if (taps_per_launch)
         *taps_per_launch = (double)blocks * 256.0 * iters * probe_taps_per_iter(variant);
     return check_launch();
@@ -277,7 +328,22 @@ const char* tconv_status_string(int status) {
     }
 }
 
+int tconv_device_status(void* stream) {
+    int* p = device_status_ptr();
+    if (!p) return cuda_fail(cudaGetLastError());
+    cudaStream_t st = (cudaStream_t)stream;
+    int v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, p, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (v == 0) return TCONV_OK;
+    e = cudaMemsetAsync(p, 0, sizeof(int), st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return TCONV_ERR_DEVICE_TIMEOUT;
+}
+
 const char* tconv_last_error(void) { return g_last_error; }
 const char* tconv_last_kernel(void) { return g_last_kernel; }
+long long tconv_launch_count(void) { return g_launches; }
 
 }  // extern "C"

@@ -1,12 +1,20 @@
-// Tiled forward kernels: the input halo tile and a repacked weight tile are staged
-// in shared memory (asynchronous copies, two stages), every thread keeps a block
-// of 8 output channels x Q x 4 pixels in registers and folds taps with packed
-// adds (two channels per instruction) and 3-input min / max.
+// Tiled forward kernels (fp32).
 //
-// A CTA owns TILE_K output channels x one tile of output pixels.  Pixel tiles are
-// TW columns wide and TH rows high, where rows run over the flattened (n, oh)
-// space, so a tile may span several images of a small feature map.
+// A CTA owns TILE_K output channels x one tile of output pixels and walks the
+// input channels in chunks of CC.  Per chunk the input halo tile (zero padding
+// comes from the copy engine's out-of-bounds fill) and the repacked weights of
+// the chunk are brought into shared memory by TMA: one tiled tensor copy for x,
+// one bulk copy for each weight / alpha / beta block, all signalling one mbarrier
+// per stage (two stages).  Feature maps whose rows are not 16-byte multiples, or
+// tiles that span several images of a small map, take per-element asynchronous
+// copies instead.  Every thread keeps 8 output channels x Q x 4 pixels in
+// registers and folds taps with packed adds (two channels per instruction) and
+// 3-input min / max.
 #pragma once
+#include <cuda.h>
+
+#include <cstring>
+
 #include "tconv_common.cuh"
 
 namespace tconv {
@@ -30,18 +38,80 @@ __device__ __forceinline__ void add2(float x, float wlo, float whi, float& lo, f
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(tt) : "l"(xx), "l"(ww));
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
 }
+__device__ __forceinline__ unsigned smem_u32(const void* p) {
+    return (unsigned)__cvta_generic_to_shared(p);
+}
 __device__ __forceinline__ void cp_async4(void* smem, const void* gmem, bool valid) {
-    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
     const int n = valid ? 4 : 0;  // 0 source bytes: the destination is zero-filled
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(s), "l"(gmem), "r"(n));
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(smem)), "l"(gmem), "r"(n) : "memory");
 }
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem)), "l"(gmem) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N));
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// mbarrier + TMA (single-CTA use; no multicast anywhere)
+__device__ __forceinline__ void mbar_init(void* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(void* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait: gives up after a fixed number of polls and reports failure.
+__device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity) {
+    const unsigned addr = smem_u32(bar);
+    for (int i = 0; i < (1 << 20); ++i) {
+        unsigned ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_3d(void* smem, const CUtensorMap* map, int c0, int c1,
+                                            int c2, void* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(smem)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* smem, const void* gmem, unsigned bytes, void* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(smem)), "l"(gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// L floats starting SHIFT floats past a 16-byte aligned shared-memory address, with the
+// widest aligned vector loads the position allows.
+template <int SHIFT, int L, int I = 0>
+__device__ __forceinline__ void load_segment(const float* base, float* out) {
+    if constexpr (I < L) {
+        constexpr int pos = SHIFT + I;
+        if constexpr ((pos % 4 == 0) && (I + 4 <= L)) {
+            const float4 v = *reinterpret_cast<const float4*>(base + pos);
+            out[I] = v.x; out[I + 1] = v.y; out[I + 2] = v.z; out[I + 3] = v.w;
+            load_segment<SHIFT, L, I + 4>(base, out);
+        } else if constexpr ((pos % 2 == 0) && (I + 2 <= L)) {
+            const float2 v = *reinterpret_cast<const float2*>(base + pos);
+            out[I] = v.x; out[I + 1] = v.y;
+            load_segment<SHIFT, L, I + 2>(base, out);
+        } else {
+            out[I] = base[pos];
+            load_segment<SHIFT, L, I + 1>(base, out);
+        }
+    }
+}
+__device__ __forceinline__ void load8(const float* p, float* out) {
+    const float4 a = *reinterpret_cast<const float4*>(p);
+    const float4 b = *reinterpret_cast<const float4*>(p + 4);
+    out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+    out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
 }
 
 // ----------------------------------------------------------------------------------
@@ -92,23 +162,33 @@ struct TiledParams {
     const float* bias;
     void* y;
     void* winners;
-    int TW, QPR, TH;   // tile: output columns, quads per row, rows of the flattened (n, oh) space
+    int* status;       // device status word: set non-zero when a bounded wait gives up
+    int TW, QPR, TH;   // tile: output columns, quads per row, output rows
     int n_col_tiles, n_row_tiles;
+    int tiles_per_img; // > 0: row tiles stay inside one image; 0: rows run over the flattened (n, oh) space
     int total_rows;    // N * OH
     int NSLOTS, XW, XP;  // staged input rows per tile, staged columns, row pitch (floats)
-    int GAP;           // extra input-row slots between two images of one tile
+    int GAP;           // extra input-row slots between two images of one tile (flattened tiles)
     int CC, Cpad, nchunks;
+    int stage_floats, x_stage, w_stage, ab_stage;  // shared-memory layout of one stage (floats)
 };
 
-// fp32 tiled forward.  MODE: tconv_mode_t, CHAN: CH_SUM / CH_MAX / CH_MIN, WIN: emit winners.
+// Column shift of the TMA path: the tile's first input column ow0*SW - pw is rounded
+// down to a multiple of 4 floats so that the copy starts on a 16-byte boundary.  The
+// TMA path is used with "same" padding pw = (S-1)*DW/2 only, which fixes the shift.
+template <int S, int DW> struct TmaShift { static constexpr int value = (4 - (((S - 1) * DW / 2) % 4)) % 4; };
+
+// MODE: tconv_mode_t, CHAN: CH_SUM / CH_MAX / CH_MIN, WIN: emit winners, XTMA: x tile by TMA.
 // Q quads of 4 pixels per thread, KG groups of 8 output channels and PW pixel warps per CTA.
-template <int MODE, int CHAN, bool WIN, int R, int S, int SW, int DW, int Q, int KG, int PW>
+template <int MODE, int CHAN, bool WIN, bool XTMA, int R, int S, int SW, int DW, int Q, int KG, int PW>
 __global__ void __launch_bounds__(KG * PW * 32)
-fwd_tiled_f32_kernel(const TiledParams p) {
+fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams p) {
     constexpr int RS = R * S;
     constexpr int TILE_K = KG * 8;
     constexpr int NT = KG * PW * 32;
+    constexpr int NWARPS = KG * PW;
     constexpr int L = 3 * SW + (S - 1) * DW + 1;  // input columns one quad touches per row
+    constexpr int SHIFT = XTMA ? TmaShift<S, DW>::value : 0;
     constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
     constexpr bool PAR = (MODE == TCONV_PARALLEL);
     constexpr bool TAP_MIN = (MODE == TCONV_MIN_PLUS);  // tap-level extremum of single-branch modes
@@ -118,13 +198,10 @@ fwd_tiled_f32_kernel(const TiledParams p) {
                               (MODE == TCONV_MIN_PLUS && CHAN == CH_MIN));
     const Geo& g = p.g;
 
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int x_stage = p.CC * p.NSLOTS * p.XP;          // floats
-    const int w_stage = p.CC * RS * TILE_K;              // floats
-    const int ab_stage = TWO ? p.CC * TILE_K : 0;        // floats (each of alpha, beta)
-    const int stage_floats = x_stage + w_stage * (PAR ? 2 : 1) + 2 * ab_stage;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     float* stage0 = reinterpret_cast<float*>(smem_raw);
-    int* slot_off = reinterpret_cast<int*>(stage0 + 2 * stage_floats);
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(stage0 + 2 * p.stage_floats);
+    int* slot_off = reinterpret_cast<int*>(bars + 2);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int kg = warp % KG, wp = warp / KG;
@@ -132,15 +209,30 @@ fwd_tiled_f32_kernel(const TiledParams p) {
     const int rt = blockIdx.x / p.n_col_tiles;
     const int kt = blockIdx.y;
     const int ow0 = ct * p.TW;
-    const int row0 = rt * p.TH;
+    int row0, rows_here;
+    if (p.tiles_per_img > 0) {
+        const int n = rt / p.tiles_per_img;
+        const int oh0 = (rt - n * p.tiles_per_img) * p.TH;
+        row0 = n * g.OH + oh0;
+        rows_here = min(p.TH, g.OH - oh0);
+    } else {
+        row0 = rt * p.TH;
+        rows_here = min(p.TH, p.total_rows - row0);
+    }
     const int iw0 = ow0 * SW - g.pw;
     const int n0 = row0 / g.OH;
+    const int oh_first = row0 - n0 * g.OH;
 
-    // input-row slot table: element offset of the row start inside x (per channel 0), or -1
-    for (int sl = tid; sl < p.NSLOTS; sl += NT) slot_off[sl] = -1;
-    __syncthreads();
-    {
-        const int rows_here = min(p.TH, p.total_rows - row0);
+    if constexpr (XTMA) {
+        if (tid == 0) {
+            mbar_init(&bars[0], 1);
+            mbar_init(&bars[1], 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+    } else {
+        // input-row slot table: element offset of the row start inside x (channel 0), or -1
+        for (int sl = tid; sl < p.NSLOTS; sl += NT) slot_off[sl] = -1;
+        __syncthreads();
         const int span = (R - 1) * g.dh + 1;
         for (int e = tid; e < rows_here * span; e += NT) {
             const int lr = e / span, dr = e - lr * span;
@@ -148,7 +240,7 @@ fwd_tiled_f32_kernel(const TiledParams p) {
             const int n = gr / g.OH, oh = gr - n * g.OH;
             const int ih = oh * g.sh - g.ph + dr;
             const int sl = lr * g.sh + (n - n0) * p.GAP + dr;
-            if (ih >= 0 && ih < g.H) slot_off[sl] = (n * g.C * g.H + ih) * g.W;  // several writers, one value
+            if (ih >= 0 && ih < g.H) slot_off[sl] = (n * g.C * g.H + ih) * g.W;  // writers agree
         }
     }
     __syncthreads();
@@ -162,7 +254,7 @@ fwd_tiled_f32_kernel(const TiledParams p) {
         const int qi = wp * 32 + lane + q * (32 * PW);
         int lr = qi / p.QPR;
         const int qx = qi - lr * p.QPR;
-        const bool ok = (lr < p.TH) && (row0 + lr < p.total_rows);
+        const bool ok = (lr < rows_here);
         if (!ok) lr = 0;
         const int gr = row0 + lr;
         const int n = gr / g.OH;
@@ -177,39 +269,57 @@ fwd_tiled_f32_kernel(const TiledParams p) {
     const float* wt2_k = PAR ? p.wt2 + (size_t)kt * p.Cpad * RS * TILE_K : nullptr;
     const float* at_k = TWO ? p.at + (size_t)kt * p.Cpad * TILE_K : nullptr;
     const float* bt_k = TWO ? p.bt + (size_t)kt * p.Cpad * TILE_K : nullptr;
+    const int w_off = p.x_stage, w2_off = p.x_stage + p.w_stage;
+    const int a_off = p.x_stage + p.w_stage * (PAR ? 2 : 1), b_off = a_off + p.ab_stage;
 
-    auto issue_chunk = [&](int ch, float* st) {
+    auto issue_chunk = [&](int ch, int s) {
+        float* st = stage0 + s * p.stage_floats;
         const int c0 = ch * p.CC;
-        // x halo tile: one warp per (channel, slot) row, lanes along the columns
-        float* xs = st;
-        for (int rowi = warp; rowi < p.CC * p.NSLOTS; rowi += KG * PW) {
-            const int cc = rowi / p.NSLOTS, sl = rowi - cc * p.NSLOTS;
-            const int off = slot_off[sl];
-            const bool rok = (off >= 0) && (c0 + cc < g.C);
-            const float* src_row = xg + (rok ? (size_t)off + (size_t)(c0 + cc) * chw : 0);
-            float* dst_row = xs + (size_t)rowi * p.XP;
-            for (int col = lane; col < p.XW; col += 32) {
-                const int iw = iw0 + col;
-                const bool ok = rok && iw >= 0 && iw < g.W;
-                cp_async4(dst_row + col, ok ? src_row + iw : xg, ok);
+        if constexpr (XTMA) {
+            if (tid == 0) {
+                const unsigned bytes = (unsigned)((p.CC * p.NSLOTS * p.XP + p.w_stage * (PAR ? 2 : 1) + 2 * p.ab_stage) * sizeof(float));
+                mbar_expect_tx(&bars[s], bytes);
+                tma_load_3d(st, &xmap, iw0 - SHIFT, oh_first * g.sh - g.ph, n0 * g.C + c0, &bars[s]);
+                bulk_load(st + w_off, wt_k + (size_t)c0 * RS * TILE_K, p.w_stage * sizeof(float), &bars[s]);
+                if (PAR) bulk_load(st + w2_off, wt2_k + (size_t)c0 * RS * TILE_K, p.w_stage * sizeof(float), &bars[s]);
+                if (TWO) {
+                    bulk_load(st + a_off, at_k + (size_t)c0 * TILE_K, p.ab_stage * sizeof(float), &bars[s]);
+                    bulk_load(st + b_off, bt_k + (size_t)c0 * TILE_K, p.ab_stage * sizeof(float), &bars[s]);
+                }
             }
-        }
-        // weights (and alpha, beta): contiguous blocks, 16 bytes per copy
-        float* ws = st + x_stage;
-        const float* wsrc = wt_k + (size_t)c0 * RS * TILE_K;
-        for (int e = tid; e < w_stage / 4; e += NT) cp_async16(ws + e * 4, wsrc + e * 4);
-        if (PAR) {
-            const float* wsrc2 = wt2_k + (size_t)c0 * RS * TILE_K;
-            for (int e = tid; e < w_stage / 4; e += NT) cp_async16(ws + w_stage + e * 4, wsrc2 + e * 4);
-        }
-        if (TWO) {
-            float* as = st + x_stage + w_stage * (PAR ? 2 : 1);
-            for (int e = tid; e < ab_stage / 4; e += NT) {
-                cp_async16(as + e * 4, at_k + (size_t)c0 * TILE_K + e * 4);
-                cp_async16(as + ab_stage + e * 4, bt_k + (size_t)c0 * TILE_K + e * 4);
+        } else {
+            // x halo tile: one warp per (channel, slot) row, lanes along the columns
+            for (int cc = 0; cc < p.CC; ++cc) {
+                const bool cok = (c0 + cc < g.C);
+                const float* src_c = xg + (size_t)(cok ? c0 + cc : 0) * chw;
+                float* dst_c = st + (size_t)cc * p.NSLOTS * p.XP;
+                for (int sl = warp; sl < p.NSLOTS; sl += NWARPS) {
+                    const int off = slot_off[sl];
+                    const bool rok = cok && (off >= 0);
+                    const float* src_row = src_c + (rok ? off : 0);
+                    float* dst_row = dst_c + sl * p.XP;
+                    for (int col = lane; col < p.XW; col += 32) {
+                        const int iw = iw0 + col;
+                        const bool ok = rok && iw >= 0 && iw < g.W;
+                        cp_async4(dst_row + col, ok ? src_row + iw : xg, ok);
+                    }
+                }
             }
+            // weights (and alpha, beta): contiguous blocks, 16 bytes per copy
+            const float* wsrc = wt_k + (size_t)c0 * RS * TILE_K;
+            for (int e = tid; e < p.w_stage / 4; e += NT) cp_async16(st + w_off + e * 4, wsrc + e * 4);
+            if (PAR) {
+                const float* wsrc2 = wt2_k + (size_t)c0 * RS * TILE_K;
+                for (int e = tid; e < p.w_stage / 4; e += NT) cp_async16(st + w2_off + e * 4, wsrc2 + e * 4);
+            }
+            if (TWO) {
+                for (int e = tid; e < p.ab_stage / 4; e += NT) {
+                    cp_async16(st + a_off + e * 4, at_k + (size_t)c0 * TILE_K + e * 4);
+                    cp_async16(st + b_off + e * 4, bt_k + (size_t)c0 * TILE_K + e * 4);
+                }
+            }
+            cp_async_commit();
         }
-        cp_async_commit();
     };
 
     // accumulators
@@ -226,20 +336,30 @@ fwd_tiled_f32_kernel(const TiledParams p) {
             }
 
     const size_t plane = (size_t)g.OH * g.OW;
-    issue_chunk(0, stage0);
+    const int row_step = g.dh * p.XP;
+    const int chan_step = p.NSLOTS * p.XP;
+    issue_chunk(0, 0);
     for (int ch = 0; ch < p.nchunks; ++ch) {
-        float* st = stage0 + (ch & 1) * stage_floats;
-        if (ch + 1 < p.nchunks) {
-            issue_chunk(ch + 1, stage0 + ((ch + 1) & 1) * stage_floats);
-            cp_async_wait<1>();
+        const int s = ch & 1;
+        float* st = stage0 + s * p.stage_floats;
+        if (ch + 1 < p.nchunks) issue_chunk(ch + 1, s ^ 1);
+        if constexpr (XTMA) {
+            if (!mbar_wait(&bars[s], (ch >> 1) & 1)) {
+                // the copy did not land in time: flag it, give the copies in flight one more
+                // bounded chance to finish, and leave
+                if (p.status) *p.status = 1;
+                mbar_wait(&bars[s], (ch >> 1) & 1);
+                if (ch + 1 < p.nchunks) mbar_wait(&bars[s ^ 1], ((ch + 1) >> 1) & 1);
+                return;
+            }
         } else {
-            cp_async_wait<0>();
+            if (ch + 1 < p.nchunks) cp_async_wait<1>(); else cp_async_wait<0>();
+            __syncthreads();
         }
-        __syncthreads();
-        const float* xs = st;
-        const float* ws = st + x_stage + kg * 8;
-        const float* ws2 = ws + w_stage;
-        const float* as = st + x_stage + w_stage * (PAR ? 2 : 1) + kg * 8;
+        const float* ws = st + w_off + kg * 8;
+        const float* ws2 = st + w2_off + kg * 8;
+        const float* as = st + a_off + kg * 8;
+        const float* bs = st + b_off + kg * 8;
         const int nc = min(p.CC, g.C - ch * p.CC);
         for (int cc = 0; cc < nc; ++cc) {
             // the R rows of input this thread's quads touch in channel cc
@@ -247,21 +367,10 @@ fwd_tiled_f32_kernel(const TiledParams p) {
 #pragma unroll
             for (int q = 0; q < Q; ++q)
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const float* src = xs + (size_t)cc * p.NSLOTS * p.XP + xoff[q] + r * g.dh * p.XP;
-#pragma unroll
-                    for (int i = 0; i + 4 <= L; i += 4) {
-                        const float4 v = *reinterpret_cast<const float4*>(src + i);
-                        xr[q][r][i] = v.x; xr[q][r][i + 1] = v.y; xr[q][r][i + 2] = v.z; xr[q][r][i + 3] = v.w;
-                    }
-                    if constexpr ((L & 3) >= 2) {
-                        const float2 v = *reinterpret_cast<const float2*>(src + (L & ~3));
-                        xr[q][r][L & ~3] = v.x; xr[q][r][(L & ~3) + 1] = v.y;
-                    }
-                    if constexpr (L & 1) xr[q][r][L - 1] = src[L - 1];
-                }
-            const float* wc = ws + (size_t)cc * RS * TILE_K;
-            const float* wc2 = ws2 + (size_t)cc * RS * TILE_K;
+                for (int r = 0; r < R; ++r)
+                    load_segment<SHIFT, L>(st + cc * chan_step + xoff[q] + r * row_step, xr[q][r]);
+            const float* wc = ws + cc * (RS * TILE_K);
+            const float* wc2 = ws2 + cc * (RS * TILE_K);
 
             float mx[CARRIED ? 1 : 8][Q][4];           // per-channel extremum (max branch / single branch)
             float mn[TWO ? 8 : 1][Q][4];               // per-channel minimum (two-branch modes)
@@ -271,25 +380,15 @@ fwd_tiled_f32_kernel(const TiledParams p) {
                 // winner codes per (output, channel): every tap is compared on its own
 #pragma unroll
                 for (int tap = 0; tap < RS; ++tap) {
-                    const int r = tap / S, s = tap % S;
+                    const int r = tap / S, sx = tap % S;
                     float wv[8], wv2[8];
-                    {
-                        const float4 a = *reinterpret_cast<const float4*>(wc + tap * TILE_K);
-                        const float4 b = *reinterpret_cast<const float4*>(wc + tap * TILE_K + 4);
-                        wv[0] = a.x; wv[1] = a.y; wv[2] = a.z; wv[3] = a.w;
-                        wv[4] = b.x; wv[5] = b.y; wv[6] = b.z; wv[7] = b.w;
-                    }
-                    if constexpr (PAR) {
-                        const float4 a = *reinterpret_cast<const float4*>(wc2 + tap * TILE_K);
-                        const float4 b = *reinterpret_cast<const float4*>(wc2 + tap * TILE_K + 4);
-                        wv2[0] = a.x; wv2[1] = a.y; wv2[2] = a.z; wv2[3] = a.w;
-                        wv2[4] = b.x; wv2[5] = b.y; wv2[6] = b.z; wv2[7] = b.w;
-                    }
+                    load8(wc + tap * TILE_K, wv);
+                    if constexpr (PAR) load8(wc2 + tap * TILE_K, wv2);
 #pragma unroll
                     for (int q = 0; q < Q; ++q)
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const float xv = xr[q][r][j * SW + s * DW];
+                            const float xv = xr[q][r][j * SW + sx * DW];
 #pragma unroll
                             for (int k = 0; k < 8; ++k) {
                                 const float t = __fadd_rn(xv, wv[k]);
@@ -324,16 +423,8 @@ fwd_tiled_f32_kernel(const TiledParams p) {
 #pragma unroll
                     for (int u = 0; u < 3; ++u)
                         if (u < nt) {
-                            const float4 a = *reinterpret_cast<const float4*>(wc + (t0 + u) * TILE_K);
-                            const float4 b = *reinterpret_cast<const float4*>(wc + (t0 + u) * TILE_K + 4);
-                            wv[u][0] = a.x; wv[u][1] = a.y; wv[u][2] = a.z; wv[u][3] = a.w;
-                            wv[u][4] = b.x; wv[u][5] = b.y; wv[u][6] = b.z; wv[u][7] = b.w;
-                            if constexpr (PAR) {
-                                const float4 c4 = *reinterpret_cast<const float4*>(wc2 + (t0 + u) * TILE_K);
-                                const float4 d4 = *reinterpret_cast<const float4*>(wc2 + (t0 + u) * TILE_K + 4);
-                                wv2[u][0] = c4.x; wv2[u][1] = c4.y; wv2[u][2] = c4.z; wv2[u][3] = c4.w;
-                                wv2[u][4] = d4.x; wv2[u][5] = d4.y; wv2[u][6] = d4.z; wv2[u][7] = d4.w;
-                            }
+                            load8(wc + (t0 + u) * TILE_K, wv[u]);
+                            if constexpr (PAR) load8(wc2 + (t0 + u) * TILE_K, wv2[u]);
                         }
 #pragma unroll
                     for (int q = 0; q < Q; ++q)
@@ -395,14 +486,8 @@ fwd_tiled_f32_kernel(const TiledParams p) {
             if constexpr (!CARRIED) {
                 float av[8], bv[8];
                 if constexpr (TWO) {
-                    const float4 a0 = *reinterpret_cast<const float4*>(as + cc * TILE_K);
-                    const float4 a1 = *reinterpret_cast<const float4*>(as + cc * TILE_K + 4);
-                    const float4 b0 = *reinterpret_cast<const float4*>(as + ab_stage + cc * TILE_K);
-                    const float4 b1 = *reinterpret_cast<const float4*>(as + ab_stage + cc * TILE_K + 4);
-                    av[0] = a0.x; av[1] = a0.y; av[2] = a0.z; av[3] = a0.w;
-                    av[4] = a1.x; av[5] = a1.y; av[6] = a1.z; av[7] = a1.w;
-                    bv[0] = b0.x; bv[1] = b0.y; bv[2] = b0.z; bv[3] = b0.w;
-                    bv[4] = b1.x; bv[5] = b1.y; bv[6] = b1.z; bv[7] = b1.w;
+                    load8(as + cc * TILE_K, av);
+                    load8(bs + cc * TILE_K, bv);
                 }
                 const int c = ch * p.CC + cc;
 #pragma unroll
@@ -457,7 +542,7 @@ fwd_tiled_f32_kernel(const TiledParams p) {
                 }
             }
         }
-        __syncthreads();
+        __syncthreads();  // every thread is done with this stage before it is refilled
     }
 
     // epilogue: bias, store, winner index of the Max / Min channel combines
@@ -486,7 +571,7 @@ fwd_tiled_f32_kernel(const TiledParams p) {
             }
             if constexpr (WIN && CHAN != CH_SUM) {
                 // the winning channel is known; rescan its window for the first tap that attains the
-                // extremum (same adds as the main loop, so equality is exact)
+                // extremum (same rounded adds as the main loop, so equality is exact)
                 int32_t* idx = reinterpret_cast<int32_t*>(p.winners);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -518,6 +603,7 @@ struct TiledPlan {
     int threads;
     size_t smem;
     int tile_k;
+    bool xtma;
     size_t ws_w, ws_ab;  // workspace split (bytes): each weight array, each of alpha / beta
 };
 
@@ -529,16 +615,16 @@ inline size_t tiled_ws_bytes(const Geo& g) {
     return 2 * w + 2 * ab + 1024;
 }
 
+inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
+
 template <int R, int S, int SW, int DW, int Q, int KG, int PW>
-inline bool plan_tiles(const Geo& g, bool par, bool two, TiledPlan* pl) {
+inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* pl) {
     TiledParams& p = pl->p;
     constexpr int TILE_K = KG * 8;
     constexpr int NQ = Q * 32 * PW;
     const int qpr_full = (g.OW + 3) / 4;
-    // column tiles: as wide as the row allows, at most NQ/2 quads (so a tile keeps >= 2 rows
-    // unless the row is very wide), split evenly
-    int max_qpr = NQ >= 32 ? NQ / 4 : NQ;
-    if (max_qpr < 1) max_qpr = 1;
+    // column tiles: at most NQ/4 quads wide (a tile keeps >= 4 rows unless the row is short), split evenly
+    const int max_qpr = NQ >= 32 ? NQ / 4 : NQ;
     const int ncol = (qpr_full + max_qpr - 1) / max_qpr;
     p.QPR = (qpr_full + ncol - 1) / ncol;
     p.TW = p.QPR * 4;
@@ -546,22 +632,41 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, TiledPlan* pl) {
     p.TH = NQ / p.QPR;
     if (p.TH < 1) return false;
     p.total_rows = g.N * g.OH;
-    if (p.TH > p.total_rows) p.TH = p.total_rows;
-    p.n_row_tiles = (p.total_rows + p.TH - 1) / p.TH;
-    p.GAP = (R - 1) * g.dh - g.sh + 1;
-    if (p.GAP < 0) p.GAP = 0;
-    const int max_imgs = (p.TH - 1) / g.OH + 2;
-    p.NSLOTS = (p.TH - 1) * g.sh + (R - 1) * g.dh + 1 + (max_imgs - 1) * p.GAP;
-    p.XW = (p.TW - 1) * SW + (S - 1) * DW + 1;
-    // a quad reads up to 3*SW + (S-1)*DW + 1 floats from column 4*SW*qx, rounded up to vectors
-    const int reach = (p.QPR - 1) * 4 * SW + ((3 * SW + (S - 1) * DW + 1 + 3) & ~3);
-    p.XP = ((reach > p.XW ? reach : p.XW) + 3) & ~3;
+    // TMA path: rows of x are 16-byte multiples, "same" padding along w (fixes the column shift),
+    // and tiles that stay inside one image without idling more than a quarter of the lanes
+    const int shift = TmaShift<S, DW>::value;
+    const int th_img = p.TH < g.OH ? p.TH : g.OH;
+    const int tiles_img = (g.OH + th_img - 1) / th_img;
+    const bool rows_fit = (double)g.OH / (tiles_img * th_img) >= 0.75 && th_img * p.QPR * 4 >= NQ * 3;
+    pl->xtma = ((g.W * esize) % 16 == 0) && (g.pw == (S - 1) * DW / 2) && rows_fit;
+    p.XW = (p.TW - 1) * SW + (S - 1) * DW + 1;   // == (QPR-1)*4*SW + L
+    if (pl->xtma) {
+        p.TH = th_img;
+        p.tiles_per_img = tiles_img;
+        p.n_row_tiles = g.N * tiles_img;
+        p.GAP = 0;
+        p.NSLOTS = (p.TH - 1) * g.sh + (R - 1) * g.dh + 1;
+        p.XP = round_up(p.XW + shift, 4);
+        if (p.XP > 256 || p.NSLOTS > 256) return false;
+    } else {
+        if (p.TH > p.total_rows) p.TH = p.total_rows;
+        p.tiles_per_img = 0;
+        p.n_row_tiles = (p.total_rows + p.TH - 1) / p.TH;
+        p.GAP = (R - 1) * g.dh - g.sh + 1;
+        if (p.GAP < 0) p.GAP = 0;
+        const int max_imgs = (p.TH - 1) / g.OH + 2;
+        p.NSLOTS = (p.TH - 1) * g.sh + (R - 1) * g.dh + 1 + (max_imgs - 1) * p.GAP;
+        p.XP = round_up(p.XW, 4);
+    }
     p.CC = 8;
-    p.Cpad = (g.C + p.CC - 1) / p.CC * p.CC;
+    p.Cpad = round_up(g.C, p.CC);
     p.nchunks = p.Cpad / p.CC;
-    const size_t stage = (size_t)p.CC * p.NSLOTS * p.XP + (size_t)p.CC * g.RS * TILE_K * (par ? 2 : 1) +
-                         (two ? 2 * (size_t)p.CC * TILE_K : 0);
-    pl->smem = 2 * stage * sizeof(float) + (size_t)p.NSLOTS * sizeof(int) + 16;
+    // one stage: x tile | weights | (weights 2) | alpha | beta, each block 128-byte aligned
+    p.x_stage = round_up(p.CC * p.NSLOTS * p.XP, 32);
+    p.w_stage = p.CC * g.RS * TILE_K;            // multiple of 32 floats
+    p.ab_stage = two ? p.CC * TILE_K : 0;
+    p.stage_floats = p.x_stage + p.w_stage * (par ? 2 : 1) + 2 * p.ab_stage;
+    pl->smem = 2 * (size_t)p.stage_floats * sizeof(float) + 16 + (size_t)p.NSLOTS * sizeof(int) + 16;
     if (pl->smem > 200 * 1024) return false;
     const int nkt = (g.K + TILE_K - 1) / TILE_K;
     pl->grid = dim3((unsigned)(p.n_col_tiles * p.n_row_tiles), (unsigned)nkt, 1);
@@ -572,92 +677,118 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, TiledPlan* pl) {
     return true;
 }
 
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                    CUtensorMapFloatOOBfill);
+
+inline encode_tiled_fn get_encode_tiled() {
+    static encode_tiled_fn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return (encode_tiled_fn)f;
+    }();
+    return fn;
+}
+
+// x viewed as [N*C][H][W]; box = [CC][NSLOTS][XP]; out-of-range elements read as zero.
+inline bool make_x_map(const Geo& g, const void* x, int esize, const TiledParams& p, CUtensorMap* map) {
+    encode_tiled_fn enc = get_encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N * g.C};
+    const cuuint64_t strides[2] = {(cuuint64_t)g.W * esize, (cuuint64_t)g.H * g.W * esize};
+    const cuuint32_t box[3] = {(cuuint32_t)p.XP, (cuuint32_t)p.NSLOTS, (cuuint32_t)p.CC};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUtensorMapDataType dt = esize == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    return enc(map, dt, 3, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Arguments of one forward launch (host side).
+struct FwdArgs {
+    Geo g;
+    int dtype;
+    const void *x, *w, *w2;
+    const float *alpha, *beta, *bias;
+    void* y;
+    void* winners;
+    void* ws;
+    size_t ws_bytes;
+    int* status;
+    cudaStream_t st;
+    const char* name;  // out: kernel variant
+};
+
 template <typename T, int MODE, int CHAN, bool WIN, int R, int S, int SW, int DW, int Q, int KG, int PW>
-int launch_tiled_variant(const Geo& g, const T* x, const T* w, const T* w2, const float* alpha,
-                         const float* beta, const float* bias, T* y, void* winners, void* ws,
-                         size_t ws_bytes, cudaStream_t st) {
+int launch_tiled_variant(FwdArgs& a) {
     constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
     constexpr bool PAR = (MODE == TCONV_PARALLEL);
+    const Geo& g = a.g;
     TiledPlan pl;
     pl.p.g = g;
-    if (!plan_tiles<R, S, SW, DW, Q, KG, PW>(g, PAR, TWO, &pl)) return TCONV_ERR_UNSUPPORTED;
+    if (!plan_tiles<R, S, SW, DW, Q, KG, PW>(g, PAR, TWO, (int)sizeof(T), &pl)) return TCONV_ERR_UNSUPPORTED;
     const size_t need = pl.ws_w * (PAR ? 2 : 1) + (TWO ? 2 * pl.ws_ab : 0);
-    if (!ws || ws_bytes < need) return TCONV_ERR_WORKSPACE_TOO_SMALL;
-    float* wt = reinterpret_cast<float*>(ws);
+    if (!a.ws || a.ws_bytes < need) return TCONV_ERR_WORKSPACE_TOO_SMALL;
+    float* wt = reinterpret_cast<float*>(a.ws);
     float* wt2 = PAR ? wt + pl.ws_w / sizeof(float) : nullptr;
     float* at = TWO ? wt + (pl.ws_w * (PAR ? 2 : 1)) / sizeof(float) : nullptr;
     float* bt = TWO ? at + pl.ws_ab / sizeof(float) : nullptr;
+    CUtensorMap xmap;
+    memset(&xmap, 0, sizeof(xmap));
+    if (pl.xtma && !make_x_map(g, a.x, (int)sizeof(T), pl.p, &xmap)) return TCONV_ERR_CUDA;
     const int nkt = pl.grid.y;
     const size_t nrep = (size_t)nkt * pl.p.Cpad * g.RS * pl.tile_k;
-    repack_weights_kernel<T><<<(unsigned)((nrep + 255) / 256), 256, 0, st>>>(
-        g.K, g.C, g.RS, pl.tile_k, pl.p.Cpad, nkt, w, w2, alpha, beta, wt, wt2, at, bt);
-    pl.p.x = x; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
-    pl.p.bias = bias; pl.p.y = y; pl.p.winners = winners;
-    auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, R, S, SW, DW, Q, KG, PW>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-        return TCONV_ERR_CUDA;
-    kern<<<pl.grid, pl.threads, pl.smem, st>>>(pl.p);
+    repack_weights_kernel<T><<<(unsigned)((nrep + 255) / 256), 256, 0, a.st>>>(
+        g.K, g.C, g.RS, pl.tile_k, pl.p.Cpad, nkt, (const T*)a.w, (const T*)a.w2, a.alpha, a.beta, wt, wt2, at, bt);
+    pl.p.x = a.x; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
+    pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
+    if (pl.xtma) {
+        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, true, R, S, SW, DW, Q, KG, PW>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+            return TCONV_ERR_CUDA;
+        kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);
+        a.name = WIN ? "fwd_tiled_f32_tma_win" : "fwd_tiled_f32_tma";
+    } else {
+        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, false, R, S, SW, DW, Q, KG, PW>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+            return TCONV_ERR_CUDA;
+        kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);
+        a.name = WIN ? "fwd_tiled_f32_win" : "fwd_tiled_f32";
+    }
     return TCONV_OK;
 }
 
 // Geometry families with a tiled kernel: 3x3 windows with (stride_w, dil_w) in
 // {(1,1), (2,1), (1,2)}.
 template <typename T, int MODE, int CHAN, bool WIN>
-int launch_tiled_geom(const Geo& g, const T* x, const T* w, const T* w2, const float* alpha,
-                      const float* beta, const float* bias, T* y, void* winners, void* ws,
-                      size_t ws_bytes, cudaStream_t st) {
+int launch_tiled_geom(FwdArgs& a) {
     constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
     // two quads per thread where one running value per output suffices (the carried
     // extremum of layers (iv), (v) without winners), else one
     constexpr bool CARRIED = !TWO && !WIN && ((MODE == TCONV_MAX_PLUS && CHAN == CH_MAX) ||
                                               (MODE == TCONV_MIN_PLUS && CHAN == CH_MIN));
     constexpr int Q = CARRIED ? 2 : 1;
+    const Geo& g = a.g;
     if (g.R == 3 && g.S == 3) {
-        if (g.sw == 1 && g.dw == 1)
-            return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 1, Q, 4, 1>(g, x, w, w2, alpha, beta, bias, y, winners, ws, ws_bytes, st);
-        if (g.sw == 2 && g.dw == 1)
-            return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 2, 1, Q, 4, 1>(g, x, w, w2, alpha, beta, bias, y, winners, ws, ws_bytes, st);
-        if (g.sw == 1 && g.dw == 2)
-            return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 2, Q, 4, 1>(g, x, w, w2, alpha, beta, bias, y, winners, ws, ws_bytes, st);
+        if (g.sw == 1 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 1, Q, 4, 1>(a);
+        if (g.sw == 2 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 2, 1, Q, 4, 1>(a);
+        if (g.sw == 1 && g.dw == 2) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 2, Q, 4, 1>(a);
     }
     return TCONV_ERR_UNSUPPORTED;
 }
 
-template <typename T, bool WIN>
-int launch_tiled_mode(const Geo& g, const T* x, const T* w, const T* w2, const float* alpha,
-                      const float* beta, const float* bias, T* y, void* winners, void* ws,
-                      size_t ws_bytes, cudaStream_t st) {
-#define TCONV_GO(M, CH) \
-    return launch_tiled_geom<T, M, CH, WIN>(g, x, w, w2, alpha, beta, bias, y, winners, ws, ws_bytes, st)
-    if (g.mode == TCONV_COMPOUND) TCONV_GO(TCONV_COMPOUND, CH_SUM);
-    if (g.mode == TCONV_PARALLEL) TCONV_GO(TCONV_PARALLEL, CH_SUM);
-    if (g.mode == TCONV_MAX_PLUS) {
-        if (g.chan == CH_MAX) TCONV_GO(TCONV_MAX_PLUS, CH_MAX);
-        if (g.chan == CH_MIN) TCONV_GO(TCONV_MAX_PLUS, CH_MIN);
-        TCONV_GO(TCONV_MAX_PLUS, CH_SUM);
-    }
-    if (g.chan == CH_MAX) TCONV_GO(TCONV_MIN_PLUS, CH_MAX);
-    if (g.chan == CH_MIN) TCONV_GO(TCONV_MIN_PLUS, CH_MIN);
-    TCONV_GO(TCONV_MIN_PLUS, CH_SUM);
-#undef TCONV_GO
-}
-
-// Launches the tiled forward kernel that covers this geometry.  Returns
-// TCONV_ERR_UNSUPPORTED when none does (the caller then uses the any-shape kernel).
-template <typename T>
-int launch_fwd_tiled(const Geo& g, const T* x, const T* w, const T* w2, const float* alpha,
-                     const float* beta, const float* bias, T* y, void* winners, void* ws,
-                     size_t ws_bytes, cudaStream_t st, const char** name) {
-    if constexpr (sizeof(T) != 4) {
-        return TCONV_ERR_UNSUPPORTED;  // bf16: separate kernel
-    } else {
-    if (g.wide) return TCONV_ERR_UNSUPPORTED;
-    if ((double)g.N * g.C * g.H * g.W >= 2.0e9) return TCONV_ERR_UNSUPPORTED;  // 32-bit offsets
-    *name = winners ? "fwd_tiled_f32_win" : "fwd_tiled_f32";
-    if (winners)
-        return launch_tiled_mode<T, true>(g, x, w, w2, alpha, beta, bias, y, winners, ws, ws_bytes, st);
-    return launch_tiled_mode<T, false>(g, x, w, w2, alpha, beta, bias, y, winners, ws, ws_bytes, st);
-    }
+// One instance per (mode, channel combine): compiled in its own translation unit.
+template <int MODE, int CHAN>
+int launch_fwd_tiled_inst(FwdArgs& a) {
+    if (a.dtype != TCONV_F32) return TCONV_ERR_UNSUPPORTED;  // bf16: separate kernel
+    if (a.g.wide) return TCONV_ERR_UNSUPPORTED;
+    if ((double)a.g.N * a.g.C * a.g.H * a.g.W >= 2.0e9) return TCONV_ERR_UNSUPPORTED;  // 32-bit offsets
+    if (a.winners) return launch_tiled_geom<float, MODE, CHAN, true>(a);
+    return launch_tiled_geom<float, MODE, CHAN, false>(a);
 }
 
 }  // namespace tconv

@@ -23,7 +23,8 @@ TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
 # every symbol include/tconv.h declares
 SYMBOLS = ("tconv_output_shape", "tconv_winner_bytes", "tconv_workspace_bytes", "tconv_forward",
            "tconv_backward", "tconv_paper_ops", "tconv_alu_probe", "tconv_alu_probe_name",
-           "tconv_status_string", "tconv_last_error", "tconv_last_kernel")
+           "tconv_device_status", "tconv_status_string", "tconv_last_error", "tconv_last_kernel",
+           "tconv_launch_count")
 
 
 class TconvError(RuntimeError):
@@ -64,10 +65,13 @@ def _load() -> ctypes.CDLL:
     lib.tconv_alu_probe.restype = ctypes.c_int
     lib.tconv_alu_probe_name.argtypes = [ctypes.c_int]
     lib.tconv_alu_probe_name.restype = ctypes.c_char_p
+    lib.tconv_device_status.argtypes = [vp]
+    lib.tconv_device_status.restype = ctypes.c_int
     lib.tconv_status_string.argtypes = [ctypes.c_int]
     lib.tconv_status_string.restype = ctypes.c_char_p
     lib.tconv_last_error.restype = ctypes.c_char_p
     lib.tconv_last_kernel.restype = ctypes.c_char_p
+    lib.tconv_launch_count.restype = ctypes.c_longlong
     return lib
 
 
@@ -142,6 +146,11 @@ def tconv_alu_probe_name(variant: int):
     return None if s is None else s.decode()
 
 
+def tconv_device_status(stream=None) -> int:
+    """Synchronise the stream and report (and clear) a device-side wait that gave up."""
+    return _lib.tconv_device_status(_stream(stream))
+
+
 def tconv_status_string(status: int) -> str:
     return _lib.tconv_status_string(status).decode()
 
@@ -152,6 +161,10 @@ def tconv_last_error() -> str:
 
 def tconv_last_kernel() -> str:
     return _lib.tconv_last_kernel().decode()
+
+
+def tconv_launch_count() -> int:
+    return int(_lib.tconv_launch_count())
 
 
 # ---- convenience: allocate outputs with torch, check the status ----------------------

@@ -59,6 +59,25 @@ def test_multi_tile_ragged(mode, chan):
                        recompute=False)
 
 
+@pytest.mark.parametrize("mode,chan", ALL_MODES)
+def test_tma_staged_shapes(mode, chan):
+    """Shapes whose input rows are 16-byte multiples with 'same' padding take the TMA-staged
+    kernels: several channel chunks, ragged K and C, partial row tiles, stride 2, dilation 2."""
+    from paper_2504_06881_b200 import tconv
+    cases = [inputs.layer(3, 19, 20, 32, 41, 3, 3, stride=1, pad=1, mode=mode, chan=chan),
+             inputs.layer(2, 10, 30, 56, 35, 3, 3, stride=2, pad=1, mode=mode, chan=chan),
+             inputs.layer(2, 9, 24, 64, 33, 3, 3, stride=1, pad=2, dil=2, mode=mode, chan=chan),
+             inputs.layer(2, 17, 28, 28, 16, 3, 3, stride=1, pad=1, mode=mode, chan=chan),
+             inputs.layer(1, 8, 6, 128, 8, 3, 3, stride=1, pad=1, mode=mode, chan=chan)]
+    for i, d in enumerate(cases):
+        t = inputs.draw(d, 450 + i)
+        parity.check_forward(d, t, check_winners=False)
+        assert "tma" in tconv.tconv_last_kernel(), tconv.tconv_last_kernel()
+        assert tconv.tconv_device_status() == 0
+        parity.check_layer(d, None, 460 + i, recompute=False)
+        parity.check_layer(d, TIES, 470 + i, recompute=False, stored_winners=(i == 0))
+
+
 def test_other_window_sizes():
     """1x1, 1x3, 5x5 (more than 16 taps: wide winner codes), 7x7 windows."""
     for (R, S, pad) in ((1, 1, 0), (1, 3, 1), (5, 5, 2), (7, 7, 3), (4, 4, 1)):
