@@ -1,0 +1,394 @@
+"""Benchmark of the tropical-convolution hot path on B200.
+
+One step = forward + backward of one layer of each mode (max_plus, min_plus, compound,
+parallel) at N=128, C=K=64, 32x32, 3x3, stride 1, pad 1, fp32 (the configuration the
+headline metric is quoted on), on seeded synthetic tensors.  The metric is tropical
+Gop/s: operations of the paper's complexity analysis (additions + comparisons +
+multiplications, Section 4.1), forward and backward each credited with the forward
+count, divided by device time.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+`--impl reference` times the CPU checker under oracle/ (as it stands) on the host cores
+on a bounded sample of the same workload.  With N > 1 (torchrun) every rank runs the same
+independent replica: the path has no inter-GPU exchange.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+MODES = [("max_plus", "default"), ("min_plus", "default"), ("compound", "default"),
+         ("parallel", "default")]
+WORKLOAD = "cfg2: one layer of each mode fwd+bwd fp32, N=128 C=K=64 32x32 3x3 s1 p1"
+# probe variants whose best gives the add+max/min peak of a mode's instruction mix
+PROBES = {"max_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
+          "min_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
+          "compound": ("f32_add_minmax2", "f32_add_minmax3", "f32_add2_minmax3"),
+          "parallel": ("f32_2add_minmax2", "f32_2add_minmax3", "f32_2add2_minmax3")}
+
+
+def layer_ops(d):
+    """Operations of Section 4.1 for one forward pass (python restatement for the CPU arm)."""
+    from paper_2504_06881_b200 import inputs
+    OH, OW = inputs.output_hw(d)
+    P = d["N"] * d["K"] * OH * OW
+    C, RS = d["C"], d["R"] * d["S"]
+    if d["mode"] == "compound":
+        return ((RS * C + 2 * C - 1) + 2 * (RS - 1) * C + 2 * C) * P
+    if d["mode"] == "parallel":
+        return ((2 * RS * C + 2 * C - 1) + 2 * (RS - 1) * C + 2 * C) * P
+    chan = d["chan"] if d["chan"] != "default" else "full"
+    if chan == "sum":
+        return ((C - 1 + RS * C) + (RS - 1) * C) * P
+    return (RS * C + (RS * C - 1)) * P
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 6:
+                self.samples.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            try:
+                sm.append(float(s[0])); mx = float(s[1])
+            except ValueError:
+                continue
+            for name, v in zip(names, s[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------ CPU arm (the checker)
+def time_oracle_sample(n_sample: int):
+    """One fwd+bwd of each mode on an n_sample-image slice of the workload, on the host cores."""
+    from oracle import tconv_oracle as ora
+    from paper_2504_06881_b200 import inputs
+    t_total, ops = 0.0, 0.0
+    for i, (mode, chan) in enumerate(MODES):
+        d, dist = inputs.cfg2(mode, chan, N=n_sample)
+        t = inputs.draw(d, 1020 + i, **dist)
+        two = mode in ("compound", "parallel")
+        w2 = t["w2"] if mode == "parallel" else None
+        al, be = (t["alpha"], t["beta"]) if two else (None, None)
+        t0 = time.perf_counter()
+        ora.forward(d, t["x"], t["w"], w2, al, be, t["bias"])
+        ora.backward(d, t["x"], t["w"], t["g"], w2, al, be)
+        t_total += time.perf_counter() - t0
+        ops += 2 * layer_ops(d)
+    return t_total, ops
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import tconv_oracle as ora
+    ora.build()
+    cores = ora.threads()
+    # the checker's backward runs one thread per image: one image per core keeps every
+    # core busy and makes a step a few seconds of CPU work
+    n_sample = max(1, min(128, cores))
+    for _ in range(args.warmup):
+        time_oracle_sample(1)
+    t_sum, ops_sum = 0.0, 0.0
+    for _ in range(args.steps):
+        t, ops = time_oracle_sample(n_sample)
+        t_sum += t; ops_sum += ops
+    value = ops_sum / t_sum / 1e9
+    sample = f"{n_sample} of 128 images of each layer per step (fwd+bwd, all four modes)"
+    line = {"impl": "reference", "metric": "tropical conv fwd+bwd Gop/s", "value": value, "unit": "Gop/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * t_sum / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "Gop/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "Gop/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------ GPU arm
+class Layer:
+    """Device-resident tensors of one layer plus its outputs, allocated once."""
+
+    def __init__(self, mode, chan, seed, torch, tconv, inputs, dev):
+        self.d, dist = inputs.cfg2(mode, chan)
+        d = self.d
+        t = inputs.draw(d, seed, **dist)
+        self.host = {k: torch.from_numpy(v).pin_memory() for k, v in t.items()}
+        self.two = mode in ("compound", "parallel")
+        self.par = mode == "parallel"
+        self.dev = {k: v.to(dev, non_blocking=True) for k, v in self.host.items()}
+        N, C, H, W, K = d["N"], d["C"], d["H"], d["W"], d["K"]
+        OH, OW = tconv.tconv_output_shape(d)
+        f32 = torch.float32
+        self.y = torch.empty((N, K, OH, OW), dtype=f32, device=dev)
+        self.win = tconv.winner_buffer(d, dev)
+        self.ws = torch.empty(tconv.tconv_workspace_bytes(d, True), dtype=torch.uint8, device=dev)
+        self.gx = torch.empty((N, C, H, W), dtype=f32, device=dev)
+        self.gw = torch.empty((K, C, 3, 3), dtype=f32, device=dev)
+        self.gw2 = torch.empty((K, C, 3, 3), dtype=f32, device=dev) if self.par else None
+        self.ga = torch.empty((K, C), dtype=f32, device=dev) if self.two else None
+        self.gb = torch.empty((K, C), dtype=f32, device=dev) if self.two else None
+        self.gbias = torch.empty((K,), dtype=f32, device=dev)
+        self.ops = 2 * tconv.tconv_paper_ops(d)
+        self.taps = N * K * OH * OW * C * 9
+        self.tconv = tconv
+        # pinned host landing buffers of the end-to-end leg
+        self.h_y = torch.empty((N, K, OH, OW), dtype=f32).pin_memory()
+        self.h_gx = torch.empty((N, C, H, W), dtype=f32).pin_memory()
+        self.h_small = {k: torch.empty_like(getattr(self, k), device="cpu").pin_memory()
+                        for k in ("gw", "gw2", "ga", "gb", "gbias") if getattr(self, k) is not None}
+
+    def fwd(self, with_winners=True):
+        v = self.dev
+        rc = self.tconv.tconv_forward(self.d, v["x"], v["w"], v["w2"] if self.par else None,
+                                      v["alpha"] if self.two else None, v["beta"] if self.two else None,
+                                      v["bias"], self.y, self.win if with_winners else None, self.ws)
+        if rc != 0:
+            raise self.tconv.TconvError(rc, "tconv_forward")
+
+    def bwd(self):
+        v = self.dev
+        rc = self.tconv.tconv_backward(self.d, v["x"], v["w"], v["w2"] if self.par else None,
+                                       v["alpha"] if self.two else None, v["beta"] if self.two else None,
+                                       v["g"], self.win, self.gx, self.gw, self.gw2, self.ga, self.gb,
+                                       self.gbias, self.ws)
+        if rc != 0:
+            raise self.tconv.TconvError(rc, "tconv_backward")
+
+    def e2e_step(self):
+        """Host buffers in, host buffers out: copies inside the timed region."""
+        names = ["x", "w", "bias", "g"] + (["w2"] if self.par else []) + (["alpha", "beta"] if self.two else [])
+        for k in names:
+            self.dev[k].copy_(self.host[k], non_blocking=True)
+        self.fwd()
+        self.bwd()
+        self.h_y.copy_(self.y, non_blocking=True)
+        self.h_gx.copy_(self.gx, non_blocking=True)
+        for k, h in self.h_small.items():
+            h.copy_(getattr(self, k), non_blocking=True)
+        h2d = sum(self.host[k].numel() * 4 for k in names)
+        d2h = (self.h_y.numel() + self.h_gx.numel() + sum(h.numel() for h in self.h_small.values())) * 4
+        return h2d, d2h
+
+
+def measure_alu_peak(torch, tconv):
+    """Best measured taps/s over the candidate instruction mixes, per mode."""
+    sink = torch.zeros(4, device="cuda")
+    names, i = {}, 0
+    while tconv.tconv_alu_probe_name(i) is not None:
+        names[tconv.tconv_alu_probe_name(i)] = i
+        i += 1
+    rate = {}
+    for name, v in names.items():
+        for _ in range(2):
+            tconv.tconv_alu_probe(v, 2000, sink)
+        best = None
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); taps = tconv.tconv_alu_probe(v, 2000, sink); e1.record()
+            torch.cuda.synchronize()
+            r = taps / (e0.elapsed_time(e1) * 1e-3)
+            best = r if best is None else max(best, r)
+        rate[name] = best
+    return {m: max(rate[p] for p in ps) for m, ps in PROBES.items()}, rate
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2504_06881_b200 import inputs, tconv
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    layers = [Layer(m, c, 1020 + i, torch, tconv, inputs, dev) for i, (m, c) in enumerate(MODES)]
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        for L in layers:
+            L.fwd()
+            L.bwd()
+
+    # ---- device-resident timing: W warm-up steps, then exactly K steps
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = tconv.tconv_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = tconv.tconv_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if tconv.tconv_device_status() != 0:
+        raise SystemExit("a device-side wait timed out during the timed region")
+
+    # ---- end to end: host buffers in and out, copies inside the timed region
+    for _ in range(2):
+        for L in layers:
+            L.e2e_step()
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h2d = d2h = 0
+    f0.record()
+    for _ in range(args.steps):
+        h2d = d2h = 0
+        for L in layers:
+            a, b = L.e2e_step()
+            h2d += a; d2h += b
+    f1.record()
+    barrier()
+    ms_e2e = f0.elapsed_time(f1)
+
+    # ---- per-call times of every mode (for the roofline of the dominant kernel)
+    per = {}
+    for L in layers:
+        rec = {}
+        for what, fn in (("fwd", lambda: L.fwd(False)), ("fwd_winners", L.fwd), ("bwd", L.bwd)):
+            ts = []
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record(); torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            rec[what] = float(np.median(ts))
+            rec[what + "_kernel"] = tconv.tconv_last_kernel()
+        per[L.d["mode"]] = rec
+    peaks, probe_rates = measure_alu_peak(torch, tconv)
+
+    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ops_step = sum(L.ops for L in layers)
+    value = world * ops_step * args.steps / (ms * 1e-3) / 1e9
+    e2e_value = world * ops_step * args.steps / (ms_e2e * 1e-3) / 1e9
+
+    # dominant kernel = the call with the largest time in a step; its roofline is the
+    # add+max/min ALU peak of that mode (a tap = one x+w term folded into min and/or max)
+    dom_mode, dom_what = max(((m, w) for m in per for w in ("fwd_winners", "bwd")),
+                             key=lambda mw: per[mw[0]][mw[1]])
+    L = next(x for x in layers if x.d["mode"] == dom_mode)
+    achieved = L.taps / (per[dom_mode][dom_what] * 1e-3) / 1e12
+    roofline = {"bound": "alu", "kernel": per[dom_mode][dom_what + "_kernel"], "call": f"{dom_mode} {dom_what}",
+                "achieved": achieved, "peak": peaks[dom_mode] / 1e12, "unit": "Ttap/s",
+                "frac": achieved / (peaks[dom_mode] / 1e12), "traffic": None,
+                "peak_source": "measured in this run: best register-only add+max/min probe of the mode"}
+    fwd_frac = {m: {"ms": per[m]["fwd"], "Ttap_s": L2.taps / (per[m]["fwd"] * 1e-3) / 1e12,
+                    "frac_of_alu_peak": L2.taps / (per[m]["fwd"] * 1e-3) / peaks[m],
+                    "kernel": per[m]["fwd_kernel"]}
+                for m, L2 in ((x.d["mode"], x) for x in layers)}
+
+    # ---- CPU baseline: the checker as it stands, bounded sample, host cores of this machine
+    from oracle import tconv_oracle as ora
+    ora.build()
+    n_sample = max(1, min(128, 2 * ora.threads()))   # two images per core: about 10 s
+    tc, opsc = time_oracle_sample(n_sample)
+    cpu = {"value": opsc / tc / 1e9, "unit": "Gop/s", "cores": ora.threads(), "kind": "oracle",
+           "sample": f"{n_sample} of 128 images of each layer, fwd+bwd, all four modes ({tc:.1f} s)"}
+
+    line = {"metric": "tropical conv fwd+bwd Gop/s", "value": value, "unit": "Gop/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "l2": "per-step working set ~1.6 GB exceeds the 126 MB L2",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": "Gop/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu,
+            "per_mode_ms": per, "forward_vs_alu_peak": fwd_frac,
+            "alu_probe_Ttap_s": {k: v / 1e12 for k, v in probe_rates.items()}}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
