@@ -6,6 +6,7 @@
 
 #include "alu_probe.cuh"
 #include "tconv_common.cuh"
+#include "tconv_bwd.cuh"
 #include "tconv_generic.cuh"
 #include "tconv_tiled.cuh"
 
@@ -155,29 +156,115 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                const float* beta, const void* gy, const void* winners, void* gx, float* gw,
                float* gw2, float* galpha, float* gbeta, float* gbias, void* ws, size_t ws_bytes,
                cudaStream_t st) {
-    (void)ws; (void)ws_bytes;
     const bool twob = two_branch(g.mode);
-    if (gx) {
-        const size_t total = (size_t)g.N * g.C * g.H * g.W;
-        bwd_gx_generic_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
-            g, alpha, beta, (const T*)gy, winners, (T*)gx);
-        g_launches += 1;
+    const bool tiled = !force_generic();
+    const char* name = "bwd_generic";
+    bool bias_done = false;
+    if (g.chan != CH_SUM) {
+        const int32_t* idx = (const int32_t*)winners;
+        int thi = 0;
+        size_t smem = 0;
+        if (gx) {
+            if (tiled && plan_idx_gx(g, &thi, &smem)) {
+                auto kern = bwd_idx_gx_kernel<T>;
+                if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemLimit) != cudaSuccess)
+                    return cuda_fail(cudaGetLastError());
+                const int tiles = (g.H + thi - 1) / thi;
+                const unsigned magic = g.RS == 1 ? 0u : (0xFFFFFFFFu / (unsigned)g.RS) + 1u;
+                kern<<<(unsigned)(g.N * tiles), 256, smem, st>>>(g, (const T*)gy, idx, (T*)gx, thi, tiles, magic);
+                name = "bwd_idx";
+            } else {
+                const size_t total = (size_t)g.N * g.C * g.H * g.W;
+                bwd_gx_generic_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+                    g, alpha, beta, (const T*)gy, winners, (T*)gx);
+            }
+            g_launches += 1;
+        }
+        int chunks = 0;
+        if ((gw || gbias) && tiled && plan_idx_gw(g, &chunks, &smem) && ws && ws_bytes >= bwd_ws_bytes(g)) {
+            const size_t CRS = (size_t)g.C * g.RS;
+            float* pw = (float*)ws;
+            float* pb = pw + (size_t)chunks * g.K * CRS;
+            auto kern = bwd_idx_gw_kernel<T>;
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemLimit) != cudaSuccess)
+                return cuda_fail(cudaGetLastError());
+            const int npc = (g.N + chunks - 1) / chunks;
+            kern<<<dim3((unsigned)g.K, (unsigned)chunks), 256, smem, st>>>(g, (const T*)gy, idx, pw, pb, npc);
+            g_launches += 1;
+            if (gw) {
+                const size_t len = (size_t)g.K * CRS;
+                bwd_reduce_partials_kernel<<<(unsigned)((len + 255) / 256), 256, 0, st>>>(pw, gw, len, chunks);
+                g_launches += 1;
+            }
+            if (gbias) {
+                bwd_reduce_partials_kernel<<<(unsigned)((g.K + 255) / 256), 256, 0, st>>>(pb, gbias, (size_t)g.K, chunks);
+                g_launches += 1;
+                bias_done = true;
+            }
+            name = "bwd_idx";
+        } else if (gw) {
+            bwd_gw_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C * g.RS), 256, 0, st>>>(
+                g, alpha, beta, (const T*)gy, winners, gw, gw2);
+            g_launches += 1;
+        }
+    } else {
+        const uint8_t* codes = (const uint8_t*)winners;
+        const int br = twob ? 0 : (g.mode == TCONV_MIN_PLUS ? 1 : 2);
+        CodeGxPlan pl;
+        if (gx) {
+            if (tiled && plan_code_gx(g, &pl)) {
+                const dim3 grid((unsigned)(g.N * pl.tiles_per_img), (unsigned)((g.C + pl.CB - 1) / pl.CB));
+#define TCONV_GX(BR)                                                                                 \
+    {                                                                                                \
+        auto kern = bwd_code_gx_kernel<T, BR>;                                                       \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemLimit) != cudaSuccess) \
+            return cuda_fail(cudaGetLastError());                                                    \
+        kern<<<grid, 256, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);          \
     }
-    if (gw || gw2) {
-        bwd_gw_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C * g.RS), 256, 0, st>>>(
-            g, alpha, beta, (const T*)gy, winners, gw, gw2);
-        g_launches += 1;
+                if (br == 0) TCONV_GX(0) else if (br == 1) TCONV_GX(1) else TCONV_GX(2)
+#undef TCONV_GX
+                name = "bwd_code";
+            } else {
+                const size_t total = (size_t)g.N * g.C * g.H * g.W;
+                bwd_gx_generic_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+                    g, alpha, beta, (const T*)gy, winners, (T*)gx);
+            }
+            g_launches += 1;
+        }
+        if (gw || gw2 || galpha || gbeta) {
+            if (tiled && !g.wide && code_gw_smem(g) <= kBwdSmemLimit) {
+                const size_t smem = code_gw_smem(g);
+#define TCONV_GW(BR)                                                                                 \
+    {                                                                                                \
+        auto kern = bwd_code_gw_kernel<T, BR>;                                                       \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemLimit) != cudaSuccess) \
+            return cuda_fail(cudaGetLastError());                                                    \
+        kern<<<(unsigned)((size_t)g.K * g.C), 256, smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
+                                                      (const T*)gy, codes, gw, gw2, galpha, gbeta); \
     }
-    if (twob && (galpha || gbeta)) {
-        bwd_gab_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C), 256, 0, st>>>(
-            g, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, winners, galpha, gbeta);
-        g_launches += 1;
+                if (br == 0) TCONV_GW(0) else if (br == 1) TCONV_GW(1) else TCONV_GW(2)
+#undef TCONV_GW
+                g_launches += 1;
+                name = "bwd_code";
+            } else {
+                if (gw || gw2) {
+                    bwd_gw_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C * g.RS), 256, 0, st>>>(
+                        g, alpha, beta, (const T*)gy, winners, gw, gw2);
+                    g_launches += 1;
+                }
+                if (twob && (galpha || gbeta)) {
+                    bwd_gab_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C), 256, 0, st>>>(
+                        g, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, winners, galpha, gbeta);
+                    g_launches += 1;
+                }
+            }
+        }
     }
-    if (gbias) {
+    if (gbias && !bias_done) {
         bwd_bias_kernel<T><<<(unsigned)g.K, 256, 0, st>>>(g, (const T*)gy, gbias);
         g_launches += 1;
     }
-    snprintf(g_last_kernel, sizeof(g_last_kernel), "bwd_generic");
+    snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", name);
     return check_launch();
 }
 
@@ -205,8 +292,10 @@ size_t tconv_workspace_bytes(const tconv_desc_t* desc, int backward) {
     if (make_geo(desc, &g) != TCONV_OK) return 0;
     const size_t fwd = align_up(tiled_ws_bytes(g), 256);  // repacked weights, alpha, beta
     if (!backward) return fwd;
-    // winners recomputed (by a forward pass) into the workspace when the caller passes none
-    return align_up(winner_bytes(g), 256) + fwd;
+    // winners recomputed (by a forward pass) into the workspace when the caller passes none;
+    // the forward scratch and the backward partial sums are not live at the same time
+    const size_t bwd = align_up(bwd_ws_bytes(g), 256);
+    return align_up(winner_bytes(g), 256) + (fwd > bwd ? fwd : bwd);
 }
 
 int tconv_forward(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,
