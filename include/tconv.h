@@ -148,6 +148,40 @@ int tconv_backward(const tconv_desc_t *desc, const void *x, const void *w, const
                    size_t workspace_bytes, void *stream);
 
 /*
+ * Forward pass for callers that cannot allocate device memory.  (The paper has no
+ * counterpart of this entry point; it exists for the library's users.)
+ *
+ * Some callers have no way to hand over a workspace: code that runs inside a region
+ * where the CUDA allocator must not be touched (for example between the capture calls
+ * of a stream, or in a real-time loop that was given a fixed memory budget), plug-ins
+ * whose host application owns all device memory, and small C programs that link this
+ * library without a tensor framework.  For them this variant of tconv_forward takes
+ * its scratch (the repacked weights, alpha and beta of the tiled kernels) from a fixed
+ * array inside the library image instead of a caller workspace.  It calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   - Arguments are those of tconv_forward without workspace / workspace_bytes; the
+ *     caller still owns and passes every input and output.
+ *   - The built-in scratch holds tconv_forward_noalloc_max_scratch() bytes (8 MiB; every
+ *     GPU that loads the library holds that much until the process exits).  A layer with
+ *     tconv_workspace_bytes(desc, 0) above that is rejected with TCONV_ERR_TOO_LARGE and
+ *     a message in tconv_last_error(); nothing is launched.
+ *   - The first call on each device looks up the device address of the scratch (with
+ *     that device current).  Make that first call before starting any stream capture.
+ *   - All calls share the one array.  Each call rewrites every byte of it that it later
+ *     reads, so nothing depends on earlier contents; but two calls whose kernels overlap
+ *     on the GPU (different streams, or different host threads) race on it.  Serialise
+ *     them on one stream or with events.
+ * Results are identical to tconv_forward's.
+ */
+int tconv_forward_noalloc(const tconv_desc_t *desc, const void *x, const void *w, const void *w2,
+                          const float *alpha, const float *beta, const float *bias, void *y,
+                          void *winners, void *stream);
+
+/* Capacity in bytes of the scratch tconv_forward_noalloc uses.  Host call. */
+size_t tconv_forward_noalloc_max_scratch(void);
+
+/*
  * Number of operations the paper's complexity analysis (Section 4.1) assigns to
  * one forward pass of the layer: additions + comparisons + multiplications
  * (theta = 1).  Host call; 0 for an invalid descriptor.

@@ -431,6 +431,55 @@ int tconv_device_status(void* stream) {
     return TCONV_ERR_DEVICE_TIMEOUT;
 }
 
+// ---- forward pass for callers that cannot allocate device memory --------------------
+// Scratch of the allocation-free entry point: lives in the library image, so every GPU
+// that loads the library holds these bytes until the process exits.
+#define TCONV_NOALLOC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TCONV_NOALLOC_SCRATCH_BYTES];
+
+size_t tconv_forward_noalloc_max_scratch(void) { return TCONV_NOALLOC_SCRATCH_BYTES; }
+
+int tconv_forward_noalloc(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,
+                          const float* alpha, const float* beta, const float* bias, void* y,
+                          void* winners, void* stream) {
+    Geo g;
+    int rc = make_geo(desc, &g);
+    if (rc != TCONV_OK) return rc;
+    if (!x || !w || !y) return TCONV_ERR_INVALID_ARG;
+    if (g.mode == TCONV_PARALLEL && !w2) return TCONV_ERR_INVALID_ARG;
+    if (misaligned(x) || misaligned(w) || misaligned(w2) || misaligned(alpha) || misaligned(beta) ||
+        misaligned(bias) || misaligned(y) || misaligned(winners))
+        return TCONV_ERR_MISALIGNED;
+    const size_t need = tconv_workspace_bytes(desc, 0);
+    if (need > TCONV_NOALLOC_SCRATCH_BYTES) {
+        snprintf(g_last_error, sizeof(g_last_error),
+                 "layer needs %zu bytes of scratch, the built-in scratch holds %u", need,
+                 (unsigned)TCONV_NOALLOC_SCRATCH_BYTES);
+        return TCONV_ERR_TOO_LARGE;
+    }
+    // In host code the array's name is only a stand-in; the device address comes from the
+    // runtime, once per device, with that device current.
+    static void* scratch_ptr[64] = {nullptr};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return TCONV_ERR_UNSUPPORTED;
+    if (!scratch_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress((void**)&p, g_noalloc_scratch);
+        if (e != cudaSuccess) return cuda_fail(e);
+        scratch_ptr[dev] = p;
+    }
+    if (!two_branch(g.mode)) { alpha = nullptr; beta = nullptr; }
+    cudaStream_t st = (cudaStream_t)stream;
+    g_last_error[0] = 0;
+    if (desc->dtype == TCONV_F32)
+        return forward_t<float>(g, x, w, w2, alpha, beta, bias, y, winners, scratch_ptr[dev],
+                                TCONV_NOALLOC_SCRATCH_BYTES, st);
+    return forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, bias, y, winners, scratch_ptr[dev],
+                                    TCONV_NOALLOC_SCRATCH_BYTES, st);
+}
+
 const char* tconv_last_error(void) { return g_last_error; }
 const char* tconv_last_kernel(void) { return g_last_kernel; }
 long long tconv_launch_count(void) { return g_launches; }

@@ -22,7 +22,7 @@ TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
 
 # every symbol include/tconv.h declares
 SYMBOLS = ("tconv_output_shape", "tconv_winner_bytes", "tconv_workspace_bytes", "tconv_forward",
-           "tconv_backward", "tconv_paper_ops", "tconv_alu_probe", "tconv_alu_probe_name",
+           "tconv_backward", "tconv_forward_noalloc", "tconv_forward_noalloc_max_scratch", "tconv_paper_ops", "tconv_alu_probe", "tconv_alu_probe_name",
            "tconv_device_status", "tconv_status_string", "tconv_last_error", "tconv_last_kernel",
            "tconv_launch_count")
 
@@ -59,6 +59,9 @@ def _load() -> ctypes.CDLL:
     lib.tconv_forward.restype = ctypes.c_int
     lib.tconv_backward.argtypes = [dp, vp, vp, vp, fp, fp, vp, vp, vp, fp, fp, fp, fp, fp, vp, sz, vp]
     lib.tconv_backward.restype = ctypes.c_int
+    lib.tconv_forward_noalloc.argtypes = [dp, vp, vp, vp, fp, fp, fp, vp, vp, vp]
+    lib.tconv_forward_noalloc.restype = ctypes.c_int
+    lib.tconv_forward_noalloc_max_scratch.restype = sz
     lib.tconv_paper_ops.argtypes = [dp]
     lib.tconv_paper_ops.restype = ctypes.c_double
     lib.tconv_alu_probe.argtypes = [ctypes.c_int, ctypes.c_int, vp, ctypes.POINTER(ctypes.c_double), vp]
@@ -130,6 +133,17 @@ def tconv_backward(d: dict, x, w, w2, alpha, beta, grad_y, winners, grad_x, grad
                                _p(beta), _p(grad_y), _p(winners), _p(grad_x), _p(grad_w),
                                _p(grad_w2), _p(grad_alpha), _p(grad_beta), _p(grad_bias),
                                _p(workspace), nbytes, _stream(stream))
+
+
+def tconv_forward_noalloc(d: dict, x, w, w2, alpha, beta, bias, y, winners=None, stream=None) -> int:
+    """Raw call of the allocation-free forward: no workspace argument; the library's built-in
+    scratch is used.  For callers that must not touch the device allocator.  Returns the status."""
+    return _lib.tconv_forward_noalloc(ctypes.byref(make_desc(d)), _p(x), _p(w), _p(w2), _p(alpha),
+                                      _p(beta), _p(bias), _p(y), _p(winners), _stream(stream))
+
+
+def tconv_forward_noalloc_max_scratch() -> int:
+    return int(_lib.tconv_forward_noalloc_max_scratch())
 
 
 def tconv_alu_probe(variant: int, iters: int, sink, stream=None) -> float:
