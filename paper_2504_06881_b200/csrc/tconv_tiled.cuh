@@ -170,13 +170,16 @@ struct TiledParams {
     int NSLOTS, XW, XP;  // staged input rows per tile, staged columns, row pitch (floats)
     int GAP;           // extra input-row slots between two images of one tile (flattened tiles)
     int CC, Cpad, nchunks;
-    int stage_floats, x_stage, w_stage, ab_stage;  // shared-memory layout of one stage (floats)
+    int stage_floats, x_stage, w_stage, ab_stage;  // shared-memory layout of one stage (4-byte words)
 };
 
 // Column shift of the TMA path: the tile's first input column ow0*SW - pw is rounded
 // down to a multiple of 4 floats so that the copy starts on a 16-byte boundary.  The
 // TMA path is used with "same" padding pw = (S-1)*DW/2 only, which fixes the shift.
-template <int S, int DW> struct TmaShift { static constexpr int value = (4 - (((S - 1) * DW / 2) % 4)) % 4; };
+template <int S, int DW, int ESIZE = 4> struct TmaShift {
+    static constexpr int unit = 16 / ESIZE;  // elements per 16 bytes
+    static constexpr int value = (unit - (((S - 1) * DW / 2) % unit)) % unit;
+};
 
 // MODE: tconv_mode_t, CHAN: CH_SUM / CH_MAX / CH_MIN, WIN: emit winners, XTMA: x tile by TMA.
 // Q quads of 4 pixels per thread, KG groups of 8 output channels and PW pixel warps per CTA.
@@ -627,6 +630,9 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* p
     const int max_qpr = NQ >= 32 ? NQ / 4 : NQ;
     const int ncol = (qpr_full + max_qpr - 1) / max_qpr;
     p.QPR = (qpr_full + ncol - 1) / ncol;
+    // every column tile must start on a 16-byte boundary of the input row (TMA): with 2-byte
+    // elements that needs an even number of 8-byte quads per tile
+    if (esize == 2 && ncol > 1 && ((p.QPR * SW) & 1)) p.QPR += 1;
     p.TW = p.QPR * 4;
     p.n_col_tiles = (g.OW + p.TW - 1) / p.TW;
     p.TH = NQ / p.QPR;
@@ -634,7 +640,8 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* p
     p.total_rows = g.N * g.OH;
     // TMA path: rows of x are 16-byte multiples, "same" padding along w (fixes the column shift),
     // and tiles that stay inside one image without idling more than a quarter of the lanes
-    const int shift = TmaShift<S, DW>::value;
+    const int unit = 16 / esize;                                     // elements per 16 bytes
+    const int shift = esize == 4 ? TmaShift<S, DW, 4>::value : TmaShift<S, DW, 2>::value;
     const int th_img = p.TH < g.OH ? p.TH : g.OH;
     const int tiles_img = (g.OH + th_img - 1) / th_img;
     const bool rows_fit = (double)g.OH / (tiles_img * th_img) >= 0.75 && th_img * p.QPR * 4 >= NQ * 3;
@@ -646,7 +653,7 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* p
         p.n_row_tiles = g.N * tiles_img;
         p.GAP = 0;
         p.NSLOTS = (p.TH - 1) * g.sh + (R - 1) * g.dh + 1;
-        p.XP = round_up(p.XW + shift, 4);
+        p.XP = round_up(p.XW + shift, unit);
         if (p.XP > 256 || p.NSLOTS > 256) return false;
     } else {
         if (p.TH > p.total_rows) p.TH = p.total_rows;
@@ -656,13 +663,14 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* p
         if (p.GAP < 0) p.GAP = 0;
         const int max_imgs = (p.TH - 1) / g.OH + 2;
         p.NSLOTS = (p.TH - 1) * g.sh + (R - 1) * g.dh + 1 + (max_imgs - 1) * p.GAP;
-        p.XP = round_up(p.XW, 4);
+        p.XP = round_up(p.XW, unit);
     }
     p.CC = 8;
     p.Cpad = round_up(g.C, p.CC);
     p.nchunks = p.Cpad / p.CC;
-    // one stage: x tile | weights | (weights 2) | alpha | beta, each block 128-byte aligned
-    p.x_stage = round_up(p.CC * p.NSLOTS * p.XP, 32);
+    // one stage: x tile | weights | (weights 2) | alpha | beta, each block 128-byte aligned;
+    // sizes in 4-byte words (XP counts elements of esize bytes)
+    p.x_stage = round_up(p.CC * p.NSLOTS * p.XP * esize / 4, 32);
     p.w_stage = p.CC * g.RS * TILE_K;            // multiple of 32 floats
     p.ab_stage = two ? p.CC * TILE_K : 0;
     p.stage_floats = p.x_stage + p.w_stage * (par ? 2 : 1) + 2 * p.ab_stage;

@@ -59,20 +59,26 @@ def test_multi_tile_ragged(mode, chan):
                        recompute=False)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("mode,chan", ALL_MODES)
-def test_tma_staged_shapes(mode, chan):
+def test_tma_staged_shapes(mode, chan, dtype):
     """Shapes whose input rows are 16-byte multiples with 'same' padding take the TMA-staged
-    kernels: several channel chunks, ragged K and C, partial row tiles, stride 2, dilation 2."""
+    kernels: several channel chunks, ragged K and C, partial row tiles, several column tiles,
+    stride 2, dilation 2."""
     from paper_2504_06881_b200 import tconv
-    cases = [inputs.layer(3, 19, 20, 32, 41, 3, 3, stride=1, pad=1, mode=mode, chan=chan),
-             inputs.layer(2, 10, 30, 56, 35, 3, 3, stride=2, pad=1, mode=mode, chan=chan),
-             inputs.layer(2, 9, 24, 64, 33, 3, 3, stride=1, pad=2, dil=2, mode=mode, chan=chan),
-             inputs.layer(2, 17, 28, 28, 16, 3, 3, stride=1, pad=1, mode=mode, chan=chan),
-             inputs.layer(1, 8, 6, 128, 8, 3, 3, stride=1, pad=1, mode=mode, chan=chan)]
+    mk = lambda *a, **k: inputs.layer(*a, mode=mode, chan=chan, dtype=dtype, **k)
+    cases = [mk(3, 19, 20, 32, 41, 3, 3, stride=1, pad=1),
+             mk(2, 10, 30, 56, 35, 3, 3, stride=2, pad=1),
+             mk(2, 9, 24, 64, 33, 3, 3, stride=1, pad=2, dil=2),
+             mk(2, 17, 28, 28, 16, 3, 3, stride=1, pad=1),
+             mk(1, 8, 6, 128, 8, 3, 3, stride=1, pad=1),
+             mk(1, 5, 9, 40, 8, 3, 3, stride=1, pad=1)]
     for i, d in enumerate(cases):
         t = inputs.draw(d, 450 + i)
         parity.check_forward(d, t, check_winners=False)
-        assert "tma" in tconv.tconv_last_kernel(), tconv.tconv_last_kernel()
+        expect_tma = (d["W"] * (4 if dtype == "f32" else 2)) % 16 == 0
+        assert ("tma" in tconv.tconv_last_kernel()) == expect_tma, tconv.tconv_last_kernel()
+        assert "tiled" in tconv.tconv_last_kernel()
         assert tconv.tconv_device_status() == 0
         parity.check_layer(d, None, 460 + i, recompute=False)
         parity.check_layer(d, TIES, 470 + i, recompute=False, stored_winners=(i == 0))
