@@ -183,8 +183,17 @@ template <int S, int DW, int ESIZE = 4> struct TmaShift {
 
 // MODE: tconv_mode_t, CHAN: CH_SUM / CH_MAX / CH_MIN, WIN: emit winners, XTMA: x tile by TMA.
 // Q quads of 4 pixels per thread, KG groups of 8 output channels and PW pixel warps per CTA.
+// Resident CTAs per SM the register allocation aims at: the winner-free kernels are bound by
+// the ALU / FMA pipes and want four or more warps per scheduler to hide their latencies.
+#ifndef TCONV_MINB_SINGLE
+#define TCONV_MINB_SINGLE 4
+#endif
+#ifndef TCONV_Q_CARRIED
+#define TCONV_Q_CARRIED 2
+#endif
 template <int MODE, int CHAN, bool WIN, bool XTMA, int R, int S, int SW, int DW, int Q, int KG, int PW>
-__global__ void __launch_bounds__(KG * PW * 32)
+__global__ void __launch_bounds__(KG * PW * 32,
+                                  (WIN || MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL) ? 1 : TCONV_MINB_SINGLE)
 fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams p) {
     constexpr int RS = R * S;
     constexpr int TILE_K = KG * 8;
@@ -779,7 +788,7 @@ int launch_tiled_geom(FwdArgs& a) {
     // extremum of layers (iv), (v) without winners), else one
     constexpr bool CARRIED = !TWO && !WIN && ((MODE == TCONV_MAX_PLUS && CHAN == CH_MAX) ||
                                               (MODE == TCONV_MIN_PLUS && CHAN == CH_MIN));
-    constexpr int Q = CARRIED ? 2 : 1;
+    constexpr int Q = CARRIED ? TCONV_Q_CARRIED : 1;
     const Geo& g = a.g;
     if (g.R == 3 && g.S == 3) {
         if (g.sw == 1 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 1, Q, 4, 1>(a);
