@@ -167,7 +167,7 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
         if (gx) {
             if (tiled && plan_idx_gx(g, &thi, &smem)) {
                 auto kern = bwd_idx_gx_kernel<T>;
-                if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemLimit) != cudaSuccess)
+                if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess)
                     return cuda_fail(cudaGetLastError());
                 const int tiles = (g.H + thi - 1) / thi;
                 const unsigned magic = g.RS == 1 ? 0u : (0xFFFFFFFFu / (unsigned)g.RS) + 1u;
@@ -186,7 +186,7 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
             float* pw = (float*)ws;
             float* pb = pw + (size_t)chunks * g.K * CRS;
             auto kern = bwd_idx_gw_kernel<T>;
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemLimit) != cudaSuccess)
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess)
                 return cuda_fail(cudaGetLastError());
             const int npc = (g.N + chunks - 1) / chunks;
             kern<<<dim3((unsigned)g.K, (unsigned)chunks), 256, smem, st>>>(g, (const T*)gy, idx, pw, pb, npc);
@@ -217,7 +217,7 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
 #define TCONV_GX(BR)                                                                                 \
     {                                                                                                \
         auto kern = bwd_code_gx_kernel<T, BR>;                                                       \
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemLimit) != cudaSuccess) \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<grid, 256, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);          \
     }
@@ -232,17 +232,32 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
             g_launches += 1;
         }
         if (gw || gw2 || galpha || gbeta) {
-            if (tiled && !g.wide && code_gw_smem(g) <= kBwdSmemLimit) {
-                const size_t smem = code_gw_smem(g);
-#define TCONV_GW(BR)                                                                                 \
+            CodeGwPlan gp;
+            plan_code_gw(g, &gp);
+            if (tiled && !g.wide && gp.smem <= kBwdSmemLimit) {
+                // zero-padded copy of x for the branch values of grad_alpha / grad_beta, placed after
+                // the grad_bias partials in the workspace
+                const size_t bias_part = ((size_t)16 * g.K * sizeof(float) + 255) / 256 * 256;
+                const size_t pad_bytes = padded_x_bytes(g, (int)sizeof(T));
+                if (br == 0 && (galpha || gbeta) && ws && ws_bytes >= bias_part + pad_bytes &&
+                    (double)g.N * g.C * gp.HP * gp.WP < 2.0e9) {
+                    T* xpad = (T*)((char*)ws + bias_part);
+                    const size_t total = (size_t)g.N * g.C * gp.HP * gp.WP;
+                    pad_input_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, (const T*)x, xpad, gp.HP, gp.WP);
+                    g_launches += 1;
+                    gp.xs_elems = gp.HP * gp.WP;
+                    gp.xpad = xpad;
+                }
+#define TCONV_GW(BR, XSV)                                                                            \
     {                                                                                                \
-        auto kern = bwd_code_gw_kernel<T, BR>;                                                       \
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemLimit) != cudaSuccess) \
+        auto kern = bwd_code_gw_kernel<T, BR, XSV>;                                                  \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
-        kern<<<(unsigned)((size_t)g.K * g.C), 256, smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
-                                                      (const T*)gy, codes, gw, gw2, galpha, gbeta); \
+        kern<<<(unsigned)((size_t)g.K * g.C), 256, gp.smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
+                                                      (const T*)gy, codes, gw, gw2, galpha, gbeta, gp); \
     }
-                if (br == 0) TCONV_GW(0) else if (br == 1) TCONV_GW(1) else TCONV_GW(2)
+                if (br == 0) { if (gp.xs_elems) TCONV_GW(0, true) else TCONV_GW(0, false) }
+                else if (br == 1) TCONV_GW(1, false) else TCONV_GW(2, false)
 #undef TCONV_GW
                 g_launches += 1;
                 name = "bwd_code";
@@ -261,8 +276,19 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
         }
     }
     if (gbias && !bias_done) {
-        bwd_bias_kernel<T><<<(unsigned)g.K, 256, 0, st>>>(g, (const T*)gy, gbias);
-        g_launches += 1;
+        int chunks = g.N < 16 ? g.N : 16;
+        if (tiled && ws && ws_bytes >= (size_t)chunks * g.K * sizeof(float)) {
+            const int npc = (g.N + chunks - 1) / chunks;
+            chunks = (g.N + npc - 1) / npc;
+            bwd_bias_partial_kernel<T><<<dim3((unsigned)g.K, (unsigned)chunks), 256, 0, st>>>(
+                g, (const T*)gy, (float*)ws, npc);
+            bwd_reduce_partials_kernel<<<(unsigned)((g.K + 255) / 256), 256, 0, st>>>((const float*)ws, gbias,
+                                                                                   (size_t)g.K, chunks);
+            g_launches += 2;
+        } else {
+            bwd_bias_kernel<T><<<(unsigned)g.K, 256, 0, st>>>(g, (const T*)gy, gbias);
+            g_launches += 1;
+        }
     }
     snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", name);
     return check_launch();

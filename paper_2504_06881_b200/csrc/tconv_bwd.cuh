@@ -130,6 +130,8 @@ __global__ void bwd_reduce_partials_kernel(const float* __restrict__ partial, fl
 }
 
 // ---------------------------------------------------------------------------------- codes: grad_x
+constexpr int kGxCB = 2;   // most channels a CTA of bwd_code_gx_kernel handles
+
 struct CodeGxPlan {
     int THI, tiles_per_img;  // owned input rows per CTA
     int CB;                  // channels per CTA
@@ -143,7 +145,7 @@ __global__ void __launch_bounds__(256)
 bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
                    CodeGxPlan pl) {
-    extern __shared__ float A[];  // [CB][RS][4][NQpad]
+    extern __shared__ float A[];  // [CB][RS][4][NQpad], then alpha / beta of this CTA's channels [K][CB] each
     const int tile_i = blockIdx.x % pl.tiles_per_img;
     const int n = blockIdx.x / pl.tiles_per_img;
     const int c0 = blockIdx.y * pl.CB;
@@ -156,7 +158,18 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     const int NR = oh_hi - oh_lo + 1;
     const int NQ = NR * pl.QPR;
     const int NQp = pl.NQpad;
-    for (int e = threadIdx.x; e < pl.CB * g.RS * 4 * NQp; e += blockDim.x) A[e] = 0.0f;
+    const int nacc = pl.CB * g.RS * 4 * NQp;
+    float* a_s = A + nacc;
+    float* b_s = a_s + g.K * pl.CB;
+    for (int e = threadIdx.x; e < nacc; e += blockDim.x) A[e] = 0.0f;
+    if constexpr (BR == 0) {
+        for (int e = threadIdx.x; e < g.K * pl.CB; e += blockDim.x) {
+            const int k = e / pl.CB, cb = e - k * pl.CB;
+            const bool ok = cb < ncb;
+            a_s[e] = (ok && alpha) ? alpha[(size_t)k * g.C + c0 + cb] : 1.0f;
+            b_s[e] = (ok && beta) ? beta[(size_t)k * g.C + c0 + cb] : 1.0f;
+        }
+    }
     __syncthreads();
     const size_t plane = (size_t)g.OH * g.OW;
     const bool vec = (g.OW & 3) == 0;
@@ -165,15 +178,16 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
         const int ow0 = (q - orow * pl.QPR) * 4;
         const size_t pix = (size_t)(oh_lo + orow) * g.OW + ow0;
         float* Aq = A + q;
-        for (int k = 0; k < g.K; ++k) {
+        // operands of output channel k: 4 gradients and the code words of the CTA's channels;
+        // the loads of k+1 are issued before the accumulators of k are updated
+        auto load_k = [&](int k, float* gv, unsigned* cw) {
             const size_t ob = ((size_t)n * g.K + k) * plane + pix;
-            float gv[4];
             if (vec) {
                 if constexpr (sizeof(T) == 4) {
-                    const float4 v = *reinterpret_cast<const float4*>(gy + ob);
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(gy + ob));
                     gv[0] = v.x; gv[1] = v.y; gv[2] = v.z; gv[3] = v.w;
                 } else {
-                    const uint2 v = *reinterpret_cast<const uint2*>(gy + ob);
+                    const uint2 v = __ldg(reinterpret_cast<const uint2*>(gy + ob));
                     gv[0] = __uint_as_float(v.x << 16); gv[1] = __uint_as_float(v.x & 0xffff0000u);
                     gv[2] = __uint_as_float(v.y << 16); gv[3] = __uint_as_float(v.y & 0xffff0000u);
                 }
@@ -181,37 +195,52 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
 #pragma unroll
                 for (int j = 0; j < 4; ++j) gv[j] = (ow0 + j < g.OW) ? to_f32(gy[ob + j]) : 0.0f;
             }
-            for (int cb = 0; cb < ncb; ++cb) {
-                const int c = c0 + cb;
-                const size_t cbase = (((size_t)n * g.K + k) * g.C + c) * plane + pix;
-                unsigned cw;
-                if (vec) {
-                    cw = *reinterpret_cast<const unsigned*>(codes + cbase);
-                } else {
-                    cw = 0;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (ow0 + j < g.OW) cw |= (unsigned)codes[cbase + j] << (8 * j);
+            for (int cb = 0; cb < kGxCB; ++cb) {
+                cw[cb] = 0;
+                if (cb < ncb) {
+                    const size_t cbase = (((size_t)n * g.K + k) * g.C + c0 + cb) * plane + pix;
+                    if (vec) {
+                        cw[cb] = __ldg(reinterpret_cast<const unsigned*>(codes + cbase));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (ow0 + j < g.OW) cw[cb] |= (unsigned)codes[cbase + j] << (8 * j);
+                    }
                 }
+            }
+        };
+        float gv_cur[4], gv_nxt[4];
+        unsigned cw_cur[kGxCB], cw_nxt[kGxCB];
+        load_k(0, gv_cur, cw_cur);
+        for (int k = 0; k < g.K; ++k) {
+            if (k + 1 < g.K) load_k(k + 1, gv_nxt, cw_nxt);
+#pragma unroll
+            for (int cb = 0; cb < kGxCB; ++cb) {
+                if (cb >= ncb) break;
                 float a = 1.0f, b = 1.0f;
                 if constexpr (BR == 0) {
-                    if (alpha) a = __ldg(alpha + (size_t)k * g.C + c);
-                    if (beta) b = __ldg(beta + (size_t)k * g.C + c);
+                    a = a_s[k * pl.CB + cb];
+                    b = b_s[k * pl.CB + cb];
                 }
                 float* Ac = Aq + (size_t)cb * g.RS * 4 * NQp;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const unsigned code = (cw >> (8 * j)) & 0xffu;
+                    const unsigned code = (cw_cur[cb] >> (8 * j)) & 0xffu;
                     if constexpr (BR == 0 || BR == 1) {
                         const int t = code & 15u;
-                        Ac[(t * 4 + j) * NQp] += (BR == 0 ? a * gv[j] : gv[j]);
+                        Ac[(t * 4 + j) * NQp] += (BR == 0 ? a * gv_cur[j] : gv_cur[j]);
                     }
                     if constexpr (BR == 0 || BR == 2) {
                         const int t = code >> 4;
-                        Ac[(t * 4 + j) * NQp] += (BR == 0 ? b * gv[j] : gv[j]);
+                        Ac[(t * 4 + j) * NQp] += (BR == 0 ? b * gv_cur[j] : gv_cur[j]);
                     }
                 }
             }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) gv_cur[j] = gv_nxt[j];
+#pragma unroll
+            for (int cb = 0; cb < kGxCB; ++cb) cw_cur[cb] = cw_nxt[cb];
         }
     }
     __syncthreads();
@@ -243,14 +272,37 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
 }
 
 // ---------------------------------------------------------------------------------- codes: grad_w, grad_alpha, grad_beta
-template <typename T, int BR>
+// One CTA per (k, c).  XS: a zero-padded copy of x (made once per backward call by
+// pad_input_kernel) is available, so that the branch values x[winner] + w[winner] of
+// grad_alpha / grad_beta are gathered without bounds checks.
+struct CodeGwPlan {
+    int HP, WP;      // padded plane extent covering every tap of every output
+    int xs_elems;    // elements of one padded plane (0: no padded copy)
+    size_t smem;
+    const void* xpad;
+};
+
+// xpad[n][c][HP][WP] = x with ph rows / pw columns of zeros in front (and zeros behind)
+template <typename T>
+__global__ void pad_input_kernel(Geo g, const T* __restrict__ x, T* __restrict__ xpad, int HP, int WP) {
+    const size_t total = (size_t)g.N * g.C * HP * WP;
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int pc = (int)(i % WP);
+    const int pr = (int)((i / WP) % HP);
+    const size_t nc = i / ((size_t)WP * HP);
+    const int ih = pr - g.ph, iw = pc - g.pw;
+    xpad[i] = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? x[(nc * g.H + ih) * g.W + iw] : zero_of<T>();
+}
+
+template <typename T, int BR, bool XS>
 __global__ void __launch_bounds__(256)
 bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
                    const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes,
                    float* __restrict__ gw, float* __restrict__ gw2, float* __restrict__ galpha,
-                   float* __restrict__ gbeta) {
-    extern __shared__ float S[];  // [2*RS + 2][256] private columns, then tap tables
+                   float* __restrict__ gbeta, CodeGwPlan pl) {
+    extern __shared__ float S[];  // [2*RS + 2][256] private columns | tap tables | weights | x planes
     const int c = blockIdx.x % g.C;
     const int k = blockIdx.x / g.C;
     const int tid = threadIdx.x;
@@ -258,24 +310,30 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
     float* col = S + tid;
     int* tap_dh = reinterpret_cast<int*>(S + NB * 256);
     int* tap_dw = tap_dh + g.RS;
-    float* wmin_s = reinterpret_cast<float*>(tap_dw + g.RS);
+    int* tap_off = tap_dw + g.RS;
+    float* wmin_s = reinterpret_cast<float*>(tap_off + g.RS);
     float* wmax_s = wmin_s + g.RS;
     for (int b = 0; b < NB; ++b) col[b * 256] = 0.0f;
     if (tid < g.RS) {
-        tap_dh[tid] = (tid / g.S) * g.dh - g.ph;
-        tap_dw[tid] = (tid % g.S) * g.dw - g.pw;
-        wmin_s[tid] = to_f32(w[((size_t)k * g.C + c) * g.RS + tid]);
-        wmax_s[tid] = to_f32((g.mode == TCONV_PARALLEL ? w2 : w)[((size_t)k * g.C + c) * g.RS + tid]);
+        const int r = tid / g.S, sx = tid % g.S;
+        tap_dh[tid] = r * g.dh - g.ph;
+        tap_dw[tid] = sx * g.dw - g.pw;
+        tap_off[tid] = r * g.dh * pl.WP + sx * g.dw;
+        const size_t wi = ((size_t)k * g.C + c) * g.RS + tid;
+        wmin_s[tid] = to_f32(w[wi]);
+        wmax_s[tid] = to_f32((g.mode == TCONV_PARALLEL ? w2 : w)[wi]);
     }
-    __syncthreads();
     const bool need_ab = (BR == 0) && (galpha || gbeta);
     const int QPR = (g.OW + 3) >> 2;
     const int NQ = g.OH * QPR;
     const size_t plane = (size_t)g.OH * g.OW;
     const bool vec = (g.OW & 3) == 0;
     float sa = 0.0f, sb = 0.0f;
+
+    __syncthreads();
     for (int n = 0; n < g.N; ++n) {
         const T* xc = x + ((size_t)n * g.C + c) * g.H * g.W;
+        const T* xsn = reinterpret_cast<const T*>(pl.xpad) + ((size_t)n * g.C + c) * pl.xs_elems;
         const size_t obase = ((size_t)n * g.K + k) * plane;
         const size_t cbase = (((size_t)n * g.K + k) * g.C + c) * plane;
         for (int q = tid; q < NQ; q += 256) {
@@ -285,12 +343,12 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
             float gv[4];
             unsigned cw;
             if (vec) {
-                cw = *reinterpret_cast<const unsigned*>(codes + cbase + pix);
+                cw = __ldg(reinterpret_cast<const unsigned*>(codes + cbase + pix));
                 if constexpr (sizeof(T) == 4) {
-                    const float4 v = *reinterpret_cast<const float4*>(gy + obase + pix);
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(gy + obase + pix));
                     gv[0] = v.x; gv[1] = v.y; gv[2] = v.z; gv[3] = v.w;
                 } else {
-                    const uint2 v = *reinterpret_cast<const uint2*>(gy + obase + pix);
+                    const uint2 v = __ldg(reinterpret_cast<const uint2*>(gy + obase + pix));
                     gv[0] = __uint_as_float(v.x << 16); gv[1] = __uint_as_float(v.x & 0xffff0000u);
                     gv[2] = __uint_as_float(v.y << 16); gv[3] = __uint_as_float(v.y & 0xffff0000u);
                 }
@@ -303,6 +361,7 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
                     if (ok) cw |= (unsigned)codes[cbase + pix + j] << (8 * j);
                 }
             }
+            const int xbase = oh * g.sh * pl.WP + ow0 * g.sw;   // staged-plane index of tap (0, 0) of pixel ow0
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 if (!vec && ow0 + j >= g.OW) continue;
@@ -312,9 +371,13 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
                     const int t = code & 15u;
                     col[t * 256] += gv[j];
                     if (need_ab) {
-                        const int ih = oh * g.sh + tap_dh[t], iw = ow * g.sw + tap_dw[t];
-                        T xv = zero_of<T>();
-                        if (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) xv = xc[(size_t)ih * g.W + iw];
+                        T xv;
+                        if constexpr (XS) {
+                            xv = xsn[xbase + j * g.sw + tap_off[t]];
+                        } else {
+                            const int ih = oh * g.sh + tap_dh[t], iw = ow * g.sw + tap_dw[t];
+                            xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xc[(size_t)ih * g.W + iw] : zero_of<T>();
+                        }
                         sa = __fmaf_rn(gv[j], tap_add(xv, from_f32<T>(wmin_s[t])), sa);
                     }
                 }
@@ -322,9 +385,13 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
                     const int t = code >> 4;
                     col[(g.RS + t) * 256] += gv[j];
                     if (need_ab) {
-                        const int ih = oh * g.sh + tap_dh[t], iw = ow * g.sw + tap_dw[t];
-                        T xv = zero_of<T>();
-                        if (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) xv = xc[(size_t)ih * g.W + iw];
+                        T xv;
+                        if constexpr (XS) {
+                            xv = xsn[xbase + j * g.sw + tap_off[t]];
+                        } else {
+                            const int ih = oh * g.sh + tap_dh[t], iw = ow * g.sw + tap_dw[t];
+                            xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xc[(size_t)ih * g.W + iw] : zero_of<T>();
+                        }
                         sb = __fmaf_rn(gv[j], tap_add(xv, from_f32<T>(wmax_s[t])), sb);
                     }
                 }
@@ -362,14 +429,49 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
     }
 }
 
+// grad_bias partials: grid (K, chunks); partial[chunk][k] = sum of grad_y over the chunk's images
+template <typename T>
+__global__ void __launch_bounds__(256)
+bwd_bias_partial_kernel(Geo g, const T* __restrict__ gy, float* __restrict__ partial, int n_per_chunk) {
+    __shared__ float red[256];
+    const int k = blockIdx.x, chunk = blockIdx.y;
+    const size_t plane = (size_t)g.OH * g.OW;
+    const int n_lo = chunk * n_per_chunk, n_hi = min(g.N, n_lo + n_per_chunk);
+    float s = 0.0f;
+    for (int n = n_lo; n < n_hi; ++n) {
+        const T* src = gy + ((size_t)n * g.K + k) * plane;
+        for (size_t j = threadIdx.x; j < plane; j += blockDim.x) s += to_f32(src[j]);
+    }
+    const float t = block_sum(s, red);
+    if (threadIdx.x == 0) partial[chunk * g.K + k] = t;
+}
+
 // ---------------------------------------------------------------------------------- host side
+inline void plan_code_gw(const Geo& g, CodeGwPlan* pl) {
+    pl->smem = ((size_t)(2 * g.RS + 2) * 256 + 5 * (size_t)g.RS + 4) * sizeof(float);
+    pl->HP = (g.OH - 1) * g.sh + (g.R - 1) * g.dh + 1;
+    pl->WP = (g.OW - 1) * g.sw + (g.S - 1) * g.dw + 1;
+    if (pl->HP < g.H + g.ph) pl->HP = g.H + g.ph;   // rows / columns no output reaches still hold x
+    if (pl->WP < g.W + g.pw) pl->WP = g.W + g.pw;
+    pl->xs_elems = 0;
+    pl->xpad = nullptr;
+}
+inline size_t padded_x_bytes(const Geo& g, int esize) {
+    if (!two_branch(g.mode)) return 0;
+    CodeGwPlan pl;
+    plan_code_gw(g, &pl);
+    return ((size_t)g.N * g.C * pl.HP * pl.WP * esize + 255) / 256 * 256;
+}
+
 inline size_t bwd_ws_bytes(const Geo& g) {
-    // partial histograms of the Max / Min combine: at most 16 chunks of [K][C*RS + 1] floats
-    if (g.chan == CH_SUM) return 0;
+    // partial histograms of the Max / Min combine: at most 16 chunks of [K][C*RS + 1] floats;
+    // Sum forms: 16 chunks of grad_bias partials
+    if (g.chan == CH_SUM) return (size_t)16 * g.K * sizeof(float) + 256 + padded_x_bytes(g, 4);
     return (size_t)16 * g.K * ((size_t)g.C * g.RS + 1) * sizeof(float) + 256;
 }
 
-constexpr size_t kBwdSmemLimit = 160 * 1024;
+constexpr size_t kBwdSmemLimit = 160 * 1024;   // planning budget per CTA
+constexpr int kBwdSmemAttr = 200 * 1024;       // opt-in ceiling set on the kernels
 
 // Plans for the winner-driven kernels; false when the shape does not fit (the caller then
 // uses the any-shape kernels).
@@ -403,7 +505,7 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
     if (g.wide) return false;
     pl->QPR = (g.OW + 3) / 4;
     const int halo = (g.R - 1) * g.dh;
-    for (int cb = 2; cb >= 1; --cb) {
+    for (int cb = kGxCB; cb >= 1; --cb) {
         // rows of output quads that fit: CB * RS * 4 floats per quad
         const size_t per_quad = (size_t)cb * g.RS * 4 * sizeof(float);
         const long maxq = (long)(kBwdSmemLimit / per_quad) / 32 * 32;
@@ -424,15 +526,11 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
         pl->tiles_per_img = (g.H + thi - 1) / thi;
         pl->NRmax = (int)nr;
         pl->NQpad = (int)(((long)nr * pl->QPR + 31) / 32 * 32);
-        pl->smem = (size_t)cb * g.RS * 4 * pl->NQpad * sizeof(float);
-        if (pl->smem > kBwdSmemLimit) continue;
+        pl->smem = ((size_t)cb * g.RS * 4 * pl->NQpad + 2 * (size_t)g.K * cb) * sizeof(float);
+        if (pl->smem > kBwdSmemLimit + 16 * 1024) continue;
         return true;
     }
     return false;
-}
-
-inline size_t code_gw_smem(const Geo& g) {
-    return (size_t)(2 * g.RS + 2) * 256 * sizeof(float) + (size_t)g.RS * 4 * sizeof(int);
 }
 
 }  // namespace tconv
