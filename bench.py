@@ -194,12 +194,16 @@ class Layer:
         if rc != 0:
             raise self.tconv.TconvError(rc, "tconv_forward")
 
-    def bwd(self):
+    def bwd(self, parts="all"):
+        """parts: "all", "x" (grad_x only) or "params" (every parameter gradient)."""
         v = self.dev
+        gx = self.gx if parts in ("all", "x") else None
+        P = parts in ("all", "params")
         rc = self.tconv.tconv_backward(self.d, v["x"], v["w"], v["w2"] if self.par else None,
                                        v["alpha"] if self.two else None, v["beta"] if self.two else None,
-                                       v["g"], self.win, self.gx, self.gw, self.gw2, self.ga, self.gb,
-                                       self.gbias, self.ws)
+                                       v["g"], self.win, gx, self.gw if P else None,
+                                       self.gw2 if P else None, self.ga if P else None,
+                                       self.gb if P else None, self.gbias if P else None, self.ws)
         if rc != 0:
             raise self.tconv.TconvError(rc, "tconv_backward")
 
@@ -312,7 +316,8 @@ def run_gpu(args):
     per = {}
     for L in layers:
         rec = {}
-        for what, fn in (("fwd", lambda: L.fwd(False)), ("fwd_winners", L.fwd), ("bwd", L.bwd)):
+        for what, fn in (("fwd", lambda: L.fwd(False)), ("fwd_winners", L.fwd), ("bwd", L.bwd),
+                         ("bwd_grad_x", lambda: L.bwd("x")), ("bwd_params", lambda: L.bwd("params"))):
             ts = []
             for _ in range(5):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -338,7 +343,7 @@ def run_gpu(args):
 
     # dominant kernel = the call with the largest time in a step; its roofline is the
     # add+max/min ALU peak of that mode (a tap = one x+w term folded into min and/or max)
-    dom_mode, dom_what = max(((m, w) for m in per for w in ("fwd_winners", "bwd")),
+    dom_mode, dom_what = max(((m, w) for m in per for w in ("fwd_winners", "bwd_grad_x", "bwd_params")),
                              key=lambda mw: per[mw[0]][mw[1]])
     L = next(x for x in layers if x.d["mode"] == dom_mode)
     achieved = L.taps / (per[dom_mode][dom_what] * 1e-3) / 1e12

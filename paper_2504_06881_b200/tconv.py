@@ -238,7 +238,10 @@ def backward(d: dict, x, w, grad_y, w2=None, alpha=None, beta=None, winners=None
     if "grad_bias" in need:
         out["grad_bias"] = torch.empty((K,), dtype=f32, device=dev)
     nws = tconv_workspace_bytes(d, True)
-    ws = torch.empty(nws, dtype=torch.uint8, device=dev) if nws else None
+    if winners is not None:
+        # the figure includes room for recomputed winners, not needed when they are passed
+        nws -= (tconv_winner_bytes(d) + 255) // 256 * 256
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev) if nws > 0 else None
     rc = tconv_backward(d, x, w, w2, alpha, beta, grad_y, winners, out.get("grad_x"),
                         out.get("grad_w"), out.get("grad_w2"), out.get("grad_alpha"),
                         out.get("grad_beta"), out.get("grad_bias"), ws, stream)
