@@ -157,21 +157,24 @@ def run_reference(args):
 class Layer:
     """Device-resident tensors of one layer plus its outputs, allocated once."""
 
-    def __init__(self, mode, chan, seed, torch, tconv, inputs, dev):
-        self.d, dist = inputs.cfg2(mode, chan)
+    def __init__(self, mode, chan, seed, torch, tconv, inputs, dev, n_images=128, dtype="f32"):
+        self.d, dist = inputs.cfg2(mode, chan, N=n_images)
+        self.d = dict(self.d, dtype=dtype)
         d = self.d
         t = inputs.draw(d, seed, **dist)
-        self.host = {k: torch.from_numpy(v).pin_memory() for k, v in t.items()}
+        dt = tconv.TORCH_DTYPE[dtype]
+        self.host = {k: torch.from_numpy(v).to(dt if k in ("x", "w", "w2", "g") else torch.float32).pin_memory()
+                     for k, v in t.items()}
         self.two = mode in ("compound", "parallel")
         self.par = mode == "parallel"
         self.dev = {k: v.to(dev, non_blocking=True) for k, v in self.host.items()}
         N, C, H, W, K = d["N"], d["C"], d["H"], d["W"], d["K"]
         OH, OW = tconv.tconv_output_shape(d)
         f32 = torch.float32
-        self.y = torch.empty((N, K, OH, OW), dtype=f32, device=dev)
+        self.y = torch.empty((N, K, OH, OW), dtype=dt, device=dev)
         self.win = tconv.winner_buffer(d, dev)
         self.ws = torch.empty(tconv.tconv_workspace_bytes(d, True), dtype=torch.uint8, device=dev)
-        self.gx = torch.empty((N, C, H, W), dtype=f32, device=dev)
+        self.gx = torch.empty((N, C, H, W), dtype=dt, device=dev)
         self.gw = torch.empty((K, C, 3, 3), dtype=f32, device=dev)
         self.gw2 = torch.empty((K, C, 3, 3), dtype=f32, device=dev) if self.par else None
         self.ga = torch.empty((K, C), dtype=f32, device=dev) if self.two else None
@@ -181,8 +184,8 @@ class Layer:
         self.taps = N * K * OH * OW * C * 9
         self.tconv = tconv
         # pinned host landing buffers of the end-to-end leg
-        self.h_y = torch.empty((N, K, OH, OW), dtype=f32).pin_memory()
-        self.h_gx = torch.empty((N, C, H, W), dtype=f32).pin_memory()
+        self.h_y = torch.empty((N, K, OH, OW), dtype=dt).pin_memory()
+        self.h_gx = torch.empty((N, C, H, W), dtype=dt).pin_memory()
         self.h_small = {k: torch.empty_like(getattr(self, k), device="cpu").pin_memory()
                         for k in ("gw", "gw2", "ga", "gb", "gbias") if getattr(self, k) is not None}
 
@@ -218,8 +221,8 @@ class Layer:
         self.h_gx.copy_(self.gx, non_blocking=True)
         for k, h in self.h_small.items():
             h.copy_(getattr(self, k), non_blocking=True)
-        h2d = sum(self.host[k].numel() * 4 for k in names)
-        d2h = (self.h_y.numel() + self.h_gx.numel() + sum(h.numel() for h in self.h_small.values())) * 4
+        h2d = sum(self.host[k].numel() * self.host[k].element_size() for k in names)
+        d2h = sum(h.numel() * h.element_size() for h in [self.h_y, self.h_gx] + list(self.h_small.values()))
         return h2d, d2h
 
 
@@ -382,15 +385,46 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_single(args):
+    """One call of one layer, repeated: the small, single-kernel case the ncu captures under
+    profiles/ are taken on (`--only MODE --what fwd|fwd_winners|bwd --images N [--dtype bf16]`)."""
+    import torch
+    from paper_2504_06881_b200 import inputs, tconv
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    L = Layer(args.only, "default", 1020, torch, tconv, inputs, dev, n_images=args.images, dtype=args.dtype)
+    fn = {"fwd": lambda: L.fwd(False), "fwd_winners": L.fwd, "bwd": L.bwd}[args.what]
+    L.fwd()
+    for _ in range(max(args.warmup, 1)):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    print(json.dumps({"only": args.only, "what": args.what, "images": args.images, "dtype": args.dtype,
+                      "ms": ms, "Ttap_s": L.taps / (ms * 1e-3) / 1e12, "kernel": tconv.tconv_last_kernel()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--only", default=None, choices=["max_plus", "min_plus", "compound", "parallel"],
+                    help="profile helper: run one layer's call instead of the benchmark step")
+    ap.add_argument("--what", default="fwd", choices=["fwd", "fwd_winners", "bwd"])
+    ap.add_argument("--images", type=int, default=128)
+    ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.only:
+        run_single(args)
     else:
         run_gpu(args)
 

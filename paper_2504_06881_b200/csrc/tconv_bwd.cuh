@@ -480,9 +480,10 @@ inline bool plan_idx_gx(const Geo& g, int* THI, size_t* smem) {
     if (row == 0 || row > kBwdSmemLimit) return false;
     int t = (int)(kBwdSmemLimit / row);
     if (t > g.H) t = g.H;
-    // keep at least ~2 CTAs per SM worth of tiles when the batch is small
-    while (t > 4 && (size_t)g.N * ((g.H + t - 1) / t) < 296) t = (t + 1) / 2;
+    // keep at least ~2 CTAs per SM worth of tiles when the batch is small, but never bands so thin
+    // that most scanned rows are halo
     const int halo = (g.R - 1) * g.dh;
+    while ((t + 1) / 2 >= 2 * halo && (t + 1) / 2 >= 4 && (size_t)g.N * ((g.H + t - 1) / t) < 296) t = (t + 1) / 2;
     if (t < g.H && t < 2 * halo) return false;  // too much redundant scanning
     *THI = t;
     *smem = row * t;
