@@ -214,14 +214,21 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
         if (gx) {
             if (tiled && plan_code_gx(g, &pl)) {
                 const dim3 grid((unsigned)(g.N * pl.tiles_per_img), (unsigned)((g.C + pl.CB - 1) / pl.CB));
-#define TCONV_GX(BR)                                                                                 \
+#define TCONV_GX(BR, CBV, VECV)                                                                      \
     {                                                                                                \
-        auto kern = bwd_code_gx_kernel<T, BR>;                                                       \
+        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV>;                                            \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<grid, 256, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);          \
     }
-                if (br == 0) TCONV_GX(0) else if (br == 1) TCONV_GX(1) else TCONV_GX(2)
+#define TCONV_GX2(BR)                                                                                \
+    {                                                                                                \
+        if (pl.CB == 2) { if (vec) TCONV_GX(BR, 2, true) else TCONV_GX(BR, 2, false) }               \
+        else { if (vec) TCONV_GX(BR, 1, true) else TCONV_GX(BR, 1, false) }                           \
+    }
+                const bool vec = (g.OW & 3) == 0;
+                if (br == 0) TCONV_GX2(0) else if (br == 1) TCONV_GX2(1) else TCONV_GX2(2)
+#undef TCONV_GX2
 #undef TCONV_GX
                 name = "bwd_code";
             } else {
@@ -248,16 +255,19 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                     gp.xs_elems = gp.HP * gp.WP;
                     gp.xpad = xpad;
                 }
-#define TCONV_GW(BR, XSV)                                                                            \
+#define TCONV_GW(BR, XSV, VECV)                                                                      \
     {                                                                                                \
-        auto kern = bwd_code_gw_kernel<T, BR, XSV>;                                                  \
+        auto kern = bwd_code_gw_kernel<T, BR, XSV, VECV>;                                            \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<(unsigned)((size_t)g.K * g.C), 256, gp.smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
                                                       (const T*)gy, codes, gw, gw2, galpha, gbeta, gp); \
     }
-                if (br == 0) { if (gp.xs_elems) TCONV_GW(0, true) else TCONV_GW(0, false) }
-                else if (br == 1) TCONV_GW(1, false) else TCONV_GW(2, false)
+#define TCONV_GWV(BR, XSV) { if (vecw) TCONV_GW(BR, XSV, true) else TCONV_GW(BR, XSV, false) }
+                const bool vecw = (g.OW & 3) == 0;
+                if (br == 0) { if (gp.xs_elems) TCONV_GWV(0, true) else TCONV_GWV(0, false) }
+                else if (br == 1) TCONV_GWV(1, false) else TCONV_GWV(2, false)
+#undef TCONV_GWV
 #undef TCONV_GW
                 g_launches += 1;
                 name = "bwd_code";

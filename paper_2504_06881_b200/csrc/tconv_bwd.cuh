@@ -139,8 +139,41 @@ struct CodeGxPlan {
     size_t smem;
 };
 
+// Loads 4 horizontally adjacent gradients (VEC: one aligned vector load).
+template <typename T, bool VEC>
+__device__ __forceinline__ void load_g4(const T* p, int ow0, int OW, float* gv) {
+    if constexpr (VEC) {
+        if constexpr (sizeof(T) == 4) {
+            const float4 v = __ldg(reinterpret_cast<const float4*>(p));
+            gv[0] = v.x; gv[1] = v.y; gv[2] = v.z; gv[3] = v.w;
+        } else {
+            const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+            gv[0] = __uint_as_float(v.x << 16); gv[1] = __uint_as_float(v.x & 0xffff0000u);
+            gv[2] = __uint_as_float(v.y << 16); gv[3] = __uint_as_float(v.y & 0xffff0000u);
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) gv[j] = (ow0 + j < OW) ? to_f32(p[j]) : 0.0f;
+    }
+}
+// Loads the 4 winner codes of a quad as one word (VEC: one aligned 32-bit load).
+template <bool VEC>
+__device__ __forceinline__ unsigned load_c4(const uint8_t* p, int ow0, int OW) {
+    if constexpr (VEC) {
+        return __ldg(reinterpret_cast<const unsigned*>(p));
+    } else {
+        unsigned cw = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (ow0 + j < OW) cw |= (unsigned)p[j] << (8 * j);
+        return cw;
+    }
+}
+
 // BR: 0 = both branches (compound / parallel), 1 = min branch only, 2 = max branch only.
-template <typename T, int BR>
+// CB channels per CTA (the CTA's last channel block may hold fewer: those lanes idle).
+// VEC: OW is a multiple of 4 (aligned vector loads of grad_y and of the codes).
+template <typename T, int BR, int CB, bool VEC>
 __global__ void __launch_bounds__(256)
 bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
@@ -148,8 +181,8 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     extern __shared__ float A[];  // [CB][RS][4][NQpad], then alpha / beta of this CTA's channels [K][CB] each
     const int tile_i = blockIdx.x % pl.tiles_per_img;
     const int n = blockIdx.x / pl.tiles_per_img;
-    const int c0 = blockIdx.y * pl.CB;
-    const int ncb = min(pl.CB, g.C - c0);
+    const int c0 = blockIdx.y * CB;
+    const int ncb = min(CB, g.C - c0);
     const int ih0 = tile_i * pl.THI;
     const int rows = min(pl.THI, g.H - ih0);
     const int num = ih0 + g.ph - (g.R - 1) * g.dh;
@@ -158,89 +191,76 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     const int NR = oh_hi - oh_lo + 1;
     const int NQ = NR * pl.QPR;
     const int NQp = pl.NQpad;
-    const int nacc = pl.CB * g.RS * 4 * NQp;
+    const int nacc = CB * g.RS * 4 * NQp;
     float* a_s = A + nacc;
-    float* b_s = a_s + g.K * pl.CB;
+    float* b_s = a_s + g.K * CB;
     for (int e = threadIdx.x; e < nacc; e += blockDim.x) A[e] = 0.0f;
     if constexpr (BR == 0) {
-        for (int e = threadIdx.x; e < g.K * pl.CB; e += blockDim.x) {
-            const int k = e / pl.CB, cb = e - k * pl.CB;
+        for (int e = threadIdx.x; e < g.K * CB; e += blockDim.x) {
+            const int k = e / CB, cb = e - k * CB;
             const bool ok = cb < ncb;
-            a_s[e] = (ok && alpha) ? alpha[(size_t)k * g.C + c0 + cb] : 1.0f;
-            b_s[e] = (ok && beta) ? beta[(size_t)k * g.C + c0 + cb] : 1.0f;
+            a_s[e] = (ok && alpha) ? alpha[(size_t)k * g.C + c0 + cb] : (ok ? 1.0f : 0.0f);
+            b_s[e] = (ok && beta) ? beta[(size_t)k * g.C + c0 + cb] : (ok ? 1.0f : 0.0f);
         }
     }
     __syncthreads();
     const size_t plane = (size_t)g.OH * g.OW;
-    const bool vec = (g.OW & 3) == 0;
+    const size_t cstep = (size_t)g.C * plane;        // codes: one output channel k further
+    const unsigned tstride = 4u * NQp * sizeof(float); // bytes between the accumulators of two taps
     for (int q = threadIdx.x; q < NQ; q += blockDim.x) {
         const int orow = q / pl.QPR;
         const int ow0 = (q - orow * pl.QPR) * 4;
         const size_t pix = (size_t)(oh_lo + orow) * g.OW + ow0;
-        float* Aq = A + q;
-        // operands of output channel k: 4 gradients and the code words of the CTA's channels;
-        // the loads of k+1 are issued before the accumulators of k are updated
-        auto load_k = [&](int k, float* gv, unsigned* cw) {
-            const size_t ob = ((size_t)n * g.K + k) * plane + pix;
-            if (vec) {
-                if constexpr (sizeof(T) == 4) {
-                    const float4 v = __ldg(reinterpret_cast<const float4*>(gy + ob));
-                    gv[0] = v.x; gv[1] = v.y; gv[2] = v.z; gv[3] = v.w;
-                } else {
-                    const uint2 v = __ldg(reinterpret_cast<const uint2*>(gy + ob));
-                    gv[0] = __uint_as_float(v.x << 16); gv[1] = __uint_as_float(v.x & 0xffff0000u);
-                    gv[2] = __uint_as_float(v.y << 16); gv[3] = __uint_as_float(v.y & 0xffff0000u);
-                }
-            } else {
+        const T* gp = gy + (size_t)n * g.K * plane + pix;
+        // a channel past C reads channel C-1 again; its alpha = beta = 0 (or it is skipped below)
+        const uint8_t* cp[CB];
+        char* Ab[CB];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) gv[j] = (ow0 + j < g.OW) ? to_f32(gy[ob + j]) : 0.0f;
-            }
-#pragma unroll
-            for (int cb = 0; cb < kGxCB; ++cb) {
-                cw[cb] = 0;
-                if (cb < ncb) {
-                    const size_t cbase = (((size_t)n * g.K + k) * g.C + c0 + cb) * plane + pix;
-                    if (vec) {
-                        cw[cb] = __ldg(reinterpret_cast<const unsigned*>(codes + cbase));
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            if (ow0 + j < g.OW) cw[cb] |= (unsigned)codes[cbase + j] << (8 * j);
-                    }
-                }
-            }
-        };
+        for (int cb = 0; cb < CB; ++cb) {
+            const int c = min(c0 + cb, g.C - 1);
+            cp[cb] = codes + ((size_t)n * g.K * g.C + c) * plane + pix;
+            Ab[cb] = reinterpret_cast<char*>(A + (size_t)cb * g.RS * 4 * NQp + q);
+        }
         float gv_cur[4], gv_nxt[4];
-        unsigned cw_cur[kGxCB], cw_nxt[kGxCB];
-        load_k(0, gv_cur, cw_cur);
-        for (int k = 0; k < g.K; ++k) {
-            if (k + 1 < g.K) load_k(k + 1, gv_nxt, cw_nxt);
+        unsigned cw_cur[CB], cw_nxt[CB];
+        load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
 #pragma unroll
-            for (int cb = 0; cb < kGxCB; ++cb) {
-                if (cb >= ncb) break;
+        for (int cb = 0; cb < CB; ++cb) cw_cur[cb] = load_c4<VEC>(cp[cb], ow0, g.OW);
+        for (int k = 0; k < g.K; ++k) {
+            if (k + 1 < g.K) {
+                gp += plane;
+                load_g4<T, VEC>(gp, ow0, g.OW, gv_nxt);
+#pragma unroll
+                for (int cb = 0; cb < CB; ++cb) {
+                    cp[cb] += cstep;
+                    cw_nxt[cb] = load_c4<VEC>(cp[cb], ow0, g.OW);
+                }
+            }
+#pragma unroll
+            for (int cb = 0; cb < CB; ++cb) {
+                if (BR != 0 && cb >= ncb) continue;   // single-branch layers have no zero coefficient to hide behind
                 float a = 1.0f, b = 1.0f;
                 if constexpr (BR == 0) {
-                    a = a_s[k * pl.CB + cb];
-                    b = b_s[k * pl.CB + cb];
+                    a = a_s[k * CB + cb];
+                    b = b_s[k * CB + cb];
                 }
-                float* Ac = Aq + (size_t)cb * g.RS * 4 * NQp;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const unsigned code = (cw_cur[cb] >> (8 * j)) & 0xffu;
                     if constexpr (BR == 0 || BR == 1) {
-                        const int t = code & 15u;
-                        Ac[(t * 4 + j) * NQp] += (BR == 0 ? a * gv_cur[j] : gv_cur[j]);
+                        float* dst = reinterpret_cast<float*>(Ab[cb] + (code & 15u) * tstride + j * NQp * sizeof(float));
+                        *dst = (BR == 0) ? __fmaf_rn(a, gv_cur[j], *dst) : (*dst + gv_cur[j]);
                     }
                     if constexpr (BR == 0 || BR == 2) {
-                        const int t = code >> 4;
-                        Ac[(t * 4 + j) * NQp] += (BR == 0 ? b * gv_cur[j] : gv_cur[j]);
+                        float* dst = reinterpret_cast<float*>(Ab[cb] + (code >> 4) * tstride + j * NQp * sizeof(float));
+                        *dst = (BR == 0) ? __fmaf_rn(b, gv_cur[j], *dst) : (*dst + gv_cur[j]);
                     }
                 }
             }
 #pragma unroll
             for (int j = 0; j < 4; ++j) gv_cur[j] = gv_nxt[j];
 #pragma unroll
-            for (int cb = 0; cb < kGxCB; ++cb) cw_cur[cb] = cw_nxt[cb];
+            for (int cb = 0; cb < CB; ++cb) cw_cur[cb] = cw_nxt[cb];
         }
     }
     __syncthreads();
@@ -295,111 +315,109 @@ __global__ void pad_input_kernel(Geo g, const T* __restrict__ x, T* __restrict__
     xpad[i] = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? x[(nc * g.H + ih) * g.W + iw] : zero_of<T>();
 }
 
-template <typename T, int BR, bool XS>
+template <typename T, int BR, bool XS, bool VEC>
 __global__ void __launch_bounds__(256)
 bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
                    const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes,
                    float* __restrict__ gw, float* __restrict__ gw2, float* __restrict__ galpha,
                    float* __restrict__ gbeta, CodeGwPlan pl) {
-    extern __shared__ float S[];  // [2*RS + 2][256] private columns | tap tables | weights | x planes
+    extern __shared__ float S[];  // [2*RS + 2][256] private columns | per-tap tables
     const int c = blockIdx.x % g.C;
     const int k = blockIdx.x / g.C;
     const int tid = threadIdx.x;
     const int NB = 2 * g.RS + 2;
-    float* col = S + tid;
+    char* colb = reinterpret_cast<char*>(S + tid);
     int* tap_dh = reinterpret_cast<int*>(S + NB * 256);
     int* tap_dw = tap_dh + g.RS;
-    int* tap_off = tap_dw + g.RS;
-    float* wmin_s = reinterpret_cast<float*>(tap_off + g.RS);
-    float* wmax_s = wmin_s + g.RS;
-    for (int b = 0; b < NB; ++b) col[b * 256] = 0.0f;
+    // {offset of the tap inside the padded plane, weight of the tap}: min branch, max branch
+    int2* tapw_min = reinterpret_cast<int2*>(tap_dw + g.RS + ((g.RS & 1) ? 0 : 0) + (((2 * g.RS) & 1) ? 1 : 0));
+    int2* tapw_max = tapw_min + g.RS;
+    for (int b = 0; b < NB; ++b) S[b * 256 + tid] = 0.0f;
     if (tid < g.RS) {
         const int r = tid / g.S, sx = tid % g.S;
         tap_dh[tid] = r * g.dh - g.ph;
         tap_dw[tid] = sx * g.dw - g.pw;
-        tap_off[tid] = r * g.dh * pl.WP + sx * g.dw;
         const size_t wi = ((size_t)k * g.C + c) * g.RS + tid;
-        wmin_s[tid] = to_f32(w[wi]);
-        wmax_s[tid] = to_f32((g.mode == TCONV_PARALLEL ? w2 : w)[wi]);
+        const int off = r * g.dh * pl.WP + sx * g.dw;
+        tapw_min[tid] = make_int2(off, __float_as_int(to_f32(w[wi])));
+        tapw_max[tid] = make_int2(off, __float_as_int(to_f32((g.mode == TCONV_PARALLEL ? w2 : w)[wi])));
     }
+    __syncthreads();
     const bool need_ab = (BR == 0) && (galpha || gbeta);
     const int QPR = (g.OW + 3) >> 2;
     const int NQ = g.OH * QPR;
     const size_t plane = (size_t)g.OH * g.OW;
-    const bool vec = (g.OW & 3) == 0;
+    const size_t gstep = (size_t)g.K * plane;            // grad_y: one image further
+    const size_t cstep = (size_t)g.K * g.C * plane;      // codes: one image further
+    const size_t xstep = (size_t)g.C * pl.xs_elems;      // padded x: one image further
     float sa = 0.0f, sb = 0.0f;
-
-    __syncthreads();
-    for (int n = 0; n < g.N; ++n) {
-        const T* xc = x + ((size_t)n * g.C + c) * g.H * g.W;
-        const T* xsn = reinterpret_cast<const T*>(pl.xpad) + ((size_t)n * g.C + c) * pl.xs_elems;
-        const size_t obase = ((size_t)n * g.K + k) * plane;
-        const size_t cbase = (((size_t)n * g.K + k) * g.C + c) * plane;
-        for (int q = tid; q < NQ; q += 256) {
-            const int oh = q / QPR;
-            const int ow0 = (q - oh * QPR) * 4;
-            const size_t pix = (size_t)oh * g.OW + ow0;
-            float gv[4];
-            unsigned cw;
-            if (vec) {
-                cw = __ldg(reinterpret_cast<const unsigned*>(codes + cbase + pix));
-                if constexpr (sizeof(T) == 4) {
-                    const float4 v = __ldg(reinterpret_cast<const float4*>(gy + obase + pix));
-                    gv[0] = v.x; gv[1] = v.y; gv[2] = v.z; gv[3] = v.w;
-                } else {
-                    const uint2 v = __ldg(reinterpret_cast<const uint2*>(gy + obase + pix));
-                    gv[0] = __uint_as_float(v.x << 16); gv[1] = __uint_as_float(v.x & 0xffff0000u);
-                    gv[2] = __uint_as_float(v.y << 16); gv[3] = __uint_as_float(v.y & 0xffff0000u);
-                }
-            } else {
-                cw = 0;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const bool ok = ow0 + j < g.OW;
-                    gv[j] = ok ? to_f32(gy[obase + pix + j]) : 0.0f;
-                    if (ok) cw |= (unsigned)codes[cbase + pix + j] << (8 * j);
-                }
+    for (int q = tid; q < NQ; q += 256) {
+        const int oh = q / QPR;
+        const int ow0 = (q - oh * QPR) * 4;
+        const size_t pix = (size_t)oh * g.OW + ow0;
+        const T* gp = gy + (size_t)k * plane + pix;
+        const uint8_t* cp = codes + ((size_t)k * g.C + c) * plane + pix;
+        const T* xp = XS ? reinterpret_cast<const T*>(pl.xpad) + (size_t)c * pl.xs_elems +
+                               (size_t)oh * g.sh * pl.WP + ow0 * g.sw
+                         : x + (size_t)c * g.H * g.W;
+        float gv_cur[4], gv_nxt[4];
+        unsigned cw_cur, cw_nxt = 0;
+        load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
+        cw_cur = load_c4<VEC>(cp, ow0, g.OW);
+        for (int n = 0; n < g.N; ++n) {
+            if (n + 1 < g.N) {
+                gp += gstep;
+                cp += cstep;
+                load_g4<T, VEC>(gp, ow0, g.OW, gv_nxt);
+                cw_nxt = load_c4<VEC>(cp, ow0, g.OW);
             }
-            const int xbase = oh * g.sh * pl.WP + ow0 * g.sw;   // staged-plane index of tap (0, 0) of pixel ow0
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                if (!vec && ow0 + j >= g.OW) continue;
-                const unsigned code = (cw >> (8 * j)) & 0xffu;
-                const int ow = ow0 + j;
+                if (!VEC && ow0 + j >= g.OW) continue;
+                const unsigned code = (cw_cur >> (8 * j)) & 0xffu;
+                const float gvj = gv_cur[j];
                 if constexpr (BR == 0 || BR == 1) {
-                    const int t = code & 15u;
-                    col[t * 256] += gv[j];
+                    const unsigned t = code & 15u;
+                    float* dst = reinterpret_cast<float*>(colb + t * 1024u);
+                    *dst += gvj;
                     if (need_ab) {
+                        const int2 tw = tapw_min[t];
                         T xv;
                         if constexpr (XS) {
-                            xv = xsn[xbase + j * g.sw + tap_off[t]];
+                            xv = xp[j * g.sw + tw.x];
                         } else {
-                            const int ih = oh * g.sh + tap_dh[t], iw = ow * g.sw + tap_dw[t];
-                            xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xc[(size_t)ih * g.W + iw] : zero_of<T>();
+                            const int ih = oh * g.sh + tap_dh[t], iw = (ow0 + j) * g.sw + tap_dw[t];
+                            xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xp[(size_t)ih * g.W + iw] : zero_of<T>();
                         }
-                        sa = __fmaf_rn(gv[j], tap_add(xv, from_f32<T>(wmin_s[t])), sa);
+                        sa = __fmaf_rn(gvj, tap_add(xv, from_f32<T>(__int_as_float(tw.y))), sa);
                     }
                 }
                 if constexpr (BR == 0 || BR == 2) {
-                    const int t = code >> 4;
-                    col[(g.RS + t) * 256] += gv[j];
+                    const unsigned t = code >> 4;
+                    float* dst = reinterpret_cast<float*>(colb + (g.RS + t) * 1024u);
+                    *dst += gvj;
                     if (need_ab) {
+                        const int2 tw = tapw_max[t];
                         T xv;
                         if constexpr (XS) {
-                            xv = xsn[xbase + j * g.sw + tap_off[t]];
+                            xv = xp[j * g.sw + tw.x];
                         } else {
-                            const int ih = oh * g.sh + tap_dh[t], iw = ow * g.sw + tap_dw[t];
-                            xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xc[(size_t)ih * g.W + iw] : zero_of<T>();
+                            const int ih = oh * g.sh + tap_dh[t], iw = (ow0 + j) * g.sw + tap_dw[t];
+                            xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xp[(size_t)ih * g.W + iw] : zero_of<T>();
                         }
-                        sb = __fmaf_rn(gv[j], tap_add(xv, from_f32<T>(wmax_s[t])), sb);
+                        sb = __fmaf_rn(gvj, tap_add(xv, from_f32<T>(__int_as_float(tw.y))), sb);
                     }
                 }
             }
+            xp += XS ? xstep : (size_t)g.C * g.H * g.W;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) gv_cur[j] = gv_nxt[j];
+            cw_cur = cw_nxt;
         }
     }
-    col[(2 * g.RS) * 256] = sa;
-    col[(2 * g.RS + 1) * 256] = sb;
+    S[(2 * g.RS) * 256 + tid] = sa;
+    S[(2 * g.RS + 1) * 256 + tid] = sb;
     __syncthreads();
     // fixed tree over the 256 columns of every bin
     for (int step = 128; step > 0; step >>= 1) {
@@ -448,7 +466,7 @@ bwd_bias_partial_kernel(Geo g, const T* __restrict__ gy, float* __restrict__ par
 
 // ---------------------------------------------------------------------------------- host side
 inline void plan_code_gw(const Geo& g, CodeGwPlan* pl) {
-    pl->smem = ((size_t)(2 * g.RS + 2) * 256 + 5 * (size_t)g.RS + 4) * sizeof(float);
+    pl->smem = ((size_t)(2 * g.RS + 2) * 256 + 6 * (size_t)g.RS + 4) * sizeof(float);
     pl->HP = (g.OH - 1) * g.sh + (g.R - 1) * g.dh + 1;
     pl->WP = (g.OW - 1) * g.sw + (g.S - 1) * g.dw + 1;
     if (pl->HP < g.H + g.ph) pl->HP = g.H + g.ph;   // rows / columns no output reaches still hold x
@@ -527,7 +545,7 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
         pl->tiles_per_img = (g.H + thi - 1) / thi;
         pl->NRmax = (int)nr;
         pl->NQpad = (int)(((long)nr * pl->QPR + 31) / 32 * 32);
-        pl->smem = ((size_t)cb * g.RS * 4 * pl->NQpad + 2 * (size_t)g.K * cb) * sizeof(float);
+        pl->smem = ((size_t)cb * g.RS * 4 * pl->NQpad + 2 * (size_t)g.K * kGxCB) * sizeof(float);
         if (pl->smem > kBwdSmemLimit + 16 * 1024) continue;
         return true;
     }
