@@ -265,29 +265,37 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     }
     __syncthreads();
     // gather: every owned input element sums, over the taps, the accumulator of the output
-    // pixel that reads it through that tap
-    const int per_c = rows * g.W;
-    for (int e = threadIdx.x; e < ncb * per_c; e += blockDim.x) {
-        const int cb = e / per_c;
-        const int rem = e - cb * per_c;
-        const int ih = ih0 + rem / g.W, iw = rem % g.W;
+    // pixel that reads it through that tap (one warp per input row, lanes along the columns)
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool unit_stride = (g.sh == 1 && g.sw == 1);
+    for (int cb = 0; cb < ncb; ++cb) {
         const float* Ac = A + (size_t)cb * g.RS * 4 * NQp;
-        float s = 0.0f;
-        for (int r = 0; r < g.R; ++r) {
-            const int nh = ih + g.ph - r * g.dh;
-            if (nh < 0 || nh % g.sh != 0) continue;
-            const int oh = nh / g.sh;
-            if (oh < oh_lo || oh > oh_hi) continue;
-            for (int sx = 0; sx < g.S; ++sx) {
-                const int nw = iw + g.pw - sx * g.dw;
-                if (nw < 0 || nw % g.sw != 0) continue;
-                const int ow = nw / g.sw;
-                if (ow >= g.OW) continue;
-                const int q = (oh - oh_lo) * pl.QPR + (ow >> 2);
-                s += Ac[((r * g.S + sx) * 4 + (ow & 3)) * NQp + q];
+        T* gxc = gx + ((size_t)n * g.C + c0 + cb) * g.H * g.W;
+        for (int row = warp; row < rows; row += 8) {
+            const int ih = ih0 + row;
+            for (int iw = lane; iw < g.W; iw += 32) {
+                float s = 0.0f;
+                for (int r = 0; r < g.R; ++r) {
+                    int oh = ih + g.ph - r * g.dh;
+                    if (!unit_stride) {
+                        if (oh < 0 || oh % g.sh != 0) continue;
+                        oh /= g.sh;
+                    }
+                    if (oh < oh_lo || oh > oh_hi) continue;
+                    const float* Ar = Ac + (oh - oh_lo) * pl.QPR;
+                    for (int sx = 0; sx < g.S; ++sx) {
+                        int ow = iw + g.pw - sx * g.dw;
+                        if (!unit_stride) {
+                            if (ow < 0 || ow % g.sw != 0) continue;
+                            ow /= g.sw;
+                        }
+                        if (ow < 0 || ow >= g.OW) continue;
+                        s += Ar[((r * g.S + sx) * 4 + (ow & 3)) * NQp + (ow >> 2)];
+                    }
+                }
+                gxc[(size_t)ih * g.W + iw] = from_f32<T>(s);
             }
         }
-        gx[((size_t)n * g.C + c0 + cb) * g.H * g.W + (size_t)ih * g.W + iw] = from_f32<T>(s);
     }
 }
 
