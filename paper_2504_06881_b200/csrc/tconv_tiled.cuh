@@ -38,6 +38,15 @@ __device__ __forceinline__ void add2(float x, float wlo, float whi, float& lo, f
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(tt) : "l"(xx), "l"(ww));
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
 }
+// {c0, c1} = a * {v0, v1} + {c0, c1}: one packed fused multiply-add (scalar a splat)
+__device__ __forceinline__ void fma2s(float a, float v0, float v1, float& c0, float& c1) {
+    unsigned long long aa, vv, cc;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(aa) : "f"(a));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(vv) : "f"(v0), "f"(v1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(cc) : "f"(c0), "f"(c1));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(cc) : "l"(aa), "l"(vv));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(c0), "=f"(c1) : "l"(cc));
+}
 __device__ __forceinline__ unsigned smem_u32(const void* p) {
     return (unsigned)__cvta_generic_to_shared(p);
 }
@@ -105,6 +114,15 @@ __device__ __forceinline__ void load_segment(const float* base, float* out) {
             out[I] = base[pos];
             load_segment<SHIFT, L, I + 1>(base, out);
         }
+    }
+}
+template <int N>
+__device__ __forceinline__ void loadn(const float* p, float* out) {
+    static_assert(N % 4 == 0, "vector loads");
+#pragma unroll
+    for (int i = 0; i < N; i += 4) {
+        const float4 a = *reinterpret_cast<const float4*>(p + i);
+        out[i] = a.x; out[i + 1] = a.y; out[i + 2] = a.z; out[i + 3] = a.w;
     }
 }
 __device__ __forceinline__ void load8(const float* p, float* out) {
@@ -191,12 +209,14 @@ template <int S, int DW, int ESIZE = 4> struct TmaShift {
 #ifndef TCONV_Q_CARRIED
 #define TCONV_Q_CARRIED 2
 #endif
-template <int MODE, int CHAN, bool WIN, bool XTMA, int R, int S, int SW, int DW, int Q, int KG, int PW>
+template <int MODE, int CHAN, bool WIN, bool XTMA, int R, int S, int SW, int DW, int Q, int KG, int PW, int TK>
 __global__ void __launch_bounds__(KG * PW * 32,
-                                  (WIN || MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL) ? 1 : TCONV_MINB_SINGLE)
+                                  (WIN && CHAN == CH_SUM) ? 3
+                                  : (WIN || MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL) ? 1 : TCONV_MINB_SINGLE)
 fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams p) {
+    static_assert(TK == 4 || TK == 8, "output channels per thread");
     constexpr int RS = R * S;
-    constexpr int TILE_K = KG * 8;
+    constexpr int TILE_K = KG * TK;
     constexpr int NT = KG * PW * 32;
     constexpr int NWARPS = KG * PW;
     constexpr int L = 3 * SW + (S - 1) * DW + 1;  // input columns one quad touches per row
@@ -335,10 +355,10 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
     };
 
     // accumulators
-    float acc[8][Q][4];   // Sum forms: running sum; Max/Min combine: running best
-    int cbest[WIN && CHAN != CH_SUM ? 8 : 1][Q][4];
+    float acc[TK][Q][4];   // Sum forms: running sum; Max/Min combine: running best
+    int cbest[WIN && CHAN != CH_SUM ? TK : 1][Q][4];
 #pragma unroll
-    for (int k = 0; k < 8; ++k)
+    for (int k = 0; k < TK; ++k)
 #pragma unroll
         for (int q = 0; q < Q; ++q)
 #pragma unroll
@@ -368,10 +388,10 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
             if (ch + 1 < p.nchunks) cp_async_wait<1>(); else cp_async_wait<0>();
             __syncthreads();
         }
-        const float* ws = st + w_off + kg * 8;
-        const float* ws2 = st + w2_off + kg * 8;
-        const float* as = st + a_off + kg * 8;
-        const float* bs = st + b_off + kg * 8;
+        const float* ws = st + w_off + kg * TK;
+        const float* ws2 = st + w2_off + kg * TK;
+        const float* as = st + a_off + kg * TK;
+        const float* bs = st + b_off + kg * TK;
         const int nc = min(p.CC, g.C - ch * p.CC);
         for (int cc = 0; cc < nc; ++cc) {
             // the R rows of input this thread's quads touch in channel cc
@@ -384,46 +404,10 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
             const float* wc = ws + cc * (RS * TILE_K);
             const float* wc2 = ws2 + cc * (RS * TILE_K);
 
-            float mx[CARRIED ? 1 : 8][Q][4];           // per-channel extremum (max branch / single branch)
-            float mn[TWO ? 8 : 1][Q][4];               // per-channel minimum (two-branch modes)
-            int amx[WIN && CHAN == CH_SUM ? 8 : 1][Q][4], amn[WIN && TWO ? 8 : 1][Q][4];
+            float mx[CARRIED ? 1 : TK][Q][4];           // per-channel extremum (max branch / single branch)
+            float mn[TWO ? TK : 1][Q][4];               // per-channel minimum (two-branch modes)
 
-            if constexpr (WIN && CHAN == CH_SUM) {
-                // winner codes per (output, channel): every tap is compared on its own
-#pragma unroll
-                for (int tap = 0; tap < RS; ++tap) {
-                    const int r = tap / S, sx = tap % S;
-                    float wv[8], wv2[8];
-                    load8(wc + tap * TILE_K, wv);
-                    if constexpr (PAR) load8(wc2 + tap * TILE_K, wv2);
-#pragma unroll
-                    for (int q = 0; q < Q; ++q)
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float xv = xr[q][r][j * SW + sx * DW];
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                const float t = __fadd_rn(xv, wv[k]);
-                                const float t2 = PAR ? __fadd_rn(xv, wv2[k]) : t;
-                                if constexpr (TWO) {
-                                    if (tap == 0) {
-                                        mn[k][q][j] = t; amn[k][q][j] = 0;
-                                        mx[k][q][j] = t2; amx[k][q][j] = 0;
-                                    } else {
-                                        if (t < mn[k][q][j]) { mn[k][q][j] = t; amn[k][q][j] = tap; }
-                                        if (t2 > mx[k][q][j]) { mx[k][q][j] = t2; amx[k][q][j] = tap; }
-                                    }
-                                } else {
-                                    if (tap == 0) {
-                                        mx[k][q][j] = t; amx[k][q][j] = 0;
-                                    } else if (TAP_MIN ? (t < mx[k][q][j]) : (t > mx[k][q][j])) {
-                                        mx[k][q][j] = t; amx[k][q][j] = tap;
-                                    }
-                                }
-                            }
-                        }
-                }
-            } else {
+            {
                 // taps folded in groups: a fresh chain opens with 3 taps, later groups take 2
                 constexpr int FIRST = CARRIED ? 2 : (RS >= 3 ? 3 : RS);
                 constexpr int NG = 1 + (RS - FIRST + 1) / 2;
@@ -431,12 +415,12 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                 for (int gi = 0; gi < NG; ++gi) {
                     const int t0 = (gi == 0) ? 0 : FIRST + 2 * (gi - 1);
                     const int nt = (gi == 0) ? (FIRST < RS ? FIRST : RS) : ((RS - t0) < 2 ? (RS - t0) : 2);
-                    float wv[3][8], wv2[PAR ? 3 : 1][8];
+                    float wv[3][TK], wv2[PAR ? 3 : 1][TK];
 #pragma unroll
                     for (int u = 0; u < 3; ++u)
                         if (u < nt) {
-                            load8(wc + (t0 + u) * TILE_K, wv[u]);
-                            if constexpr (PAR) load8(wc2 + (t0 + u) * TILE_K, wv2[u]);
+                            loadn<TK>(wc + (t0 + u) * TILE_K, wv[u]);
+                            if constexpr (PAR) loadn<TK>(wc2 + (t0 + u) * TILE_K, wv2[u]);
                         }
 #pragma unroll
                     for (int q = 0; q < Q; ++q)
@@ -450,7 +434,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                                     xv[u] = xr[q][tap / S][j * SW + (tap % S) * DW];
                                 }
 #pragma unroll
-                            for (int kp = 0; kp < 4; ++kp) {
+                            for (int kp = 0; kp < TK / 2; ++kp) {
                                 float ta[3][2], tb[3][2];
 #pragma unroll
                                 for (int u = 0; u < 3; ++u)
@@ -496,14 +480,14 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
 
             // channel combine
             if constexpr (!CARRIED) {
-                float av[8], bv[8];
+                float av[TK], bv[TK];
                 if constexpr (TWO) {
-                    load8(as + cc * TILE_K, av);
-                    load8(bs + cc * TILE_K, bv);
+                    loadn<TK>(as + cc * TILE_K, av);
+                    loadn<TK>(bs + cc * TILE_K, bv);
                 }
                 const int c = ch * p.CC + cc;
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
+                for (int k = 0; k < TK; ++k)
 #pragma unroll
                     for (int q = 0; q < Q; ++q)
 #pragma unroll
@@ -522,6 +506,96 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                             }
                         }
                 if constexpr (WIN && CHAN == CH_SUM) {
+                    // Winning taps, recovered on the FMA pipe.  With m the exact extremum of the
+                    // channel, d = (t - m) * 2^30 is computed with one rounding and is zero exactly for
+                    // the taps that attain m; key = |d| * (-2^125) + (RS - tap) is RS - tap for those
+                    // taps and hugely negative otherwise, so the maximum key belongs to the lowest
+                    // winning tap.  The sums t are the same rounded adds as in the first pass; the
+                    // extrema have been folded into acc above and are rescaled in place.
+                    // (|x + w| < 2^97 is assumed.)
+                    constexpr float kS = 1073741824.0f;                 // 2^30
+                    constexpr float kH = 4.253529586511731e37f;         // 2^125
+                    float kmn[TWO ? TK : 1][Q][4], kmx[TK][Q][4];
+#pragma unroll
+                    for (int k = 0; k < TK; ++k)
+#pragma unroll
+                        for (int q = 0; q < Q; ++q)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                mx[k][q][j] = -mx[k][q][j] * kS;
+                                if constexpr (TWO) mn[k][q][j] = -mn[k][q][j] * kS;
+                            }
+                    constexpr int FIRST2 = (RS >= 3 ? 3 : RS);
+                    constexpr int NG2 = 1 + (RS - FIRST2 + 1) / 2;
+#pragma unroll
+                    for (int gi = 0; gi < NG2; ++gi) {
+                        const int t0 = (gi == 0) ? 0 : FIRST2 + 2 * (gi - 1);
+                        const int nt = (gi == 0) ? (FIRST2 < RS ? FIRST2 : RS) : ((RS - t0) < 2 ? (RS - t0) : 2);
+                        float wv[3][TK], wv2[PAR ? 3 : 1][TK];
+#pragma unroll
+                        for (int u = 0; u < 3; ++u)
+                            if (u < nt) {
+                                loadn<TK>(wc + (t0 + u) * TILE_K, wv[u]);
+                                if constexpr (PAR) loadn<TK>(wc2 + (t0 + u) * TILE_K, wv2[u]);
+                            }
+#pragma unroll
+                        for (int q = 0; q < Q; ++q)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                float xv[3];
+#pragma unroll
+                                for (int u = 0; u < 3; ++u)
+                                    if (u < nt) {
+                                        const int tap = t0 + u;
+                                        xv[u] = xr[q][tap / S][j * SW + (tap % S) * DW];
+                                    }
+#pragma unroll
+                                for (int kp = 0; kp < TK / 2; ++kp) {
+                                    float ka[3][2], kb[3][2];   // keys of the min branch / max branch
+#pragma unroll
+                                    for (int u = 0; u < 3; ++u)
+                                        if (u < nt) {
+                                            const float rank = (float)(RS - (t0 + u));
+                                            float ta0, ta1, tb0, tb1;
+                                            add2(xv[u], wv[u][2 * kp], wv[u][2 * kp + 1], ta0, ta1);
+                                            if constexpr (PAR) add2(xv[u], wv2[u][2 * kp], wv2[u][2 * kp + 1], tb0, tb1);
+                                            else { tb0 = ta0; tb1 = ta1; }
+                                            if constexpr (TWO) {
+                                                float d0 = mn[2 * kp][q][j], d1 = mn[2 * kp + 1][q][j];
+                                                fma2s(kS, ta0, ta1, d0, d1);            // >= 0
+                                                ka[u][0] = rank; ka[u][1] = rank;
+                                                fma2s(-kH, d0, d1, ka[u][0], ka[u][1]);
+                                                float e0 = mx[2 * kp][q][j], e1 = mx[2 * kp + 1][q][j];
+                                                fma2s(kS, tb0, tb1, e0, e1);            // <= 0
+                                                kb[u][0] = rank; kb[u][1] = rank;
+                                                fma2s(kH, e0, e1, kb[u][0], kb[u][1]);
+                                            } else {
+                                                float e0 = mx[2 * kp][q][j], e1 = mx[2 * kp + 1][q][j];
+                                                fma2s(kS, ta0, ta1, e0, e1);
+                                                kb[u][0] = rank; kb[u][1] = rank;
+                                                fma2s(TAP_MIN ? -kH : kH, e0, e1, kb[u][0], kb[u][1]);
+                                            }
+                                        }
+#pragma unroll
+                                    for (int h = 0; h < 2; ++h) {
+                                        const int k = 2 * kp + h;
+                                        if (gi == 0) {
+                                            kmx[k][q][j] = nt == 3 ? ext3(kb[0][h], kb[1][h], kb[2][h], false)
+                                                           : nt == 2 ? ext2(kb[0][h], kb[1][h], false) : kb[0][h];
+                                            if constexpr (TWO)
+                                                kmn[k][q][j] = nt == 3 ? ext3(ka[0][h], ka[1][h], ka[2][h], false)
+                                                               : nt == 2 ? ext2(ka[0][h], ka[1][h], false) : ka[0][h];
+                                        } else {
+                                            kmx[k][q][j] = nt == 2 ? ext3(kmx[k][q][j], kb[0][h], kb[1][h], false)
+                                                                   : ext2(kmx[k][q][j], kb[0][h], false);
+                                            if constexpr (TWO)
+                                                kmn[k][q][j] = nt == 2 ? ext3(kmn[k][q][j], ka[0][h], ka[1][h], false)
+                                                                       : ext2(kmn[k][q][j], ka[0][h], false);
+                                        }
+                                    }
+                                }
+                            }
+                    }
                     // one byte per (n, k, c, oh, ow): low nibble argmin tap, high nibble argmax tap
                     uint8_t* codes = reinterpret_cast<uint8_t*>(p.winners);
 #pragma unroll
@@ -529,17 +603,18 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                         if (out_row[q] < 0) continue;
                         const int n = out_row[q] / g.OH, oh = out_row[q] - n * g.OH;
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const int kk = kt * TILE_K + kg * 8 + k;
+                        for (int k = 0; k < TK; ++k) {
+                            const int kk = kt * TILE_K + kg * TK + k;
                             if (kk >= g.K) continue;
                             uint8_t* dst = codes + (((size_t)n * g.K + kk) * g.C + c) * plane +
                                            (size_t)oh * g.OW + qcol[q];
                             unsigned packed = 0;
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
+                                const unsigned tmax = (unsigned)(RS - __float2int_rn(kmx[k][q][j]));
                                 unsigned code;
-                                if constexpr (TWO) code = amn[k][q][j] | (amx[k][q][j] << 4);
-                                else code = TAP_MIN ? amx[k][q][j] : (amx[k][q][j] << 4);
+                                if constexpr (TWO) code = (unsigned)(RS - __float2int_rn(kmn[k][q][j])) | (tmax << 4);
+                                else code = TAP_MIN ? tmax : (tmax << 4);
                                 packed |= code << (8 * j);
                             }
                             if (qcol[q] + 3 < g.OW && ((g.OW & 3) == 0)) {
@@ -564,8 +639,8 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
         if (out_row[q] < 0) continue;
         const int n = out_row[q] / g.OH, oh = out_row[q] - n * g.OH;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int kk = kt * TILE_K + kg * 8 + k;
+        for (int k = 0; k < TK; ++k) {
+            const int kk = kt * TILE_K + kg * TK + k;
             if (kk >= g.K) continue;
             const float bk = p.bias ? p.bias[kk] : 0.0f;
             const size_t o = ((size_t)n * g.K + kk) * plane + (size_t)oh * g.OW + qcol[q];
@@ -591,7 +666,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                     if (ow >= g.OW) continue;
                     const int c = cbest[k][q][j];
                     const float* xc = xg + ((size_t)n * g.C + c) * chw;
-                    const float* wk = wt_k + ((size_t)c * RS) * TILE_K + kg * 8 + k;
+                    const float* wk = wt_k + ((size_t)c * RS) * TILE_K + kg * TK + k;
                     int tapw = 0;
 #pragma unroll
                     for (int tap = RS - 1; tap >= 0; --tap) {
@@ -629,10 +704,10 @@ inline size_t tiled_ws_bytes(const Geo& g) {
 
 inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
 
-template <int R, int S, int SW, int DW, int Q, int KG, int PW>
+template <int R, int S, int SW, int DW, int Q, int KG, int PW, int TK = 8>
 inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* pl) {
     TiledParams& p = pl->p;
-    constexpr int TILE_K = KG * 8;
+    constexpr int TILE_K = KG * TK;
     constexpr int NQ = Q * 32 * PW;
     const int qpr_full = (g.OW + 3) / 4;
     // column tiles: at most NQ/4 quads wide (a tile keeps >= 4 rows unless the row is short), split evenly
@@ -740,14 +815,14 @@ struct FwdArgs {
     const char* name;  // out: kernel variant
 };
 
-template <typename T, int MODE, int CHAN, bool WIN, int R, int S, int SW, int DW, int Q, int KG, int PW>
+template <typename T, int MODE, int CHAN, bool WIN, int R, int S, int SW, int DW, int Q, int KG, int PW, int TK>
 int launch_tiled_variant(FwdArgs& a) {
     constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
     constexpr bool PAR = (MODE == TCONV_PARALLEL);
     const Geo& g = a.g;
     TiledPlan pl;
     pl.p.g = g;
-    if (!plan_tiles<R, S, SW, DW, Q, KG, PW>(g, PAR, TWO, (int)sizeof(T), &pl)) return TCONV_ERR_UNSUPPORTED;
+    if (!plan_tiles<R, S, SW, DW, Q, KG, PW, TK>(g, PAR, TWO, (int)sizeof(T), &pl)) return TCONV_ERR_UNSUPPORTED;
     const size_t need = pl.ws_w * (PAR ? 2 : 1) + (TWO ? 2 * pl.ws_ab : 0);
     if (!a.ws || a.ws_bytes < need) return TCONV_ERR_WORKSPACE_TOO_SMALL;
     float* wt = reinterpret_cast<float*>(a.ws);
@@ -764,13 +839,13 @@ int launch_tiled_variant(FwdArgs& a) {
     pl.p.x = a.x; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
     if (pl.xtma) {
-        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, true, R, S, SW, DW, Q, KG, PW>;
+        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, true, R, S, SW, DW, Q, KG, PW, TK>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
             return TCONV_ERR_CUDA;
         kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);
         a.name = WIN ? "fwd_tiled_f32_tma_win" : "fwd_tiled_f32_tma";
     } else {
-        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, false, R, S, SW, DW, Q, KG, PW>;
+        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, false, R, S, SW, DW, Q, KG, PW, TK>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
             return TCONV_ERR_CUDA;
         kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);
@@ -789,11 +864,13 @@ int launch_tiled_geom(FwdArgs& a) {
     constexpr bool CARRIED = !TWO && !WIN && ((MODE == TCONV_MAX_PLUS && CHAN == CH_MAX) ||
                                               (MODE == TCONV_MIN_PLUS && CHAN == CH_MIN));
     constexpr int Q = CARRIED ? TCONV_Q_CARRIED : 1;
+    // the winner pass of the Sum forms keeps two extra values per output: 4 channels per thread
+    constexpr int TK = (WIN && CHAN == CH_SUM) ? 4 : 8;
     const Geo& g = a.g;
     if (g.R == 3 && g.S == 3) {
-        if (g.sw == 1 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 1, Q, 4, 1>(a);
-        if (g.sw == 2 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 2, 1, Q, 4, 1>(a);
-        if (g.sw == 1 && g.dw == 2) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 2, Q, 4, 1>(a);
+        if (g.sw == 1 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 1, Q, 4, 1, TK>(a);
+        if (g.sw == 2 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 2, 1, Q, 4, 1, TK>(a);
+        if (g.sw == 1 && g.dw == 2) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 2, Q, 4, 1, TK>(a);
     }
     return TCONV_ERR_UNSUPPORTED;
 }
