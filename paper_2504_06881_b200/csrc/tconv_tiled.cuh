@@ -38,6 +38,15 @@ __device__ __forceinline__ void add2(float x, float wlo, float whi, float& lo, f
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(tt) : "l"(xx), "l"(ww));
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
 }
+// The same packed add, opaque to common-subexpression elimination: the winner pass recomputes
+// the tap sums instead of keeping all of them alive since the first pass.
+__device__ __forceinline__ void add2_again(float x, float wlo, float whi, float& lo, float& hi) {
+    unsigned long long xx, ww, tt;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(xx) : "f"(x));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ww) : "f"(wlo), "f"(whi));
+    asm volatile("add.rn.f32x2 %0, %1, %2;" : "=l"(tt) : "l"(xx), "l"(ww));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
+}
 // {c0, c1} = a * {v0, v1} + {c0, c1}: one packed fused multiply-add (scalar a splat)
 __device__ __forceinline__ void fma2s(float a, float v0, float v1, float& c0, float& c1) {
     unsigned long long aa, vv, cc;
@@ -557,8 +566,8 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                                         if (u < nt) {
                                             const float rank = (float)(RS - (t0 + u));
                                             float ta0, ta1, tb0, tb1;
-                                            add2(xv[u], wv[u][2 * kp], wv[u][2 * kp + 1], ta0, ta1);
-                                            if constexpr (PAR) add2(xv[u], wv2[u][2 * kp], wv2[u][2 * kp + 1], tb0, tb1);
+                                            add2_again(xv[u], wv[u][2 * kp], wv[u][2 * kp + 1], ta0, ta1);
+                                            if constexpr (PAR) add2_again(xv[u], wv2[u][2 * kp], wv2[u][2 * kp + 1], tb0, tb1);
                                             else { tb0 = ta0; tb1 = ta1; }
                                             if constexpr (TWO) {
                                                 float d0 = mn[2 * kp][q][j], d1 = mn[2 * kp + 1][q][j];
