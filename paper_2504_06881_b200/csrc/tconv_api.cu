@@ -166,12 +166,26 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
         size_t smem = 0;
         if (gx) {
             if (tiled && plan_idx_gx(g, &thi, &smem)) {
-                auto kern = bwd_idx_gx_kernel<T>;
-                if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess)
-                    return cuda_fail(cudaGetLastError());
                 const int tiles = (g.H + thi - 1) / thi;
                 const unsigned magic = g.RS == 1 ? 0u : (0xFFFFFFFFu / (unsigned)g.RS) + 1u;
-                kern<<<(unsigned)(g.N * tiles), 256, smem, st>>>(g, (const T*)gy, idx, (T*)gx, thi, tiles, magic);
+                if (g.RS <= 15) {
+                    // the phases of this form are latency-bound: aim at three resident CTAs per SM
+                    int thi2 = thi;
+                    while ((size_t)g.C * g.W * sizeof(float) * thi2 > 72 * 1024 &&
+                           (thi2 + 1) / 2 >= 2 * (g.R - 1) * g.dh && thi2 > 4)
+                        thi2 = (thi2 + 1) / 2;
+                    auto kern = bwd_idx_gx2_kernel<T>;
+                    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess)
+                        return cuda_fail(cudaGetLastError());
+                    const int tiles2 = (g.H + thi2 - 1) / thi2;
+                    kern<<<(unsigned)(g.N * tiles2), 256, (size_t)g.C * g.W * sizeof(float) * thi2, st>>>(
+                        g, (const T*)gy, idx, (T*)gx, thi2, tiles2, magic);
+                } else {
+                    auto kern = bwd_idx_gx_kernel<T>;
+                    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess)
+                        return cuda_fail(cudaGetLastError());
+                    kern<<<(unsigned)(g.N * tiles), 256, smem, st>>>(g, (const T*)gy, idx, (T*)gx, thi, tiles, magic);
+                }
                 name = "bwd_idx";
             } else {
                 const size_t total = (size_t)g.N * g.C * g.H * g.W;

@@ -72,6 +72,102 @@ bwd_idx_gx_kernel(Geo g, const T* __restrict__ gy, const int32_t* __restrict__ i
     }
 }
 
+// Second form of the same kernel for R*S <= 15: a thread reads the winners of its pixel once
+// (batches of independent loads) and keeps only their taps, 4 bits each, in registers (blocks of
+// 64 output channels).  In the phase of tap t it finds the channels whose winner is t with a few
+// bit operations and touches only those: it reloads their winner (for the input channel) and
+// their grad_y, the loads of the next match in flight while the current one is accumulated.
+template <typename T>
+__global__ void __launch_bounds__(256)
+bwd_idx_gx2_kernel(Geo g, const T* __restrict__ gy, const int32_t* __restrict__ idx,
+                   T* __restrict__ gx, int THI, int tiles_per_img, unsigned magic) {
+    extern __shared__ float tile[];  // [C][THI][W]
+    const int n = blockIdx.x / tiles_per_img;
+    const int ih0 = (blockIdx.x - n * tiles_per_img) * THI;
+    const int rows = min(THI, g.H - ih0);
+    const int cstride = THI * g.W;
+    for (int e = threadIdx.x; e < g.C * cstride; e += blockDim.x) tile[e] = 0.0f;
+    const int num = ih0 + g.ph - (g.R - 1) * g.dh;
+    const int oh_lo = num <= 0 ? 0 : (num + g.sh - 1) / g.sh;
+    const int oh_hi = min(g.OH - 1, (ih0 + rows - 1 + g.ph) / g.sh);
+    const int npix = (oh_hi - oh_lo + 1) * g.OW;
+    const size_t plane = (size_t)g.OH * g.OW;
+    const size_t img = (size_t)n * g.K * plane + (size_t)oh_lo * g.OW;   // first contributing pixel, k = 0
+    __syncthreads();
+    for (int pp0 = 0; pp0 < npix; pp0 += blockDim.x) {
+        const int pp = pp0 + threadIdx.x;
+        const bool live = pp < npix;
+        const int orow = live ? pp / g.OW : 0;
+        const int oh = oh_lo + orow, ow = live ? pp - orow * g.OW : 0;
+        for (int kb0 = 0; kb0 < g.K; kb0 += 64) {
+            const int kn = min(64, g.K - kb0);
+            const int32_t* ip = idx + img + (size_t)kb0 * plane + pp;
+            const T* gp = gy + img + (size_t)kb0 * plane + pp;
+            // taps of the 64 winners, 4 bits each; 15 marks "no channel here"
+            unsigned taps4[8];
+#pragma unroll
+            for (int wq = 0; wq < 8; ++wq) {
+                unsigned id[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    id[i] = (live && wq * 8 + i < kn) ? (unsigned)__ldg(ip + (size_t)(wq * 8 + i) * plane) : 0xffffffffu;
+                unsigned packed = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const unsigned c = magic ? __umulhi(id[i], magic) : id[i];
+                    const unsigned tap = (id[i] == 0xffffffffu) ? 15u : (id[i] - c * g.RS);
+                    packed |= tap << (4 * i);
+                }
+                taps4[wq] = packed;
+            }
+            for (int tap = 0; tap < g.RS; ++tap) {
+                const int r = tap / g.S, sx = tap - r * g.S;
+                const int ih = oh * g.sh - g.ph + r * g.dh;
+                const int iw = ow * g.sw - g.pw + sx * g.dw;
+                if (live && ih >= ih0 && ih < ih0 + rows && iw >= 0 && iw < g.W) {
+                    float* dst = tile + (ih - ih0) * g.W + iw;
+                    const unsigned pat = 0x11111111u * (unsigned)tap;
+                    // software pipeline over the matches: (id, gv) of the next one are loaded first
+                    bool have = false;
+                    unsigned id_cur = 0;
+                    float gv_cur = 0.0f;
+#pragma unroll
+                    for (int wq = 0; wq < 8; ++wq) {
+                        unsigned z = taps4[wq] ^ pat;       // nibble == 0 where the tap matches
+                        z |= z >> 1;
+                        z |= z >> 2;
+                        unsigned m = ~z & 0x11111111u;      // bit 4*i set where nibble i matches
+                        while (m) {
+                            const int kk = wq * 8 + ((__ffs(m) - 1) >> 2);
+                            m &= m - 1;
+                            const unsigned id_nxt = (unsigned)__ldg(ip + (size_t)kk * plane);
+                            const float gv_nxt = to_f32(gp[(size_t)kk * plane]);
+                            if (have) {
+                                const unsigned c = magic ? __umulhi(id_cur, magic) : id_cur;
+                                dst[c * cstride] += gv_cur;
+                            }
+                            id_cur = id_nxt;
+                            gv_cur = gv_nxt;
+                            have = true;
+                        }
+                    }
+                    if (have) {
+                        const unsigned c = magic ? __umulhi(id_cur, magic) : id_cur;
+                        dst[c * cstride] += gv_cur;
+                    }
+                }
+                __syncthreads();
+            }
+        }
+    }
+    for (int e = threadIdx.x; e < g.C * rows * g.W; e += blockDim.x) {
+        const int c = e / (rows * g.W);
+        const int rem = e - c * rows * g.W;
+        gx[((size_t)n * g.C + c) * g.H * g.W + (size_t)ih0 * g.W + rem] =
+            from_f32<T>(tile[c * cstride + rem]);
+    }
+}
+
 // ---------------------------------------------------------------------------------- idx: grad_w, grad_bias
 template <typename T>
 __global__ void __launch_bounds__(256)
