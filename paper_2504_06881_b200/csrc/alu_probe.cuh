@@ -1,9 +1,11 @@
 // Register-only throughput probes of the add + max/min instruction mixes the
 // tropical kernels can be built from.  Each thread keeps a TK x TP block of
 // running extrema and folds taps x[j] + w[i] into them, exactly the inner loop of
-// the forward pass minus its memory traffic.  An empty asm statement that names
-// x and w as read-write operands stops the compiler from hoisting the adds out
-// of the loop without costing an instruction.
+// the forward pass minus its memory traffic.  The x operands are advanced by a
+// real add in every iteration (TP + 1 extra adds per TK * TP * 2 taps): an empty
+// asm barrier is not enough, because the assembler, which never sees it, would
+// hoist the loop-invariant tap sums out of the loop and the probe would measure
+// min/max alone.
 #pragma once
 #include "tconv_common.cuh"
 
@@ -74,6 +76,7 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
         constexpr int KP = 4, PX = 8;
         __nv_bfloat162 x[PX + 1], wa[KP], wb[KP], va[KP], vb[KP];
         __nv_bfloat162 mn[KP][PX], mx[KP][PX];
+        const __nv_bfloat162 dx2 = __float2bfloat162_rn(seed * 0.0078125f);
         for (int j = 0; j <= PX; ++j) x[j] = __float2bfloat162_rn(seed * (float)(j + threadIdx.x));
         for (int i = 0; i < KP; ++i) {
             wa[i] = __float2bfloat162_rn(seed * (float)(i + 3));
@@ -84,7 +87,7 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
         }
         for (int it = 0; it < iters; ++it) {
 #pragma unroll
-            for (int j = 0; j <= PX; ++j) TCONV_OPAQUE_R(*reinterpret_cast<unsigned*>(&x[j]));
+            for (int j = 0; j <= PX; ++j) x[j] = __hadd2(x[j], dx2);   // operands change every iteration
 #pragma unroll
             for (int i = 0; i < KP; ++i) {
                 TCONV_OPAQUE_R(*reinterpret_cast<unsigned*>(&wa[i]));
@@ -118,6 +121,7 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
     } else {
         float x[TP + 1], w0[TK], w1[TK], v0[TK], v1[TK];
         float mn[TK][TP], mx[TK][TP];
+        const float dx = seed * 1.0e-3f;
         for (int j = 0; j <= TP; ++j) x[j] = seed * (float)(j + threadIdx.x);
         for (int i = 0; i < TK; ++i) {
             w0[i] = seed * (float)(i + 3);
@@ -128,7 +132,7 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
         }
         for (int it = 0; it < iters; ++it) {
 #pragma unroll
-            for (int j = 0; j <= TP; ++j) TCONV_OPAQUE_F(x[j]);
+            for (int j = 0; j <= TP; ++j) x[j] = __fadd_rn(x[j], dx);    // operands change every iteration
 #pragma unroll
             for (int i = 0; i < TK; ++i) {
                 TCONV_OPAQUE_F(w0[i]); TCONV_OPAQUE_F(w1[i]);

@@ -433,8 +433,16 @@ int tconv_alu_probe(int variant, int iters, void* sink, double* taps_per_launch,
     const unsigned blocks = (unsigned)sms * 8u;
     cudaStream_t st = (cudaStream_t)stream;
     const float seed = 1.0009765625f;
-#define TCONV_PROBE_CASE(V) \
-    case V: alu_probe_kernel<V><<<blocks, 256, 0, st>>>(iters, seed, (float*)sink); break;
+    // debug switch: dynamic shared memory per block, to limit the resident blocks per SM
+    static const size_t probe_smem = [] {
+        const char* e = getenv("TCONV_PROBE_SMEM");
+        return e ? (size_t)atol(e) : (size_t)0;
+    }();
+#define TCONV_PROBE_CASE(V)                                                                          \
+    case V:                                                                                          \
+        if (probe_smem) cudaFuncSetAttribute(alu_probe_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)probe_smem); \
+        alu_probe_kernel<V><<<blocks, 256, probe_smem, st>>>(iters, seed, (float*)sink);             \
+        break;
     switch (variant) {
         TCONV_PROBE_CASE(0) TCONV_PROBE_CASE(1) TCONV_PROBE_CASE(2) TCONV_PROBE_CASE(3)
         TCONV_PROBE_CASE(4) TCONV_PROBE_CASE(5) TCONV_PROBE_CASE(6) TCONV_PROBE_CASE(7)
