@@ -422,6 +422,53 @@ def run_single(args):
                       "ms": ms, "Ttap_s": L.taps / (ms * 1e-3) / 1e12, "kernel": tconv.tconv_last_kernel()}))
 
 
+def run_cfg5(args):
+    """Training step of the ResNet-18-shaped hybrid network (N=64, 224x224, stages 2-4 tropical,
+    bf16 tropical kernels): step time, summed tropical-layer time and tropical Gop/s."""
+    import torch
+    from paper_2504_06881_b200 import tconv
+    from paper_2504_06881_b200.nn import HybridResNet18, TropicalConvFn
+    torch.cuda.set_device(0)
+    torch.manual_seed(1050)
+    rs = np.random.RandomState(1050)
+    N = 64
+    net = HybridResNet18(mode=args.only or "compound", dtype="bf16").cuda()
+    x = torch.from_numpy(rs.standard_normal((N, 3, 224, 224)).astype(np.float32)).cuda()
+    labels = torch.from_numpy(rs.randint(0, 1000, N)).cuda()
+    opt = torch.optim.SGD(net.parameters(), lr=0.01, momentum=0.9)
+
+    def step():
+        loss = torch.nn.functional.cross_entropy(net(x), labels)
+        opt.zero_grad()
+        loss.backward()
+        opt.step()
+        return loss
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    TropicalConvFn.events = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        loss = step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    ev = TropicalConvFn.events
+    TropicalConvFn.events = None
+    t_fwd = sum(a.elapsed_time(b) for k, d, a, b in ev if k == "fwd") / args.steps
+    t_bwd = sum(a.elapsed_time(b) for k, d, a, b in ev if k == "bwd") / args.steps
+    ops = sum(2 * tconv.tconv_paper_ops(d) for k, d, a, b in ev if k == "fwd") / args.steps
+    taps = sum(d["N"] * d["K"] * d["C"] * 9 * tconv.tconv_output_shape(d)[0] * tconv.tconv_output_shape(d)[1]
+               for k, d, a, b in ev if k == "fwd") / args.steps
+    print(json.dumps({"workload": "cfg5: ResNet-18-shaped hybrid net, N=64, 224x224, stages 2-4 tropical (bf16 kernels)",
+                      "mode": args.only or "compound", "step_ms": ms, "tropical_fwd_ms": t_fwd,
+                      "tropical_bwd_ms": t_bwd, "tropical_layers": len([1 for e in ev if e[0] == "fwd"]) // args.steps,
+                      "tropical_taps_fwd": taps, "tropical_Gop_s_fwd_bwd": ops / ((t_fwd + t_bwd) * 1e-3) / 1e9,
+                      "loss": float(loss)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -433,9 +480,13 @@ def main():
     ap.add_argument("--what", default="fwd", choices=["fwd", "fwd_winners", "bwd"])
     ap.add_argument("--images", type=int, default=128)
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5"],
+                    help="cfg5: report the hybrid ResNet-18 training step instead (use --only compound|parallel)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "cfg5":
+        run_cfg5(args)
     elif args.only:
         run_single(args)
     else:

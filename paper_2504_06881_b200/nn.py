@@ -1,0 +1,179 @@
+"""PyTorch glue over the C ABI: an autograd Function, a drop-in layer and the
+ResNet-18-shaped hybrid network of benchmark configuration 5.
+
+Everything tropical runs in the library's CUDA kernels (forward with winners, winner-routed
+backward); PyTorch supplies BatchNorm, the standard convolutions of the stem / stage 1 /
+1x1 downsamples, the loss and the optimiser, none of which is on the tropical hot path.
+The layer follows the paper's usage (Appendix "Compatibility with PyTorch"): same constructor
+arguments as ``nn.Conv2d``; ``mode`` selects max_plus / min_plus / compound / parallel.
+"""
+from __future__ import annotations
+
+import math
+
+import torch
+import torch.nn as nn
+
+from . import tconv
+
+
+class TropicalConvFn(torch.autograd.Function):
+    """y = tconv_forward(x, w, w2, alpha, beta, bias); backward = tconv_backward with the stored winners.
+
+    Master parameters may be fp32 while the layer computes in bf16: the cast happens here and the
+    parameter gradients come back in fp32.  When ``TropicalConvFn.events`` is a list, every library
+    call is bracketed by a pair of CUDA events appended to it (for the benchmark's per-layer times)."""
+
+    events = None
+
+    @staticmethod
+    def forward(ctx, x, w, w2, alpha, beta, bias, geom):
+        mode, chan, dtype, stride, pad, dil = geom
+        dt = tconv.TORCH_DTYPE[dtype]
+        N, C, H, W = x.shape
+        K, _, R, S = w.shape
+        d = dict(N=N, C=C, H=H, W=W, K=K, R=R, S=S, stride_h=stride[0], stride_w=stride[1],
+                 pad_h=pad[0], pad_w=pad[1], dil_h=dil[0], dil_w=dil[1], mode=mode, chan=chan, dtype=dtype)
+        xc = x.detach().to(dt).contiguous()
+        wc = w.detach().to(dt).contiguous()
+        w2c = w2.detach().to(dt).contiguous() if w2 is not None else None
+        al = alpha.detach().float().contiguous() if alpha is not None else None
+        be = beta.detach().float().contiguous() if beta is not None else None
+        bi = bias.detach().float().contiguous() if bias is not None else None
+        need_grad = any(t is not None and t.requires_grad for t in (x, w, w2, alpha, beta, bias))
+        ev = TropicalConvFn.events
+        if ev is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        y, winners = tconv.forward(d, xc, wc, w2c, al, be, bi, want_winners=need_grad)
+        if ev is not None:
+            e1.record()
+            ev.append(("fwd", d, e0, e1))
+        ctx.d = d
+        ctx.in_dtype = x.dtype
+        ctx.save_for_backward(xc, wc, w2c, al, be, winners)
+        ctx.has = (w2 is not None, alpha is not None, beta is not None, bias is not None)
+        return y.to(x.dtype) if x.dtype != dt else y
+
+    @staticmethod
+    def backward(ctx, gy):
+        xc, wc, w2c, al, be, winners = ctx.saved_tensors
+        d = ctx.d
+        dt = tconv.TORCH_DTYPE[d["dtype"]]
+        g = gy.to(dt).contiguous()
+        ev = TropicalConvFn.events
+        if ev is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        grads = tconv.backward(d, xc, wc, g, w2c, al, be, winners)
+        if ev is not None:
+            e1.record()
+            ev.append(("bwd", d, e0, e1))
+        has_w2, has_a, has_b, has_bias = ctx.has
+        gx = grads["grad_x"].to(ctx.in_dtype)
+        return (gx, grads["grad_w"], grads.get("grad_w2") if has_w2 else None,
+                grads.get("grad_alpha") if has_a else None, grads.get("grad_beta") if has_b else None,
+                grads["grad_bias"] if has_bias else None, None)
+
+
+class TropicalConv2d(nn.Module):
+    """Tropical convolution layer with ``nn.Conv2d``'s constructor arguments.
+
+    mode: "max_plus" | "min_plus" | "compound" | "parallel"; chan: "default" | "sum" | "max" | "min".
+    params (compound / parallel): "2p" learnable alpha and beta per (c_out, c_in); "1p" the
+    complementary-weight specialisation beta = 1 - alpha; "0p" alpha = beta = 1 (no scalars).
+    dtype: arithmetic type of the kernels ("f32" or "bf16"); parameters stay fp32."""
+
+    def __init__(self, in_channels, out_channels, kernel_size, stride=1, padding=0, dilation=1,
+                 bias=True, mode="compound", chan="default", params="2p", dtype="f32"):
+        super().__init__()
+        two = lambda v: (v, v) if isinstance(v, int) else tuple(v)
+        self.kernel_size, self.stride, self.padding, self.dilation = map(two, (kernel_size, stride, padding, dilation))
+        self.in_channels, self.out_channels = in_channels, out_channels
+        self.mode, self.chan, self.params, self.dtype = mode, chan, params, dtype
+        R, S = self.kernel_size
+        self.weight = nn.Parameter(torch.empty(out_channels, in_channels, R, S))
+        self.weight2 = nn.Parameter(torch.empty(out_channels, in_channels, R, S)) if mode == "parallel" else None
+        two_branch = mode in ("compound", "parallel")
+        self.alpha = nn.Parameter(torch.empty(out_channels, in_channels)) if two_branch and params in ("1p", "2p") else None
+        self.beta = nn.Parameter(torch.empty(out_channels, in_channels)) if two_branch and params == "2p" else None
+        self.bias = nn.Parameter(torch.zeros(out_channels)) if bias else None
+        self.reset_parameters()
+
+    def reset_parameters(self):
+        fan_in = self.in_channels * self.kernel_size[0] * self.kernel_size[1]
+        bound = 1.0 / math.sqrt(fan_in)
+        for w in (self.weight, self.weight2):
+            if w is not None:
+                nn.init.uniform_(w, -bound, bound)
+        # the paper gives no initial values for alpha / beta: start from the normalised average of
+        # the two branches divided by the fan-in of the channel sum
+        for a in (self.alpha, self.beta):
+            if a is not None:
+                nn.init.constant_(a, 0.5 / self.in_channels)
+
+    def extra_repr(self):
+        return (f"{self.in_channels}, {self.out_channels}, kernel_size={self.kernel_size}, stride={self.stride}, "
+                f"padding={self.padding}, dilation={self.dilation}, mode={self.mode}, chan={self.chan}, "
+                f"params={self.params}, dtype={self.dtype}")
+
+    def forward(self, x):
+        alpha, beta = self.alpha, self.beta
+        if self.mode in ("compound", "parallel") and self.params == "1p":
+            beta = 1.0 - alpha
+        geom = (self.mode, self.chan, self.dtype, self.stride, self.padding, self.dilation)
+        return TropicalConvFn.apply(x, self.weight, self.weight2, alpha, beta, self.bias, geom)
+
+
+class TropicalBasicBlock(nn.Module):
+    """The paper's TCNN basic block 2: Tropical - BN - Tropical - BN, intermediate ReLU removed,
+    identity (or 1x1 standard-convolution) shortcut, ReLU after the sum."""
+
+    def __init__(self, cin, cout, stride, mode, dtype):
+        super().__init__()
+        self.conv1 = TropicalConv2d(cin, cout, 3, stride=stride, padding=1, bias=False, mode=mode, dtype=dtype)
+        self.bn1 = nn.BatchNorm2d(cout)
+        self.conv2 = TropicalConv2d(cout, cout, 3, stride=1, padding=1, bias=False, mode=mode, dtype=dtype)
+        self.bn2 = nn.BatchNorm2d(cout)
+        self.down = None
+        if stride != 1 or cin != cout:
+            self.down = nn.Sequential(nn.Conv2d(cin, cout, 1, stride=stride, bias=False), nn.BatchNorm2d(cout))
+
+    def forward(self, x):
+        out = self.bn2(self.conv2(self.bn1(self.conv1(x))))
+        return torch.relu(out + (x if self.down is None else self.down(x)))
+
+
+class StandardBasicBlock(nn.Module):
+    def __init__(self, cin, cout, stride):
+        super().__init__()
+        self.conv1 = nn.Conv2d(cin, cout, 3, stride=stride, padding=1, bias=False)
+        self.bn1 = nn.BatchNorm2d(cout)
+        self.conv2 = nn.Conv2d(cout, cout, 3, padding=1, bias=False)
+        self.bn2 = nn.BatchNorm2d(cout)
+
+    def forward(self, x):
+        return torch.relu(self.bn2(self.conv2(torch.relu(self.bn1(self.conv1(x))))) + x)
+
+
+class HybridResNet18(nn.Module):
+    """ResNet-18 shape; every 3x3 convolution of stages 2-4 is a tropical layer of the given mode
+    (stem, stage 1 and the 1x1 downsamples are standard convolutions)."""
+
+    def __init__(self, mode="compound", dtype="bf16", num_classes=1000):
+        super().__init__()
+        self.stem = nn.Sequential(nn.Conv2d(3, 64, 7, stride=2, padding=3, bias=False), nn.BatchNorm2d(64),
+                                  nn.ReLU(inplace=True), nn.MaxPool2d(3, stride=2, padding=1))
+        self.layer1 = nn.Sequential(StandardBasicBlock(64, 64, 1), StandardBasicBlock(64, 64, 1))
+        self.layer2 = nn.Sequential(TropicalBasicBlock(64, 128, 2, mode, dtype), TropicalBasicBlock(128, 128, 1, mode, dtype))
+        self.layer3 = nn.Sequential(TropicalBasicBlock(128, 256, 2, mode, dtype), TropicalBasicBlock(256, 256, 1, mode, dtype))
+        self.layer4 = nn.Sequential(TropicalBasicBlock(256, 512, 2, mode, dtype), TropicalBasicBlock(512, 512, 1, mode, dtype))
+        self.head = nn.Sequential(nn.AdaptiveAvgPool2d(1), nn.Flatten(), nn.Linear(512, num_classes))
+
+    def forward(self, x):
+        x = self.layer1(self.stem(x))
+        x = self.layer4(self.layer3(self.layer2(x)))
+        return self.head(x)
+
+    def tropical_layers(self):
+        return [m for m in self.modules() if isinstance(m, TropicalConv2d)]
