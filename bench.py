@@ -466,7 +466,7 @@ def run_cfg5(args):
                       "mode": args.only or "compound", "step_ms": ms, "tropical_fwd_ms": t_fwd,
                       "tropical_bwd_ms": t_bwd, "tropical_layers": len([1 for e in ev if e[0] == "fwd"]) // args.steps,
                       "tropical_taps_fwd": taps, "tropical_Gop_s_fwd_bwd": ops / ((t_fwd + t_bwd) * 1e-3) / 1e9,
-                      "loss": float(loss)}))
+                      "loss": float(loss.detach())}))
 
 
 def main():

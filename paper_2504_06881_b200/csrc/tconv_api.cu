@@ -227,7 +227,8 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
         CodeGxPlan pl;
         if (gx) {
             if (tiled && plan_code_gx(g, &pl)) {
-                const dim3 grid((unsigned)(g.N * pl.tiles_per_img), (unsigned)((g.C + pl.CB - 1) / pl.CB));
+                const dim3 grid((unsigned)(((g.N + pl.imgs - 1) / pl.imgs) * pl.tiles_per_img),
+                                (unsigned)((g.C + pl.CB - 1) / pl.CB));
 #define TCONV_GX(BR, CBV, VECV)                                                                      \
     {                                                                                                \
         auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV>;                                            \

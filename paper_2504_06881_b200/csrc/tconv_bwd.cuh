@@ -229,6 +229,7 @@ __global__ void bwd_reduce_partials_kernel(const float* __restrict__ partial, fl
 constexpr int kGxCB = 2;   // most channels a CTA of bwd_code_gx_kernel handles
 
 struct CodeGxPlan {
+    int imgs;                // images per CTA (> 1 only when a CTA owns whole images of a small map)
     int THI, tiles_per_img;  // owned input rows per CTA
     int CB;                  // channels per CTA
     int NRmax, QPR, NQpad;   // contributing output rows (max), quads per row, padded quad count
@@ -275,8 +276,11 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
                    CodeGxPlan pl) {
     extern __shared__ float A[];  // [CB][RS][4][NQpad], then alpha / beta of this CTA's channels [K][CB] each
+    // a CTA owns either a band of input rows of one image or pl.imgs whole images of a small map;
+    // its output quads are numbered image by image
     const int tile_i = blockIdx.x % pl.tiles_per_img;
-    const int n = blockIdx.x / pl.tiles_per_img;
+    const int n_first = (blockIdx.x / pl.tiles_per_img) * pl.imgs;
+    const int nimg = min(pl.imgs, g.N - n_first);
     const int c0 = blockIdx.y * CB;
     const int ncb = min(CB, g.C - c0);
     const int ih0 = tile_i * pl.THI;
@@ -285,7 +289,8 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     const int oh_lo = num <= 0 ? 0 : (num + g.sh - 1) / g.sh;
     const int oh_hi = min(g.OH - 1, (ih0 + rows - 1 + g.ph) / g.sh);
     const int NR = oh_hi - oh_lo + 1;
-    const int NQ = NR * pl.QPR;
+    const int NQ1 = NR * pl.QPR;          // quads of one image
+    const int NQ = NQ1 * nimg;
     const int NQp = pl.NQpad;
     const int nacc = CB * g.RS * 4 * NQp;
     float* a_s = A + nacc;
@@ -304,8 +309,11 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     const size_t cstep = (size_t)g.C * plane;        // codes: one output channel k further
     const unsigned tstride = 4u * NQp * sizeof(float); // bytes between the accumulators of two taps
     for (int q = threadIdx.x; q < NQ; q += blockDim.x) {
-        const int orow = q / pl.QPR;
-        const int ow0 = (q - orow * pl.QPR) * 4;
+        const int il = q / NQ1;
+        const int q1 = q - il * NQ1;
+        const int n = n_first + il;
+        const int orow = q1 / pl.QPR;
+        const int ow0 = (q1 - orow * pl.QPR) * 4;
         const size_t pix = (size_t)(oh_lo + orow) * g.OW + ow0;
         const T* gp = gy + (size_t)n * g.K * plane + pix;
         // a channel past C reads channel C-1 again; its alpha = beta = 0 (or it is skipped below)
@@ -364,9 +372,10 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     // pixel that reads it through that tap (one warp per input row, lanes along the columns)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool unit_stride = (g.sh == 1 && g.sw == 1);
+    for (int il = 0; il < nimg; ++il)
     for (int cb = 0; cb < ncb; ++cb) {
-        const float* Ac = A + (size_t)cb * g.RS * 4 * NQp;
-        T* gxc = gx + ((size_t)n * g.C + c0 + cb) * g.H * g.W;
+        const float* Ac = A + (size_t)cb * g.RS * 4 * NQp + il * NQ1;
+        T* gxc = gx + ((size_t)(n_first + il) * g.C + c0 + cb) * g.H * g.W;
         for (int row = warp; row < rows; row += 8) {
             const int ih = ih0 + row;
             for (int iw = lane; iw < g.W; iw += 32) {
@@ -456,68 +465,117 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
     const size_t cstep = (size_t)g.K * g.C * plane;      // codes: one image further
     const size_t xstep = (size_t)g.C * pl.xs_elems;      // padded x: one image further
     float sa = 0.0f, sb = 0.0f;
-    for (int q = tid; q < NQ; q += 256) {
-        const int oh = q / QPR;
-        const int ow0 = (q - oh * QPR) * 4;
-        const size_t pix = (size_t)oh * g.OW + ow0;
-        const T* gp = gy + (size_t)k * plane + pix;
-        const uint8_t* cp = codes + ((size_t)k * g.C + c) * plane + pix;
-        const T* xp = XS ? reinterpret_cast<const T*>(pl.xpad) + (size_t)c * pl.xs_elems +
-                               (size_t)oh * g.sh * pl.WP + ow0 * g.sw
-                         : x + (size_t)c * g.H * g.W;
-        float gv_cur[4], gv_nxt[4];
-        unsigned cw_cur, cw_nxt = 0;
-        load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
-        cw_cur = load_c4<VEC>(cp, ow0, g.OW);
-        for (int n = 0; n < g.N; ++n) {
-            if (n + 1 < g.N) {
-                gp += gstep;
-                cp += cstep;
-                load_g4<T, VEC>(gp, ow0, g.OW, gv_nxt);
-                cw_nxt = load_c4<VEC>(cp, ow0, g.OW);
-            }
+    // one (image, quad) item: 4 gradients gv, 4 winner codes cw, padded-x pointer xp of the item
+    auto accumulate = [&](int oh, int ow0, const float* gv, unsigned cw, const T* xp) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (!VEC && ow0 + j >= g.OW) continue;
-                const unsigned code = (cw_cur >> (8 * j)) & 0xffu;
-                const float gvj = gv_cur[j];
-                if constexpr (BR == 0 || BR == 1) {
-                    const unsigned t = code & 15u;
-                    float* dst = reinterpret_cast<float*>(colb + t * 1024u);
-                    *dst += gvj;
-                    if (need_ab) {
-                        const int2 tw = tapw_min[t];
-                        T xv;
-                        if constexpr (XS) {
-                            xv = xp[j * g.sw + tw.x];
-                        } else {
-                            const int ih = oh * g.sh + tap_dh[t], iw = (ow0 + j) * g.sw + tap_dw[t];
-                            xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xp[(size_t)ih * g.W + iw] : zero_of<T>();
-                        }
-                        sa = __fmaf_rn(gvj, tap_add(xv, from_f32<T>(__int_as_float(tw.y))), sa);
+        for (int j = 0; j < 4; ++j) {
+            if (!VEC && ow0 + j >= g.OW) continue;
+            const unsigned code = (cw >> (8 * j)) & 0xffu;
+            const float gvj = gv[j];
+            if constexpr (BR == 0 || BR == 1) {
+                const unsigned t = code & 15u;
+                float* dst = reinterpret_cast<float*>(colb + t * 1024u);
+                *dst += gvj;
+                if (need_ab) {
+                    const int2 tw = tapw_min[t];
+                    T xv;
+                    if constexpr (XS) {
+                        xv = xp[j * g.sw + tw.x];
+                    } else {
+                        const int ih = oh * g.sh + tap_dh[t], iw = (ow0 + j) * g.sw + tap_dw[t];
+                        xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xp[(size_t)ih * g.W + iw] : zero_of<T>();
                     }
-                }
-                if constexpr (BR == 0 || BR == 2) {
-                    const unsigned t = code >> 4;
-                    float* dst = reinterpret_cast<float*>(colb + (g.RS + t) * 1024u);
-                    *dst += gvj;
-                    if (need_ab) {
-                        const int2 tw = tapw_max[t];
-                        T xv;
-                        if constexpr (XS) {
-                            xv = xp[j * g.sw + tw.x];
-                        } else {
-                            const int ih = oh * g.sh + tap_dh[t], iw = (ow0 + j) * g.sw + tap_dw[t];
-                            xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xp[(size_t)ih * g.W + iw] : zero_of<T>();
-                        }
-                        sb = __fmaf_rn(gvj, tap_add(xv, from_f32<T>(__int_as_float(tw.y))), sb);
-                    }
+                    sa = __fmaf_rn(gvj, tap_add(xv, from_f32<T>(__int_as_float(tw.y))), sa);
                 }
             }
-            xp += XS ? xstep : (size_t)g.C * g.H * g.W;
+            if constexpr (BR == 0 || BR == 2) {
+                const unsigned t = code >> 4;
+                float* dst = reinterpret_cast<float*>(colb + (g.RS + t) * 1024u);
+                *dst += gvj;
+                if (need_ab) {
+                    const int2 tw = tapw_max[t];
+                    T xv;
+                    if constexpr (XS) {
+                        xv = xp[j * g.sw + tw.x];
+                    } else {
+                        const int ih = oh * g.sh + tap_dh[t], iw = (ow0 + j) * g.sw + tap_dw[t];
+                        xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xp[(size_t)ih * g.W + iw] : zero_of<T>();
+                    }
+                    sb = __fmaf_rn(gvj, tap_add(xv, from_f32<T>(__int_as_float(tw.y))), sb);
+                }
+            }
+        }
+    };
+    if (NQ >= 192) {
+        // large maps: a thread keeps its quad and walks the images (constant pointer strides)
+        for (int q = tid; q < NQ; q += 256) {
+            const int oh = q / QPR;
+            const int ow0 = (q - oh * QPR) * 4;
+            const size_t pix = (size_t)oh * g.OW + ow0;
+            const T* gp = gy + (size_t)k * plane + pix;
+            const uint8_t* cp = codes + ((size_t)k * g.C + c) * plane + pix;
+            const T* xp = XS ? reinterpret_cast<const T*>(pl.xpad) + (size_t)c * pl.xs_elems +
+                                   (size_t)oh * g.sh * pl.WP + ow0 * g.sw
+                             : x + (size_t)c * g.H * g.W;
+            float gv_cur[4], gv_nxt[4];
+            unsigned cw_cur, cw_nxt = 0;
+            load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
+            cw_cur = load_c4<VEC>(cp, ow0, g.OW);
+            for (int n = 0; n < g.N; ++n) {
+                if (n + 1 < g.N) {
+                    gp += gstep;
+                    cp += cstep;
+                    load_g4<T, VEC>(gp, ow0, g.OW, gv_nxt);
+                    cw_nxt = load_c4<VEC>(cp, ow0, g.OW);
+                }
+                accumulate(oh, ow0, gv_cur, cw_cur, xp);
+                xp += XS ? xstep : (size_t)g.C * g.H * g.W;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) gv_cur[j] = gv_nxt[j];
+                cw_cur = cw_nxt;
+            }
+        }
+    } else {
+        // small maps: the threads walk the flattened (image, quad) pairs with a stride of 256
+        const int dn = 256 / NQ, dq = 256 - dn * NQ;
+        int n = tid / NQ, q = tid - n * NQ;
+        float gv_cur[4], gv_nxt[4];
+        unsigned cw_cur = 0, cw_nxt = 0;
+        auto item_ptrs = [&](int n_, int q_, int& oh, int& ow0, const T*& gp, const uint8_t*& cp, const T*& xp) {
+            oh = q_ / QPR;
+            ow0 = (q_ - oh * QPR) * 4;
+            const size_t pix = (size_t)oh * g.OW + ow0;
+            gp = gy + ((size_t)n_ * g.K + k) * plane + pix;
+            cp = codes + (((size_t)n_ * g.K + k) * g.C + c) * plane + pix;
+            xp = XS ? reinterpret_cast<const T*>(pl.xpad) + ((size_t)n_ * g.C + c) * pl.xs_elems +
+                          (size_t)oh * g.sh * pl.WP + ow0 * g.sw
+                    : x + ((size_t)n_ * g.C + c) * g.H * g.W;
+        };
+        int oh = 0, ow0 = 0;
+        const T* gp = nullptr; const uint8_t* cp = nullptr; const T* xp = nullptr;
+        bool have = n < g.N;
+        if (have) {
+            item_ptrs(n, q, oh, ow0, gp, cp, xp);
+            load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
+            cw_cur = load_c4<VEC>(cp, ow0, g.OW);
+        }
+        while (have) {
+            int n2 = n + dn, q2 = q + dq;
+            if (q2 >= NQ) { q2 -= NQ; ++n2; }
+            const bool more = n2 < g.N;
+            int oh2 = 0, ow2 = 0;
+            const T* gp2 = nullptr; const uint8_t* cp2 = nullptr; const T* xp2 = nullptr;
+            if (more) {
+                item_ptrs(n2, q2, oh2, ow2, gp2, cp2, xp2);
+                load_g4<T, VEC>(gp2, ow2, g.OW, gv_nxt);
+                cw_nxt = load_c4<VEC>(cp2, ow2, g.OW);
+            }
+            accumulate(oh, ow0, gv_cur, cw_cur, xp);
+            n = n2; q = q2; oh = oh2; ow0 = ow2; xp = xp2;
 #pragma unroll
             for (int j = 0; j < 4; ++j) gv_cur[j] = gv_nxt[j];
             cw_cur = cw_nxt;
+            have = more;
         }
     }
     S[(2 * g.RS) * 256 + tid] = sa;
@@ -635,9 +693,16 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
         long nr = maxq / pl->QPR;
         if (nr < 1) continue;
         int thi;
+        pl->imgs = 1;
         if (nr >= g.OH) {
             thi = g.H;                      // the whole image: no redundant rows
             nr = g.OH;
+            // small maps: several whole images per CTA so that its 256 threads have quads to own
+            const long q1 = (long)g.OH * pl->QPR;
+            long im = 256 / q1;
+            if (im > maxq / q1) im = maxq / q1;
+            if (im > g.N) im = g.N;
+            if (im > 1) pl->imgs = (int)im;
         } else {
             // NR = ceil((THI + halo) / sh) + 1 at most
             thi = (int)((nr - 2) * g.sh) - halo;
@@ -648,7 +713,7 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
         pl->THI = thi;
         pl->tiles_per_img = (g.H + thi - 1) / thi;
         pl->NRmax = (int)nr;
-        pl->NQpad = (int)(((long)nr * pl->QPR + 31) / 32 * 32);
+        pl->NQpad = (int)(((long)nr * pl->QPR * pl->imgs + 31) / 32 * 32);
         pl->smem = ((size_t)cb * g.RS * 4 * pl->NQpad + 2 * (size_t)g.K * kGxCB) * sizeof(float);
         if (pl->smem > kBwdSmemLimit + 16 * 1024) continue;
         return true;
