@@ -229,13 +229,15 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
             if (tiled && plan_code_gx(g, &pl)) {
                 const dim3 grid((unsigned)(((g.N + pl.imgs - 1) / pl.imgs) * pl.tiles_per_img),
                                 (unsigned)((g.C + pl.CB - 1) / pl.CB));
-#define TCONV_GX(BR, CBV, VECV)                                                                      \
+#define TCONV_GXM(BR, CBV, VECV, MULTI)                                                              \
     {                                                                                                \
-        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV>;                                            \
+        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV, MULTI>;                                     \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<grid, 256, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);          \
     }
+#define TCONV_GX(BR, CBV, VECV)                                                                      \
+    { if (pl.imgs > 1) TCONV_GXM(BR, CBV, VECV, true) else TCONV_GXM(BR, CBV, VECV, false) }
 #define TCONV_GX2(BR)                                                                                \
     {                                                                                                \
         if (pl.CB == 2) { if (vec) TCONV_GX(BR, 2, true) else TCONV_GX(BR, 2, false) }               \
@@ -245,6 +247,7 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                 if (br == 0) TCONV_GX2(0) else if (br == 1) TCONV_GX2(1) else TCONV_GX2(2)
 #undef TCONV_GX2
 #undef TCONV_GX
+#undef TCONV_GXM
                 name = "bwd_code";
             } else {
                 const size_t total = (size_t)g.N * g.C * g.H * g.W;

@@ -270,7 +270,8 @@ __device__ __forceinline__ unsigned load_c4(const uint8_t* p, int ow0, int OW) {
 // BR: 0 = both branches (compound / parallel), 1 = min branch only, 2 = max branch only.
 // CB channels per CTA (the CTA's last channel block may hold fewer: those lanes idle).
 // VEC: OW is a multiple of 4 (aligned vector loads of grad_y and of the codes).
-template <typename T, int BR, int CB, bool VEC>
+// MULTI: the CTA owns pl.imgs whole images (small maps); else one band of rows of one image.
+template <typename T, int BR, int CB, bool VEC, bool MULTI>
 __global__ void __launch_bounds__(256)
 bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
@@ -279,8 +280,8 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     // a CTA owns either a band of input rows of one image or pl.imgs whole images of a small map;
     // its output quads are numbered image by image
     const int tile_i = blockIdx.x % pl.tiles_per_img;
-    const int n_first = (blockIdx.x / pl.tiles_per_img) * pl.imgs;
-    const int nimg = min(pl.imgs, g.N - n_first);
+    const int n_first = MULTI ? (blockIdx.x / pl.tiles_per_img) * pl.imgs : blockIdx.x / pl.tiles_per_img;
+    const int nimg = MULTI ? min(pl.imgs, g.N - n_first) : 1;
     const int c0 = blockIdx.y * CB;
     const int ncb = min(CB, g.C - c0);
     const int ih0 = tile_i * pl.THI;
@@ -309,7 +310,7 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     const size_t cstep = (size_t)g.C * plane;        // codes: one output channel k further
     const unsigned tstride = 4u * NQp * sizeof(float); // bytes between the accumulators of two taps
     for (int q = threadIdx.x; q < NQ; q += blockDim.x) {
-        const int il = q / NQ1;
+        const int il = MULTI ? q / NQ1 : 0;
         const int q1 = q - il * NQ1;
         const int n = n_first + il;
         const int orow = q1 / pl.QPR;

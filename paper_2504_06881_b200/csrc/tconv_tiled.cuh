@@ -38,14 +38,18 @@ __device__ __forceinline__ void add2(float x, float wlo, float whi, float& lo, f
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(tt) : "l"(xx), "l"(ww));
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
 }
-// The same packed add, opaque to common-subexpression elimination: the winner pass recomputes
-// the tap sums instead of keeping all of them alive since the first pass.
-__device__ __forceinline__ void add2_again(float x, float wlo, float whi, float& lo, float& hi) {
-    unsigned long long xx, ww, tt;
-    asm("mov.b64 %0, {%1, %1};" : "=l"(xx) : "f"(x));
-    asm("mov.b64 %0, {%1, %2};" : "=l"(ww) : "f"(wlo), "f"(whi));
-    asm volatile("add.rn.f32x2 %0, %1, %2;" : "=l"(tt) : "l"(xx), "l"(ww));
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
+// Extremum of v[0..RS)[h] with 3-input min / max: a fresh chain opens with three values,
+// every later step folds two more.
+template <int RS>
+__device__ __forceinline__ float fold_taps(const float (*v)[2], int h, bool is_min) {
+    float m;
+    if constexpr (RS >= 3) m = ext3(v[0][h], v[1][h], v[2][h], is_min);
+    else if constexpr (RS == 2) m = ext2(v[0][h], v[1][h], is_min);
+    else m = v[0][h];
+#pragma unroll
+    for (int i = 3; i + 1 < RS; i += 2) m = ext3(m, v[i][h], v[i + 1][h], is_min);
+    if constexpr (RS > 3 && ((RS - 3) & 1)) m = ext2(m, v[RS - 1][h], is_min);
+    return m;
 }
 // {c0, c1} = a * {v0, v1} + {c0, c1}: one packed fused multiply-add (scalar a splat)
 __device__ __forceinline__ void fma2s(float a, float v0, float v1, float& c0, float& c1) {
@@ -127,7 +131,12 @@ __device__ __forceinline__ void load_segment(const float* base, float* out) {
 }
 template <int N>
 __device__ __forceinline__ void loadn(const float* p, float* out) {
-    static_assert(N % 4 == 0, "vector loads");
+    static_assert(N == 2 || N % 4 == 0, "vector loads");
+    if constexpr (N == 2) {
+        const float2 a = *reinterpret_cast<const float2*>(p);
+        out[0] = a.x; out[1] = a.y;
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < N; i += 4) {
         const float4 a = *reinterpret_cast<const float4*>(p + i);
@@ -215,17 +224,20 @@ template <int S, int DW, int ESIZE = 4> struct TmaShift {
 #ifndef TCONV_MINB_SINGLE
 #define TCONV_MINB_SINGLE 4
 #endif
+#ifndef TCONV_MINB_WINSUM
+#define TCONV_MINB_WINSUM 3
+#endif
 #ifndef TCONV_Q_CARRIED
 #define TCONV_Q_CARRIED 2
 #endif
 template <int MODE, int CHAN, bool WIN, bool XTMA, int R, int S, int SW, int DW, int Q, int KG, int PW, int TK>
 __global__ void __launch_bounds__(KG * PW * 32,
-                                  (WIN && CHAN == CH_SUM) ? 3
+                                  (WIN && CHAN == CH_SUM) ? TCONV_MINB_WINSUM
                                   : WIN ? 1
                                   : (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL) ? (TK == 4 ? 4 : 1)
                                   : TCONV_MINB_SINGLE)
 fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams p) {
-    static_assert(TK == 4 || TK == 8, "output channels per thread");
+    static_assert(TK == 2 || TK == 4 || TK == 8, "output channels per thread");
     constexpr int RS = R * S;
     constexpr int TILE_K = KG * TK;
     constexpr int NT = KG * PW * 32;
@@ -379,6 +391,17 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
             }
 
     const size_t plane = (size_t)g.OH * g.OW;
+    // Sum forms with winners: where this thread's codes of (its first output channel, input channel 0) go
+    uint8_t* code_base[Q];
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+        code_base[q] = nullptr;
+        if (WIN && CHAN == CH_SUM && out_row[q] >= 0) {
+            const int n = out_row[q] / g.OH, oh = out_row[q] - n * g.OH;
+            code_base[q] = reinterpret_cast<uint8_t*>(p.winners) +
+                           ((size_t)n * g.K + (size_t)kt * TILE_K) * g.C * plane + (size_t)oh * g.OW + qcol[q];
+        }
+    }
     const int row_step = g.dh * p.XP;
     const int chan_step = p.NSLOTS * p.XP;
     issue_chunk(0, 0);
@@ -415,6 +438,121 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
             const float* wc = ws + cc * (RS * TILE_K);
             const float* wc2 = ws2 + cc * (RS * TILE_K);
 
+            if constexpr (WIN && CHAN == CH_SUM) {
+                // Sum forms that emit winners.  Per pair of output channels and per pixel the RS tap
+                // sums stay in registers, feed the extrema, and then give the winning taps on the
+                // FMA pipe: with m the exact extremum, d = (t - m) * 2^32 is computed with one
+                // rounding and is zero exactly for the taps that attain m;
+                // key = |d| * (-2^125) + (2^23 + rank(tap)) equals 2^23 + rank for those taps and is
+                // below 2^23 for every other tap, so the largest key belongs to the lowest winning
+                // tap when rank decreases with the tap, and the low mantissa bits of that key are
+                // rank itself: 15 - tap for the min branch (low nibble of the code), 16 * (15 - tap)
+                // for the max branch (high nibble), both read back with one complement-and-mask.
+                // (a non-zero |d| * 2^125 is at least 256 > 240, the largest rank; |x + w| < 2^95 is assumed.)
+                constexpr float kS = 4294967296.0f;          // 2^32
+                constexpr float kH = 4.253529586511731e37f;  // 2^125
+                constexpr float kB = 8388608.0f;             // 2^23
+                constexpr bool DO_MIN = TWO || TAP_MIN, DO_MAX = TWO || !TAP_MIN;
+                const int c = ch * p.CC + cc;
+                float av[TK], bv[TK];
+                if constexpr (TWO) {
+                    loadn<TK>(as + cc * TILE_K, av);
+                    loadn<TK>(bs + cc * TILE_K, bv);
+                }
+#pragma unroll
+                for (int kp = 0; kp < TK / 2; ++kp) {
+                    float wa[RS][2], wb[PAR ? RS : 1][2];
+#pragma unroll
+                    for (int tap = 0; tap < RS; ++tap) {
+                        loadn<2>(wc + tap * TILE_K + 2 * kp, wa[tap]);
+                        if constexpr (PAR) loadn<2>(wc2 + tap * TILE_K + 2 * kp, wb[tap]);
+                    }
+#pragma unroll
+                    for (int q = 0; q < Q; ++q) {
+                        unsigned packed[2] = {0u, 0u};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            float ta[RS][2], tb[PAR ? RS : 1][2];
+#pragma unroll
+                            for (int tap = 0; tap < RS; ++tap) {
+                                const float xv = xr[q][tap / S][j * SW + (tap % S) * DW];
+                                add2(xv, wa[tap][0], wa[tap][1], ta[tap][0], ta[tap][1]);
+                                if constexpr (PAR) add2(xv, wb[tap][0], wb[tap][1], tb[tap][0], tb[tap][1]);
+                            }
+                            const float (*tm)[2] = PAR ? tb : ta;   // sums of the max branch
+                            unsigned bits_min[2] = {0u, 0u}, bits_max[2] = {0u, 0u};
+                            float lo[2] = {0.0f, 0.0f}, hi[2] = {0.0f, 0.0f};
+                            if constexpr (DO_MIN) {
+                                lo[0] = fold_taps<RS>(ta, 0, true);
+                                lo[1] = fold_taps<RS>(ta, 1, true);
+                            }
+                            if constexpr (DO_MAX) {
+                                hi[0] = fold_taps<RS>(tm, 0, false);
+                                hi[1] = fold_taps<RS>(tm, 1, false);
+                            }
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                float& a = acc[2 * kp + h][q][j];
+                                if constexpr (TWO) {
+                                    a = __fmaf_rn(av[2 * kp + h], lo[h], a);
+                                    a = __fmaf_rn(bv[2 * kp + h], hi[h], a);
+                                } else {
+                                    a = __fadd_rn(a, TAP_MIN ? lo[h] : hi[h]);
+                                }
+                            }
+                            if constexpr (DO_MIN) {
+                                const float e0 = -lo[0] * kS, e1 = -lo[1] * kS;
+                                float key[RS][2];
+#pragma unroll
+                                for (int tap = 0; tap < RS; ++tap) {
+                                    float d0 = e0, d1 = e1;
+                                    fma2s(kS, ta[tap][0], ta[tap][1], d0, d1);             // >= 0
+                                    key[tap][0] = key[tap][1] = kB + (float)(15 - tap);
+                                    fma2s(-kH, d0, d1, key[tap][0], key[tap][1]);
+                                }
+                                bits_min[0] = __float_as_uint(fold_taps<RS>(key, 0, false));
+                                bits_min[1] = __float_as_uint(fold_taps<RS>(key, 1, false));
+                            }
+                            if constexpr (DO_MAX) {
+                                const float e0 = -hi[0] * kS, e1 = -hi[1] * kS;
+                                float key[RS][2];
+#pragma unroll
+                                for (int tap = 0; tap < RS; ++tap) {
+                                    float d0 = e0, d1 = e1;
+                                    fma2s(kS, tm[tap][0], tm[tap][1], d0, d1);             // <= 0
+                                    key[tap][0] = key[tap][1] = kB + (float)(16 * (15 - tap));
+                                    fma2s(kH, d0, d1, key[tap][0], key[tap][1]);
+                                }
+                                bits_max[0] = __float_as_uint(fold_taps<RS>(key, 0, false));
+                                bits_max[1] = __float_as_uint(fold_taps<RS>(key, 1, false));
+                            }
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                unsigned code;
+                                if constexpr (TWO) code = (~bits_min[h] & 0x0fu) | (~bits_max[h] & 0xf0u);
+                                else code = TAP_MIN ? (~bits_min[h] & 0x0fu) : (~bits_max[h] & 0xf0u);
+                                packed[h] |= code << (8 * j);
+                            }
+                        }
+                        // one byte per (n, k, c, oh, ow): low nibble argmin tap, high nibble argmax tap
+                        if (out_row[q] >= 0) {
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const int kl = kg * TK + 2 * kp + h;
+                                if (kt * TILE_K + kl >= g.K) continue;
+                                uint8_t* dst = code_base[q] + ((size_t)kl * g.C + c) * plane;
+                                if (qcol[q] + 3 < g.OW && ((g.OW & 3) == 0)) {
+                                    *reinterpret_cast<unsigned*>(dst) = packed[h];
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j)
+                                        if (qcol[q] + j < g.OW) dst[j] = (uint8_t)(packed[h] >> (8 * j));
+                                }
+                            }
+                        }
+                    }
+                }
+            } else {
             float mx[CARRIED ? 1 : TK][Q][4];           // per-channel extremum (max branch / single branch)
             float mn[TWO ? TK : 1][Q][4];               // per-channel minimum (two-branch modes)
 
@@ -516,128 +654,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                                 acc[k][q][j] = ext2(acc[k][q][j], mx[k][q][j], CHAN == CH_MIN);
                             }
                         }
-                if constexpr (WIN && CHAN == CH_SUM) {
-                    // Winning taps, recovered on the FMA pipe.  With m the exact extremum of the
-                    // channel, d = (t - m) * 2^30 is computed with one rounding and is zero exactly for
-                    // the taps that attain m; key = |d| * (-2^125) + (RS - tap) is RS - tap for those
-                    // taps and hugely negative otherwise, so the maximum key belongs to the lowest
-                    // winning tap.  The sums t are the same rounded adds as in the first pass; the
-                    // extrema have been folded into acc above and are rescaled in place.
-                    // (|x + w| < 2^97 is assumed.)
-                    constexpr float kS = 1073741824.0f;                 // 2^30
-                    constexpr float kH = 4.253529586511731e37f;         // 2^125
-                    float kmn[TWO ? TK : 1][Q][4], kmx[TK][Q][4];
-#pragma unroll
-                    for (int k = 0; k < TK; ++k)
-#pragma unroll
-                        for (int q = 0; q < Q; ++q)
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                mx[k][q][j] = -mx[k][q][j] * kS;
-                                if constexpr (TWO) mn[k][q][j] = -mn[k][q][j] * kS;
-                            }
-                    constexpr int FIRST2 = (RS >= 3 ? 3 : RS);
-                    constexpr int NG2 = 1 + (RS - FIRST2 + 1) / 2;
-#pragma unroll
-                    for (int gi = 0; gi < NG2; ++gi) {
-                        const int t0 = (gi == 0) ? 0 : FIRST2 + 2 * (gi - 1);
-                        const int nt = (gi == 0) ? (FIRST2 < RS ? FIRST2 : RS) : ((RS - t0) < 2 ? (RS - t0) : 2);
-                        float wv[3][TK], wv2[PAR ? 3 : 1][TK];
-#pragma unroll
-                        for (int u = 0; u < 3; ++u)
-                            if (u < nt) {
-                                loadn<TK>(wc + (t0 + u) * TILE_K, wv[u]);
-                                if constexpr (PAR) loadn<TK>(wc2 + (t0 + u) * TILE_K, wv2[u]);
-                            }
-#pragma unroll
-                        for (int q = 0; q < Q; ++q)
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                float xv[3];
-#pragma unroll
-                                for (int u = 0; u < 3; ++u)
-                                    if (u < nt) {
-                                        const int tap = t0 + u;
-                                        xv[u] = xr[q][tap / S][j * SW + (tap % S) * DW];
-                                    }
-#pragma unroll
-                                for (int kp = 0; kp < TK / 2; ++kp) {
-                                    float ka[3][2], kb[3][2];   // keys of the min branch / max branch
-#pragma unroll
-                                    for (int u = 0; u < 3; ++u)
-                                        if (u < nt) {
-                                            const float rank = (float)(RS - (t0 + u));
-                                            float ta0, ta1, tb0, tb1;
-                                            add2_again(xv[u], wv[u][2 * kp], wv[u][2 * kp + 1], ta0, ta1);
-                                            if constexpr (PAR) add2_again(xv[u], wv2[u][2 * kp], wv2[u][2 * kp + 1], tb0, tb1);
-                                            else { tb0 = ta0; tb1 = ta1; }
-                                            if constexpr (TWO) {
-                                                float d0 = mn[2 * kp][q][j], d1 = mn[2 * kp + 1][q][j];
-                                                fma2s(kS, ta0, ta1, d0, d1);            // >= 0
-                                                ka[u][0] = rank; ka[u][1] = rank;
-                                                fma2s(-kH, d0, d1, ka[u][0], ka[u][1]);
-                                                float e0 = mx[2 * kp][q][j], e1 = mx[2 * kp + 1][q][j];
-                                                fma2s(kS, tb0, tb1, e0, e1);            // <= 0
-                                                kb[u][0] = rank; kb[u][1] = rank;
-                                                fma2s(kH, e0, e1, kb[u][0], kb[u][1]);
-                                            } else {
-                                                float e0 = mx[2 * kp][q][j], e1 = mx[2 * kp + 1][q][j];
-                                                fma2s(kS, ta0, ta1, e0, e1);
-                                                kb[u][0] = rank; kb[u][1] = rank;
-                                                fma2s(TAP_MIN ? -kH : kH, e0, e1, kb[u][0], kb[u][1]);
-                                            }
-                                        }
-#pragma unroll
-                                    for (int h = 0; h < 2; ++h) {
-                                        const int k = 2 * kp + h;
-                                        if (gi == 0) {
-                                            kmx[k][q][j] = nt == 3 ? ext3(kb[0][h], kb[1][h], kb[2][h], false)
-                                                           : nt == 2 ? ext2(kb[0][h], kb[1][h], false) : kb[0][h];
-                                            if constexpr (TWO)
-                                                kmn[k][q][j] = nt == 3 ? ext3(ka[0][h], ka[1][h], ka[2][h], false)
-                                                               : nt == 2 ? ext2(ka[0][h], ka[1][h], false) : ka[0][h];
-                                        } else {
-                                            kmx[k][q][j] = nt == 2 ? ext3(kmx[k][q][j], kb[0][h], kb[1][h], false)
-                                                                   : ext2(kmx[k][q][j], kb[0][h], false);
-                                            if constexpr (TWO)
-                                                kmn[k][q][j] = nt == 2 ? ext3(kmn[k][q][j], ka[0][h], ka[1][h], false)
-                                                                       : ext2(kmn[k][q][j], ka[0][h], false);
-                                        }
-                                    }
-                                }
-                            }
-                    }
-                    // one byte per (n, k, c, oh, ow): low nibble argmin tap, high nibble argmax tap
-                    uint8_t* codes = reinterpret_cast<uint8_t*>(p.winners);
-#pragma unroll
-                    for (int q = 0; q < Q; ++q) {
-                        if (out_row[q] < 0) continue;
-                        const int n = out_row[q] / g.OH, oh = out_row[q] - n * g.OH;
-#pragma unroll
-                        for (int k = 0; k < TK; ++k) {
-                            const int kk = kt * TILE_K + kg * TK + k;
-                            if (kk >= g.K) continue;
-                            uint8_t* dst = codes + (((size_t)n * g.K + kk) * g.C + c) * plane +
-                                           (size_t)oh * g.OW + qcol[q];
-                            unsigned packed = 0;
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const unsigned tmax = (unsigned)(RS - __float2int_rn(kmx[k][q][j]));
-                                unsigned code;
-                                if constexpr (TWO) code = (unsigned)(RS - __float2int_rn(kmn[k][q][j])) | (tmax << 4);
-                                else code = TAP_MIN ? tmax : (tmax << 4);
-                                packed |= code << (8 * j);
-                            }
-                            if (qcol[q] + 3 < g.OW && ((g.OW & 3) == 0)) {
-                                *reinterpret_cast<unsigned*>(dst) = packed;
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 4; ++j)
-                                    if (qcol[q] + j < g.OW) dst[j] = (uint8_t)(packed >> (8 * j));
-                            }
-                        }
-                    }
-                }
+            }
             }
         }
         __syncthreads();  // every thread is done with this stage before it is refilled
@@ -875,13 +892,16 @@ int launch_tiled_geom(FwdArgs& a) {
     constexpr bool CARRIED = !TWO && !WIN && ((MODE == TCONV_MAX_PLUS && CHAN == CH_MAX) ||
                                               (MODE == TCONV_MIN_PLUS && CHAN == CH_MIN));
     constexpr int Q = CARRIED ? TCONV_Q_CARRIED : 1;
-    // the winner pass of the Sum forms keeps two extra values per output: 4 channels per thread
-    // two-branch kernels keep three values per output: 4 channels per thread leave room for
+    // Sum forms that emit winners work on one pair of output channels at a time: 4 channels per
+    // thread (2 or 8 measured no faster); two-branch kernels keep three values per output: 4 channels per thread leave room for
     // four resident CTAs per SM (measured 3-6 % faster than 8 channels per thread)
 #ifndef TCONV_TK_TWO
 #define TCONV_TK_TWO 4
 #endif
-    constexpr int TK = (WIN && CHAN == CH_SUM) ? 4 : (TWO ? TCONV_TK_TWO : 8);
+#ifndef TCONV_TK_WINSUM
+#define TCONV_TK_WINSUM 4
+#endif
+    constexpr int TK = (WIN && CHAN == CH_SUM) ? TCONV_TK_WINSUM : (TWO ? TCONV_TK_TWO : 8);
     const Geo& g = a.g;
     if (g.R == 3 && g.S == 3) {
         if (g.sw == 1 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 1, Q, 4, 1, TK>(a);
