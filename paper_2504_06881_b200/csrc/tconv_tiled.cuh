@@ -135,12 +135,12 @@ __device__ __forceinline__ void loadn(const float* p, float* out) {
     if constexpr (N == 2) {
         const float2 a = *reinterpret_cast<const float2*>(p);
         out[0] = a.x; out[1] = a.y;
-        return;
-    }
+    } else {
 #pragma unroll
-    for (int i = 0; i < N; i += 4) {
-        const float4 a = *reinterpret_cast<const float4*>(p + i);
-        out[i] = a.x; out[i + 1] = a.y; out[i + 2] = a.z; out[i + 3] = a.w;
+        for (int i = 0; i < N; i += 4) {
+            const float4 a = *reinterpret_cast<const float4*>(p + i);
+            out[i] = a.x; out[i + 1] = a.y; out[i + 2] = a.z; out[i + 3] = a.w;
+        }
     }
 }
 __device__ __forceinline__ void load8(const float* p, float* out) {
@@ -787,6 +787,8 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* p
     p.ab_stage = two ? p.CC * TILE_K : 0;
     p.stage_floats = p.x_stage + p.w_stage * (par ? 2 : 1) + 2 * p.ab_stage;
     pl->smem = 2 * (size_t)p.stage_floats * sizeof(float) + 16 + (size_t)p.NSLOTS * sizeof(int) + 16;
+    // 2-byte elements without TMA: a table of source offsets for one channel plane of the tile
+    if (!pl->xtma && esize == 2) pl->smem += ((size_t)p.NSLOTS * p.XP + 4) * sizeof(int);
     if (pl->smem > 200 * 1024) return false;
     const int nkt = (g.K + TILE_K - 1) / TILE_K;
     pl->grid = dim3((unsigned)(p.n_col_tiles * p.n_row_tiles), (unsigned)nkt, 1);

@@ -144,6 +144,7 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
     unsigned* stage0 = reinterpret_cast<unsigned*>(smem_raw);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(stage0 + 2 * p.stage_floats);
     int* slot_off = reinterpret_cast<int*>(bars + 2);
+    int* src_tab = slot_off + ((p.NSLOTS + 3) & ~3);   // staging table of the non-TMA path
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int kg = warp % KG, wp = warp / KG;
@@ -182,6 +183,14 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
             const int ih = oh * g.sh - g.ph + dr;
             const int sl = lr * g.sh + (n - n0) * p.GAP + dr;
             if (ih >= 0 && ih < g.H) slot_off[sl] = (n * g.C * g.H + ih) * g.W;
+        }
+        __syncthreads();
+        // element offsets inside x (channel 0 of the tile's first image row space), -1 = zero
+        for (int i = tid; i < p.NSLOTS * p.XP; i += NT) {
+            const int sl = i / p.XP, col = i - sl * p.XP;
+            const int iw = iw0 + col;
+            const int off = slot_off[sl];
+            src_tab[i] = (off >= 0 && iw >= 0 && iw < g.W) ? off + iw : -1;
         }
     }
     __syncthreads();
@@ -230,23 +239,20 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                 }
             }
         } else {
-            // x halo tile by plain 2-byte loads (rows are not 16-byte multiples here)
+            // x halo tile by plain 2-byte loads (rows are not 16-byte multiples here): the source
+            // offset of every element of one channel plane comes from a table built once per CTA,
+            // and the loads of the chunk's channels are issued together before any is stored
             unsigned short* xs = reinterpret_cast<unsigned short*>(st);
-            for (int cc = 0; cc < p.CC; ++cc) {
-                const bool cok = (c0 + cc < g.C);
-                const unsigned short* src_c = xg + (size_t)(cok ? c0 + cc : 0) * chw;
-                unsigned short* dst_c = xs + (size_t)cc * p.NSLOTS * p.XP;
-                for (int sl = warp; sl < p.NSLOTS; sl += NWARPS) {
-                    const int off = slot_off[sl];
-                    const bool rok = cok && (off >= 0);
-                    const unsigned short* src_row = src_c + (rok ? off : 0);
-                    unsigned short* dst_row = dst_c + sl * p.XP;
-                    for (int col = lane; col < p.XP; col += 32) {
-                        const int iw = iw0 + col;
-                        const bool ok = rok && iw >= 0 && iw < g.W;
-                        dst_row[col] = ok ? src_row[iw] : (unsigned short)0;
-                    }
-                }
+            const int per_c = p.NSLOTS * p.XP;
+            for (int i = tid; i < per_c; i += NT) {
+                const int so = src_tab[i];
+                unsigned short v[8];
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc)
+                    v[cc] = (so >= 0 && cc < p.CC && c0 + cc < g.C) ? xg[(size_t)(c0 + cc) * chw + so] : (unsigned short)0;
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc)
+                    if (cc < p.CC) xs[cc * per_c + i] = v[cc];
             }
             const unsigned* wsrc = wt_k + (size_t)c0 * RS * TILE_K;
             for (int e = tid; e < p.w_stage / 4; e += NT) cp_async16(st + w_off + e * 4, wsrc + e * 4);
