@@ -45,6 +45,8 @@ PROBES = {"max_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
           "min_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
           "compound": ("f32_add_minmax2", "f32_add_minmax3", "f32_add2_minmax3"),
           "parallel": ("f32_2add_minmax2", "f32_2add_minmax3", "f32_2add2_minmax3")}
+# register-only probes of the winner-emitting Sum-form inner loop (sums, extrema, FMA keys, key fold)
+WIN_PROBES = {"compound": "f32_win_compound", "parallel": "f32_win_parallel"}
 
 
 def layer_ops(d):
@@ -358,15 +360,21 @@ def run_gpu(args):
                              key=lambda mw: per[mw[0]][mw[1]])
     L = next(x for x in layers if x.d["mode"] == dom_mode)
     achieved = L.taps / (per[dom_mode][dom_what] * 1e-3) / 1e12
+    win_mix = dom_what == "fwd_winners" and dom_mode in WIN_PROBES
+    peak = probe_rates[WIN_PROBES[dom_mode]] if win_mix else peaks[dom_mode]
     roofline = {"bound": "alu", "kernel": per[dom_mode][dom_what + "_kernel"], "call": f"{dom_mode} {dom_what}",
-                "achieved": achieved, "peak": peaks[dom_mode] / 1e12, "unit": "Ttap/s",
-                "frac": achieved / (peaks[dom_mode] / 1e12),
+                "achieved": achieved, "peak": peak / 1e12, "unit": "Ttap/s",
+                "frac": achieved / (peak / 1e12),
                 "traffic": (4 * DRAM_BYTES_N32[(dom_mode, dom_what)]
                             if (dom_mode, dom_what) in DRAM_BYTES_N32 else None),
                 "traffic_note": "DRAM bytes per launch, ncu capture at N=32 scaled x4 (see profiles/)",
-                "peak_source": "measured in this run: best register-only add+max/min probe of the mode "
-                               "(taps/s of the winner-free instruction mix; a winner-emitting or backward "
-                               "kernel does more work per tap than that mix)"}
+                "peak_source": ("measured in this run: register-only probe of the winner-emitting inner loop of "
+                                "the mode (tap sums, extrema, two fused multiply-adds per tap and branch for "
+                                "the winner keys, key fold)" if win_mix else
+                                "measured in this run: best register-only add+max/min probe of the mode "
+                                "(taps/s of the winner-free instruction mix; a backward kernel does other "
+                                "work per tap than that mix)"),
+                "frac_of_winner_free_peak": achieved / (peaks[dom_mode] / 1e12)}
     fwd_frac = {m: {"ms": per[m]["fwd"], "Ttap_s": L2.taps / (per[m]["fwd"] * 1e-3) / 1e12,
                     "frac_of_alu_peak": L2.taps / (per[m]["fwd"] * 1e-3) / peaks[m],
                     "kernel": per[m]["fwd_kernel"]}

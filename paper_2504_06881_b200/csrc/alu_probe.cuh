@@ -21,6 +21,20 @@ __device__ __forceinline__ float min3f(float a, float b, float c) {
     asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
+// {c0, c1} = a * {v0, v1} + {c0, c1}: one packed fused multiply-add
+__device__ __forceinline__ void fma2f(float a, float v0, float v1, float& c0, float& c1) {
+    unsigned long long aa, vv, cc;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(aa) : "f"(a));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(vv) : "f"(v0), "f"(v1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(cc) : "f"(c0), "f"(c1));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(cc) : "l"(aa), "l"(vv));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(c0), "=f"(c1) : "l"(cc));
+}
+// extremum of nine values with a 3-input chain (3 + 2 + 2 + 2)
+__device__ __forceinline__ float fold9(const float (*v)[2], int h, bool is_min) {
+    if (is_min) return min3f(min3f(min3f(min3f(v[0][h], v[1][h], v[2][h]), v[3][h], v[4][h]), v[5][h], v[6][h]), v[7][h], v[8][h]);
+    return max3f(max3f(max3f(max3f(v[0][h], v[1][h], v[2][h]), v[3][h], v[4][h]), v[5][h], v[6][h]), v[7][h], v[8][h]);
+}
 // Packed fp32 add: {lo, hi} = {x + wlo, x + whi}, one instruction for two taps.
 __device__ __forceinline__ void add2f(float x, float wlo, float whi, float& lo, float& hi) {
     unsigned long long xx, ww, tt;
@@ -46,6 +60,9 @@ enum {
     PROBE_F32_ADD_ONLY,          // adds alone (sum-reduced), the FP32 pipe by itself
     PROBE_F32_MAX2_ONLY,         // 2-input max alone
     PROBE_F32_MAX3_ONLY,         // 3-input max alone
+    PROBE_F32_WIN_SINGLE,        // Sum form with winners, one branch: sums, extremum, FMA keys, key fold
+    PROBE_F32_WIN_COMPOUND,      // the same for compound (shared sums, two branches)
+    PROBE_F32_WIN_PARALLEL,      // the same for parallel (two sets of sums)
     PROBE_COUNT
 };
 
@@ -53,7 +70,8 @@ static const char* const kProbeNames[PROBE_COUNT] = {
     "f32_add_max2",       "f32_add_max3",      "f32_add2_max3",   "f32_add_minmax2",
     "f32_add_minmax3",    "f32_add2_minmax3",  "f32_2add_minmax2", "f32_2add_minmax3",
     "f32_2add2_minmax3",  "bf16x2_add_max",    "bf16x2_add_minmax", "bf16x2_2add_minmax",
-    "f32_add_only",       "f32_max2_only",     "f32_max3_only"};
+    "f32_add_only",       "f32_max2_only",     "f32_max3_only",   "f32_win_single",
+    "f32_win_compound",   "f32_win_parallel"};
 
 // Taps folded per thread per loop iteration, by variant (must match the kernel).
 __host__ inline int probe_taps_per_iter(int v) {
@@ -61,6 +79,9 @@ __host__ inline int probe_taps_per_iter(int v) {
         case PROBE_BF16X2_ADD_MAX:
         case PROBE_BF16X2_ADD_MINMAX:
         case PROBE_BF16X2_2ADD_MINMAX: return 4 * 8 * 2 * 2;  // 4 channel pairs x 8 pixels x 2 lanes x 2 taps
+        case PROBE_F32_WIN_SINGLE:
+        case PROBE_F32_WIN_COMPOUND:
+        case PROBE_F32_WIN_PARALLEL: return 4 * 4 * 9;        // 4 channels x 4 pixels x a 3x3 window
         default: return 8 * 4 * 2;                            // 8 channels x 4 pixels x 2 taps
     }
 }
@@ -118,6 +139,95 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
         for (int i = 0; i < KP; ++i)
             for (int j = 0; j < PX; ++j) r = __hadd2(r, __hadd2(mx[i][j], mn[i][j]));
         if (__low2float(r) == 12345.678f) sink[0] = __high2float(r);
+    } else if constexpr (V == PROBE_F32_WIN_SINGLE || V == PROBE_F32_WIN_COMPOUND || V == PROBE_F32_WIN_PARALLEL) {
+        // The winner-emitting Sum-form inner loop on registers only: per pair of output channels
+        // and pixel, nine packed tap sums, their extrema, the channel combine, two packed fused
+        // multiply-adds per tap and branch for the keys, the key fold and the code byte.
+        constexpr bool TWOB = (V != PROBE_F32_WIN_SINGLE), PARB = (V == PROBE_F32_WIN_PARALLEL);
+        constexpr float kS = 4294967296.0f, kH = 4.253529586511731e37f, kB = 8388608.0f;
+        float x[12], wa[2][9][2], wb[PARB ? 2 : 1][9][2], acc[4][4], al[4], be[4];
+        unsigned codes = 0u;
+        const float dx = seed * 1.0e-3f;
+        for (int j = 0; j < 12; ++j) x[j] = seed * (float)(j + threadIdx.x);
+        for (int kp = 0; kp < 2; ++kp)
+            for (int t = 0; t < 9; ++t)
+                for (int h = 0; h < 2; ++h) {
+                    wa[kp][t][h] = seed * (float)(kp * 18 + t * 2 + h + 3);
+                    if (PARB) wb[kp][t][h] = seed * (float)(kp * 18 + t * 2 + h + 5);
+                }
+        for (int k = 0; k < 4; ++k) {
+            al[k] = seed * (float)(k + 1); be[k] = seed * (float)(k + 2);
+            for (int j = 0; j < 4; ++j) acc[k][j] = 0.0f;
+        }
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int j = 0; j < 12; ++j) x[j] = __fadd_rn(x[j], dx);     // operands change every iteration
+#pragma unroll
+            for (int kp = 0; kp < 2; ++kp)
+#pragma unroll
+                for (int t = 0; t < 9; ++t) {
+                    TCONV_OPAQUE_F(wa[kp][t][0]); TCONV_OPAQUE_F(wa[kp][t][1]);
+                    if constexpr (PARB) { TCONV_OPAQUE_F(wb[kp][t][0]); TCONV_OPAQUE_F(wb[kp][t][1]); }
+                }
+#pragma unroll
+            for (int kp = 0; kp < 2; ++kp)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float ta[9][2], tb[PARB ? 9 : 1][2];
+#pragma unroll
+                    for (int t = 0; t < 9; ++t) {
+                        add2f(x[j + t], wa[kp][t][0], wa[kp][t][1], ta[t][0], ta[t][1]);
+                        if constexpr (PARB) add2f(x[j + t], wb[kp][t][0], wb[kp][t][1], tb[t][0], tb[t][1]);
+                    }
+                    const float (*tm)[2] = PARB ? tb : ta;
+                    float lo[2] = {0.0f, 0.0f}, hi[2];
+                    unsigned bmn[2] = {0u, 0u}, bmx[2];
+                    hi[0] = fold9(tm, 0, false); hi[1] = fold9(tm, 1, false);
+                    if constexpr (TWOB) { lo[0] = fold9(ta, 0, true); lo[1] = fold9(ta, 1, true); }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if constexpr (TWOB) {
+                            acc[2 * kp + h][j] = __fmaf_rn(al[2 * kp + h], lo[h], acc[2 * kp + h][j]);
+                            acc[2 * kp + h][j] = __fmaf_rn(be[2 * kp + h], hi[h], acc[2 * kp + h][j]);
+                        } else {
+                            acc[2 * kp + h][j] = __fadd_rn(acc[2 * kp + h][j], hi[h]);
+                        }
+                    }
+                    if constexpr (TWOB) {
+                        const float e0 = -lo[0] * kS, e1 = -lo[1] * kS;
+                        float key[9][2];
+#pragma unroll
+                        for (int t = 0; t < 9; ++t) {
+                            float d0 = e0, d1 = e1;
+                            fma2f(kS, ta[t][0], ta[t][1], d0, d1);
+                            key[t][0] = key[t][1] = kB + (float)(15 - t);
+                            fma2f(-kH, d0, d1, key[t][0], key[t][1]);
+                        }
+                        bmn[0] = __float_as_uint(fold9(key, 0, false));
+                        bmn[1] = __float_as_uint(fold9(key, 1, false));
+                    }
+                    {
+                        const float e0 = -hi[0] * kS, e1 = -hi[1] * kS;
+                        float key[9][2];
+#pragma unroll
+                        for (int t = 0; t < 9; ++t) {
+                            float d0 = e0, d1 = e1;
+                            fma2f(kS, tm[t][0], tm[t][1], d0, d1);
+                            key[t][0] = key[t][1] = kB + (float)(16 * (15 - t));
+                            fma2f(kH, d0, d1, key[t][0], key[t][1]);
+                        }
+                        bmx[0] = __float_as_uint(fold9(key, 0, false));
+                        bmx[1] = __float_as_uint(fold9(key, 1, false));
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        codes ^= ((~bmn[h] & 0x0fu) | (~bmx[h] & 0xf0u)) << (8 * j);
+                }
+        }
+        float r = __uint_as_float(codes);
+        for (int k = 0; k < 4; ++k)
+            for (int j = 0; j < 4; ++j) r += acc[k][j];
+        if (r == 12345.678f) sink[0] = r;
     } else {
         float x[TP + 1], w0[TK], w1[TK], v0[TK], v1[TK];
         float mn[TK][TP], mx[TK][TP];

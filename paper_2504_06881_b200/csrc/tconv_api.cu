@@ -451,7 +451,8 @@ int tconv_alu_probe(int variant, int iters, void* sink, double* taps_per_launch,
         TCONV_PROBE_CASE(0) TCONV_PROBE_CASE(1) TCONV_PROBE_CASE(2) TCONV_PROBE_CASE(3)
         TCONV_PROBE_CASE(4) TCONV_PROBE_CASE(5) TCONV_PROBE_CASE(6) TCONV_PROBE_CASE(7)
         TCONV_PROBE_CASE(8) TCONV_PROBE_CASE(9) TCONV_PROBE_CASE(10) TCONV_PROBE_CASE(11)
-        TCONV_PROBE_CASE(12) TCONV_PROBE_CASE(13) TCONV_PROBE_CASE(14)
+        TCONV_PROBE_CASE(12) TCONV_PROBE_CASE(13) TCONV_PROBE_CASE(14) TCONV_PROBE_CASE(15)
+        TCONV_PROBE_CASE(16) TCONV_PROBE_CASE(17)
     }
 #undef TCONV_PROBE_CASE
     g_launches += 1;
