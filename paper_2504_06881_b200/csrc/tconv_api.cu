@@ -227,17 +227,20 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
         CodeGxPlan pl;
         if (gx) {
             if (tiled && plan_code_gx(g, &pl)) {
-                const dim3 grid((unsigned)(((g.N + pl.imgs - 1) / pl.imgs) * pl.tiles_per_img),
-                                (unsigned)((g.C + pl.CB - 1) / pl.CB));
-#define TCONV_GXM(BR, CBV, VECV, MULTI)                                                              \
+                const dim3 grid(pl.grid);
+#define TCONV_GXM(BR, CBV, VECV, MULTI, NTH)                                                         \
     {                                                                                                \
-        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV, MULTI>;                                     \
+        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV, MULTI, NTH>;                                \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
-        kern<<<grid, 256, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);          \
+        kern<<<grid, pl.threads, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);   \
     }
 #define TCONV_GX(BR, CBV, VECV)                                                                      \
-    { if (pl.imgs > 1) TCONV_GXM(BR, CBV, VECV, true) else TCONV_GXM(BR, CBV, VECV, false) }
+    {                                                                                                \
+        if (pl.imgs > 1) TCONV_GXM(BR, CBV, VECV, true, 256)                                         \
+        else if (pl.threads > 256) TCONV_GXM(BR, CBV, VECV, false, 1024)                             \
+        else TCONV_GXM(BR, CBV, VECV, false, 256)                                                    \
+    }
 #define TCONV_GX2(BR)                                                                                \
     {                                                                                                \
         if (pl.CB == 2) { if (vec) TCONV_GX(BR, 2, true) else TCONV_GX(BR, 2, false) }               \

@@ -233,6 +233,9 @@ struct CodeGxPlan {
     int THI, tiles_per_img;  // owned input rows per CTA
     int CB;                  // channels per CTA
     int NRmax, QPR, NQpad;   // contributing output rows (max), quads per row, padded quad count
+    int threads;             // CTA size: 256, or more where the tile leaves room for only 1-2 CTAs per SM
+    int ncblk;               // channel blocks (the fastest-varying part of the CTA index)
+    unsigned grid;           // CTAs: image groups x row bands x channel blocks
     size_t smem;
 };
 
@@ -271,18 +274,21 @@ __device__ __forceinline__ unsigned load_c4(const uint8_t* p, int ow0, int OW) {
 // CB channels per CTA (the CTA's last channel block may hold fewer: those lanes idle).
 // VEC: OW is a multiple of 4 (aligned vector loads of grad_y and of the codes).
 // MULTI: the CTA owns pl.imgs whole images (small maps); else one band of rows of one image.
-template <typename T, int BR, int CB, bool VEC, bool MULTI>
-__global__ void __launch_bounds__(256)
+// NTH: upper bound of the CTA size (256, or 1024 for tiles that leave room for one or two CTAs per SM).
+template <typename T, int BR, int CB, bool VEC, bool MULTI, int NTH>
+__global__ void __launch_bounds__(NTH)
 bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
                    CodeGxPlan pl) {
     extern __shared__ float A[];  // [CB][RS][4][NQpad], then alpha / beta of this CTA's channels [K][CB] each
     // a CTA owns either a band of input rows of one image or pl.imgs whole images of a small map;
     // its output quads are numbered image by image
-    const int tile_i = blockIdx.x % pl.tiles_per_img;
-    const int n_first = MULTI ? (blockIdx.x / pl.tiles_per_img) * pl.imgs : blockIdx.x / pl.tiles_per_img;
+    // channel blocks vary fastest over the grid: CTAs that run together share one band of grad_y
+    const int cblk = blockIdx.x % pl.ncblk, xt = blockIdx.x / pl.ncblk;
+    const int tile_i = xt % pl.tiles_per_img;
+    const int n_first = MULTI ? (xt / pl.tiles_per_img) * pl.imgs : xt / pl.tiles_per_img;
     const int nimg = MULTI ? min(pl.imgs, g.N - n_first) : 1;
-    const int c0 = blockIdx.y * CB;
+    const int c0 = cblk * CB;
     const int ncb = min(CB, g.C - c0);
     const int ih0 = tile_i * pl.THI;
     const int rows = min(pl.THI, g.H - ih0);
@@ -326,58 +332,68 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
             cp[cb] = codes + ((size_t)n * g.K * g.C + c) * plane + pix;
             Ab[cb] = reinterpret_cast<char*>(A + (size_t)cb * g.RS * 4 * NQp + q);
         }
-        float gv_cur[4], gv_nxt[4];
-        unsigned cw_cur[CB], cw_nxt[CB];
-        load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
+        // operands of output channel k + PF are requested while channel k is consumed
+        constexpr int PF = 4;
+        float gv[PF][4];
+        unsigned cw[PF][CB];
 #pragma unroll
-        for (int cb = 0; cb < CB; ++cb) cw_cur[cb] = load_c4<VEC>(cp[cb], ow0, g.OW);
-        for (int k = 0; k < g.K; ++k) {
-            if (k + 1 < g.K) {
-                gp += plane;
-                load_g4<T, VEC>(gp, ow0, g.OW, gv_nxt);
+        for (int u = 0; u < PF; ++u)
+            if (u < g.K) {
+                load_g4<T, VEC>(gp + (size_t)u * plane, ow0, g.OW, gv[u]);
+#pragma unroll
+                for (int cb = 0; cb < CB; ++cb) cw[u][cb] = load_c4<VEC>(cp[cb] + (size_t)u * cstep, ow0, g.OW);
+            }
+        gp += (size_t)PF * plane;          // the next channel to request
+#pragma unroll
+        for (int cb = 0; cb < CB; ++cb) cp[cb] += (size_t)PF * cstep;
+        for (int k0 = 0; k0 < g.K; k0 += PF) {
+#pragma unroll
+            for (int u = 0; u < PF; ++u) {
+                const int k = k0 + u;
+                if (k >= g.K) break;
 #pragma unroll
                 for (int cb = 0; cb < CB; ++cb) {
-                    cp[cb] += cstep;
-                    cw_nxt[cb] = load_c4<VEC>(cp[cb], ow0, g.OW);
-                }
-            }
-#pragma unroll
-            for (int cb = 0; cb < CB; ++cb) {
-                if (BR != 0 && cb >= ncb) continue;   // single-branch layers have no zero coefficient to hide behind
-                float a = 1.0f, b = 1.0f;
-                if constexpr (BR == 0) {
-                    a = a_s[k * CB + cb];
-                    b = b_s[k * CB + cb];
-                }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const unsigned code = (cw_cur[cb] >> (8 * j)) & 0xffu;
-                    if constexpr (BR == 0 || BR == 1) {
-                        float* dst = reinterpret_cast<float*>(Ab[cb] + (code & 15u) * tstride + j * NQp * sizeof(float));
-                        *dst = (BR == 0) ? __fmaf_rn(a, gv_cur[j], *dst) : (*dst + gv_cur[j]);
+                    if (BR != 0 && cb >= ncb) continue;   // single-branch layers have no zero coefficient to hide behind
+                    float a = 1.0f, b = 1.0f;
+                    if constexpr (BR == 0) {
+                        a = a_s[k * CB + cb];
+                        b = b_s[k * CB + cb];
                     }
-                    if constexpr (BR == 0 || BR == 2) {
-                        float* dst = reinterpret_cast<float*>(Ab[cb] + (code >> 4) * tstride + j * NQp * sizeof(float));
-                        *dst = (BR == 0) ? __fmaf_rn(b, gv_cur[j], *dst) : (*dst + gv_cur[j]);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const unsigned code = (cw[u][cb] >> (8 * j)) & 0xffu;
+                        if constexpr (BR == 0 || BR == 1) {
+                            float* dst = reinterpret_cast<float*>(Ab[cb] + (code & 15u) * tstride + j * NQp * sizeof(float));
+                            *dst = (BR == 0) ? __fmaf_rn(a, gv[u][j], *dst) : (*dst + gv[u][j]);
+                        }
+                        if constexpr (BR == 0 || BR == 2) {
+                            float* dst = reinterpret_cast<float*>(Ab[cb] + (code >> 4) * tstride + j * NQp * sizeof(float));
+                            *dst = (BR == 0) ? __fmaf_rn(b, gv[u][j], *dst) : (*dst + gv[u][j]);
+                        }
                     }
                 }
+                if (k + PF < g.K) {
+                    load_g4<T, VEC>(gp, ow0, g.OW, gv[u]);
+#pragma unroll
+                    for (int cb = 0; cb < CB; ++cb) {
+                        cw[u][cb] = load_c4<VEC>(cp[cb], ow0, g.OW);
+                        cp[cb] += cstep;
+                    }
+                    gp += plane;
+                }
             }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) gv_cur[j] = gv_nxt[j];
-#pragma unroll
-            for (int cb = 0; cb < CB; ++cb) cw_cur[cb] = cw_nxt[cb];
         }
     }
     __syncthreads();
     // gather: every owned input element sums, over the taps, the accumulator of the output
     // pixel that reads it through that tap (one warp per input row, lanes along the columns)
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     const bool unit_stride = (g.sh == 1 && g.sw == 1);
     for (int il = 0; il < nimg; ++il)
     for (int cb = 0; cb < ncb; ++cb) {
         const float* Ac = A + (size_t)cb * g.RS * 4 * NQp + il * NQ1;
         T* gxc = gx + ((size_t)(n_first + il) * g.C + c0 + cb) * g.H * g.W;
-        for (int row = warp; row < rows; row += 8) {
+        for (int row = warp; row < rows; row += nwarps) {
             const int ih = ih0 + row;
             for (int iw = lane; iw < g.W; iw += 32) {
                 float s = 0.0f;
@@ -717,6 +733,19 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
         pl->NQpad = (int)(((long)nr * pl->QPR * pl->imgs + 31) / 32 * 32);
         pl->smem = ((size_t)cb * g.RS * 4 * pl->NQpad + 2 * (size_t)g.K * kGxCB) * sizeof(float);
         if (pl->smem > kBwdSmemLimit + 16 * 1024) continue;
+        // a large tile leaves one or two CTAs per SM: give them the warps the SM can hold, in
+        // equal passes over the tile's quads
+        const int per_sm = (int)((227 * 1024) / (pl->smem + 1024));
+        int cap = per_sm >= 3 ? 256 : (per_sm == 2 ? 512 : 1024);
+        const int nq = (int)nr * pl->QPR * pl->imgs;
+        const int passes = (nq + cap - 1) / cap;
+        int th = ((nq + passes - 1) / passes + 31) / 32 * 32;
+        if (th < 256) th = 256;
+        pl->threads = th < cap ? th : cap;
+        pl->ncblk = (g.C + cb - 1) / cb;
+        const size_t nct = (size_t)((g.N + pl->imgs - 1) / pl->imgs) * pl->tiles_per_img * pl->ncblk;
+        if (nct > 0x7fffffffu) return false;
+        pl->grid = (unsigned)nct;
         return true;
     }
     return false;
