@@ -13,6 +13,7 @@
 #pragma once
 #include <cuda.h>
 
+#include <cstdlib>
 #include <cstring>
 
 #include "tconv_common.cuh"
@@ -203,6 +204,12 @@ struct TiledParams {
     int n_col_tiles, n_row_tiles;
     int tiles_per_img; // > 0: row tiles stay inside one image; 0: rows run over the flattened (n, oh) space
     int total_rows;    // N * OH
+    int ragged;        // 1: a tile is NQ consecutive quads of the flattened (n, oh, quad) space (rows whose
+                       //    quads do not divide the lanes of a warp), 0: a tile is TH whole rows
+    int total_quads;   // N * OH * QPR
+    int xbox;          // elements of one staged x block (channels x rows x pitch)
+    int xblock;        // ragged TMA tiles: elements between the staged blocks of the tile's two images
+                       // (xbox rounded up so that the second block starts on a 128-byte boundary)
     int NSLOTS, XW, XP;  // staged input rows per tile, staged columns, row pitch (floats)
     int GAP;           // extra input-row slots between two images of one tile (flattened tiles)
     int CC, Cpad, nchunks;
@@ -230,7 +237,7 @@ template <int S, int DW, int ESIZE = 4> struct TmaShift {
 #ifndef TCONV_Q_CARRIED
 #define TCONV_Q_CARRIED 2
 #endif
-template <int MODE, int CHAN, bool WIN, bool XTMA, int R, int S, int SW, int DW, int Q, int KG, int PW, int TK>
+template <int MODE, int CHAN, bool WIN, bool XTMA, bool RAG, int R, int S, int SW, int DW, int Q, int KG, int PW, int TK>
 __global__ void __launch_bounds__(KG * PW * 32,
                                   (WIN && CHAN == CH_SUM) ? TCONV_MINB_WINSUM
                                   : WIN ? 1
@@ -264,8 +271,14 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
     const int rt = blockIdx.x / p.n_col_tiles;
     const int kt = blockIdx.y;
     const int ow0 = ct * p.TW;
-    int row0, rows_here;
-    if (p.tiles_per_img > 0) {
+    constexpr int NQ_TILE = Q * 32 * PW;   // quads per tile
+    int row0, rows_here, qfirst = 0;       // qfirst: ragged tiles start this many quads into row0
+    if constexpr (RAG) {
+        const int q0 = rt * NQ_TILE;
+        row0 = q0 / p.QPR;
+        qfirst = q0 - row0 * p.QPR;
+        rows_here = (min(q0 + NQ_TILE, p.total_quads) - 1) / p.QPR - row0 + 1;
+    } else if (p.tiles_per_img > 0) {
         const int n = rt / p.tiles_per_img;
         const int oh0 = (rt - n * p.tiles_per_img) * p.TH;
         row0 = n * g.OH + oh0;
@@ -277,6 +290,8 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
     const int iw0 = ow0 * SW - g.pw;
     const int n0 = row0 / g.OH;
     const int oh_first = row0 - n0 * g.OH;
+    // a ragged TMA tile may run into the next image, which is staged as a second block
+    const bool two_imgs = XTMA && RAG && (row0 + rows_here - 1) / g.OH > n0;
 
     if constexpr (XTMA) {
         if (tid == 0) {
@@ -307,15 +322,19 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
         const int qi = wp * 32 + lane + q * (32 * PW);
-        int lr = qi / p.QPR;
-        const int qx = qi - lr * p.QPR;
-        const bool ok = (lr < rows_here);
+        const int qq = qi + qfirst;
+        int lr = qq / p.QPR;
+        const int qx = qq - lr * p.QPR;
+        const bool ok = RAG ? (rt * NQ_TILE + qi < p.total_quads) : (lr < rows_here);
         if (!ok) lr = 0;
         const int gr = row0 + lr;
         const int n = gr / g.OH;
         out_row[q] = ok ? gr : -1;
         qcol[q] = ow0 + qx * 4;
-        xoff[q] = (lr * g.sh + (n - n0) * p.GAP) * p.XP + qx * 4 * SW;
+        if constexpr (XTMA && RAG)
+            xoff[q] = (n == n0 ? lr * g.sh * p.XP : p.xblock + (gr - (n0 + 1) * g.OH) * g.sh * p.XP) + qx * 4 * SW;
+        else
+            xoff[q] = (lr * g.sh + (n - n0) * p.GAP) * p.XP + qx * 4 * SW;
     }
 
     const float* xg = reinterpret_cast<const float*>(p.x);
@@ -332,9 +351,10 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
         const int c0 = ch * p.CC;
         if constexpr (XTMA) {
             if (tid == 0) {
-                const unsigned bytes = (unsigned)((p.CC * p.NSLOTS * p.XP + p.w_stage * (PAR ? 2 : 1) + 2 * p.ab_stage) * sizeof(float));
+                const unsigned bytes = (unsigned)((p.xbox * (two_imgs ? 2 : 1) + p.w_stage * (PAR ? 2 : 1) + 2 * p.ab_stage) * sizeof(float));
                 mbar_expect_tx(&bars[s], bytes);
                 tma_load_3d(st, &xmap, iw0 - SHIFT, oh_first * g.sh - g.ph, n0 * g.C + c0, &bars[s]);
+                if (two_imgs) tma_load_3d(st + p.xblock, &xmap, iw0 - SHIFT, -g.ph, (n0 + 1) * g.C + c0, &bars[s]);
                 bulk_load(st + w_off, wt_k + (size_t)c0 * RS * TILE_K, p.w_stage * sizeof(float), &bars[s]);
                 if (PAR) bulk_load(st + w2_off, wt2_k + (size_t)c0 * RS * TILE_K, p.w_stage * sizeof(float), &bars[s]);
                 if (TWO) {
@@ -732,8 +752,9 @@ inline size_t tiled_ws_bytes(const Geo& g) {
 
 inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
 
+// One candidate plan: ragged tiles allowed or not, cc input channels per staged chunk.
 template <int R, int S, int SW, int DW, int Q, int KG, int PW, int TK = 8>
-inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* pl) {
+inline bool plan_tiles_opt(const Geo& g, bool par, bool two, int esize, bool allow_ragged, int cc, TiledPlan* pl) {
     TiledParams& p = pl->p;
     constexpr int TILE_K = KG * TK;
     constexpr int NQ = Q * 32 * PW;
@@ -750,16 +771,32 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* p
     p.TH = NQ / p.QPR;
     if (p.TH < 1) return false;
     p.total_rows = g.N * g.OH;
+    p.total_quads = p.total_rows * p.QPR;
+    p.xblock = 0;
+    // rows whose quads do not divide the lanes: tiles of NQ consecutive quads of the flattened
+    // (n, oh, quad) space instead of whole rows, so that every lane owns a quad
+    p.ragged = (allow_ragged && ncol == 1 && NQ % p.QPR != 0 && p.total_quads > NQ) ? 1 : 0;
+    const int rows_max = p.ragged ? (p.QPR - 1 + NQ - 1) / p.QPR + 1 : p.TH;   // rows one tile can touch
     // TMA path: rows of x are 16-byte multiples, "same" padding along w (fixes the column shift),
     // and tiles that stay inside one image without idling more than a quarter of the lanes
+    // (ragged tiles: inside two images, each staged by its own copy)
     const int unit = 16 / esize;                                     // elements per 16 bytes
     const int shift = esize == 4 ? TmaShift<S, DW, 4>::value : TmaShift<S, DW, 2>::value;
     const int th_img = p.TH < g.OH ? p.TH : g.OH;
     const int tiles_img = (g.OH + th_img - 1) / th_img;
-    const bool rows_fit = (double)g.OH / (tiles_img * th_img) >= 0.75 && th_img * p.QPR * 4 >= NQ * 3;
+    const bool rows_fit = p.ragged ? (g.OH * p.QPR >= NQ)
+                                   : ((double)g.OH / (tiles_img * th_img) >= 0.75 && th_img * p.QPR * 4 >= NQ * 3);
     pl->xtma = ((g.W * esize) % 16 == 0) && (g.pw == (S - 1) * DW / 2) && rows_fit;
     p.XW = (p.TW - 1) * SW + (S - 1) * DW + 1;   // == (QPR-1)*4*SW + L
-    if (pl->xtma) {
+    if (pl->xtma && p.ragged) {
+        p.TH = rows_max;
+        p.tiles_per_img = 0;
+        p.n_row_tiles = (p.total_quads + NQ - 1) / NQ;
+        p.GAP = 0;
+        p.NSLOTS = (rows_max - 1) * g.sh + (R - 1) * g.dh + 1;
+        p.XP = round_up(p.XW + shift, unit);
+        if (p.XP > 256 || p.NSLOTS > 256) return false;
+    } else if (pl->xtma) {
         p.TH = th_img;
         p.tiles_per_img = tiles_img;
         p.n_row_tiles = g.N * tiles_img;
@@ -768,21 +805,24 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* p
         p.XP = round_up(p.XW + shift, unit);
         if (p.XP > 256 || p.NSLOTS > 256) return false;
     } else {
+        if (p.ragged) p.TH = rows_max;
         if (p.TH > p.total_rows) p.TH = p.total_rows;
         p.tiles_per_img = 0;
-        p.n_row_tiles = (p.total_rows + p.TH - 1) / p.TH;
+        p.n_row_tiles = p.ragged ? (p.total_quads + NQ - 1) / NQ : (p.total_rows + p.TH - 1) / p.TH;
         p.GAP = (R - 1) * g.dh - g.sh + 1;
         if (p.GAP < 0) p.GAP = 0;
         const int max_imgs = (p.TH - 1) / g.OH + 2;
         p.NSLOTS = (p.TH - 1) * g.sh + (R - 1) * g.dh + 1 + (max_imgs - 1) * p.GAP;
         p.XP = round_up(p.XW, unit);
     }
-    p.CC = 8;
+    p.CC = cc;
     p.Cpad = round_up(g.C, p.CC);
     p.nchunks = p.Cpad / p.CC;
     // one stage: x tile | weights | (weights 2) | alpha | beta, each block 128-byte aligned;
     // sizes in 4-byte words (XP counts elements of esize bytes)
-    p.x_stage = round_up(p.CC * p.NSLOTS * p.XP * esize / 4, 32);
+    p.xbox = p.CC * p.NSLOTS * p.XP;
+    p.xblock = round_up(p.xbox, 128 / esize);
+    p.x_stage = round_up(((pl->xtma && p.ragged) ? p.xblock + p.xbox : p.xbox) * esize / 4, 32);
     p.w_stage = p.CC * g.RS * TILE_K;            // multiple of 32 floats
     p.ab_stage = two ? p.CC * TILE_K : 0;
     p.stage_floats = p.x_stage + p.w_stage * (par ? 2 : 1) + 2 * p.ab_stage;
@@ -797,6 +837,28 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* p
     pl->ws_w = (size_t)nkt * p.Cpad * g.RS * TILE_K * sizeof(float);
     pl->ws_ab = (size_t)nkt * p.Cpad * TILE_K * sizeof(float);
     return true;
+}
+
+// Picks the plan: ragged tiles keep every lane busy but stage taller (and, with TMA, two) input
+// blocks; the first candidate whose two stages leave room for four resident CTAs per SM wins, in
+// the order ragged / whole rows, 8 / 4 channels per chunk; else whole rows with 8 channels.
+template <int R, int S, int SW, int DW, int Q, int KG, int PW, int TK = 8>
+inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* pl) {
+    static const char* force = getenv("TCONV_PLAN");   // debug switch: "r8", "r4", "n8", "n4"
+    if (force && (force[0] == 'r' || force[0] == 'n') && (force[1] == '8' || force[1] == '4'))
+        return plan_tiles_opt<R, S, SW, DW, Q, KG, PW, TK>(g, par, two, esize, force[0] == 'r', force[1] - '0', pl);
+    // 8 channels per chunk when four CTAs stay resident, else 4 channels when three do (measured
+    // on the stride-2 56 -> 28 layer: 8.06 against 7.86 Ttap/s for whole-row tiles at four CTAs)
+    for (int cc = 8; cc >= 4; cc -= 4) {
+        const size_t budget = (cc == 8 ? 56 : 74) * 1024;
+        TiledPlan cand = *pl;
+        if (plan_tiles_opt<R, S, SW, DW, Q, KG, PW, TK>(g, par, two, esize, true, cc, &cand) && cand.p.ragged &&
+            cand.smem <= budget) {
+            *pl = cand;
+            return true;
+        }
+    }
+    return plan_tiles_opt<R, S, SW, DW, Q, KG, PW, TK>(g, par, two, esize, false, 8, pl);
 }
 
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -868,19 +930,21 @@ int launch_tiled_variant(FwdArgs& a) {
         g.K, g.C, g.RS, pl.tile_k, pl.p.Cpad, nkt, (const T*)a.w, (const T*)a.w2, a.alpha, a.beta, wt, wt2, at, bt);
     pl.p.x = a.x; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
+#define TCONV_LAUNCH_F32(XTMAV, RAGV)                                                                 \
+    {                                                                                                \
+        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, TK>; \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) \
+            return TCONV_ERR_CUDA;                                                                   \
+        kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);                                    \
+    }
     if (pl.xtma) {
-        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, true, R, S, SW, DW, Q, KG, PW, TK>;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-            return TCONV_ERR_CUDA;
-        kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);
+        if (pl.p.ragged) TCONV_LAUNCH_F32(true, true) else TCONV_LAUNCH_F32(true, false)
         a.name = WIN ? "fwd_tiled_f32_tma_win" : "fwd_tiled_f32_tma";
     } else {
-        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, false, R, S, SW, DW, Q, KG, PW, TK>;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-            return TCONV_ERR_CUDA;
-        kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);
+        if (pl.p.ragged) TCONV_LAUNCH_F32(false, true) else TCONV_LAUNCH_F32(false, false)
         a.name = WIN ? "fwd_tiled_f32_win" : "fwd_tiled_f32";
     }
+#undef TCONV_LAUNCH_F32
     return TCONV_OK;
 }
 

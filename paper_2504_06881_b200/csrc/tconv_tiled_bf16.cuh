@@ -117,7 +117,7 @@ __global__ void repack_weights_bf16_kernel(int K, int C, int RS, int tile_k, int
     }
 }
 
-template <int MODE, int CHAN, bool WIN, bool XTMA, int R, int S, int SW, int DW, int Q, int KG, int PW>
+template <int MODE, int CHAN, bool WIN, bool XTMA, bool RAG, int R, int S, int SW, int DW, int Q, int KG, int PW>
 __global__ void __launch_bounds__(KG * PW * 32)
 fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams p) {
     static_assert(S == 3, "the pixel-pair selection below is written for 3 taps per row");
@@ -152,8 +152,14 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
     const int rt = blockIdx.x / p.n_col_tiles;
     const int kt = blockIdx.y;
     const int ow0 = ct * p.TW;
-    int row0, rows_here;
-    if (p.tiles_per_img > 0) {
+    constexpr int NQ_TILE = Q * 32 * PW;   // quads per tile
+    int row0, rows_here, qfirst = 0;       // qfirst: ragged tiles start this many quads into row0
+    if constexpr (RAG) {
+        const int q0 = rt * NQ_TILE;
+        row0 = q0 / p.QPR;
+        qfirst = q0 - row0 * p.QPR;
+        rows_here = (min(q0 + NQ_TILE, p.total_quads) - 1) / p.QPR - row0 + 1;
+    } else if (p.tiles_per_img > 0) {
         const int n = rt / p.tiles_per_img;
         const int oh0 = (rt - n * p.tiles_per_img) * p.TH;
         row0 = n * g.OH + oh0;
@@ -165,6 +171,8 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
     const int iw0 = ow0 * SW - g.pw;
     const int n0 = row0 / g.OH;
     const int oh_first = row0 - n0 * g.OH;
+    // a ragged TMA tile may run into the next image, which is staged as a second block
+    const bool two_imgs = XTMA && RAG && (row0 + rows_here - 1) / g.OH > n0;
 
     if constexpr (XTMA) {
         if (tid == 0) {
@@ -202,15 +210,19 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
         const int qi = wp * 32 + lane + q * (32 * PW);
-        int lr = qi / p.QPR;
-        const int qx = qi - lr * p.QPR;
-        const bool ok = (lr < rows_here);
+        const int qq = qi + qfirst;
+        int lr = qq / p.QPR;
+        const int qx = qq - lr * p.QPR;
+        const bool ok = RAG ? (rt * NQ_TILE + qi < p.total_quads) : (lr < rows_here);
         if (!ok) lr = 0;
         const int gr = row0 + lr;
         const int n = gr / g.OH;
         out_row[q] = ok ? gr : -1;
         qcol[q] = ow0 + qx * 4;
-        xoff[q] = (lr * g.sh + (n - n0) * p.GAP) * pitch_w + qx * 2 * SW;
+        if constexpr (XTMA && RAG)
+            xoff[q] = (n == n0 ? lr * g.sh * pitch_w : p.xblock / 2 + (gr - (n0 + 1) * g.OH) * g.sh * pitch_w) + qx * 2 * SW;
+        else
+            xoff[q] = (lr * g.sh + (n - n0) * p.GAP) * pitch_w + qx * 2 * SW;
     }
 
     const unsigned short* xg = reinterpret_cast<const unsigned short*>(p.x);
@@ -227,10 +239,11 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
         const int c0 = ch * p.CC;
         if constexpr (XTMA) {
             if (tid == 0) {
-                const unsigned bytes = (unsigned)(p.CC * p.NSLOTS * p.XP * 2 +
+                const unsigned bytes = (unsigned)(p.xbox * 2 * (two_imgs ? 2 : 1) +
                                                   (p.w_stage * (PAR ? 2 : 1) + 2 * p.ab_stage) * 4);
                 mbar_expect_tx(&bars[s], bytes);
                 tma_load_3d(st, &xmap, iw0 - SHIFT, oh_first * g.sh - g.ph, n0 * g.C + c0, &bars[s]);
+                if (two_imgs) tma_load_3d(st + p.xblock / 2, &xmap, iw0 - SHIFT, -g.ph, (n0 + 1) * g.C + c0, &bars[s]);
                 bulk_load(st + w_off, wt_k + (size_t)c0 * RS * TILE_K, p.w_stage * 4, &bars[s]);
                 if (PAR) bulk_load(st + w2_off, wt2_k + (size_t)c0 * RS * TILE_K, p.w_stage * 4, &bars[s]);
                 if (TWO) {
@@ -606,19 +619,21 @@ int launch_tiled_variant_bf16(FwdArgs& a) {
         a.alpha, a.beta, (unsigned*)wt, (unsigned*)wt2, at, bt);
     pl.p.x = a.x; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
+#define TCONV_LAUNCH_BF16(XTMAV, RAGV)                                                                \
+    {                                                                                                \
+        auto kern = fwd_tiled_bf16_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW>;    \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) \
+            return TCONV_ERR_CUDA;                                                                   \
+        kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);                                    \
+    }
     if (pl.xtma) {
-        auto kern = fwd_tiled_bf16_kernel<MODE, CHAN, WIN, true, R, S, SW, DW, Q, KG, PW>;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-            return TCONV_ERR_CUDA;
-        kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);
+        if (pl.p.ragged) TCONV_LAUNCH_BF16(true, true) else TCONV_LAUNCH_BF16(true, false)
         a.name = WIN ? "fwd_tiled_bf16_tma_win" : "fwd_tiled_bf16_tma";
     } else {
-        auto kern = fwd_tiled_bf16_kernel<MODE, CHAN, WIN, false, R, S, SW, DW, Q, KG, PW>;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-            return TCONV_ERR_CUDA;
-        kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);
+        if (pl.p.ragged) TCONV_LAUNCH_BF16(false, true) else TCONV_LAUNCH_BF16(false, false)
         a.name = WIN ? "fwd_tiled_bf16_win" : "fwd_tiled_bf16";
     }
+#undef TCONV_LAUNCH_BF16
     return TCONV_OK;
 }
 

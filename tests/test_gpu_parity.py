@@ -84,6 +84,28 @@ def test_tma_staged_shapes(mode, chan, dtype):
         parity.check_layer(d, TIES, 470 + i, recompute=False, stored_winners=(i == 0))
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("mode,chan", ALL_MODES)
+def test_ragged_quad_tiles(mode, chan, dtype):
+    """Rows of 6 or 7 quads do not divide a warp's 32 lanes: a tile is then 32 consecutive quads of
+    the flattened (image, row, quad) space.  Tiles that start in mid-row, cross into the next image
+    (second staged block), cover the last partial tile, and maps so small that a tile spans three
+    images (per-element staging)."""
+    from paper_2504_06881_b200 import tconv
+    mk = lambda *a, **k: inputs.layer(*a, mode=mode, chan=chan, dtype=dtype, **k)
+    cases = [mk(3, 9, 10, 24, 12, 3, 3, stride=1, pad=1),      # 6 quads per row, 60 per image
+             mk(5, 8, 6, 24, 8, 3, 3, stride=1, pad=1),        # 36 quads per image: most tiles cross images
+             mk(6, 8, 4, 24, 8, 3, 3, stride=1, pad=1),        # 24 quads per image: a tile spans three
+             mk(3, 10, 28, 28, 20, 3, 3, stride=1, pad=1),     # 7 quads per row
+             mk(2, 9, 24, 56, 16, 3, 3, stride=2, pad=1),      # stride 2 onto 12 x 28
+             mk(2, 9, 14, 24, 16, 3, 3, stride=1, pad=2, dil=2)]
+    for i, d in enumerate(cases):
+        parity.check_layer(d, None, 480 + i, recompute=False)
+        assert "tiled" in tconv.tconv_last_kernel() or "bwd" in tconv.tconv_last_kernel()
+        assert tconv.tconv_device_status() == 0
+        parity.check_layer(d, TIES, 490 + i, recompute=False)
+
+
 def test_other_window_sizes():
     """1x1, 1x3, 5x5 (more than 16 taps: wide winner codes), 7x7 windows."""
     for (R, S, pad) in ((1, 1, 0), (1, 3, 1), (5, 5, 2), (7, 7, 3), (4, 4, 1)):
