@@ -32,14 +32,13 @@ sys.path.insert(0, str(ROOT))
 MODES = [("max_plus", "default"), ("min_plus", "default"), ("compound", "default"),
          ("parallel", "default")]
 WORKLOAD = "cfg2: one layer of each mode fwd+bwd fp32, N=128 C=K=64 32x32 3x3 s1 p1"
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch at N=32, from the ncu
-# captures summarised under profiles/ (fwd_tiled_f32_win_parallel_cfg2_n32.md,
-# bwd_code_kernels_compound_cfg2_n32.md, bwd_idx_gx_maxplus_cfg2_n32.md); a full-size launch
-# (N=128) processes 4x the units and its traffic grows in proportion.
-DRAM_BYTES_N32 = {("parallel", "fwd_winners"): 105.13e6, ("compound", "fwd_winners"): 105.13e6,
-                  ("compound", "bwd_params"): 157.28e6, ("parallel", "bwd_params"): 157.28e6,
-                  ("compound", "bwd_grad_x"): 150.11e6, ("parallel", "bwd_grad_x"): 150.11e6,
-                  ("max_plus", "bwd_grad_x"): 16.82e6, ("min_plus", "bwd_grad_x"): 16.82e6}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch at the bench's full size
+# (N=128), from one-pass ncu captures of those two counters, summarised in
+# profiles/dram_traffic_cfg2_n128.md.  bwd_params is the grad_w kernel of the call.
+DRAM_BYTES_FULL = {("parallel", "fwd_winners"): 645.29e6, ("compound", "fwd_winners"): 647.10e6,
+                   ("compound", "bwd_params"): 789.41e6, ("parallel", "bwd_params"): 789.41e6,
+                   ("compound", "bwd_grad_x"): 609.60e6, ("parallel", "bwd_grad_x"): 609.60e6,
+                   ("max_plus", "bwd_grad_x"): 70.30e6, ("min_plus", "bwd_grad_x"): 70.30e6}
 # probe variants whose best gives the add+max/min peak of a mode's instruction mix
 PROBES = {"max_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
           "min_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
@@ -365,9 +364,8 @@ def run_gpu(args):
     roofline = {"bound": "alu", "kernel": per[dom_mode][dom_what + "_kernel"], "call": f"{dom_mode} {dom_what}",
                 "achieved": achieved, "peak": peak / 1e12, "unit": "Ttap/s",
                 "frac": achieved / (peak / 1e12),
-                "traffic": (4 * DRAM_BYTES_N32[(dom_mode, dom_what)]
-                            if (dom_mode, dom_what) in DRAM_BYTES_N32 else None),
-                "traffic_note": "DRAM bytes per launch, ncu capture at N=32 scaled x4 (see profiles/)",
+                "traffic": DRAM_BYTES_FULL.get((dom_mode, dom_what)),
+                "traffic_note": "DRAM bytes per launch, one-pass ncu capture at this size (profiles/dram_traffic_cfg2_n128.md)",
                 "peak_source": ("measured in this run: register-only probe of the winner-emitting inner loop of "
                                 "the mode (tap sums, extrema, two fused multiply-adds per tap and branch for "
                                 "the winner keys, key fold)" if win_mix else
