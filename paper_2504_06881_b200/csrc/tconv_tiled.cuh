@@ -844,13 +844,13 @@ inline bool plan_tiles_opt(const Geo& g, bool par, bool two, int esize, bool all
 // the order ragged / whole rows, 8 / 4 channels per chunk; else whole rows with 8 channels.
 template <int R, int S, int SW, int DW, int Q, int KG, int PW, int TK = 8>
 inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* pl) {
-    static const char* force = getenv("TCONV_PLAN");   // debug switch: "r8", "r4", "n8", "n4"
-    if (force && (force[0] == 'r' || force[0] == 'n') && (force[1] == '8' || force[1] == '4'))
+    static const char* force = getenv("TCONV_PLAN");   // debug switch: "r8", "r6", "r4", "n8", "n6", "n4"
+    if (force && (force[0] == 'r' || force[0] == 'n') && (force[1] == '8' || force[1] == '6' || force[1] == '4'))
         return plan_tiles_opt<R, S, SW, DW, Q, KG, PW, TK>(g, par, two, esize, force[0] == 'r', force[1] - '0', pl);
     // 8 channels per chunk when four CTAs stay resident, else 4 channels when three do (measured
     // on the stride-2 56 -> 28 layer: 8.06 against 7.86 Ttap/s for whole-row tiles at four CTAs)
-    for (int cc = 8; cc >= 4; cc -= 4) {
-        const size_t budget = (cc == 8 ? 56 : 74) * 1024;
+    for (int cc = 8; cc >= 4; cc -= 2) {
+        const size_t budget = (cc == 4 ? 74 : 56) * 1024;
         TiledPlan cand = *pl;
         if (plan_tiles_opt<R, S, SW, DW, Q, KG, PW, TK>(g, par, two, esize, true, cc, &cand) && cand.p.ragged &&
             cand.smem <= budget) {

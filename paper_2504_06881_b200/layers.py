@@ -1,0 +1,36 @@
+"""The paper's layer names over ``TropicalConv2d`` (Section 3.1 layers (i)-(vi), Sections 3.4 / 3.5,
+Appendix "Compatibility with PyTorch"): every class takes ``nn.Conv2d``'s constructor arguments.
+
+Base operator + channel combine:  MinPlusSumConv2d (ii), MaxPlusSumConv2d (i), MinPlusMaxConv2d
+(iii), MaxPlusMinConv2d (vi), MinPlusMinConv2d (iv), MaxPlusMaxConv2d (v).
+Compound / parallel with 0, 1 (beta = 1 - alpha) or 2 learnable scalar sets per (c_out, c_in).
+"""
+from __future__ import annotations
+
+from .nn import TropicalConv2d
+
+
+def _named(name, mode, chan="default", params="2p", doc=""):
+    def __init__(self, in_channels, out_channels, kernel_size, stride=1, padding=0, dilation=1,
+                 bias=True, dtype="f32", **kw):
+        TropicalConv2d.__init__(self, in_channels, out_channels, kernel_size, stride=stride,
+                                padding=padding, dilation=dilation, bias=bias, mode=mode, chan=chan,
+                                params=kw.pop("params", params), dtype=dtype, **kw)
+    return type(name, (TropicalConv2d,), {"__init__": __init__, "__doc__": doc})
+
+
+MaxPlusSumConv2d = _named("MaxPlusSumConv2d", "max_plus", "sum", doc="layer (i): sum over channels of the max-plus window")
+MinPlusSumConv2d = _named("MinPlusSumConv2d", "min_plus", "sum", doc="layer (ii): sum over channels of the min-plus window")
+MinPlusMaxConv2d = _named("MinPlusMaxConv2d", "min_plus", "max", doc="layer (iii): max over channels of the min-plus window")
+MinPlusMinConv2d = _named("MinPlusMinConv2d", "min_plus", "min", doc="layer (iv): min over channels and window")
+MaxPlusMaxConv2d = _named("MaxPlusMaxConv2d", "max_plus", "max", doc="layer (v): max over channels and window")
+MaxPlusMinConv2d = _named("MaxPlusMinConv2d", "max_plus", "min", doc="layer (vi): min over channels of the max-plus window")
+
+CompoundMinMaxPlusSumConv2d0p = _named("CompoundMinMaxPlusSumConv2d0p", "compound", params="0p", doc="compound mode, alpha = beta = 1")
+CompoundMinMaxPlusSumConv2d1p = _named("CompoundMinMaxPlusSumConv2d1p", "compound", params="1p", doc="compound mode, beta = 1 - alpha")
+CompoundMinMaxPlusSumConv2d2p = _named("CompoundMinMaxPlusSumConv2d2p", "compound", params="2p", doc="compound mode, learnable alpha and beta")
+ParallelMinMaxPlusSumConv2d0p = _named("ParallelMinMaxPlusSumConv2d0p", "parallel", params="0p", doc="parallel mode, alpha = beta = 1")
+ParallelMinMaxPlusSumConv2d1p = _named("ParallelMinMaxPlusSumConv2d1p", "parallel", params="1p", doc="parallel mode, beta = 1 - alpha")
+ParallelMinMaxPlusSumConv2d2p = _named("ParallelMinMaxPlusSumConv2d2p", "parallel", params="2p", doc="parallel mode, learnable alpha and beta")
+
+__all__ = [n for n in dir() if n.endswith(("Conv2d", "0p", "1p", "2p"))]

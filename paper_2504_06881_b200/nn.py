@@ -80,12 +80,16 @@ class TropicalConv2d(nn.Module):
     """Tropical convolution layer with ``nn.Conv2d``'s constructor arguments.
 
     mode: "max_plus" | "min_plus" | "compound" | "parallel"; chan: "default" | "sum" | "max" | "min".
-    params (compound / parallel): "2p" learnable alpha and beta per (c_out, c_in); "1p" the
-    complementary-weight specialisation beta = 1 - alpha; "0p" alpha = beta = 1 (no scalars).
+    params (compound / parallel; the specialisations of Section 3.6): "2p" learnable alpha and beta
+    per (c_out, c_in); "1p" complementary weights beta = 1 - alpha; "shared" beta = alpha;
+    "opposite" beta = -alpha; "0p" alpha = beta = 1 (no scalars); "fixed" the constants
+    ``fixed=(alpha, beta)``, e.g. (0.5, 0.5) or (1, -1), held as buffers.
     dtype: arithmetic type of the kernels ("f32" or "bf16"); parameters stay fp32."""
 
+    PARAMS = ("0p", "1p", "2p", "shared", "opposite", "fixed")
+
     def __init__(self, in_channels, out_channels, kernel_size, stride=1, padding=0, dilation=1,
-                 bias=True, mode="compound", chan="default", params="2p", dtype="f32"):
+                 bias=True, mode="compound", chan="default", params="2p", dtype="f32", fixed=(0.5, 0.5)):
         super().__init__()
         two = lambda v: (v, v) if isinstance(v, int) else tuple(v)
         self.kernel_size, self.stride, self.padding, self.dilation = map(two, (kernel_size, stride, padding, dilation))
@@ -95,8 +99,14 @@ class TropicalConv2d(nn.Module):
         self.weight = nn.Parameter(torch.empty(out_channels, in_channels, R, S))
         self.weight2 = nn.Parameter(torch.empty(out_channels, in_channels, R, S)) if mode == "parallel" else None
         two_branch = mode in ("compound", "parallel")
-        self.alpha = nn.Parameter(torch.empty(out_channels, in_channels)) if two_branch and params in ("1p", "2p") else None
+        if params not in self.PARAMS:
+            raise ValueError(f"params must be one of {self.PARAMS}")
+        learn_a = two_branch and params in ("1p", "2p", "shared", "opposite")
+        self.alpha = nn.Parameter(torch.empty(out_channels, in_channels)) if learn_a else None
         self.beta = nn.Parameter(torch.empty(out_channels, in_channels)) if two_branch and params == "2p" else None
+        if two_branch and params == "fixed":
+            self.register_buffer("alpha_fixed", torch.full((out_channels, in_channels), float(fixed[0])))
+            self.register_buffer("beta_fixed", torch.full((out_channels, in_channels), float(fixed[1])))
         self.bias = nn.Parameter(torch.zeros(out_channels)) if bias else None
         self.reset_parameters()
 
@@ -119,8 +129,15 @@ class TropicalConv2d(nn.Module):
 
     def forward(self, x):
         alpha, beta = self.alpha, self.beta
-        if self.mode in ("compound", "parallel") and self.params == "1p":
-            beta = 1.0 - alpha
+        if self.mode in ("compound", "parallel"):
+            if self.params == "1p":
+                beta = 1.0 - alpha
+            elif self.params == "shared":
+                beta = alpha
+            elif self.params == "opposite":
+                beta = -alpha
+            elif self.params == "fixed":
+                alpha, beta = self.alpha_fixed, self.beta_fixed
         geom = (self.mode, self.chan, self.dtype, self.stride, self.padding, self.dilation)
         return TropicalConvFn.apply(x, self.weight, self.weight2, alpha, beta, self.bias, geom)
 

@@ -1,0 +1,105 @@
+"""The named layer set (Section 3.1 layers (i)-(vi), compound / parallel with 0p / 1p / 2p scalars,
+the alpha / beta specialisations of Section 3.6)."""
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2504_06881_b200 import inputs, layers
+
+
+def _golden():
+    out = {}
+    for line in (Path(__file__).parent / "golden" / "lenet_param_counts.txt").read_text().splitlines():
+        if line and not line.startswith("#"):
+            name, n = line.split()
+            out[name] = int(n)
+    return out
+
+
+def test_lenet_variants_built_from_the_named_layers_have_the_papers_parameter_counts():
+    """LeNet: conv 1->6 5x5, conv 6->16 5x5, fc 400-120-84-10 (results table of the LeNet section).
+    C / P = both convolutions compound / parallel, CM / PM = only the first one."""
+    import torch.nn as nn
+    g = _golden()
+    fc = 400 * 120 + 120 + 120 * 84 + 84 + 84 * 10 + 10
+    count = lambda *mods: sum(p.numel() for m in mods for p in m.parameters()) + fc
+    std = lambda ci, co: nn.Conv2d(ci, co, 5)
+    C1, C2 = layers.CompoundMinMaxPlusSumConv2d1p, layers.CompoundMinMaxPlusSumConv2d2p
+    P1, P2 = layers.ParallelMinMaxPlusSumConv2d1p, layers.ParallelMinMaxPlusSumConv2d2p
+    assert count(std(1, 6), std(6, 16)) == g["LeNet"]
+    assert count(layers.MinPlusSumConv2d(1, 6, 5), layers.MaxPlusSumConv2d(6, 16, 5)) == g["LeNet-F-I"]
+    assert count(C1(1, 6, 5), C1(6, 16, 5)) == g["LeNet-C-alpha"]
+    assert count(C2(1, 6, 5), C2(6, 16, 5)) == g["LeNet-C-alpha/beta"]
+    assert count(C1(1, 6, 5), std(6, 16)) == g["LeNet-CM-alpha"]
+    assert count(C2(1, 6, 5), std(6, 16)) == g["LeNet-CM-alpha/beta"]
+    assert count(P1(1, 6, 5), P1(6, 16, 5)) == g["LeNet-P-alpha"]
+    assert count(P2(1, 6, 5), P2(6, 16, 5)) == g["LeNet-P-alpha/beta"]
+    assert count(P1(1, 6, 5), std(6, 16)) == g["LeNet-PM-alpha"]
+    assert count(P2(1, 6, 5), std(6, 16)) == g["LeNet-PM-alpha/beta"]
+
+
+def test_names_map_to_modes_and_channel_combines():
+    table = {"MaxPlusSumConv2d": ("max_plus", "sum"), "MinPlusSumConv2d": ("min_plus", "sum"),
+             "MinPlusMaxConv2d": ("min_plus", "max"), "MinPlusMinConv2d": ("min_plus", "min"),
+             "MaxPlusMaxConv2d": ("max_plus", "max"), "MaxPlusMinConv2d": ("max_plus", "min")}
+    for name, (mode, chan) in table.items():
+        m = getattr(layers, name)(3, 4, 3, padding=1)
+        assert (m.mode, m.chan) == (mode, chan)
+        assert m.alpha is None and m.beta is None and m.weight2 is None
+    for fam, mode in (("Compound", "compound"), ("Parallel", "parallel")):
+        for np_, (has_a, has_b) in (("0p", (False, False)), ("1p", (True, False)), ("2p", (True, True))):
+            m = getattr(layers, f"{fam}MinMaxPlusSumConv2d{np_}")(3, 4, 3)
+            assert m.mode == mode and m.params == np_
+            assert (m.alpha is not None, m.beta is not None) == (has_a, has_b)
+            assert (m.weight2 is not None) == (mode == "parallel")
+    with pytest.raises(ValueError):
+        layers.TropicalConv2d(3, 4, 3, params="3p")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("mode", ["compound", "parallel"])
+@pytest.mark.parametrize("params", ["0p", "1p", "2p", "shared", "opposite", "fixed"])
+def test_specialisations_against_the_oracle(mode, params):
+    """Forward bit-exact and the chained alpha gradient (beta = f(alpha)) against the oracle run
+    with the alpha / beta arrays the specialisation implies."""
+    from oracle import tconv_oracle as ora
+    d = inputs.layer(2, 5, 9, 12, 7, 3, 3, stride=1, pad=1, mode=mode)
+    t = inputs.draw(d, 2100)
+    m = layers.TropicalConv2d(5, 7, 3, padding=1, mode=mode, params=params, fixed=(1.0, -1.0)).cuda()
+    with torch.no_grad():
+        m.weight.copy_(torch.from_numpy(t["w"]))
+        m.bias.copy_(torch.from_numpy(t["bias"]))
+        if m.weight2 is not None:
+            m.weight2.copy_(torch.from_numpy(t["w2"]))
+        if m.alpha is not None:
+            m.alpha.copy_(torch.from_numpy(t["alpha"]))
+        if m.beta is not None:
+            m.beta.copy_(torch.from_numpy(t["beta"]))
+    a = t["alpha"]
+    ab = {"0p": (np.ones_like(a), np.ones_like(a)), "1p": (a, (1.0 - torch.from_numpy(a)).numpy()), "2p": (a, t["beta"]),
+          "shared": (a, a), "opposite": (a, -a),
+          "fixed": (np.full_like(a, 1.0), np.full_like(a, -1.0))}[params]
+    w2 = t["w2"] if mode == "parallel" else None
+    ref = ora.forward(d, t["x"], t["w"], w2, ab[0], ab[1], t["bias"])
+    x = torch.from_numpy(t["x"]).cuda().requires_grad_(True)
+    y = m(x)
+    assert np.array_equal(y.detach().cpu().numpy().view(np.uint32), ref["y"].view(np.uint32))
+    y.backward(torch.from_numpy(t["g"]).cuda())
+    gref = ora.backward(d, t["x"], t["w"], t["g"], w2, ab[0], ab[1])   # name -> (gradient, sum of |contributions|)
+
+    def close(got, want, scale):
+        return (np.abs(got.detach().cpu().numpy().astype(np.float64) - want) <= 1e-5 * scale + 1e-30).all()
+
+    assert close(x.grad, *gref["grad_x"])
+    assert close(m.weight.grad, *gref["grad_w"])
+    if m.weight2 is not None:
+        assert close(m.weight2.grad, *gref["grad_w2"])
+    (ga, gaa), (gb, gba) = gref["grad_alpha"], gref["grad_beta"]
+    if m.alpha is not None:
+        # beta = f(alpha): d loss / d alpha = grad_alpha + f'(alpha) * grad_beta
+        sign = {"1p": -1.0, "2p": 0.0, "shared": 1.0, "opposite": -1.0}[params]
+        assert close(m.alpha.grad, ga + sign * gb, gaa + abs(sign) * gba)
+    if m.beta is not None:
+        assert close(m.beta.grad, gb, gba)
