@@ -177,3 +177,52 @@ def backward(d: dict, x, w, g, w2=None, alpha=None, beta=None):
         out["grad_alpha"] = (ga, gaa)
         out["grad_beta"] = (gb, gba)
     return out
+
+
+# ---------------------------------------------------------------------------------------------
+# Depthwise form (groups = C; the MobileNetV2 variants of the paper's Section 6 replace the
+# depthwise convolutions): channel c is its own group, i.e. the dense operator above with one
+# input and one output channel, applied channel by channel.  Nothing new is computed here: every
+# number comes from ``forward`` / ``backward``.  Shapes: w, w2 [C][R][S]; alpha, beta, bias [C];
+# y, g [N][C][OH][OW]; codes uint8 [N][C][OH][OW] (low nibble argmin tap, high nibble argmax tap).
+def _dw_desc(d: dict) -> dict:
+    assert d["K"] == d["C"], "depthwise: one output channel per input channel"
+    return dict(d, C=1, K=1, chan="sum")
+
+
+def depthwise_forward(d: dict, x, w, w2=None, alpha=None, beta=None, bias=None):
+    d1 = _dw_desc(d)
+    C = d["C"]
+    two, par = d["mode"] in ("compound", "parallel"), d["mode"] == "parallel"
+    ys, cs = [], []
+    for c in range(C):
+        r = forward(d1, np.ascontiguousarray(x[:, c:c + 1]), w[c][None, None],
+                    w2[c][None, None] if par else None,
+                    np.reshape(alpha[c], (1, 1)) if (two and alpha is not None) else None,
+                    np.reshape(beta[c], (1, 1)) if (two and beta is not None) else None,
+                    np.reshape(bias[c], (1,)) if bias is not None else None)
+        ys.append(r["y"][:, 0])
+        cs.append(None if r["codes"] is None else r["codes"][:, 0, 0])
+    return {"y": np.stack(ys, 1), "codes": None if cs[0] is None else np.stack(cs, 1)}
+
+
+def depthwise_backward(d: dict, x, w, g, w2=None, alpha=None, beta=None):
+    """name -> (gradient, sum of |contributions|), float64; grad_w, grad_w2 [C][R][S]; the rest [C]."""
+    d1 = _dw_desc(d)
+    C = d["C"]
+    two, par = d["mode"] in ("compound", "parallel"), d["mode"] == "parallel"
+    parts = []
+    for c in range(C):
+        parts.append(backward(d1, np.ascontiguousarray(x[:, c:c + 1]), w[c][None, None],
+                              np.ascontiguousarray(g[:, c:c + 1]), w2[c][None, None] if par else None,
+                              np.reshape(alpha[c], (1, 1)) if (two and alpha is not None) else None,
+                              np.reshape(beta[c], (1, 1)) if (two and beta is not None) else None))
+    out = {}
+    for name in parts[0]:
+        if name == "grad_x":
+            out[name] = tuple(np.concatenate([p[name][i] for p in parts], 1) for i in (0, 1))
+        elif name in ("grad_w", "grad_w2"):
+            out[name] = tuple(np.stack([p[name][i][0, 0] for p in parts], 0) for i in (0, 1))
+        else:
+            out[name] = tuple(np.stack([p[name][i].reshape(()) for p in parts], 0) for i in (0, 1))
+    return out
