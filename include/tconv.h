@@ -182,6 +182,36 @@ int tconv_forward_noalloc(const tconv_desc_t *desc, const void *x, const void *w
 size_t tconv_forward_noalloc_max_scratch(void);
 
 /*
+ * Depthwise form (groups = C): every channel is its own group, the arrangement the paper's
+ * MobileNetV2 variants use when they replace the depthwise convolutions (Section 6, "MobileNetV2
+ * Models"):
+ *   y[n][c] = alpha[c] * min_tap(x[n][c] + w[c]) + beta[c] * max_tap(x[n][c] + w2[c]) + bias[c]
+ * (compound: w2 = w; max_plus / min_plus: the one extremum, no alpha / beta).  The descriptor is the
+ * dense one with K == C (else TCONV_ERR_INVALID_ARG) and R * S <= 16 (else TCONV_ERR_UNSUPPORTED);
+ * chan is ignored (a group has one channel).  Shapes: x, grad_x [N][C][H][W]; y, grad_y
+ * [N][C][OH][OW]; w, w2, grad_w, grad_w2 [C][R][S]; alpha, beta, bias and their gradients [C].
+ * winners: uint8 [N][C][OH][OW], argmin tap r*S+s in the low nibble, argmax tap in the high nibble
+ * (tconv_dw_winner_bytes() bytes).  Tie rule, padding, evaluation order, bf16 semantics, NULL alpha /
+ * beta / bias and error behaviour are those of tconv_forward / tconv_backward; every result equals
+ * the dense layer with one input and one output channel applied channel by channel.
+ * tconv_dw_forward needs no workspace; y may be NULL when only the winners are wanted.
+ * tconv_dw_backward needs tconv_dw_workspace_bytes(desc, 1) bytes (recomputed winners when
+ * winners == NULL, and the per-chunk partial sums of the parameter gradients); any gradient pointer
+ * may be NULL; gradients are deterministic (gather form for grad_x, fixed-order reductions).
+ * Layers whose element counts exceed 2^31 - 1 are rejected with TCONV_ERR_TOO_LARGE.
+ */
+size_t tconv_dw_winner_bytes(const tconv_desc_t *desc);
+size_t tconv_dw_workspace_bytes(const tconv_desc_t *desc, int backward);
+int tconv_dw_forward(const tconv_desc_t *desc, const void *x, const void *w, const void *w2,
+                     const float *alpha, const float *beta, const float *bias, void *y,
+                     void *winners, void *stream);
+int tconv_dw_backward(const tconv_desc_t *desc, const void *x, const void *w, const void *w2,
+                      const float *alpha, const float *beta, const void *grad_y,
+                      const void *winners, void *grad_x, float *grad_w, float *grad_w2,
+                      float *grad_alpha, float *grad_beta, float *grad_bias, void *workspace,
+                      size_t workspace_bytes, void *stream);
+
+/*
  * Number of operations the paper's complexity analysis (Section 4.1) assigns to
  * one forward pass of the layer: additions + comparisons + multiplications
  * (theta = 1).  Host call; 0 for an invalid descriptor.

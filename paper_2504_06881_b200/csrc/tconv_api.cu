@@ -7,6 +7,7 @@
 #include "alu_probe.cuh"
 #include "tconv_common.cuh"
 #include "tconv_bwd.cuh"
+#include "tconv_depthwise.cuh"
 #include "tconv_generic.cuh"
 #include "tconv_tiled.cuh"
 
@@ -327,6 +328,109 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
 
 }  // namespace
 
+// ---------------------------------------------------------------------------------- depthwise form
+namespace {
+
+// Geometry of a depthwise layer: the dense descriptor with K == C, at most 16 taps, and sizes
+// whose flat indices fit 31 bits.
+int make_dw_geo(const tconv_desc_t* d, Geo* g) {
+    const int rc = make_geo(d, g);
+    if (rc != TCONV_OK) return rc;
+    if (g->K != g->C) return TCONV_ERR_INVALID_ARG;
+    if (g->RS > 16) return TCONV_ERR_UNSUPPORTED;
+    g->chan = CH_SUM;
+    const double lim = 2147483647.0;
+    if ((double)g->N * g->C * g->OH * ((g->OW + 3) / 4) > lim || (double)g->N * g->C * g->H * g->W > lim ||
+        (double)g->N * g->C * g->OH * g->OW > lim)
+        return TCONV_ERR_TOO_LARGE;
+    return TCONV_OK;
+}
+
+// Chunks of the per-channel reduction: enough CTAs to fill the GPU, at least 1024 items each.
+int dw_chunks(const Geo& g) {
+    const long items = (long)g.N * g.OH * g.OW;
+    long n = (592 + g.C - 1) / g.C;
+    const long most = (items + 1023) / 1024;
+    if (n > most) n = most;
+    if (n < 1) n = 1;
+    return (int)n;
+}
+
+template <typename T>
+int dw_forward_t(const Geo& g, const void* x, const void* w, const void* w2, const float* alpha,
+                 const float* beta, const float* bias, void* y, void* winners, cudaStream_t st) {
+    const int QPR = (g.OW + 3) / 4;
+    const size_t total = (size_t)g.N * g.C * g.OH * QPR;
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+#define TCONV_DW_FWD(MODE)                                                                            \
+    if (winners)                                                                                     \
+        dw_fwd_kernel<T, MODE, true><<<blocks, 256, 0, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
+                                                             bias, (T*)y, (uint8_t*)winners, QPR, total); \
+    else                                                                                             \
+        dw_fwd_kernel<T, MODE, false><<<blocks, 256, 0, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
+                                                              bias, (T*)y, nullptr, QPR, total);
+    switch (g.mode) {
+        case TCONV_MAX_PLUS: TCONV_DW_FWD(TCONV_MAX_PLUS) break;
+        case TCONV_MIN_PLUS: TCONV_DW_FWD(TCONV_MIN_PLUS) break;
+        case TCONV_COMPOUND: TCONV_DW_FWD(TCONV_COMPOUND) break;
+        default: TCONV_DW_FWD(TCONV_PARALLEL) break;
+    }
+#undef TCONV_DW_FWD
+    g_launches += 1;
+    snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", winners ? "dw_fwd_win" : "dw_fwd");
+    return check_launch();
+}
+
+template <typename T>
+int dw_backward_t(const Geo& g, const void* x, const void* w, const void* w2, const float* alpha,
+                  const float* beta, const void* gy, const void* winners, void* gx, float* gw,
+                  float* gw2, float* galpha, float* gbeta, float* gbias, void* ws, cudaStream_t st) {
+    const bool twob = two_branch(g.mode), par = g.mode == TCONV_PARALLEL;
+    const int br = twob ? 0 : (g.mode == TCONV_MIN_PLUS ? 1 : 2);
+    const size_t wbytes = align_up((size_t)g.N * g.C * g.OH * g.OW, 256);
+    const uint8_t* codes = (const uint8_t*)winners;
+    float* partial = (float*)((char*)ws + wbytes);
+    if (!codes) {
+        // recompute the winners into the workspace (forward without an output)
+        const int rc = dw_forward_t<T>(g, x, w, w2, alpha, beta, nullptr, nullptr, ws, st);
+        if (rc != TCONV_OK) return rc;
+        codes = (const uint8_t*)ws;
+    }
+    if (gx) {
+        const size_t total = (size_t)g.N * g.C * g.H * g.W;
+        const unsigned blocks = (unsigned)((total + 255) / 256);
+        if (br == 0) dw_bwd_gx_kernel<T, 0><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, total);
+        else if (br == 1) dw_bwd_gx_kernel<T, 1><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, total);
+        else dw_bwd_gx_kernel<T, 2><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, total);
+        g_launches += 1;
+    }
+    if (gw || gw2 || galpha || gbeta || gbias) {
+        const int nch = dw_chunks(g);
+        const dim3 grid((unsigned)g.C, (unsigned)nch);
+        const size_t smem = (size_t)kDwAcc * 256 * sizeof(float);
+        const int need_ab = (twob && (galpha || gbeta)) ? 1 : 0;
+#define TCONV_DW_PAR(BR, PARV)                                                                        \
+    {                                                                                                \
+        auto kern = dw_bwd_params_kernel<T, BR, PARV>;                                               \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) \
+            return cuda_fail(cudaGetLastError());                                                    \
+        kern<<<grid, 256, smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, codes, partial, nch, need_ab); \
+    }
+        if (br == 0) { if (par) TCONV_DW_PAR(0, true) else TCONV_DW_PAR(0, false) }
+        else if (br == 1) TCONV_DW_PAR(1, false)
+        else TCONV_DW_PAR(2, false)
+#undef TCONV_DW_PAR
+        const int n = g.C * kDwAcc;
+        dw_bwd_finish_kernel<<<(n + 255) / 256, 256, 0, st>>>(g, partial, nch, g.mode, alpha, beta, gw, gw2, galpha,
+                                                             gbeta, gbias);
+        g_launches += 2;
+    }
+    snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", "dw_bwd");
+    return check_launch();
+}
+
+}  // namespace
+
 extern "C" {
 
 int tconv_output_shape(const tconv_desc_t* desc, int32_t* OH, int32_t* OW) {
@@ -428,6 +532,56 @@ double tconv_paper_ops(const tconv_desc_t* desc) {
     if (g.mode == TCONV_PARALLEL) return ((2 * RS * C + 2 * C - 1) + 2 * (RS - 1) * C + 2 * C) * P;
     if (g.chan == CH_SUM) return ((C - 1 + RS * C) + (RS - 1) * C) * P;
     return (RS * C + (RS * C - 1)) * P;
+}
+
+// ---------------------------------------------------------------------------------- depthwise form
+size_t tconv_dw_winner_bytes(const tconv_desc_t* desc) {
+    Geo g;
+    if (make_dw_geo(desc, &g) != TCONV_OK) return 0;
+    return (size_t)g.N * g.C * g.OH * g.OW;
+}
+
+size_t tconv_dw_workspace_bytes(const tconv_desc_t* desc, int backward) {
+    Geo g;
+    if (make_dw_geo(desc, &g) != TCONV_OK || !backward) return 0;
+    return align_up((size_t)g.N * g.C * g.OH * g.OW, 256) + (size_t)dw_chunks(g) * g.C * kDwAcc * sizeof(float) + 256;
+}
+
+int tconv_dw_forward(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,
+                     const float* alpha, const float* beta, const float* bias, void* y, void* winners,
+                     void* stream) {
+    g_last_error[0] = 0;
+    Geo g;
+    const int rc = make_dw_geo(desc, &g);
+    if (rc != TCONV_OK) return rc;
+    if (!x || !w || (!y && !winners)) return TCONV_ERR_INVALID_ARG;
+    if (g.mode == TCONV_PARALLEL && !w2) return TCONV_ERR_INVALID_ARG;
+    if (misaligned(x) || misaligned(y) || misaligned(winners)) return TCONV_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    return desc->dtype == TCONV_F32
+               ? dw_forward_t<float>(g, x, w, w2, alpha, beta, bias, y, winners, st)
+               : dw_forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, bias, y, winners, st);
+}
+
+int tconv_dw_backward(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,
+                      const float* alpha, const float* beta, const void* grad_y, const void* winners,
+                      void* grad_x, float* grad_w, float* grad_w2, float* grad_alpha, float* grad_beta,
+                      float* grad_bias, void* workspace, size_t workspace_bytes, void* stream) {
+    g_last_error[0] = 0;
+    Geo g;
+    const int rc = make_dw_geo(desc, &g);
+    if (rc != TCONV_OK) return rc;
+    if (!x || !w || !grad_y) return TCONV_ERR_INVALID_ARG;
+    if (g.mode == TCONV_PARALLEL && !w2) return TCONV_ERR_INVALID_ARG;
+    if (misaligned(x) || misaligned(grad_y) || misaligned(winners) || misaligned(grad_x) || misaligned(workspace))
+        return TCONV_ERR_MISALIGNED;
+    if (!workspace || workspace_bytes < tconv_dw_workspace_bytes(desc, 1)) return TCONV_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    return desc->dtype == TCONV_F32
+               ? dw_backward_t<float>(g, x, w, w2, alpha, beta, grad_y, winners, grad_x, grad_w, grad_w2,
+                                      grad_alpha, grad_beta, grad_bias, workspace, st)
+               : dw_backward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, grad_y, winners, grad_x, grad_w,
+                                              grad_w2, grad_alpha, grad_beta, grad_bias, workspace, st);
 }
 
 int tconv_alu_probe(int variant, int iters, void* sink, double* taps_per_launch, void* stream) {

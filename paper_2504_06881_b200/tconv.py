@@ -24,7 +24,8 @@ TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
 SYMBOLS = ("tconv_output_shape", "tconv_winner_bytes", "tconv_workspace_bytes", "tconv_forward",
            "tconv_backward", "tconv_forward_noalloc", "tconv_forward_noalloc_max_scratch", "tconv_paper_ops", "tconv_alu_probe", "tconv_alu_probe_name",
            "tconv_device_status", "tconv_status_string", "tconv_last_error", "tconv_last_kernel",
-           "tconv_launch_count")
+           "tconv_launch_count", "tconv_dw_winner_bytes", "tconv_dw_workspace_bytes", "tconv_dw_forward",
+           "tconv_dw_backward")
 
 
 class TconvError(RuntimeError):
@@ -62,6 +63,14 @@ def _load() -> ctypes.CDLL:
     lib.tconv_forward_noalloc.argtypes = [dp, vp, vp, vp, fp, fp, fp, vp, vp, vp]
     lib.tconv_forward_noalloc.restype = ctypes.c_int
     lib.tconv_forward_noalloc_max_scratch.restype = sz
+    lib.tconv_dw_winner_bytes.argtypes = [dp]
+    lib.tconv_dw_winner_bytes.restype = sz
+    lib.tconv_dw_workspace_bytes.argtypes = [dp, ctypes.c_int]
+    lib.tconv_dw_workspace_bytes.restype = sz
+    lib.tconv_dw_forward.argtypes = [dp, vp, vp, vp, fp, fp, fp, vp, vp, vp]
+    lib.tconv_dw_forward.restype = ctypes.c_int
+    lib.tconv_dw_backward.argtypes = [dp, vp, vp, vp, fp, fp, vp, vp, vp, fp, fp, fp, fp, fp, vp, sz, vp]
+    lib.tconv_dw_backward.restype = ctypes.c_int
     lib.tconv_paper_ops.argtypes = [dp]
     lib.tconv_paper_ops.restype = ctypes.c_double
     lib.tconv_alu_probe.argtypes = [ctypes.c_int, ctypes.c_int, vp, ctypes.POINTER(ctypes.c_double), vp]
@@ -140,6 +149,29 @@ def tconv_forward_noalloc(d: dict, x, w, w2, alpha, beta, bias, y, winners=None,
     scratch is used.  For callers that must not touch the device allocator.  Returns the status."""
     return _lib.tconv_forward_noalloc(ctypes.byref(make_desc(d)), _p(x), _p(w), _p(w2), _p(alpha),
                                       _p(beta), _p(bias), _p(y), _p(winners), _stream(stream))
+
+
+def tconv_dw_winner_bytes(d: dict) -> int:
+    return int(_lib.tconv_dw_winner_bytes(ctypes.byref(make_desc(d))))
+
+
+def tconv_dw_workspace_bytes(d: dict, backward: bool) -> int:
+    return int(_lib.tconv_dw_workspace_bytes(ctypes.byref(make_desc(d)), int(backward)))
+
+
+def tconv_dw_forward(d: dict, x, w, w2, alpha, beta, bias, y, winners=None, stream=None) -> int:
+    """Raw call of the depthwise forward (groups = C; d["K"] == d["C"]).  Returns the status."""
+    return _lib.tconv_dw_forward(ctypes.byref(make_desc(d)), _p(x), _p(w), _p(w2), _p(alpha), _p(beta),
+                                 _p(bias), _p(y), _p(winners), _stream(stream))
+
+
+def tconv_dw_backward(d: dict, x, w, w2, alpha, beta, grad_y, winners, grad_x, grad_w, grad_w2,
+                      grad_alpha, grad_beta, grad_bias, workspace=None, stream=None) -> int:
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    return _lib.tconv_dw_backward(ctypes.byref(make_desc(d)), _p(x), _p(w), _p(w2), _p(alpha), _p(beta),
+                                  _p(grad_y), _p(winners), _p(grad_x), _p(grad_w), _p(grad_w2),
+                                  _p(grad_alpha), _p(grad_beta), _p(grad_bias), _p(workspace), nbytes,
+                                  _stream(stream))
 
 
 def tconv_forward_noalloc_max_scratch() -> int:
@@ -247,4 +279,46 @@ def backward(d: dict, x, w, grad_y, w2=None, alpha=None, beta=None, winners=None
                         out.get("grad_beta"), out.get("grad_bias"), ws, stream)
     if rc != 0:
         raise TconvError(rc, "tconv_backward")
+    return out
+
+
+def dw_forward(d: dict, x, w, w2=None, alpha=None, beta=None, bias=None, want_winners=False, stream=None):
+    """Depthwise form: allocate y (and the winner codes) and run tconv_dw_forward.  Returns (y, winners)."""
+    N, C, H, W, R, S = (d[k] for k in "NCHWRS")
+    dt = TORCH_DTYPE[d["dtype"]]
+    _check(x, (N, C, H, W), dt, "x"); _check(w, (C, R, S), dt, "w"); _check(w2, (C, R, S), dt, "w2")
+    _check(alpha, (C,), torch.float32, "alpha"); _check(beta, (C,), torch.float32, "beta")
+    _check(bias, (C,), torch.float32, "bias")
+    OH, OW = tconv_output_shape(d)
+    y = torch.empty((N, C, OH, OW), dtype=dt, device=x.device)
+    winners = torch.empty((N, C, OH, OW), dtype=torch.uint8, device=x.device) if want_winners else None
+    rc = tconv_dw_forward(d, x, w, w2, alpha, beta, bias, y, winners, stream)
+    if rc != 0:
+        raise TconvError(rc, "tconv_dw_forward")
+    return y, winners
+
+
+def dw_backward(d: dict, x, w, grad_y, w2=None, alpha=None, beta=None, winners=None, stream=None):
+    """Depthwise form: allocate every gradient the mode has and run tconv_dw_backward.  Returns a dict."""
+    N, C, H, W, R, S = (d[k] for k in "NCHWRS")
+    dt = TORCH_DTYPE[d["dtype"]]
+    OH, OW = tconv_output_shape(d)
+    _check(x, (N, C, H, W), dt, "x"); _check(w, (C, R, S), dt, "w"); _check(w2, (C, R, S), dt, "w2")
+    _check(grad_y, (N, C, OH, OW), dt, "grad_y")
+    two, par = d["mode"] in ("compound", "parallel"), d["mode"] == "parallel"
+    dev, f32 = x.device, torch.float32
+    out = {"grad_x": torch.empty((N, C, H, W), dtype=dt, device=dev),
+           "grad_w": torch.empty((C, R, S), dtype=f32, device=dev),
+           "grad_bias": torch.empty((C,), dtype=f32, device=dev)}
+    if par:
+        out["grad_w2"] = torch.empty((C, R, S), dtype=f32, device=dev)
+    if two:
+        out["grad_alpha"] = torch.empty((C,), dtype=f32, device=dev)
+        out["grad_beta"] = torch.empty((C,), dtype=f32, device=dev)
+    ws = torch.empty(tconv_dw_workspace_bytes(d, True), dtype=torch.uint8, device=dev)
+    rc = tconv_dw_backward(d, x, w, w2, alpha, beta, grad_y, winners, out["grad_x"], out["grad_w"],
+                           out.get("grad_w2"), out.get("grad_alpha"), out.get("grad_beta"),
+                           out["grad_bias"], ws, stream)
+    if rc != 0:
+        raise TconvError(rc, "tconv_dw_backward")
     return out
