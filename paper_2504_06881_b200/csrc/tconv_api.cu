@@ -360,6 +360,32 @@ template <typename T>
 int dw_forward_t(const Geo& g, const void* x, const void* w, const void* w2, const float* alpha,
                  const float* beta, const float* bias, void* y, void* winners, cudaStream_t st) {
     const int QPR = (g.OW + 3) / 4;
+    if (g.R == 3 && g.S == 3 && g.dh == 1 && g.dw == 1 && g.sh == g.sw && (g.sw == 1 || g.sw == 2)) {
+        // 3x3 windows: strips of 4 columns x 6 rows with a register window of three input rows
+        const int strips = (g.OH + 5) / 6;
+        const size_t total3 = (size_t)g.N * g.C * strips * QPR;
+        const unsigned blocks3 = (unsigned)((total3 + 255) / 256);
+        const bool vec = (g.pw == 1 && (g.W & 3) == 0);
+#define TCONV_DW3(MODE, WINV, SWV, VECV)                                                              \
+    dw_fwd3_kernel<T, MODE, WINV, SWV, VECV><<<blocks3, 256, 0, st>>>(                               \
+        g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, bias, (T*)y, (uint8_t*)winners, QPR, strips, (unsigned)total3);
+#define TCONV_DW3_V(MODE, WINV, SWV) { if (vec) TCONV_DW3(MODE, WINV, SWV, true) else TCONV_DW3(MODE, WINV, SWV, false) }
+#define TCONV_DW3_S(MODE, WINV) { if (g.sw == 1) TCONV_DW3_V(MODE, WINV, 1) else TCONV_DW3_V(MODE, WINV, 2) }
+#define TCONV_DW3_W(MODE) { if (winners) TCONV_DW3_S(MODE, true) else TCONV_DW3_S(MODE, false) }
+        switch (g.mode) {
+            case TCONV_MAX_PLUS: TCONV_DW3_W(TCONV_MAX_PLUS) break;
+            case TCONV_MIN_PLUS: TCONV_DW3_W(TCONV_MIN_PLUS) break;
+            case TCONV_COMPOUND: TCONV_DW3_W(TCONV_COMPOUND) break;
+            default: TCONV_DW3_W(TCONV_PARALLEL) break;
+        }
+#undef TCONV_DW3_W
+#undef TCONV_DW3_S
+#undef TCONV_DW3_V
+#undef TCONV_DW3
+        g_launches += 1;
+        snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", winners ? "dw_fwd3_win" : "dw_fwd3");
+        return check_launch();
+    }
     const size_t total = (size_t)g.N * g.C * g.OH * QPR;
     const unsigned blocks = (unsigned)((total + 255) / 256);
 #define TCONV_DW_FWD(MODE)                                                                            \
@@ -396,12 +422,28 @@ int dw_backward_t(const Geo& g, const void* x, const void* w, const void* w2, co
         if (rc != TCONV_OK) return rc;
         codes = (const uint8_t*)ws;
     }
-    if (gx) {
+    if (gx && g.R == 3 && g.S == 3 && g.dh == 1 && g.dw == 1 && g.sh == 1 && g.sw == 1) {
+        // 3x3, stride 1: strips of 4 input columns x 6 input rows over a register window
+        const int QPRI = (g.W + 3) / 4, strips = (g.H + 5) / 6;
+        const size_t total = (size_t)g.N * g.C * strips * QPRI;
+        const unsigned blocks = (unsigned)((total + 255) / 256);
+        const bool vec = (g.pw == 1 && (g.OW & 3) == 0);
+#define TCONV_DW_GX3(BR, VECV)                                                                        \
+    dw_bwd_gx3_kernel<T, BR, VECV><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, QPRI, strips, \
+                                                           (unsigned)total);
+#define TCONV_DW_GX3_V(BR) { if (vec) TCONV_DW_GX3(BR, true) else TCONV_DW_GX3(BR, false) }
+        if (br == 0) TCONV_DW_GX3_V(0) else if (br == 1) TCONV_DW_GX3_V(1) else TCONV_DW_GX3_V(2)
+#undef TCONV_DW_GX3_V
+#undef TCONV_DW_GX3
+        g_launches += 1;
+    } else if (gx) {
         const size_t total = (size_t)g.N * g.C * g.H * g.W;
         const unsigned blocks = (unsigned)((total + 255) / 256);
-        if (br == 0) dw_bwd_gx_kernel<T, 0><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, total);
-        else if (br == 1) dw_bwd_gx_kernel<T, 1><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, total);
-        else dw_bwd_gx_kernel<T, 2><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, total);
+#define TCONV_DW_GX(BR, STV) dw_bwd_gx_kernel<T, BR, STV><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, total);
+#define TCONV_DW_GX_S(BR) { if (g.sh == 2 && g.sw == 2) TCONV_DW_GX(BR, 2) else TCONV_DW_GX(BR, 0) }
+        if (br == 0) TCONV_DW_GX_S(0) else if (br == 1) TCONV_DW_GX_S(1) else TCONV_DW_GX_S(2)
+#undef TCONV_DW_GX_S
+#undef TCONV_DW_GX
         g_launches += 1;
     }
     if (gw || gw2 || galpha || gbeta || gbias) {

@@ -7,6 +7,7 @@
 // tap in the low nibble and the argmax tap in the high nibble (R * S <= 16).
 #pragma once
 #include "tconv_common.cuh"
+#include "tconv_tiled.cuh"   // ext3 (3-input min / max)
 
 namespace tconv {
 
@@ -111,11 +112,185 @@ dw_fwd_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* 
     }
 }
 
+// ---------------------------------------------------------------------------------- forward, 3x3 windows
+// {lo, hi} = {x0 + w, x1 + w}: one packed fp32 add for two horizontally adjacent pixels.
+__device__ __forceinline__ void add2px(float x0, float x1, float w, float& lo, float& hi) {
+    unsigned long long xx, ww, tt;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(xx) : "f"(x0), "f"(x1));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(ww) : "f"(w));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(tt) : "l"(xx), "l"(ww));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
+}
+__device__ __forceinline__ void load4(const float* p, float* out) {
+    const float4 v = __ldg(reinterpret_cast<const float4*>(p));
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, __nv_bfloat16* out) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&v.x);
+    const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&v.y);
+    out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
+}
+// L consecutive elements of an input row starting at column c0 (zero outside the row; the whole
+// row is zero when xr is NULL).  VEC: c0 + 1 is a multiple of 4 and rows start on 4-element
+// boundaries, so the middle of an interior segment is read with aligned 4-element loads.
+template <typename T, int L, bool VEC>
+__device__ __forceinline__ void dw_load_row(const T* xr, int c0, int W, T* out) {
+    if (xr && c0 >= 0 && c0 + L <= W) {
+        if constexpr (VEC) {
+            out[0] = __ldg(xr + c0);
+#pragma unroll
+            for (int i = 1; i + 4 <= L; i += 4) load4(xr + c0 + i, out + i);
+#pragma unroll
+            for (int i = 1 + ((L - 1) / 4) * 4; i < L; ++i) out[i] = __ldg(xr + c0 + i);
+        } else {
+#pragma unroll
+            for (int i = 0; i < L; ++i) out[i] = __ldg(xr + c0 + i);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < L; ++i)
+            out[i] = (xr && c0 + i >= 0 && c0 + i < W) ? __ldg(xr + c0 + i) : zero_of<T>();
+    }
+}
+
+// 3x3 window, dilation 1, stride SW in both directions.  A thread owns a strip of 4 output
+// columns x RT output rows of one (n, c) plane and slides a window of three input rows held in
+// registers down the strip: every input row of the strip is loaded once per thread.  The nine
+// weights of the channel sit in registers.
+template <typename T, int MODE, bool WIN, int SW, bool VEC>
+__global__ void __launch_bounds__(256)
+dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
+               const float* __restrict__ alpha, const float* __restrict__ beta,
+               const float* __restrict__ bias, T* __restrict__ y, uint8_t* __restrict__ codes,
+               int QPR, int strips, unsigned total) {
+    constexpr int RT = 6;                       // output rows per strip
+    constexpr int L = 3 * SW + 3;               // input columns 4 outputs touch
+    constexpr int NROWS = (RT - 1) * SW + 3;    // input rows a strip touches
+    constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
+    constexpr bool PAR = (MODE == TCONV_PARALLEL);
+    constexpr bool DO_MIN = TWO || MODE == TCONV_MIN_PLUS, DO_MAX = TWO || MODE == TCONV_MAX_PLUS;
+    const unsigned q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= total) return;
+    const unsigned t = q / (unsigned)QPR;
+    const int qx = (int)(q - t * (unsigned)QPR);
+    const size_t nc = t / (unsigned)strips;
+    const int oh0 = (int)(t - (unsigned)nc * (unsigned)strips) * RT;
+    const int c = (int)((unsigned)nc % (unsigned)g.C);
+    const int ow0 = qx * 4;
+    const T* xp = x + nc * (size_t)g.H * g.W;
+    T wa[9], wb[9];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) {
+        wa[i] = __ldg(w + (size_t)c * 9 + i);
+        wb[i] = PAR ? __ldg(w2 + (size_t)c * 9 + i) : wa[i];
+    }
+    const float a = (TWO && alpha) ? alpha[c] : 1.0f, b = (TWO && beta) ? beta[c] : 1.0f;
+    const float bk = bias ? bias[c] : 0.0f;
+    const int ih0 = oh0 * SW - g.ph, c0 = ow0 * SW - g.pw;
+    const bool full = (ow0 + 3 < g.OW) && ((g.OW & 3) == 0);
+    T win[3][L];   // input row rho of the strip lives in win[rho % 3]
+    auto load = [&](int rho) {
+        const int ih = ih0 + rho;
+        dw_load_row<T, L, VEC>((ih >= 0 && ih < g.H) ? xp + (size_t)ih * g.W : nullptr, c0, g.W, win[rho % 3]);
+    };
+    load(0);
+    load(1);
+#pragma unroll
+    for (int k = 0; k < RT; ++k) {
+        if (oh0 + k >= g.OH) break;
+#pragma unroll
+        for (int rho = (k == 0 ? 2 : (k - 1) * SW + 3); rho <= k * SW + 2; ++rho) load(rho);
+        float mn[4], mx[4];
+        int amn[4] = {0, 0, 0, 0}, amx[4] = {0, 0, 0, 0};
+        if constexpr (sizeof(T) == 4 && !WIN) {
+            // packed adds over pixel pairs, 3-input min / max chains (3 + 2 + 2 + 2 taps)
+#pragma unroll
+            for (int jp = 0; jp < 2; ++jp) {
+                float ta[9][2], tb[PAR ? 9 : 1][2];
+#pragma unroll
+                for (int tap = 0; tap < 9; ++tap) {
+                    const float* row = reinterpret_cast<const float*>(win[(k * SW + tap / 3) % 3]);
+                    const float x0 = row[(2 * jp) * SW + tap % 3], x1 = row[(2 * jp + 1) * SW + tap % 3];
+                    add2px(x0, x1, to_f32(wa[tap]), ta[tap][0], ta[tap][1]);
+                    if constexpr (PAR) add2px(x0, x1, to_f32(wb[tap]), tb[tap][0], tb[tap][1]);
+                }
+                const float (*tm)[2] = PAR ? tb : ta;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if constexpr (DO_MIN) mn[2 * jp + h] = fold_taps<9>(ta, h, true);
+                    if constexpr (DO_MAX) mx[2 * jp + h] = fold_taps<9>(tm, h, false);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { mn[j] = INFINITY; mx[j] = -INFINITY; }
+#pragma unroll
+            for (int tap = 0; tap < 9; ++tap)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const T xv = win[(k * SW + tap / 3) % 3][j * SW + tap % 3];
+                    const float ta = tap_add(xv, wa[tap]);
+                    const float tb = PAR ? tap_add(xv, wb[tap]) : ta;
+                    if constexpr (WIN) {
+                        // strict compares in ascending tap order: the lowest tap wins a tie
+                        if (DO_MIN && ta < mn[j]) { mn[j] = ta; amn[j] = tap; }
+                        if (DO_MAX && tb > mx[j]) { mx[j] = tb; amx[j] = tap; }
+                    } else {
+                        if (DO_MIN) mn[j] = fminf(mn[j], ta);
+                        if (DO_MAX) mx[j] = fmaxf(mx[j], tb);
+                    }
+                }
+        }
+        const size_t o = (nc * g.OH + oh0 + k) * (size_t)g.OW + ow0;
+        if (y) {
+            float v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float acc;
+                if constexpr (TWO) acc = __fmaf_rn(b, mx[j], __fmaf_rn(a, mn[j], 0.0f));
+                else acc = __fadd_rn(0.0f, DO_MIN ? mn[j] : mx[j]);
+                v[j] = bias ? __fadd_rn(acc, bk) : acc;
+            }
+            if (full) {
+                if constexpr (sizeof(T) == 4) {
+                    *reinterpret_cast<float4*>(y + o) = make_float4(v[0], v[1], v[2], v[3]);
+                } else {
+                    const __nv_bfloat162 p01 = __floats2bfloat162_rn(v[0], v[1]);
+                    const __nv_bfloat162 p23 = __floats2bfloat162_rn(v[2], v[3]);
+                    *reinterpret_cast<uint2*>(y + o) = make_uint2(*reinterpret_cast<const unsigned*>(&p01),
+                                                                  *reinterpret_cast<const unsigned*>(&p23));
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (ow0 + j < g.OW) y[o + j] = from_f32<T>(v[j]);
+            }
+        }
+        if constexpr (WIN) {
+            unsigned packed = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const unsigned code = (DO_MIN ? (unsigned)amn[j] : 0u) | (DO_MAX ? (unsigned)amx[j] << 4 : 0u);
+                packed |= code << (8 * j);
+            }
+            if (full) {
+                *reinterpret_cast<unsigned*>(codes + o) = packed;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (ow0 + j < g.OW) codes[o + j] = (uint8_t)(packed >> (8 * j));
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------- grad_x
 // Gather form: one thread per input element visits, in ascending tap order, the outputs that read
 // it, and takes coef * grad_y from those whose winner is that tap.  No atomics, fixed order.
 // BR: 0 both branches, 1 min branch only, 2 max branch only.
-template <typename T, int BR>
+// ST: 0 = strides from the descriptor, 2 = both strides are 2 (shifts instead of divisions).
+template <typename T, int BR, int ST>
 __global__ void __launch_bounds__(256)
 dw_bwd_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
                  const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
@@ -133,13 +308,13 @@ dw_bwd_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict
     float acc = 0.0f;
     for (int r = 0; r < g.R; ++r) {
         const int nh = ih + g.ph - r * g.dh;
-        if (nh < 0 || nh % g.sh != 0) continue;
-        const int oh = nh / g.sh;
+        if (nh < 0 || (ST == 2 ? (nh & 1) : nh % g.sh) != 0) continue;
+        const int oh = ST == 2 ? nh >> 1 : nh / g.sh;
         if (oh >= g.OH) continue;
         for (int s = 0; s < g.S; ++s) {
             const int nw = iw + g.pw - s * g.dw;
-            if (nw < 0 || nw % g.sw != 0) continue;
-            const int ow = nw / g.sw;
+            if (nw < 0 || (ST == 2 ? (nw & 1) : nw % g.sw) != 0) continue;
+            const int ow = ST == 2 ? nw >> 1 : nw / g.sw;
             if (ow >= g.OW) continue;
             const unsigned tap = (unsigned)(r * g.S + s);
             const unsigned code = __ldg(cp + (size_t)oh * g.OW + ow);
@@ -149,6 +324,96 @@ dw_bwd_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict
         }
     }
     gx[i] = from_f32<T>(acc);
+}
+
+// grad_x for 3x3 windows, stride 1, dilation 1: a thread owns a strip of 4 input columns x RT
+// input rows and slides a window of three rows of (grad_y, winner code) down it.  Input (ih, iw)
+// is read by output (ih + ph - r, iw + pw - s) through tap (r, s); the contributions are taken in
+// ascending tap order.  Outputs outside the plane load as gradient 0.
+template <int L, bool VEC>
+__device__ __forceinline__ void dw_load_codes(const uint8_t* cr, int c0, int W, unsigned* out) {
+    if (cr && c0 >= 0 && c0 + L <= W) {
+        if constexpr (VEC) {
+            out[0] = __ldg(cr + c0);
+#pragma unroll
+            for (int i = 1; i + 4 <= L; i += 4) {
+                const unsigned v = __ldg(reinterpret_cast<const unsigned*>(cr + c0 + i));
+                out[i] = v & 0xffu; out[i + 1] = (v >> 8) & 0xffu; out[i + 2] = (v >> 16) & 0xffu; out[i + 3] = v >> 24;
+            }
+#pragma unroll
+            for (int i = 1 + ((L - 1) / 4) * 4; i < L; ++i) out[i] = __ldg(cr + c0 + i);
+        } else {
+#pragma unroll
+            for (int i = 0; i < L; ++i) out[i] = __ldg(cr + c0 + i);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < L; ++i) out[i] = (cr && c0 + i >= 0 && c0 + i < W) ? __ldg(cr + c0 + i) : 0u;
+    }
+}
+
+template <typename T, int BR, bool VEC>
+__global__ void __launch_bounds__(256)
+dw_bwd_gx3_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
+                  const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
+                  int QPR, int strips, unsigned total) {
+    constexpr int RT = 6, L = 6;
+    const unsigned q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= total) return;
+    const unsigned t = q / (unsigned)QPR;
+    const int qx = (int)(q - t * (unsigned)QPR);
+    const size_t nc = t / (unsigned)strips;
+    const int ih0 = (int)(t - (unsigned)nc * (unsigned)strips) * RT;
+    const int c = (int)((unsigned)nc % (unsigned)g.C);
+    const int iw0 = qx * 4;
+    const float a = (BR == 0 && alpha) ? alpha[c] : 1.0f, b = (BR == 0 && beta) ? beta[c] : 1.0f;
+    const T* gp = gy + nc * (size_t)g.OH * g.OW;
+    const uint8_t* cp = codes + nc * (size_t)g.OH * g.OW;
+    const int ob = ih0 + g.ph - 2, c0 = iw0 + g.pw - 2;   // first output row / column of the window
+    const bool full = (iw0 + 3 < g.W) && ((g.W & 3) == 0);
+    T gw_[3][L];
+    unsigned cw[3][L];
+    auto load = [&](int rho) {
+        const int oh = ob + rho;
+        const bool ok = oh >= 0 && oh < g.OH;
+        dw_load_row<T, L, VEC>(ok ? gp + (size_t)oh * g.OW : nullptr, c0, g.OW, gw_[rho % 3]);
+        dw_load_codes<L, VEC>(ok ? cp + (size_t)oh * g.OW : nullptr, c0, g.OW, cw[rho % 3]);
+    };
+    load(0);
+    load(1);
+#pragma unroll
+    for (int k = 0; k < RT; ++k) {
+        if (ih0 + k >= g.H) break;
+        load(k + 2);
+        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int r = 0; r < 3; ++r)
+#pragma unroll
+            for (int sx = 0; sx < 3; ++sx)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const unsigned code = cw[(k + 2 - r) % 3][j + 2 - sx];
+                    const float gv = to_f32(gw_[(k + 2 - r) % 3][j + 2 - sx]);
+                    const unsigned tap = (unsigned)(r * 3 + sx);
+                    if ((BR == 0 || BR == 1) && (code & 15u) == tap) acc[j] = (BR == 0) ? __fmaf_rn(a, gv, acc[j]) : acc[j] + gv;
+                    if ((BR == 0 || BR == 2) && (code >> 4) == tap) acc[j] = (BR == 0) ? __fmaf_rn(b, gv, acc[j]) : acc[j] + gv;
+                }
+        const size_t o = (nc * g.H + ih0 + k) * (size_t)g.W + iw0;
+        if (full) {
+            if constexpr (sizeof(T) == 4) {
+                *reinterpret_cast<float4*>(gx + o) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            } else {
+                const __nv_bfloat162 p01 = __floats2bfloat162_rn(acc[0], acc[1]);
+                const __nv_bfloat162 p23 = __floats2bfloat162_rn(acc[2], acc[3]);
+                *reinterpret_cast<uint2*>(gx + o) = make_uint2(*reinterpret_cast<const unsigned*>(&p01),
+                                                               *reinterpret_cast<const unsigned*>(&p23));
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (iw0 + j < g.W) gx[o + j] = from_f32<T>(acc[j]);
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------- parameter gradients
