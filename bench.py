@@ -475,6 +475,62 @@ def run_cfg5(args):
                       "loss": float(loss.detach())}))
 
 
+def run_dw(args):
+    """Depthwise (groups = C) layer of a MobileNetV2-shaped stage: N=128, C=144, 56x56, 3x3, stride 1,
+    pad 1 (the expanded 24-channel stage at t=6), mode --only (default compound), --dtype.  The form is
+    memory bound (9 taps per output): forward, forward with winner codes and backward are reported as
+    algorithmic GB/s against the measured copy bandwidth."""
+    import torch
+    from paper_2504_06881_b200 import inputs, tconv
+    torch.cuda.set_device(0)
+    mode = args.only or "compound"
+    N, C, H, W = args.images, 144, 56, 56
+    d = inputs.layer(N, C, H, W, C, 3, 3, stride=1, pad=1, mode=mode, dtype=args.dtype)
+    dt = tconv.TORCH_DTYPE[args.dtype]
+    es = 4 if args.dtype == "f32" else 2
+    rs = np.random.RandomState(1060)
+    f = lambda *sh: torch.from_numpy(rs.standard_normal(sh).astype(np.float32)).cuda()
+    x, g = f(N, C, H, W).to(dt), f(N, C, H, W).to(dt)
+    w, w2 = (0.1 * f(C, 3, 3)).to(dt), (0.1 * f(C, 3, 3)).to(dt)
+    al, be, bias = torch.rand(C, device="cuda"), torch.rand(C, device="cuda"), torch.rand(C, device="cuda")
+    two, par = mode in ("compound", "parallel"), mode == "parallel"
+    y = torch.empty(N, C, H, W, device="cuda", dtype=dt)
+    win = torch.empty(N, C, H, W, device="cuda", dtype=torch.uint8)
+    ws = torch.empty(tconv.tconv_dw_workspace_bytes(d, True), dtype=torch.uint8, device="cuda")
+    gx = torch.empty_like(x)
+    gw, gw2 = torch.empty(C, 3, 3, device="cuda"), torch.empty(C, 3, 3, device="cuda")
+    ga, gb, gbi = (torch.empty(C, device="cuda") for _ in range(3))
+    fa = (d, x, w, w2 if par else None, al if two else None, be if two else None, bias, y)
+    calls = {"fwd": lambda: tconv.tconv_dw_forward(*fa, None),
+             "fwd_winners": lambda: tconv.tconv_dw_forward(*fa, win),
+             "bwd": lambda: tconv.tconv_dw_backward(d, x, w, w2 if par else None, al if two else None,
+                                                    be if two else None, g, win, gx, gw, gw2 if par else None,
+                                                    ga if two else None, gb if two else None, gbi, ws)}
+    peaks_file = Path(__file__).parent / "MEASURED_PEAKS.json"
+    hbm, src = (json.loads(peaks_file.read_text())["hbm_gbs"], "measured") if peaks_file.exists() else (6650.0, "fallback")
+    n = N * C * H * W
+    # algorithmic bytes: x once, y once (+ one code byte per output); backward: grad_y and codes for
+    # grad_x plus grad_y, codes and x for the parameter gradients, grad_x written once
+    nbytes = {"fwd": 2 * n * es, "fwd_winners": 2 * n * es + n, "bwd": (n * es + n + n * es) + (2 * n * es + n)}
+    out = {"workload": f"depthwise {mode} {args.dtype}: N={N} C={C} {H}x{W} 3x3 s1 p1", "hbm_peak_GB_s": hbm,
+           "hbm_peak_source": src}
+    for name, fn in calls.items():
+        assert fn() == 0, tconv.tconv_last_error()
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(max(args.steps, 5)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        ms = float(np.median(ts))
+        out[name] = {"ms": ms, "GB_s": nbytes[name] / ms / 1e6, "frac_of_hbm": nbytes[name] / ms / 1e6 / hbm,
+                     "kernel": tconv.tconv_last_kernel()}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -486,13 +542,16 @@ def main():
     ap.add_argument("--what", default="fwd", choices=["fwd", "fwd_winners", "bwd"])
     ap.add_argument("--images", type=int, default=128)
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5"],
-                    help="cfg5: report the hybrid ResNet-18 training step instead (use --only compound|parallel)")
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5", "dw"],
+                    help="cfg5: report the hybrid ResNet-18 training step instead (use --only compound|parallel); "
+                         "dw: a depthwise (groups = C) layer against the HBM roofline")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "cfg5":
         run_cfg5(args)
+    elif args.workload == "dw":
+        run_dw(args)
     elif args.only:
         run_single(args)
     else:

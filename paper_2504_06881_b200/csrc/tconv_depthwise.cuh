@@ -131,26 +131,36 @@ __device__ __forceinline__ void load4(const __nv_bfloat16* p, __nv_bfloat16* out
     const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&v.y);
     out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
 }
-// L consecutive elements of an input row starting at column c0 (zero outside the row; the whole
-// row is zero when xr is NULL).  VEC: c0 + 1 is a multiple of 4 and rows start on 4-element
-// boundaries, so the middle of an interior segment is read with aligned 4-element loads.
+// L consecutive elements of a row, starting at column c0, in a single code path: bit i of `mask`
+// says whether column c0 + i lies inside the row (computed once per thread); `rp` points at column
+// c0 of the row (it is dereferenced only where the mask allows); a row outside the plane
+// (row_ok false) reads as zero.  VEC: c0 + 1 is a multiple of 4 and rows start on 4-element
+// boundaries, so every group of 4 from c0 + 1 on is wholly inside or wholly outside the row and
+// is read with one aligned load.
+__device__ __forceinline__ unsigned dw_col_mask(int c0, int L, int W) {
+    unsigned m = 0;
+    for (int i = 0; i < L; ++i)
+        if (c0 + i >= 0 && c0 + i < W) m |= 1u << i;
+    return m;
+}
 template <typename T, int L, bool VEC>
-__device__ __forceinline__ void dw_load_row(const T* xr, int c0, int W, T* out) {
-    if (xr && c0 >= 0 && c0 + L <= W) {
-        if constexpr (VEC) {
-            out[0] = __ldg(xr + c0);
+__device__ __forceinline__ void dw_load_row(const T* rp, bool row_ok, unsigned mask, T* out) {
+    if (!row_ok) mask = 0;
+    if constexpr (VEC) {
+        out[0] = (mask & 1u) ? __ldg(rp) : zero_of<T>();
 #pragma unroll
-            for (int i = 1; i + 4 <= L; i += 4) load4(xr + c0 + i, out + i);
-#pragma unroll
-            for (int i = 1 + ((L - 1) / 4) * 4; i < L; ++i) out[i] = __ldg(xr + c0 + i);
-        } else {
-#pragma unroll
-            for (int i = 0; i < L; ++i) out[i] = __ldg(xr + c0 + i);
+        for (int i = 1; i + 4 <= L; i += 4) {
+            if ((mask >> i) & 1u) {
+                load4(rp + i, out + i);
+            } else {
+                out[i] = out[i + 1] = out[i + 2] = out[i + 3] = zero_of<T>();
+            }
         }
+#pragma unroll
+        for (int i = 1 + ((L - 1) / 4) * 4; i < L; ++i) out[i] = ((mask >> i) & 1u) ? __ldg(rp + i) : zero_of<T>();
     } else {
 #pragma unroll
-        for (int i = 0; i < L; ++i)
-            out[i] = (xr && c0 + i >= 0 && c0 + i < W) ? __ldg(xr + c0 + i) : zero_of<T>();
+        for (int i = 0; i < L; ++i) out[i] = ((mask >> i) & 1u) ? __ldg(rp + i) : zero_of<T>();
     }
 }
 
@@ -190,9 +200,11 @@ dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T*
     const int ih0 = oh0 * SW - g.ph, c0 = ow0 * SW - g.pw;
     const bool full = (ow0 + 3 < g.OW) && ((g.OW & 3) == 0);
     T win[3][L];   // input row rho of the strip lives in win[rho % 3]
+    const unsigned cmask = dw_col_mask(c0, L, g.W);
+    const T* rp0 = xp + (ptrdiff_t)ih0 * g.W + c0;   // column c0 of the strip's first input row
     auto load = [&](int rho) {
         const int ih = ih0 + rho;
-        dw_load_row<T, L, VEC>((ih >= 0 && ih < g.H) ? xp + (size_t)ih * g.W : nullptr, c0, g.W, win[rho % 3]);
+        dw_load_row<T, L, VEC>(rp0 + rho * g.W, ih >= 0 && ih < g.H, cmask, win[rho % 3]);
     };
     load(0);
     load(1);
@@ -331,24 +343,20 @@ dw_bwd_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict
 // is read by output (ih + ph - r, iw + pw - s) through tap (r, s); the contributions are taken in
 // ascending tap order.  Outputs outside the plane load as gradient 0.
 template <int L, bool VEC>
-__device__ __forceinline__ void dw_load_codes(const uint8_t* cr, int c0, int W, unsigned* out) {
-    if (cr && c0 >= 0 && c0 + L <= W) {
-        if constexpr (VEC) {
-            out[0] = __ldg(cr + c0);
+__device__ __forceinline__ void dw_load_codes(const uint8_t* rp, bool row_ok, unsigned mask, unsigned* out) {
+    if (!row_ok) mask = 0;
+    if constexpr (VEC) {
+        out[0] = (mask & 1u) ? __ldg(rp) : 0u;
 #pragma unroll
-            for (int i = 1; i + 4 <= L; i += 4) {
-                const unsigned v = __ldg(reinterpret_cast<const unsigned*>(cr + c0 + i));
-                out[i] = v & 0xffu; out[i + 1] = (v >> 8) & 0xffu; out[i + 2] = (v >> 16) & 0xffu; out[i + 3] = v >> 24;
-            }
-#pragma unroll
-            for (int i = 1 + ((L - 1) / 4) * 4; i < L; ++i) out[i] = __ldg(cr + c0 + i);
-        } else {
-#pragma unroll
-            for (int i = 0; i < L; ++i) out[i] = __ldg(cr + c0 + i);
+        for (int i = 1; i + 4 <= L; i += 4) {
+            const unsigned v = ((mask >> i) & 1u) ? __ldg(reinterpret_cast<const unsigned*>(rp + i)) : 0u;
+            out[i] = v & 0xffu; out[i + 1] = (v >> 8) & 0xffu; out[i + 2] = (v >> 16) & 0xffu; out[i + 3] = v >> 24;
         }
+#pragma unroll
+        for (int i = 1 + ((L - 1) / 4) * 4; i < L; ++i) out[i] = ((mask >> i) & 1u) ? __ldg(rp + i) : 0u;
     } else {
 #pragma unroll
-        for (int i = 0; i < L; ++i) out[i] = (cr && c0 + i >= 0 && c0 + i < W) ? __ldg(cr + c0 + i) : 0u;
+        for (int i = 0; i < L; ++i) out[i] = ((mask >> i) & 1u) ? __ldg(rp + i) : 0u;
     }
 }
 
@@ -373,11 +381,14 @@ dw_bwd_gx3_kernel(Geo g, const float* __restrict__ alpha, const float* __restric
     const bool full = (iw0 + 3 < g.W) && ((g.W & 3) == 0);
     T gw_[3][L];
     unsigned cw[3][L];
+    const unsigned cmask = dw_col_mask(c0, L, g.OW);
+    const T* grp0 = gp + (ptrdiff_t)ob * g.OW + c0;
+    const uint8_t* crp0 = cp + (ptrdiff_t)ob * g.OW + c0;
     auto load = [&](int rho) {
         const int oh = ob + rho;
         const bool ok = oh >= 0 && oh < g.OH;
-        dw_load_row<T, L, VEC>(ok ? gp + (size_t)oh * g.OW : nullptr, c0, g.OW, gw_[rho % 3]);
-        dw_load_codes<L, VEC>(ok ? cp + (size_t)oh * g.OW : nullptr, c0, g.OW, cw[rho % 3]);
+        dw_load_row<T, L, VEC>(grp0 + rho * g.OW, ok, cmask, gw_[rho % 3]);
+        dw_load_codes<L, VEC>(crp0 + rho * g.OW, ok, cmask, cw[rho % 3]);
     };
     load(0);
     load(1);
