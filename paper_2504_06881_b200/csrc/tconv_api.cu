@@ -362,7 +362,7 @@ int dw_forward_t(const Geo& g, const void* x, const void* w, const void* w2, con
     const int QPR = (g.OW + 3) / 4;
     if (g.R == 3 && g.S == 3 && g.dh == 1 && g.dw == 1 && g.sh == g.sw && (g.sw == 1 || g.sw == 2)) {
         // 3x3 windows: strips of 4 columns x 6 rows with a register window of three input rows
-        const int strips = (g.OH + 5) / 6;
+        const int strips = (g.OH + TCONV_DW_RT - 1) / TCONV_DW_RT;
         const size_t total3 = (size_t)g.N * g.C * strips * QPR;
         const unsigned blocks3 = (unsigned)((total3 + 255) / 256);
         const bool vec = (g.pw == 1 && (g.W & 3) == 0);

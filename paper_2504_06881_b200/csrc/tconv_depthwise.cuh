@@ -113,13 +113,12 @@ dw_fwd_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* 
 }
 
 // ---------------------------------------------------------------------------------- forward, 3x3 windows
-// {lo, hi} = {x0 + w, x1 + w}: one packed fp32 add for two horizontally adjacent pixels.
-__device__ __forceinline__ void add2px(float x0, float x1, float w, float& lo, float& hi) {
-    unsigned long long xx, ww, tt;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(xx) : "f"(x0), "f"(x1));
-    asm("mov.b64 %0, {%1, %1};" : "=l"(ww) : "f"(w));
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(tt) : "l"(xx), "l"(ww));
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
+// extremum of nine values with 3-input min / max (3 + 2 + 2 + 2)
+__device__ __forceinline__ float dw_fold9(const float* v, bool is_min) {
+    float m = ext3(v[0], v[1], v[2], is_min);
+    m = ext3(m, v[3], v[4], is_min);
+    m = ext3(m, v[5], v[6], is_min);
+    return ext3(m, v[7], v[8], is_min);
 }
 __device__ __forceinline__ void load4(const float* p, float* out) {
     const float4 v = __ldg(reinterpret_cast<const float4*>(p));
@@ -174,7 +173,10 @@ dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T*
                const float* __restrict__ alpha, const float* __restrict__ beta,
                const float* __restrict__ bias, T* __restrict__ y, uint8_t* __restrict__ codes,
                int QPR, int strips, unsigned total) {
-    constexpr int RT = 6;                       // output rows per strip
+#ifndef TCONV_DW_RT
+#define TCONV_DW_RT 6
+#endif
+    constexpr int RT = TCONV_DW_RT;             // output rows per strip
     constexpr int L = 3 * SW + 3;               // input columns 4 outputs touch
     constexpr int NROWS = (RT - 1) * SW + 3;    // input rows a strip touches
     constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
@@ -213,46 +215,47 @@ dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T*
         if (oh0 + k >= g.OH) break;
 #pragma unroll
         for (int rho = (k == 0 ? 2 : (k - 1) * SW + 3); rho <= k * SW + 2; ++rho) load(rho);
+        // per pixel: nine tap sums, their extrema with 3-input min / max and, for the winner codes,
+        // the first tap that attains each extremum, recovered on the FMA pipe: d = (t - m) * 2^32 is
+        // zero exactly for winning taps, key = |d| * (-2^125) + (2^23 + rank) is 2^23 + rank for them
+        // and below 2^23 otherwise, the largest key belongs to the lowest winning tap and carries
+        // rank = 15 - tap (min branch) or 16 * (15 - tap) (max branch) in its low mantissa bits
+        // (|x + w| < 2^95 assumed)
         float mn[4], mx[4];
-        int amn[4] = {0, 0, 0, 0}, amx[4] = {0, 0, 0, 0};
-        if constexpr (sizeof(T) == 4 && !WIN) {
-            // packed adds over pixel pairs, 3-input min / max chains (3 + 2 + 2 + 2 taps)
+        unsigned code4[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int jp = 0; jp < 2; ++jp) {
-                float ta[9][2], tb[PAR ? 9 : 1][2];
+        for (int j = 0; j < 4; ++j) {
+            float ta[9], tb[PAR ? 9 : 1];
 #pragma unroll
-                for (int tap = 0; tap < 9; ++tap) {
-                    const float* row = reinterpret_cast<const float*>(win[(k * SW + tap / 3) % 3]);
-                    const float x0 = row[(2 * jp) * SW + tap % 3], x1 = row[(2 * jp + 1) * SW + tap % 3];
-                    add2px(x0, x1, to_f32(wa[tap]), ta[tap][0], ta[tap][1]);
-                    if constexpr (PAR) add2px(x0, x1, to_f32(wb[tap]), tb[tap][0], tb[tap][1]);
-                }
-                const float (*tm)[2] = PAR ? tb : ta;
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    if constexpr (DO_MIN) mn[2 * jp + h] = fold_taps<9>(ta, h, true);
-                    if constexpr (DO_MAX) mx[2 * jp + h] = fold_taps<9>(tm, h, false);
-                }
+            for (int tap = 0; tap < 9; ++tap) {
+                const T xv = win[(k * SW + tap / 3) % 3][j * SW + tap % 3];
+                ta[tap] = tap_add(xv, wa[tap]);
+                if constexpr (PAR) tb[tap] = tap_add(xv, wb[tap]);
             }
-        } else {
+            const float* tm = PAR ? tb : ta;
+            if constexpr (DO_MIN) mn[j] = dw_fold9(ta, true);
+            if constexpr (DO_MAX) mx[j] = dw_fold9(tm, false);
+            if constexpr (WIN) {
+                constexpr float kS = 4294967296.0f, kH = 4.253529586511731e37f, kB = 8388608.0f;
+                unsigned bmn = 0u, bmx = 0u;
+                if constexpr (DO_MIN) {
+                    const float e = -mn[j] * kS;
+                    float key[9];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { mn[j] = INFINITY; mx[j] = -INFINITY; }
-#pragma unroll
-            for (int tap = 0; tap < 9; ++tap)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const T xv = win[(k * SW + tap / 3) % 3][j * SW + tap % 3];
-                    const float ta = tap_add(xv, wa[tap]);
-                    const float tb = PAR ? tap_add(xv, wb[tap]) : ta;
-                    if constexpr (WIN) {
-                        // strict compares in ascending tap order: the lowest tap wins a tie
-                        if (DO_MIN && ta < mn[j]) { mn[j] = ta; amn[j] = tap; }
-                        if (DO_MAX && tb > mx[j]) { mx[j] = tb; amx[j] = tap; }
-                    } else {
-                        if (DO_MIN) mn[j] = fminf(mn[j], ta);
-                        if (DO_MAX) mx[j] = fmaxf(mx[j], tb);
-                    }
+                    for (int tap = 0; tap < 9; ++tap)
+                        key[tap] = __fmaf_rn(-kH, __fmaf_rn(kS, ta[tap], e), kB + (float)(15 - tap));
+                    bmn = __float_as_uint(dw_fold9(key, false));
                 }
+                if constexpr (DO_MAX) {
+                    const float e = -mx[j] * kS;
+                    float key[9];
+#pragma unroll
+                    for (int tap = 0; tap < 9; ++tap)
+                        key[tap] = __fmaf_rn(kH, __fmaf_rn(kS, tm[tap], e), kB + (float)(16 * (15 - tap)));
+                    bmx = __float_as_uint(dw_fold9(key, false));
+                }
+                code4[j] = (DO_MIN ? (~bmn & 0x0fu) : 0u) | (DO_MAX ? (~bmx & 0xf0u) : 0u);
+            }
         }
         const size_t o = (nc * g.OH + oh0 + k) * (size_t)g.OW + ow0;
         if (y) {
@@ -280,12 +283,7 @@ dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T*
             }
         }
         if constexpr (WIN) {
-            unsigned packed = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const unsigned code = (DO_MIN ? (unsigned)amn[j] : 0u) | (DO_MAX ? (unsigned)amx[j] << 4 : 0u);
-                packed |= code << (8 * j);
-            }
+            const unsigned packed = code4[0] | (code4[1] << 8) | (code4[2] << 16) | (code4[3] << 24);
             if (full) {
                 *reinterpret_cast<unsigned*>(codes + o) = packed;
             } else {
