@@ -34,3 +34,7 @@ ParallelMinMaxPlusSumConv2d1p = _named("ParallelMinMaxPlusSumConv2d1p", "paralle
 ParallelMinMaxPlusSumConv2d2p = _named("ParallelMinMaxPlusSumConv2d2p", "parallel", params="2p", doc="parallel mode, learnable alpha and beta")
 
 __all__ = [n for n in dir() if n.endswith(("Conv2d", "0p", "1p", "2p"))]
+
+from .nn import TropicalDepthwiseConv2d  # noqa: E402  (depthwise form of the MobileNetV2 variants)
+
+__all__.append("TropicalDepthwiseConv2d")

@@ -194,3 +194,90 @@ class HybridResNet18(nn.Module):
 
     def tropical_layers(self):
         return [m for m in self.modules() if isinstance(m, TropicalConv2d)]
+
+
+class TropicalDepthwiseFn(torch.autograd.Function):
+    """Depthwise (groups = C) form over tconv_dw_forward / tconv_dw_backward; see TropicalConvFn."""
+
+    @staticmethod
+    def forward(ctx, x, w, w2, alpha, beta, bias, geom):
+        mode, dtype, stride, pad, dil = geom
+        dt = tconv.TORCH_DTYPE[dtype]
+        N, C, H, W = x.shape
+        _, R, S = w.shape
+        d = dict(N=N, C=C, H=H, W=W, K=C, R=R, S=S, stride_h=stride[0], stride_w=stride[1],
+                 pad_h=pad[0], pad_w=pad[1], dil_h=dil[0], dil_w=dil[1], mode=mode, chan="sum", dtype=dtype)
+        xc = x.detach().to(dt).contiguous()
+        wc = w.detach().to(dt).contiguous()
+        w2c = w2.detach().to(dt).contiguous() if w2 is not None else None
+        al = alpha.detach().float().contiguous() if alpha is not None else None
+        be = beta.detach().float().contiguous() if beta is not None else None
+        bi = bias.detach().float().contiguous() if bias is not None else None
+        need_grad = any(t is not None and t.requires_grad for t in (x, w, w2, alpha, beta, bias))
+        y, winners = tconv.dw_forward(d, xc, wc, w2c, al, be, bi, want_winners=need_grad)
+        ctx.d, ctx.in_dtype = d, x.dtype
+        ctx.save_for_backward(xc, wc, w2c, al, be, winners)
+        ctx.has = (w2 is not None, alpha is not None, beta is not None, bias is not None)
+        return y.to(x.dtype) if x.dtype != dt else y
+
+    @staticmethod
+    def backward(ctx, gy):
+        xc, wc, w2c, al, be, winners = ctx.saved_tensors
+        d = ctx.d
+        g = gy.to(tconv.TORCH_DTYPE[d["dtype"]]).contiguous()
+        grads = tconv.dw_backward(d, xc, wc, g, w2c, al, be, winners)
+        has_w2, has_a, has_b, has_bias = ctx.has
+        return (grads["grad_x"].to(ctx.in_dtype), grads["grad_w"], grads.get("grad_w2") if has_w2 else None,
+                grads.get("grad_alpha") if has_a else None, grads.get("grad_beta") if has_b else None,
+                grads["grad_bias"] if has_bias else None, None)
+
+
+class TropicalDepthwiseConv2d(nn.Module):
+    """Depthwise tropical convolution (``nn.Conv2d(channels, channels, k, groups=channels)``'s place in
+    a MobileNetV2 block): per channel one window of weights, one alpha and one beta.
+
+    mode and params as in TropicalConv2d ("2p", "1p", "shared", "opposite", "0p", "fixed")."""
+
+    def __init__(self, channels, kernel_size, stride=1, padding=0, dilation=1, bias=True,
+                 mode="compound", params="2p", dtype="f32", fixed=(0.5, 0.5)):
+        super().__init__()
+        two = lambda v: (v, v) if isinstance(v, int) else tuple(v)
+        self.kernel_size, self.stride, self.padding, self.dilation = map(two, (kernel_size, stride, padding, dilation))
+        self.channels, self.mode, self.params, self.dtype = channels, mode, params, dtype
+        if params not in TropicalConv2d.PARAMS:
+            raise ValueError(f"params must be one of {TropicalConv2d.PARAMS}")
+        R, S = self.kernel_size
+        self.weight = nn.Parameter(torch.empty(channels, R, S))
+        self.weight2 = nn.Parameter(torch.empty(channels, R, S)) if mode == "parallel" else None
+        two_branch = mode in ("compound", "parallel")
+        self.alpha = nn.Parameter(torch.empty(channels)) if two_branch and params in ("1p", "2p", "shared", "opposite") else None
+        self.beta = nn.Parameter(torch.empty(channels)) if two_branch and params == "2p" else None
+        if two_branch and params == "fixed":
+            self.register_buffer("alpha_fixed", torch.full((channels,), float(fixed[0])))
+            self.register_buffer("beta_fixed", torch.full((channels,), float(fixed[1])))
+        self.bias = nn.Parameter(torch.zeros(channels)) if bias else None
+        bound = 1.0 / math.sqrt(R * S)
+        for w in (self.weight, self.weight2):
+            if w is not None:
+                nn.init.uniform_(w, -bound, bound)
+        for a in (self.alpha, self.beta):
+            if a is not None:
+                nn.init.constant_(a, 0.5)
+
+    def extra_repr(self):
+        return (f"{self.channels}, kernel_size={self.kernel_size}, stride={self.stride}, padding={self.padding}, "
+                f"dilation={self.dilation}, mode={self.mode}, params={self.params}, dtype={self.dtype}")
+
+    def forward(self, x):
+        alpha, beta = self.alpha, self.beta
+        if self.mode in ("compound", "parallel"):
+            if self.params == "1p":
+                beta = 1.0 - alpha
+            elif self.params == "shared":
+                beta = alpha
+            elif self.params == "opposite":
+                beta = -alpha
+            elif self.params == "fixed":
+                alpha, beta = self.alpha_fixed, self.beta_fixed
+        geom = (self.mode, self.dtype, self.stride, self.padding, self.dilation)
+        return TropicalDepthwiseFn.apply(x, self.weight, self.weight2, alpha, beta, self.bias, geom)

@@ -103,3 +103,47 @@ def test_specialisations_against_the_oracle(mode, params):
         assert close(m.alpha.grad, ga + sign * gb, gaa + abs(sign) * gba)
     if m.beta is not None:
         assert close(m.beta.grad, gb, gba)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("mode,params", [("compound", "2p"), ("compound", "1p"), ("parallel", "2p"), ("max_plus", "0p")])
+def test_depthwise_layer_against_the_oracle(mode, params):
+    from oracle import tconv_oracle as ora
+    from paper_2504_06881_b200.nn import TropicalDepthwiseConv2d
+    C = 6
+    d = inputs.layer(2, C, 10, 12, C, 3, 3, stride=1, pad=1, mode=mode)
+    rs = np.random.RandomState(2200)
+    x = rs.standard_normal((2, C, 10, 12)).astype(np.float32)
+    g = rs.standard_normal((2, C, 10, 12)).astype(np.float32)
+    m = TropicalDepthwiseConv2d(C, 3, padding=1, mode=mode, params=params).cuda()
+    two, par = mode in ("compound", "parallel"), mode == "parallel"
+    with torch.no_grad():
+        if m.alpha is not None:
+            m.alpha.copy_(torch.from_numpy(rs.uniform(0, 1, C).astype(np.float32)))
+        if m.beta is not None:
+            m.beta.copy_(torch.from_numpy(rs.uniform(0, 1, C).astype(np.float32)))
+        m.bias.copy_(torch.from_numpy(rs.uniform(-0.1, 0.1, C).astype(np.float32)))
+    w = m.weight.detach().cpu().numpy()
+    w2 = m.weight2.detach().cpu().numpy() if par else None
+    a = m.alpha.detach().cpu().numpy() if m.alpha is not None else None
+    b = (m.beta.detach().cpu().numpy() if m.beta is not None else (1.0 - torch.from_numpy(a)).numpy() if params == "1p" else None)
+    bias = m.bias.detach().cpu().numpy()
+    ref = ora.depthwise_forward(d, x, w, w2, a if two else None, b if two else None, bias)
+    xt = torch.from_numpy(x).cuda().requires_grad_(True)
+    y = m(xt)
+    assert np.array_equal(y.detach().cpu().numpy().view(np.uint32), ref["y"].view(np.uint32))
+    y.backward(torch.from_numpy(g).cuda())
+    gref = ora.depthwise_backward(d, x, w, g, w2, a if two else None, b if two else None)
+
+    def close(got, want, scale):
+        return (np.abs(got.detach().cpu().numpy().astype(np.float64) - want) <= 1e-5 * scale + 1e-30).all()
+
+    assert close(xt.grad, *gref["grad_x"]) and close(m.weight.grad, *gref["grad_w"]) and close(m.bias.grad, *gref["grad_bias"])
+    if par:
+        assert close(m.weight2.grad, *gref["grad_w2"])
+    if m.alpha is not None:
+        (ga, gaa), (gb, gba) = gref["grad_alpha"], gref["grad_beta"]
+        sign = -1.0 if params == "1p" else 0.0
+        assert close(m.alpha.grad, ga + sign * gb, gaa + abs(sign) * gba)
+    if m.beta is not None:
+        assert close(m.beta.grad, *gref["grad_beta"])
