@@ -197,6 +197,7 @@ class Layer:
         self.h_gx = torch.empty((N, C, H, W), dtype=dt).pin_memory()
         self.h_small = {k: torch.empty_like(getattr(self, k), device="cpu").pin_memory()
                         for k in ("gw", "gw2", "ga", "gb", "gbias") if getattr(self, k) is not None}
+        self.ev_done = self.ev_out = None   # last kernels / last device-to-host copies of the e2e leg
 
     def fwd(self, with_winners=True):
         v = self.dev
@@ -219,17 +220,36 @@ class Layer:
         if rc != 0:
             raise self.tconv.TconvError(rc, "tconv_backward")
 
-    def e2e_step(self):
-        """Host buffers in, host buffers out: copies inside the timed region."""
+    def e2e_step(self, torch, s_h2d, s_d2h):
+        """Host buffers in, host buffers out, copies inside the timed region.  The copies run on
+        their own streams so that one layer's transfers overlap the kernels of the others (each layer
+        owns its device buffers): inputs are overwritten only after the previous kernels that read
+        them, outputs only after the previous device-to-host copies of them; the kernels wait for
+        their inputs, the device-to-host copies for the kernels."""
         names = ["x", "w", "bias", "g"] + (["w2"] if self.par else []) + (["alpha", "beta"] if self.two else [])
-        for k in names:
-            self.dev[k].copy_(self.host[k], non_blocking=True)
+        cur = torch.cuda.current_stream()
+        if self.ev_done is not None:
+            s_h2d.wait_event(self.ev_done)
+        with torch.cuda.stream(s_h2d):
+            for k in names:
+                self.dev[k].copy_(self.host[k], non_blocking=True)
+            ev_in = torch.cuda.Event()
+            ev_in.record(s_h2d)
+        cur.wait_event(ev_in)
+        if self.ev_out is not None:
+            cur.wait_event(self.ev_out)
         self.fwd()
         self.bwd()
-        self.h_y.copy_(self.y, non_blocking=True)
-        self.h_gx.copy_(self.gx, non_blocking=True)
-        for k, h in self.h_small.items():
-            h.copy_(getattr(self, k), non_blocking=True)
+        self.ev_done = torch.cuda.Event()
+        self.ev_done.record(cur)
+        s_d2h.wait_event(self.ev_done)
+        with torch.cuda.stream(s_d2h):
+            self.h_y.copy_(self.y, non_blocking=True)
+            self.h_gx.copy_(self.gx, non_blocking=True)
+            for k, h in self.h_small.items():
+                h.copy_(getattr(self, k), non_blocking=True)
+            self.ev_out = torch.cuda.Event()
+            self.ev_out.record(s_d2h)
         h2d = sum(self.host[k].numel() * self.host[k].element_size() for k in names)
         d2h = sum(h.numel() * h.element_size() for h in [self.h_y, self.h_gx] + list(self.h_small.values()))
         return h2d, d2h
@@ -308,9 +328,10 @@ def run_gpu(args):
         raise SystemExit("a device-side wait timed out during the timed region")
 
     # ---- end to end: host buffers in and out, copies inside the timed region
+    s_h2d, s_d2h = torch.cuda.Stream(), torch.cuda.Stream()
     for _ in range(2):
         for L in layers:
-            L.e2e_step()
+            L.e2e_step(torch, s_h2d, s_d2h)
     barrier()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     h2d = d2h = 0
@@ -318,8 +339,10 @@ def run_gpu(args):
     for _ in range(args.steps):
         h2d = d2h = 0
         for L in layers:
-            a, b = L.e2e_step()
+            a, b = L.e2e_step(torch, s_h2d, s_d2h)
             h2d += a; d2h += b
+    for L in layers:                      # the timed region ends when the last result is on the host
+        torch.cuda.current_stream().wait_event(L.ev_out)
     f1.record()
     barrier()
     ms_e2e = f0.elapsed_time(f1)
