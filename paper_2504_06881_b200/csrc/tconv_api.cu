@@ -171,16 +171,27 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                 const unsigned magic = g.RS == 1 ? 0u : (0xFFFFFFFFu / (unsigned)g.RS) + 1u;
                 if (g.RS <= 15) {
                     // the phases of this form are latency-bound: aim at three resident CTAs per SM
+                    // (the tile shares the CTA's shared memory with the staging columns)
+                    const size_t stage = (size_t)kIdxGxKB * 256 * 2 * sizeof(float);
                     int thi2 = thi;
-                    while ((size_t)g.C * g.W * sizeof(float) * thi2 > 72 * 1024 &&
+                    while (((size_t)g.C * g.W * sizeof(float) * thi2 + stage > 73 * 1024 ||
+                            (size_t)g.C * g.W * sizeof(float) * thi2 + stage > kBwdSmemAttr) &&
                            (thi2 + 1) / 2 >= 2 * (g.R - 1) * g.dh && thi2 > 4)
                         thi2 = (thi2 + 1) / 2;
-                    auto kern = bwd_idx_gx2_kernel<T>;
+                    if ((size_t)g.C * g.W * sizeof(float) * thi2 + stage > kBwdSmemAttr) thi2 = 0;
+                    auto kern = g.RS == 9 ? bwd_idx_gx2_kernel<T, 9> : bwd_idx_gx2_kernel<T, 0>;
                     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess)
                         return cuda_fail(cudaGetLastError());
-                    const int tiles2 = (g.H + thi2 - 1) / thi2;
-                    kern<<<(unsigned)(g.N * tiles2), 256, (size_t)g.C * g.W * sizeof(float) * thi2, st>>>(
-                        g, (const T*)gy, idx, (T*)gx, thi2, tiles2, magic);
+                    if (thi2 > 0) {
+                        const int tiles2 = (g.H + thi2 - 1) / thi2;
+                        kern<<<(unsigned)(g.N * tiles2), 256, (size_t)g.C * g.W * sizeof(float) * thi2 + stage, st>>>(
+                            g, (const T*)gy, idx, (T*)gx, thi2, tiles2, magic);
+                    } else {
+                        auto kern1 = bwd_idx_gx_kernel<T>;
+                        if (cudaFuncSetAttribute(kern1, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess)
+                            return cuda_fail(cudaGetLastError());
+                        kern1<<<(unsigned)(g.N * tiles), 256, smem, st>>>(g, (const T*)gy, idx, (T*)gx, thi, tiles, magic);
+                    }
                 } else {
                     auto kern = bwd_idx_gx_kernel<T>;
                     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess)

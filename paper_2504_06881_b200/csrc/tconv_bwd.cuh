@@ -77,15 +77,23 @@ bwd_idx_gx_kernel(Geo g, const T* __restrict__ gy, const int32_t* __restrict__ i
 // 64 output channels).  In the phase of tap t it finds the channels whose winner is t with a few
 // bit operations and touches only those: it reloads their winner (for the input channel) and
 // their grad_y, the loads of the next match in flight while the current one is accumulated.
-template <typename T>
+constexpr int kIdxGxKB = 16;   // output channels per staging round of bwd_idx_gx2_kernel
+// RST: taps of the window when known at compile time (9: the tap loop unrolls and the targets of
+// the nine phases are computed once per pixel), 0: taken from the descriptor.
+template <typename T, int RST>
 __global__ void __launch_bounds__(256)
 bwd_idx_gx2_kernel(Geo g, const T* __restrict__ gy, const int32_t* __restrict__ idx,
                    T* __restrict__ gx, int THI, int tiles_per_img, unsigned magic) {
-    extern __shared__ float tile[];  // [C][THI][W]
+    constexpr int KB = kIdxGxKB;     // output channels staged per round
+    constexpr int NOFF = RST > 0 ? RST : 1;
+    extern __shared__ float tile[];  // [C][THI][W] | gs[KB][256] | cs[KB][256]
     const int n = blockIdx.x / tiles_per_img;
     const int ih0 = (blockIdx.x - n * tiles_per_img) * THI;
     const int rows = min(THI, g.H - ih0);
     const int cstride = THI * g.W;
+    // thread-private columns: gradient and winning channel of the round's output channels
+    float* gs = tile + (size_t)g.C * cstride + threadIdx.x;
+    unsigned* cs = reinterpret_cast<unsigned*>(tile + (size_t)g.C * cstride + KB * 256) + threadIdx.x;
     for (int e = threadIdx.x; e < g.C * cstride; e += blockDim.x) tile[e] = 0.0f;
     const int num = ih0 + g.ph - (g.R - 1) * g.dh;
     const int oh_lo = num <= 0 ? 0 : (num + g.sh - 1) / g.sh;
@@ -99,40 +107,54 @@ bwd_idx_gx2_kernel(Geo g, const T* __restrict__ gy, const int32_t* __restrict__ 
         const bool live = pp < npix;
         const int orow = live ? pp / g.OW : 0;
         const int oh = oh_lo + orow, ow = live ? pp - orow * g.OW : 0;
-        for (int kb0 = 0; kb0 < g.K; kb0 += 64) {
-            const int kn = min(64, g.K - kb0);
-            const int32_t* ip = idx + img + (size_t)kb0 * plane + pp;
-            const T* gp = gy + img + (size_t)kb0 * plane + pp;
-            // taps of the 64 winners, 4 bits each; 15 marks "no channel here"
-            unsigned taps4[8];
+        // element of the tile that tap t of this pixel reaches, -1 if outside the CTA's band
+        auto target = [&](int tap) {
+            const int r = tap / g.S, sx = tap - r * g.S;
+            const int ih = oh * g.sh - g.ph + r * g.dh;
+            const int iw = ow * g.sw - g.pw + sx * g.dw;
+            return (live && ih >= ih0 && ih < ih0 + rows && iw >= 0 && iw < g.W) ? (ih - ih0) * g.W + iw : -1;
+        };
+        int off[NOFF];
+        if constexpr (RST > 0) {
 #pragma unroll
-            for (int wq = 0; wq < 8; ++wq) {
-                unsigned id[8];
+            for (int tap = 0; tap < RST; ++tap) off[tap] = target(tap);
+        }
+        const int32_t* ip = idx + img + pp;
+        const T* gp = gy + img + pp;
+        for (int kb0 = 0; kb0 < g.K; kb0 += KB, ip += (size_t)KB * plane, gp += (size_t)KB * plane) {
+            const int kn = min(KB, g.K - kb0);
+            // one round: KB winners and gradients of this pixel, all loads independent; the taps
+            // stay in registers as 4-bit fields (15 marks "no channel here"), channel and gradient
+            // go to the thread's shared-memory columns so that the phases below touch no global memory
+            unsigned id[KB];
+            float gv[KB];
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    id[i] = (live && wq * 8 + i < kn) ? (unsigned)__ldg(ip + (size_t)(wq * 8 + i) * plane) : 0xffffffffu;
+            for (int i = 0; i < KB; ++i) {
+                const bool ok = live && i < kn;
+                id[i] = ok ? (unsigned)__ldg(ip + (size_t)i * plane) : 0xffffffffu;
+                gv[i] = ok ? to_f32(__ldg(gp + (size_t)i * plane)) : 0.0f;
+            }
+            unsigned taps4[KB / 8];
+#pragma unroll
+            for (int wq = 0; wq < KB / 8; ++wq) {
                 unsigned packed = 0;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const unsigned c = magic ? __umulhi(id[i], magic) : id[i];
-                    const unsigned tap = (id[i] == 0xffffffffu) ? 15u : (id[i] - c * g.RS);
+                    const unsigned v = id[wq * 8 + i];
+                    const unsigned c = magic ? __umulhi(v, magic) : v;
+                    const unsigned tap = (v == 0xffffffffu) ? 15u : (v - c * g.RS);
                     packed |= tap << (4 * i);
+                    cs[(wq * 8 + i) * 256] = c;
+                    gs[(wq * 8 + i) * 256] = gv[wq * 8 + i];
                 }
                 taps4[wq] = packed;
             }
-            for (int tap = 0; tap < g.RS; ++tap) {
-                const int r = tap / g.S, sx = tap - r * g.S;
-                const int ih = oh * g.sh - g.ph + r * g.dh;
-                const int iw = ow * g.sw - g.pw + sx * g.dw;
-                if (live && ih >= ih0 && ih < ih0 + rows && iw >= 0 && iw < g.W) {
-                    float* dst = tile + (ih - ih0) * g.W + iw;
+            auto phase = [&](int tap, int o) {
+                if (o >= 0) {
+                    float* dst = tile + o;
                     const unsigned pat = 0x11111111u * (unsigned)tap;
-                    // software pipeline over the matches: (id, gv) of the next one are loaded first
-                    bool have = false;
-                    unsigned id_cur = 0;
-                    float gv_cur = 0.0f;
 #pragma unroll
-                    for (int wq = 0; wq < 8; ++wq) {
+                    for (int wq = 0; wq < KB / 8; ++wq) {
                         unsigned z = taps4[wq] ^ pat;       // nibble == 0 where the tap matches
                         z |= z >> 1;
                         z |= z >> 2;
@@ -140,23 +162,17 @@ bwd_idx_gx2_kernel(Geo g, const T* __restrict__ gy, const int32_t* __restrict__ 
                         while (m) {
                             const int kk = wq * 8 + ((__ffs(m) - 1) >> 2);
                             m &= m - 1;
-                            const unsigned id_nxt = (unsigned)__ldg(ip + (size_t)kk * plane);
-                            const float gv_nxt = to_f32(gp[(size_t)kk * plane]);
-                            if (have) {
-                                const unsigned c = magic ? __umulhi(id_cur, magic) : id_cur;
-                                dst[c * cstride] += gv_cur;
-                            }
-                            id_cur = id_nxt;
-                            gv_cur = gv_nxt;
-                            have = true;
+                            dst[cs[kk * 256] * cstride] += gs[kk * 256];
                         }
                     }
-                    if (have) {
-                        const unsigned c = magic ? __umulhi(id_cur, magic) : id_cur;
-                        dst[c * cstride] += gv_cur;
-                    }
                 }
-                __syncthreads();
+                __syncthreads();   // inside one phase distinct pixels hit distinct inputs; phases are ordered
+            };
+            if constexpr (RST > 0) {
+#pragma unroll
+                for (int tap = 0; tap < RST; ++tap) phase(tap, off[tap]);
+            } else {
+                for (int tap = 0; tap < g.RS; ++tap) phase(tap, target(tap));
             }
         }
     }

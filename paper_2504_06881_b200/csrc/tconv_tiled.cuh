@@ -743,8 +743,8 @@ struct TiledPlan {
 };
 
 inline size_t tiled_ws_bytes(const Geo& g) {
-    // upper bound over every tile choice: K padded to 64, C padded to 8
-    const size_t Kp = ((size_t)g.K + 63) / 64 * 64, Cp = ((size_t)g.C + 7) / 8 * 8;
+    // upper bound over every tile choice: K padded to 64, C padded to the chunk size (8, 6 or 4)
+    const size_t Kp = ((size_t)g.K + 63) / 64 * 64, Cp = (size_t)g.C + 7;
     const size_t w = Kp * Cp * g.RS * sizeof(float);
     const size_t ab = Kp * Cp * sizeof(float);
     return 2 * w + 2 * ab + 1024;
