@@ -77,7 +77,7 @@ bwd_idx_gx_kernel(Geo g, const T* __restrict__ gy, const int32_t* __restrict__ i
 // 64 output channels).  In the phase of tap t it finds the channels whose winner is t with a few
 // bit operations and touches only those: it reloads their winner (for the input channel) and
 // their grad_y, the loads of the next match in flight while the current one is accumulated.
-constexpr int kIdxGxKB = 16;   // output channels per staging round of bwd_idx_gx2_kernel
+constexpr int kIdxGxKB = 8;    // output channels per staging round of bwd_idx_gx2_kernel
 // RST: taps of the window when known at compile time (9: the tap loop unrolls and the targets of
 // the nine phases are computed once per pixel), 0: taken from the descriptor.
 template <typename T, int RST>
