@@ -192,6 +192,7 @@ __global__ void repack_weights_kernel(int K, int C, int RS, int tile_k, int Cpad
 struct TiledParams {
     Geo g;
     const void* x;
+    const void* w;     // weights as the caller passed them ([K][C][R][S])
     const float* wt;   // repacked weights (min branch / the only weights)
     const float* wt2;  // repacked max-branch weights (parallel)
     const float* at;   // repacked alpha, beta
@@ -714,14 +715,15 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                     if (ow >= g.OW) continue;
                     const int c = cbest[k][q][j];
                     const float* xc = xg + ((size_t)n * g.C + c) * chw;
-                    const float* wk = wt_k + ((size_t)c * RS) * TILE_K + kg * TK + k;
+                    // the window's weights in their original layout: 9 adjacent values
+                    const float* wk = reinterpret_cast<const float*>(p.w) + ((size_t)kk * g.C + c) * RS;
                     int tapw = 0;
 #pragma unroll
                     for (int tap = RS - 1; tap >= 0; --tap) {
                         const int ih = oh * g.sh - g.ph + (tap / S) * g.dh;
                         const int iw = ow * SW - g.pw + (tap % S) * DW;
                         const float xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xc[(size_t)ih * g.W + iw] : 0.0f;
-                        if (__fadd_rn(xv, wk[tap * TILE_K]) == acc[k][q][j]) tapw = tap;
+                        if (__fadd_rn(xv, wk[tap]) == acc[k][q][j]) tapw = tap;
                     }
                     idx[o + j] = c * RS + tapw;
                 }
@@ -928,7 +930,7 @@ int launch_tiled_variant(FwdArgs& a) {
     const size_t nrep = (size_t)nkt * pl.p.Cpad * g.RS * pl.tile_k;
     repack_weights_kernel<T><<<(unsigned)((nrep + 255) / 256), 256, 0, a.st>>>(
         g.K, g.C, g.RS, pl.tile_k, pl.p.Cpad, nkt, (const T*)a.w, (const T*)a.w2, a.alpha, a.beta, wt, wt2, at, bt);
-    pl.p.x = a.x; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
+    pl.p.x = a.x; pl.p.w = a.w; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
 #define TCONV_LAUNCH_F32(XTMAV, RAGV)                                                                 \
     {                                                                                                \

@@ -575,7 +575,8 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                     const unsigned bpair = best[k][q][j >> 1];
                     const float bestv = (j & 1) ? bf_hi(bpair) : bf_lo(bpair);
                     const __nv_bfloat16* xc = xb + ((size_t)n * g.C + c) * chw;
-                    const unsigned* wk = wt_k + ((size_t)c * RS) * TILE_K + kg * 8 + k;
+                    // the window's weights in their original layout: 9 adjacent values
+                    const __nv_bfloat16* wk = reinterpret_cast<const __nv_bfloat16*>(p.w) + ((size_t)kk * g.C + c) * RS;
                     int tapw = 0;
 #pragma unroll
                     for (int tap = RS - 1; tap >= 0; --tap) {
@@ -583,9 +584,7 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                         const int iw = ow * SW - g.pw + (tap % S) * DW;
                         const __nv_bfloat16 xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W)
                                                      ? xc[(size_t)ih * g.W + iw] : __float2bfloat16_rn(0.0f);
-                        const unsigned short wbits = (unsigned short)(wk[tap * TILE_K] & 0xffffu);
-                        const __nv_bfloat16 wv = *reinterpret_cast<const __nv_bfloat16*>(&wbits);
-                        if (tap_add(xv, wv) == bestv) tapw = tap;
+                        if (tap_add(xv, wk[tap]) == bestv) tapw = tap;
                     }
                     idx[o + j] = c * RS + tapw;
                 }
@@ -617,7 +616,7 @@ int launch_tiled_variant_bf16(FwdArgs& a) {
     repack_weights_bf16_kernel<0><<<(unsigned)((nrep + 255) / 256), 256, 0, a.st>>>(
         g.K, g.C, g.RS, pl.tile_k, pl.p.Cpad, nkt, (const __nv_bfloat16*)a.w, (const __nv_bfloat16*)a.w2,
         a.alpha, a.beta, (unsigned*)wt, (unsigned*)wt2, at, bt);
-    pl.p.x = a.x; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
+    pl.p.x = a.x; pl.p.w = a.w; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
 #define TCONV_LAUNCH_BF16(XTMAV, RAGV)                                                                \
     {                                                                                                \
