@@ -35,6 +35,6 @@ ParallelMinMaxPlusSumConv2d2p = _named("ParallelMinMaxPlusSumConv2d2p", "paralle
 
 __all__ = [n for n in dir() if n.endswith(("Conv2d", "0p", "1p", "2p"))]
 
-from .nn import TropicalDepthwiseConv2d  # noqa: E402  (depthwise form of the MobileNetV2 variants)
+from .nn import TropicalConv1d, TropicalDepthwiseConv2d  # noqa: E402  (1-D form; depthwise form of the MobileNetV2 variants)
 
-__all__.append("TropicalDepthwiseConv2d")
+__all__ += ["TropicalDepthwiseConv2d", "TropicalConv1d"]

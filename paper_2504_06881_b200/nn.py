@@ -281,3 +281,20 @@ class TropicalDepthwiseConv2d(nn.Module):
                 alpha, beta = self.alpha_fixed, self.beta_fixed
         geom = (self.mode, self.dtype, self.stride, self.padding, self.dilation)
         return TropicalDepthwiseFn.apply(x, self.weight, self.weight2, alpha, beta, self.bias, geom)
+
+
+class TropicalConv1d(nn.Module):
+    """1-D tropical convolution (Section 3.2): the 2-D operator on a signal of unit height, with a
+    1 x kernel_size window.  Same arguments as ``nn.Conv1d``; mode / chan / params / dtype as in
+    TropicalConv2d.  Windows of up to 256 taps (the paper's audio networks use 80) run through the
+    any-shape kernels of the library."""
+
+    def __init__(self, in_channels, out_channels, kernel_size, stride=1, padding=0, dilation=1,
+                 bias=True, mode="compound", chan="default", params="2p", dtype="f32", fixed=(0.5, 0.5)):
+        super().__init__()
+        self.conv = TropicalConv2d(in_channels, out_channels, (1, kernel_size), stride=(1, stride),
+                                   padding=(0, padding), dilation=(1, dilation), bias=bias, mode=mode,
+                                   chan=chan, params=params, dtype=dtype, fixed=fixed)
+
+    def forward(self, x):                      # x: [N, C, L]
+        return self.conv(x.unsqueeze(2)).squeeze(2)

@@ -147,3 +147,41 @@ def test_depthwise_layer_against_the_oracle(mode, params):
         assert close(m.alpha.grad, ga + sign * gb, gaa + abs(sign) * gba)
     if m.beta is not None:
         assert close(m.beta.grad, *gref["grad_beta"])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("mode,chan", [("compound", "default"), ("parallel", "default"), ("max_plus", "default"),
+                                       ("min_plus", "sum")])
+def test_conv1d_with_a_long_window_against_the_oracle(mode, chan):
+    """Kernel length 80, stride 4 (the first layer of the paper's 1-D audio networks), as a
+    1 x 80 window on a signal of unit height."""
+    from oracle import tconv_oracle as ora
+    from paper_2504_06881_b200.nn import TropicalConv1d
+    N, C, K, Ln, S, st = 2, 3, 5, 400, 80, 4
+    d = inputs.layer(N, C, 1, Ln, K, 1, S, stride=(1, st), pad=(0, 38), mode=mode, chan=chan)
+    t = inputs.draw(d, 2300)
+    m = TropicalConv1d(C, K, S, stride=st, padding=38, mode=mode, chan=chan).cuda()
+    two, par = mode in ("compound", "parallel"), mode == "parallel"
+    with torch.no_grad():
+        m.conv.weight.copy_(torch.from_numpy(t["w"]))
+        m.conv.bias.copy_(torch.from_numpy(t["bias"]))
+        if par:
+            m.conv.weight2.copy_(torch.from_numpy(t["w2"]))
+        if two:
+            m.conv.alpha.copy_(torch.from_numpy(t["alpha"]))
+            m.conv.beta.copy_(torch.from_numpy(t["beta"]))
+    ref = ora.forward(d, t["x"], t["w"], t["w2"] if par else None, t["alpha"] if two else None,
+                      t["beta"] if two else None, t["bias"])
+    x = torch.from_numpy(t["x"][:, :, 0]).cuda().requires_grad_(True)
+    y = m(x)
+    assert np.array_equal(y.detach().cpu().numpy().view(np.uint32), ref["y"][:, :, 0].view(np.uint32))
+    y.backward(torch.from_numpy(t["g"][:, :, 0]).cuda())
+    gref = ora.backward(d, t["x"], t["w"], t["g"], t["w2"] if par else None, t["alpha"] if two else None,
+                        t["beta"] if two else None)
+
+    def close(got, want, scale):
+        return (np.abs(got.detach().cpu().numpy().astype(np.float64) - want) <= 1e-5 * scale + 1e-30).all()
+
+    assert close(x.grad.unsqueeze(2), *gref["grad_x"]) and close(m.conv.weight.grad, *gref["grad_w"])
+    if two:
+        assert close(m.conv.alpha.grad, *gref["grad_alpha"]) and close(m.conv.beta.grad, *gref["grad_beta"])
