@@ -439,44 +439,77 @@ dw_bwd_params_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, co
                      const T* __restrict__ gy, const uint8_t* __restrict__ codes,
                      float* __restrict__ partial, int nchunks, int need_ab) {
     extern __shared__ float col[];   // [kDwAcc][256]
+    __shared__ float wsm[2][16];     // the channel's weights (min branch / max branch) as fp32
     const int c = blockIdx.x, chunk = blockIdx.y, tid = threadIdx.x;
     for (int e = tid; e < kDwAcc * 256; e += 256) col[e] = 0.0f;
+    if (tid < 32) {
+        const int br = tid >> 4, tp = tid & 15;
+        const T* src = (br == 1 && PAR) ? w2 : w;
+        wsm[br][tp] = tp < g.RS ? to_f32(__ldg(src + (size_t)c * g.RS + tp)) : 0.0f;
+    }
     __syncthreads();
     const unsigned plane = (unsigned)g.OH * g.OW;
     const unsigned items = (unsigned)g.N * plane;
     const unsigned per = (items + nchunks - 1) / nchunks;
     const unsigned lo = min(items, (unsigned)chunk * per), hi = min(items, lo + per);
-    const T* wc = w + (size_t)c * g.RS;
-    const T* wc2 = PAR ? w2 + (size_t)c * g.RS : wc;
     float* mine = col + tid;
-    for (unsigned it = lo + tid; it < hi; it += 256) {
-        const unsigned n = it / plane;
-        const unsigned pix = it - n * plane;
-        const int oh = (int)(pix / (unsigned)g.OW), ow = (int)(pix - (unsigned)oh * (unsigned)g.OW);
-        const size_t o = ((size_t)n * g.C + c) * plane + pix;
-        const float gv = to_f32(__ldg(gy + o));
-        const unsigned code = __ldg(codes + o);
-        const T* xp = x + ((size_t)n * g.C + c) * (size_t)g.H * g.W;
-        mine[(2 * 16 + 2) * 256] += gv;
-        if (BR == 0 || BR == 1) {
-            const unsigned tp = code & 15u;
-            mine[tp * 256] += gv;
-            if (need_ab) {
-                const int ih = oh * g.sh - g.ph + (int)(tp / g.S) * g.dh, iw = ow * g.sw - g.pw + (int)(tp % g.S) * g.dw;
-                const T xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? __ldg(xp + (size_t)ih * g.W + iw) : zero_of<T>();
-                mine[(2 * 16) * 256] = __fmaf_rn(gv, tap_add(xv, __ldg(wc + tp)), mine[(2 * 16) * 256]);
+    float sa = 0.0f, sb = 0.0f, ss = 0.0f;   // sum g * min value, sum g * max value, sum g
+    constexpr int U = 4;                      // items in flight per thread: every load of a batch is issued first
+    for (unsigned it0 = lo + tid; it0 < hi; it0 += 256 * U) {
+        float gv[U];
+        unsigned code[U];
+        T xa[U], xb[U];
+        bool ok[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const unsigned it = it0 + u * 256;
+            ok[u] = it < hi;
+            const unsigned n = it / plane;
+            const unsigned pix = it - n * plane;
+            const size_t o = ((size_t)n * g.C + c) * plane + pix;
+            gv[u] = ok[u] ? to_f32(__ldg(gy + o)) : 0.0f;
+            code[u] = ok[u] ? (unsigned)__ldg(codes + o) : 0u;
+        }
+        if (need_ab) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const unsigned it = it0 + u * 256;
+                const unsigned n = it / plane;
+                const unsigned pix = it - n * plane;
+                const int oh = (int)(pix / (unsigned)g.OW), ow = (int)(pix - (unsigned)oh * (unsigned)g.OW);
+                const T* xp = x + ((size_t)n * g.C + c) * (size_t)g.H * g.W;
+                xa[u] = xb[u] = zero_of<T>();
+                if (BR == 0 || BR == 1) {
+                    const unsigned tp = code[u] & 15u;
+                    const int ih = oh * g.sh - g.ph + (int)(tp / g.S) * g.dh, iw = ow * g.sw - g.pw + (int)(tp % g.S) * g.dw;
+                    if (ok[u] && ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) xa[u] = __ldg(xp + (size_t)ih * g.W + iw);
+                }
+                if (BR == 0 || BR == 2) {
+                    const unsigned tp = code[u] >> 4;
+                    const int ih = oh * g.sh - g.ph + (int)(tp / g.S) * g.dh, iw = ow * g.sw - g.pw + (int)(tp % g.S) * g.dw;
+                    if (ok[u] && ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) xb[u] = __ldg(xp + (size_t)ih * g.W + iw);
+                }
             }
         }
-        if (BR == 0 || BR == 2) {
-            const unsigned tp = code >> 4;
-            mine[(16 + tp) * 256] += gv;
-            if (need_ab) {
-                const int ih = oh * g.sh - g.ph + (int)(tp / g.S) * g.dh, iw = ow * g.sw - g.pw + (int)(tp % g.S) * g.dw;
-                const T xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? __ldg(xp + (size_t)ih * g.W + iw) : zero_of<T>();
-                mine[(2 * 16 + 1) * 256] = __fmaf_rn(gv, tap_add(xv, __ldg(wc2 + tp)), mine[(2 * 16 + 1) * 256]);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (!ok[u]) continue;
+            ss += gv[u];
+            if (BR == 0 || BR == 1) {
+                const unsigned tp = code[u] & 15u;
+                mine[tp * 256] += gv[u];
+                if (need_ab) sa = __fmaf_rn(gv[u], tap_add(xa[u], from_f32<T>(wsm[0][tp])), sa);
+            }
+            if (BR == 0 || BR == 2) {
+                const unsigned tp = code[u] >> 4;
+                mine[(16 + tp) * 256] += gv[u];
+                if (need_ab) sb = __fmaf_rn(gv[u], tap_add(xb[u], from_f32<T>(wsm[1][tp])), sb);
             }
         }
     }
+    mine[(2 * 16) * 256] = sa;
+    mine[(2 * 16 + 1) * 256] = sb;
+    mine[(2 * 16 + 2) * 256] = ss;
     __syncthreads();
     // row a of the columns is summed by warp a % 8: 8 values per lane in order, then a fixed shuffle tree
     const int warp = tid >> 5, lane = tid & 31;
