@@ -288,13 +288,18 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                     gp.xs_elems = gp.HP * gp.WP;
                     gp.xpad = xpad;
                 }
-#define TCONV_GW(BR, XSV, VECV)                                                                      \
+#define TCONV_GWK(BR, XSV, VECV, WARPV, GRID)                                                         \
     {                                                                                                \
-        auto kern = bwd_code_gw_kernel<T, BR, XSV, VECV>;                                            \
+        auto kern = bwd_code_gw_kernel<T, BR, XSV, VECV, WARPV>;                                     \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
-        kern<<<(unsigned)((size_t)g.K * g.C), 256, gp.smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
+        kern<<<(unsigned)(GRID), 256, gp.smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
                                                       (const T*)gy, codes, gw, gw2, galpha, gbeta, gp); \
+    }
+#define TCONV_GW(BR, XSV, VECV)                                                                      \
+    {                                                                                                \
+        if (gp.warp) TCONV_GWK(BR, XSV, VECV, true, ((size_t)g.K * g.C + 7) / 8)                     \
+        else TCONV_GWK(BR, XSV, VECV, false, (size_t)g.K * g.C)                                      \
     }
 #define TCONV_GWV(BR, XSV) { if (vecw) TCONV_GW(BR, XSV, true) else TCONV_GW(BR, XSV, false) }
                 const bool vecw = (g.OW & 3) == 0;
@@ -302,6 +307,7 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                 else if (br == 1) TCONV_GWV(1, false) else TCONV_GWV(2, false)
 #undef TCONV_GWV
 #undef TCONV_GW
+#undef TCONV_GWK
                 g_launches += 1;
                 name = "bwd_code";
             } else {

@@ -441,9 +441,11 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
 // One CTA per (k, c).  XS: a zero-padded copy of x (made once per backward call by
 // pad_input_kernel) is available, so that the branch values x[winner] + w[winner] of
 // grad_alpha / grad_beta are gathered without bounds checks.
+constexpr int kGwTableInts = 2 * 16 + 2 + 4 * 16;   // per pair: tap_dh, tap_dw (RS <= 16 each, padded), two int2 tables
 struct CodeGwPlan {
     int HP, WP;      // padded plane extent covering every tap of every output
     int xs_elems;    // elements of one padded plane (0: no padded copy)
+    int warp;        // 1: the warp-per-pair variant of the kernel
     size_t smem;
     const void* xpad;
 };
@@ -461,35 +463,43 @@ __global__ void pad_input_kernel(Geo g, const T* __restrict__ x, T* __restrict__
     xpad[i] = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? x[(nc * g.H + ih) * g.W + iw] : zero_of<T>();
 }
 
-template <typename T, int BR, bool XS, bool VEC>
+// WARP: one warp per (k, c) pair, eight pairs per CTA, the lanes walk the pair's (image, quad)
+// items and reduce with shuffles; for maps so small that a 256-thread CTA per pair would spend its
+// time zeroing, synchronising and reducing.  Else one CTA per pair.
+template <typename T, int BR, bool XS, bool VEC, bool WARP>
 __global__ void __launch_bounds__(256)
 bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
                    const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes,
                    float* __restrict__ gw, float* __restrict__ gw2, float* __restrict__ galpha,
                    float* __restrict__ gbeta, CodeGwPlan pl) {
-    extern __shared__ float S[];  // [2*RS + 2][256] private columns | per-tap tables
-    const int c = blockIdx.x % g.C;
-    const int k = blockIdx.x / g.C;
+    extern __shared__ float S[];  // [2*RS + 2][256] private columns | per-tap tables (one set per pair)
     const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
+    const int pair = WARP ? (int)blockIdx.x * 8 + warp : (int)blockIdx.x;
+    if (WARP && pair >= g.K * g.C) return;     // whole warps leave; this variant has no block barrier
+    const int c = pair % g.C;
+    const int k = pair / g.C;
     const int NB = 2 * g.RS + 2;
+    const int me = WARP ? lane : tid;           // index of this thread among the pair's workers
+    const int nworkers = WARP ? 32 : 256;
     char* colb = reinterpret_cast<char*>(S + tid);
-    int* tap_dh = reinterpret_cast<int*>(S + NB * 256);
+    int* tap_dh = reinterpret_cast<int*>(S + NB * 256) + (WARP ? warp * kGwTableInts : 0);
     int* tap_dw = tap_dh + g.RS;
     // {offset of the tap inside the padded plane, weight of the tap}: min branch, max branch
     int2* tapw_min = reinterpret_cast<int2*>(tap_dw + g.RS + ((g.RS & 1) ? 0 : 0) + (((2 * g.RS) & 1) ? 1 : 0));
     int2* tapw_max = tapw_min + g.RS;
     for (int b = 0; b < NB; ++b) S[b * 256 + tid] = 0.0f;
-    if (tid < g.RS) {
-        const int r = tid / g.S, sx = tid % g.S;
-        tap_dh[tid] = r * g.dh - g.ph;
-        tap_dw[tid] = sx * g.dw - g.pw;
-        const size_t wi = ((size_t)k * g.C + c) * g.RS + tid;
+    if (me < g.RS) {
+        const int r = me / g.S, sx = me % g.S;
+        tap_dh[me] = r * g.dh - g.ph;
+        tap_dw[me] = sx * g.dw - g.pw;
+        const size_t wi = ((size_t)k * g.C + c) * g.RS + me;
         const int off = r * g.dh * pl.WP + sx * g.dw;
-        tapw_min[tid] = make_int2(off, __float_as_int(to_f32(w[wi])));
-        tapw_max[tid] = make_int2(off, __float_as_int(to_f32((g.mode == TCONV_PARALLEL ? w2 : w)[wi])));
+        tapw_min[me] = make_int2(off, __float_as_int(to_f32(w[wi])));
+        tapw_max[me] = make_int2(off, __float_as_int(to_f32((g.mode == TCONV_PARALLEL ? w2 : w)[wi])));
     }
-    __syncthreads();
+    if constexpr (WARP) __syncwarp(); else __syncthreads();
     const bool need_ab = (BR == 0) && (galpha || gbeta);
     const int QPR = (g.OW + 3) >> 2;
     const int NQ = g.OH * QPR;
@@ -539,7 +549,7 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
             }
         }
     };
-    if (NQ >= 192) {
+    if (!WARP && NQ >= 192) {
         // large maps: a thread keeps its quad and walks the images (constant pointer strides)
         for (int q = tid; q < NQ; q += 256) {
             const int oh = q / QPR;
@@ -569,9 +579,9 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
             }
         }
     } else {
-        // small maps: the threads walk the flattened (image, quad) pairs with a stride of 256
-        const int dn = 256 / NQ, dq = 256 - dn * NQ;
-        int n = tid / NQ, q = tid - n * NQ;
+        // small maps: the workers walk the flattened (image, quad) pairs with a stride of their number
+        const int dn = nworkers / NQ, dq = nworkers - dn * NQ;
+        int n = me / NQ, q = me - n * NQ;
         float gv_cur[4], gv_nxt[4];
         unsigned cw_cur = 0, cw_nxt = 0;
         auto item_ptrs = [&](int n_, int q_, int& oh, int& ow0, const T*& gp, const uint8_t*& cp, const T*& xp) {
@@ -611,18 +621,35 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
             have = more;
         }
     }
-    S[(2 * g.RS) * 256 + tid] = sa;
-    S[(2 * g.RS + 1) * 256 + tid] = sb;
-    __syncthreads();
-    // fixed tree over the 256 columns of every bin
-    for (int step = 128; step > 0; step >>= 1) {
-        if (tid < step)
-            for (int b = 0; b < NB; ++b) S[b * 256 + tid] += S[b * 256 + tid + step];
+    float tmin = 0.0f, tmax = 0.0f, tot_a = 0.0f, tot_b = 0.0f;
+    if constexpr (WARP) {
+        // every bin: the 32 private values of the warp, summed by a fixed butterfly; lane t keeps
+        // the totals of tap t
+        for (int b = 0; b < NB; ++b) {
+            float v = b < 2 * g.RS ? S[b * 256 + tid] : (b == 2 * g.RS ? sa : sb);
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+            if (b == lane) tmin = v;
+            if (b == g.RS + lane) tmax = v;
+            if (b == 2 * g.RS) tot_a = v;
+            if (b == 2 * g.RS + 1) tot_b = v;
+        }
+    } else {
+        S[(2 * g.RS) * 256 + tid] = sa;
+        S[(2 * g.RS + 1) * 256 + tid] = sb;
         __syncthreads();
+        // fixed tree over the 256 columns of every bin
+        for (int step = 128; step > 0; step >>= 1) {
+            if (tid < step)
+                for (int b = 0; b < NB; ++b) S[b * 256 + tid] += S[b * 256 + tid + step];
+            __syncthreads();
+        }
+        if (tid < g.RS) { tmin = S[tid * 256]; tmax = S[(g.RS + tid) * 256]; }
+        tot_a = S[(2 * g.RS) * 256];
+        tot_b = S[(2 * g.RS + 1) * 256];
     }
-    if (tid < g.RS) {
-        const float tmin = S[tid * 256], tmax = S[(g.RS + tid) * 256];
-        const size_t wi = ((size_t)k * g.C + c) * g.RS + tid;
+    if (me < g.RS) {
+        const size_t wi = ((size_t)k * g.C + c) * g.RS + me;
         if constexpr (BR == 0) {
             const float a = alpha ? alpha[(size_t)k * g.C + c] : 1.0f;
             const float b = beta ? beta[(size_t)k * g.C + c] : 1.0f;
@@ -636,9 +663,9 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
             if (gw) gw[wi] = (BR == 1) ? tmin : tmax;
         }
     }
-    if (BR == 0 && tid == 0) {
-        if (galpha) galpha[(size_t)k * g.C + c] = S[(2 * g.RS) * 256];
-        if (gbeta) gbeta[(size_t)k * g.C + c] = S[(2 * g.RS + 1) * 256];
+    if (BR == 0 && me == 0) {
+        if (galpha) galpha[(size_t)k * g.C + c] = tot_a;
+        if (gbeta) gbeta[(size_t)k * g.C + c] = tot_b;
     }
 }
 
@@ -661,7 +688,10 @@ bwd_bias_partial_kernel(Geo g, const T* __restrict__ gy, float* __restrict__ par
 
 // ---------------------------------------------------------------------------------- host side
 inline void plan_code_gw(const Geo& g, CodeGwPlan* pl) {
-    pl->smem = ((size_t)(2 * g.RS + 2) * 256 + 6 * (size_t)g.RS + 4) * sizeof(float);
+    // a warp per (k, c) pair where a pair has few (image, quad) items
+    pl->warp = ((size_t)g.N * g.OH * ((g.OW + 3) / 4) < 8192 && g.RS <= 16) ? 1 : 0;
+    pl->smem = pl->warp ? ((size_t)(2 * g.RS + 2) * 256 + 8 * (size_t)kGwTableInts) * sizeof(float)
+                        : ((size_t)(2 * g.RS + 2) * 256 + 6 * (size_t)g.RS + 4) * sizeof(float);
     pl->HP = (g.OH - 1) * g.sh + (g.R - 1) * g.dh + 1;
     pl->WP = (g.OW - 1) * g.sw + (g.S - 1) * g.dw + 1;
     if (pl->HP < g.H + g.ph) pl->HP = g.H + g.ph;   // rows / columns no output reaches still hold x
