@@ -851,8 +851,11 @@ inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* p
         return plan_tiles_opt<R, S, SW, DW, Q, KG, PW, TK>(g, par, two, esize, force[0] == 'r', force[1] - '0', pl);
     // 8 channels per chunk when four CTAs stay resident, else 4 channels when three do (measured
     // on the stride-2 56 -> 28 layer: 8.06 against 7.86 Ttap/s for whole-row tiles at four CTAs)
+    // (two-branch kernels with 8 channels per thread hold two CTAs per SM by their registers: their
+    // stages may use half of the shared memory)
+    const bool two_resident = two && TK == 8;
     for (int cc = 8; cc >= 4; cc -= 2) {
-        const size_t budget = (cc == 4 ? 74 : 56) * 1024;
+        const size_t budget = (two_resident ? 112 : (cc == 4 ? 74 : 56)) * 1024;
         TiledPlan cand = *pl;
         if (plan_tiles_opt<R, S, SW, DW, Q, KG, PW, TK>(g, par, two, esize, true, cc, &cand) && cand.p.ragged &&
             cand.smem <= budget) {
