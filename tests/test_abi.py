@@ -68,3 +68,34 @@ def test_host_side_argument_checks():
     assert tconv.tconv_status_string(-3).startswith("pointer")
     assert tconv.tconv_alu_probe_name(0) == "f32_add_max2"
     assert tconv.tconv_alu_probe_name(10_000) is None
+
+
+def test_empty_and_oversized_descriptors_are_rejected_on_the_host():
+    """Empty tensors (a zero extent) are invalid arguments; layers whose flat indices would not fit
+    the launch arithmetic are refused with TCONV_ERR_TOO_LARGE before anything is launched."""
+    d = inputs.layer(1, 1, 4, 4, 1, 3, 3, pad=1)
+    for key in ("N", "C", "K", "H", "W", "R", "S"):
+        with pytest.raises(tconv.TconvError) as e:
+            tconv.tconv_output_shape(dict(d, **{key: 0}))
+        assert e.value.status == -1
+        assert tconv.tconv_winner_bytes(dict(d, **{key: 0})) == 0
+        assert tconv.tconv_workspace_bytes(dict(d, **{key: 0}), True) == 0
+    big = inputs.layer(2_000_000, 512, 1024, 1024, 512, 3, 3, pad=1)      # 1e15 outputs
+    with pytest.raises(tconv.TconvError) as e:
+        tconv.tconv_output_shape(big)
+    assert e.value.status == -7
+    assert tconv.tconv_status_string(-7) != ""
+    with pytest.raises(tconv.TconvError) as e:                             # more than 256 taps
+        tconv.tconv_output_shape(inputs.layer(1, 1, 40, 40, 1, 17, 17))
+    assert e.value.status == -2
+
+
+def test_depthwise_descriptor_checks_on_the_host():
+    ok = inputs.layer(2, 8, 9, 9, 8, 3, 3, pad=1, mode="compound")
+    assert tconv.tconv_dw_winner_bytes(ok) == 2 * 8 * 9 * 9
+    assert tconv.tconv_dw_workspace_bytes(ok, False) == 0
+    assert tconv.tconv_dw_workspace_bytes(ok, True) >= tconv.tconv_dw_winner_bytes(ok)
+    assert tconv.tconv_dw_winner_bytes(dict(ok, K=4)) == 0                 # one output channel per input channel
+    assert tconv.tconv_dw_winner_bytes(dict(ok, R=5, S=5, pad_h=2, pad_w=2)) == 0   # a code nibble holds 16 taps
+    assert tconv.tconv_dw_winner_bytes(dict(ok, N=0)) == 0
+    assert tconv.tconv_dw_winner_bytes(inputs.layer(70_000, 1024, 64, 64, 1024, 3, 3, pad=1)) == 0   # > 2^31 - 1 elements
