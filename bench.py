@@ -277,6 +277,20 @@ def measure_alu_peak(torch, tconv):
     return {m: max(rate[p] for p in ps) for m, ps in PROBES.items()}, rate
 
 
+def max_over_ranks(torch, dist, values, device, world):
+    """The replicas' times combine as the slowest rank's (the only exchange of a run: the data
+    path itself has no collective)."""
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_value(world, ops_per_step, steps, ms):
+    """Whole-job throughput in Gop/s: every replica runs the same steps in the slowest rank's time."""
+    return world * ops_per_step * steps / (ms * 1e-3) / 1e9
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -363,18 +377,15 @@ def run_gpu(args):
         per[L.d["mode"]] = rec
     peaks, probe_rates = measure_alu_peak(torch, tconv)
 
-    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks(torch, dist, [ms, ms_e2e], dev, world)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     ops_step = sum(L.ops for L in layers)
-    value = world * ops_step * args.steps / (ms * 1e-3) / 1e9
-    e2e_value = world * ops_step * args.steps / (ms_e2e * 1e-3) / 1e9
+    value = aggregate_value(world, ops_step, args.steps, ms)
+    e2e_value = aggregate_value(world, ops_step, args.steps, ms_e2e)
 
     # dominant kernel = the call with the largest time in a step; its roofline is the
     # add+max/min ALU peak of that mode (a tap = one x+w term folded into min and/or max)
