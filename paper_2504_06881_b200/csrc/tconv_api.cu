@@ -475,7 +475,29 @@ int dw_backward_t(const Geo& g, const void* x, const void* w, const void* w2, co
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<grid, 256, smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, codes, partial, nch, need_ab); \
     }
-        if (br == 0) { if (par) TCONV_DW_PAR(0, true) else TCONV_DW_PAR(0, false) }
+        const bool k3 = g.R == 3 && g.S == 3 && g.dh == 1 && g.dw == 1 && g.sh == g.sw && (g.sw == 1 || g.sw == 2) &&
+                        nch <= g.N && g.OH * g.OW >= 100;   // tiny planes: too few strips per image
+        if (k3) {
+            // 3x3 windows: strips over a register window, the chunks are ranges of images
+            const int QPR3 = (g.OW + 3) / 4, strips3 = (g.OH + TCONV_DW_RT - 1) / TCONV_DW_RT;
+            const bool vec3 = (g.pw == 1 && (g.W & 3) == 0);
+#define TCONV_DW_P3(BR, PARV, SWV, VECV)                                                              \
+    {                                                                                                \
+        auto kern = dw_bwd_params3_kernel<T, BR, PARV, SWV, VECV>;                                   \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) \
+            return cuda_fail(cudaGetLastError());                                                    \
+        kern<<<grid, 256, smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, codes, partial, nch, \
+                                      need_ab, QPR3, strips3);                                       \
+    }
+#define TCONV_DW_P3V(BR, PARV, SWV) { if (vec3) TCONV_DW_P3(BR, PARV, SWV, true) else TCONV_DW_P3(BR, PARV, SWV, false) }
+#define TCONV_DW_P3S(BR, PARV) { if (g.sw == 1) TCONV_DW_P3V(BR, PARV, 1) else TCONV_DW_P3V(BR, PARV, 2) }
+            if (br == 0) { if (par) TCONV_DW_P3S(0, true) else TCONV_DW_P3S(0, false) }
+            else if (br == 1) TCONV_DW_P3S(1, false)
+            else TCONV_DW_P3S(2, false)
+#undef TCONV_DW_P3S
+#undef TCONV_DW_P3V
+#undef TCONV_DW_P3
+        } else if (br == 0) { if (par) TCONV_DW_PAR(0, true) else TCONV_DW_PAR(0, false) }
         else if (br == 1) TCONV_DW_PAR(1, false)
         else TCONV_DW_PAR(2, false)
 #undef TCONV_DW_PAR

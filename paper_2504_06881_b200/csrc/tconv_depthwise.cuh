@@ -523,6 +523,114 @@ dw_bwd_params_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, co
     }
 }
 
+// Parameter gradients for 3x3 windows, dilation 1, stride SW: the same strips and register window
+// as the forward.  The branch values of grad_alpha / grad_beta are the extrema recomputed from the
+// window (no gathers); the per-tap sums take the winners from the codes.  CTA (c, chunk) walks the
+// strips of its images; accumulators and reduction as in dw_bwd_params_kernel.
+template <typename T, int BR, bool PAR, int SW, bool VEC>
+__global__ void __launch_bounds__(256)
+dw_bwd_params3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
+                      const T* __restrict__ gy, const uint8_t* __restrict__ codes,
+                      float* __restrict__ partial, int nchunks, int need_ab, int QPR, int strips) {
+    constexpr int RT = TCONV_DW_RT;
+    constexpr int L = 3 * SW + 3;
+    extern __shared__ float col[];   // [kDwAcc][256]
+    const int c = blockIdx.x, chunk = blockIdx.y, tid = threadIdx.x;
+    for (int e = tid; e < kDwAcc * 256; e += 256) col[e] = 0.0f;
+    __syncthreads();
+    T wa[9], wb[9];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) {
+        wa[i] = __ldg(w + (size_t)c * 9 + i);
+        wb[i] = PAR ? __ldg(w2 + (size_t)c * 9 + i) : wa[i];
+    }
+    const int per = (g.N + nchunks - 1) / nchunks;
+    const int n_lo = min(g.N, chunk * per), n_hi = min(g.N, n_lo + per);
+    const unsigned sq = (unsigned)strips * QPR;                 // strips x quads of one plane
+    const unsigned nitems = (unsigned)(n_hi - n_lo) * sq;
+    const size_t plane = (size_t)g.OH * g.OW;
+    float* mine = col + tid;
+    float sa = 0.0f, sb = 0.0f, ss = 0.0f;
+    for (unsigned it = tid; it < nitems; it += 256) {
+        const unsigned nl = it / sq;
+        const unsigned rem = it - nl * sq;
+        const int st = (int)(rem / (unsigned)QPR), qx = (int)(rem - (unsigned)st * QPR);
+        const size_t nc = (size_t)(n_lo + nl) * g.C + c;
+        const int oh0 = st * RT, ow0 = qx * 4;
+        const T* gp = gy + nc * plane + ow0;
+        const uint8_t* cp = codes + nc * plane + ow0;
+        const bool full = (ow0 + 3 < g.OW) && ((g.OW & 3) == 0);
+        const int ih0 = oh0 * SW - g.ph, c0 = ow0 * SW - g.pw;
+        T win[3][L];
+        const unsigned cmask = need_ab ? dw_col_mask(c0, L, g.W) : 0u;
+        const T* rp0 = x + nc * (size_t)g.H * g.W + (ptrdiff_t)ih0 * g.W + c0;
+        auto load = [&](int rho) {
+            const int ih = ih0 + rho;
+            dw_load_row<T, L, VEC>(rp0 + rho * g.W, need_ab && ih >= 0 && ih < g.H, cmask, win[rho % 3]);
+        };
+        load(0);
+        load(1);
+#pragma unroll
+        for (int k = 0; k < RT; ++k) {
+            const int oh = oh0 + k;
+            if (oh >= g.OH) break;
+#pragma unroll
+            for (int rho = (k == 0 ? 2 : (k - 1) * SW + 3); rho <= k * SW + 2; ++rho) load(rho);
+            float gq[4];
+            unsigned cq;
+            if (full) {
+                T tmp[4];
+                load4(gp + (size_t)oh * g.OW, tmp);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) gq[j] = to_f32(tmp[j]);
+                cq = __ldg(reinterpret_cast<const unsigned*>(cp + (size_t)oh * g.OW));
+            } else {
+                cq = 0u;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool ok = ow0 + j < g.OW;
+                    gq[j] = ok ? to_f32(__ldg(gp + (size_t)oh * g.OW + j)) : 0.0f;
+                    if (ok) cq |= (unsigned)__ldg(cp + (size_t)oh * g.OW + j) << (8 * j);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (!full && ow0 + j >= g.OW) continue;
+                const float gv = gq[j];
+                const unsigned code = (cq >> (8 * j)) & 0xffu;
+                ss += gv;
+                if (BR == 0 || BR == 1) mine[(code & 15u) * 256] += gv;
+                if (BR == 0 || BR == 2) mine[(16 + (code >> 4)) * 256] += gv;
+                if (need_ab) {
+                    float ta[9], tb[PAR ? 9 : 1];
+#pragma unroll
+                    for (int tap = 0; tap < 9; ++tap) {
+                        const T xv = win[(k * SW + tap / 3) % 3][j * SW + tap % 3];
+                        ta[tap] = tap_add(xv, wa[tap]);
+                        if constexpr (PAR) tb[tap] = tap_add(xv, wb[tap]);
+                    }
+                    const float* tm = PAR ? tb : ta;
+                    if (BR == 0 || BR == 1) sa = __fmaf_rn(gv, dw_fold9(ta, true), sa);
+                    if (BR == 0 || BR == 2) sb = __fmaf_rn(gv, dw_fold9(tm, false), sb);
+                }
+            }
+        }
+    }
+    mine[(2 * 16) * 256] = sa;
+    mine[(2 * 16 + 1) * 256] = sb;
+    mine[(2 * 16 + 2) * 256] = ss;
+    __syncthreads();
+    const int warp = tid >> 5, lane = tid & 31;
+    for (int a = warp; a < kDwAcc; a += 8) {
+        float s = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) s += col[a * 256 + lane * 8 + e];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) s += __shfl_down_sync(0xffffffffu, s, d);
+        if (lane == 0) partial[((size_t)chunk * g.C + c) * kDwAcc + a] = s;
+    }
+}
+
 // One thread per (c, accumulator): sums the chunk partials in order and writes the gradients.
 __global__ void dw_bwd_finish_kernel(Geo g, const float* __restrict__ partial, int nchunks, int mode,
                                      const float* __restrict__ alpha, const float* __restrict__ beta,
