@@ -982,6 +982,11 @@ int launch_tiled_geom(FwdArgs& a) {
         if (g.sw == 2 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 2, 1, Q, 4, 1, TK2>(a);
         if (g.sw == 1 && g.dw == 2) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 2, Q, 4, 1, TK>(a);
     }
+    // the other windows of the paper's networks: 1 x 3 (1-D layers as signals of unit height) and 5 x 5
+    if (g.R == 1 && g.S == 3 && g.sw == 1 && g.dw == 1)
+        return launch_tiled_variant<T, MODE, CHAN, WIN, 1, 3, 1, 1, Q, 4, 1, TK>(a);
+    if (g.R == 5 && g.S == 5 && g.sw == 1 && g.dw == 1)
+        return launch_tiled_variant<T, MODE, CHAN, WIN, 5, 5, 1, 1, Q, 4, 1, TK>(a);
     return TCONV_ERR_UNSUPPORTED;
 }
 
@@ -989,7 +994,9 @@ int launch_tiled_geom(FwdArgs& a) {
 template <int MODE, int CHAN>
 int launch_fwd_tiled_inst(FwdArgs& a) {
     if (a.dtype != TCONV_F32) return TCONV_ERR_UNSUPPORTED;  // bf16: separate kernel
-    if (a.g.wide) return TCONV_ERR_UNSUPPORTED;
+    // more than 16 taps: the nibble codes of the Sum forms do not fit (the winner-free forward and
+    // the Max / Min combines do)
+    if (a.g.wide && a.winners && a.g.chan == CH_SUM) return TCONV_ERR_UNSUPPORTED;
     if ((double)a.g.N * a.g.C * a.g.H * a.g.W >= 2.0e9) return TCONV_ERR_UNSUPPORTED;  // 32-bit offsets
     if (a.winners) return launch_tiled_geom<float, MODE, CHAN, true>(a);
     return launch_tiled_geom<float, MODE, CHAN, false>(a);
