@@ -954,7 +954,7 @@ int launch_tiled_variant(FwdArgs& a) {
 }
 
 // Geometry families with a tiled kernel: 3x3 windows with (stride_w, dil_w) in
-// {(1,1), (2,1), (1,2)}.
+// {(1,1), (2,1), (1,2), (1,4)}, and the 1 x 3 and 5 x 5 windows at stride 1, dilation 1.
 template <typename T, int MODE, int CHAN, bool WIN>
 int launch_tiled_geom(FwdArgs& a) {
     constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
@@ -981,6 +981,7 @@ int launch_tiled_geom(FwdArgs& a) {
         constexpr int TK2 = (TWO && !WIN) ? 8 : TK;
         if (g.sw == 2 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 2, 1, Q, 4, 1, TK2>(a);
         if (g.sw == 1 && g.dw == 2) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 2, Q, 4, 1, TK>(a);
+        if (g.sw == 1 && g.dw == 4) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 4, Q, 4, 1, TK>(a);
     }
     // the other windows of the paper's networks: 1 x 3 (1-D layers as signals of unit height) and 5 x 5
     if (g.R == 1 && g.S == 3 && g.sw == 1 && g.dw == 1)

@@ -647,6 +647,7 @@ int launch_tiled_geom_bf16(FwdArgs& a) {
         if (g.sw == 1 && g.dw == 1) return launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 1, 1, Q, 4, 1>(a);
         if (g.sw == 2 && g.dw == 1) return launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 2, 1, Q, 4, 1>(a);
         if (g.sw == 1 && g.dw == 2) return launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 1, 2, Q, 4, 1>(a);
+        if (g.sw == 1 && g.dw == 4) return launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 1, 4, Q, 4, 1>(a);
     }
     // 1 x 3: the 1-D layers as signals of unit height
     if (g.R == 1 && g.S == 3 && g.sw == 1 && g.dw == 1)

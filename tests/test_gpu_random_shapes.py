@@ -24,7 +24,7 @@ def test_random_descriptors(seed):
         mode, chan = ALL[rs.randint(len(ALL))]
         dtype = ["f32", "bf16"][rs.randint(2)]
         R, S = WINDOWS[rs.randint(len(WINDOWS))]
-        st, dl = [1, 1, 1, 2, 2, 3][rs.randint(6)], [1, 1, 1, 2, 2, 3][rs.randint(6)]
+        st, dl = [1, 1, 1, 2, 2, 3][rs.randint(6)], [1, 1, 1, 2, 2, 3, 4, 4][rs.randint(8)]
         pad = rs.randint(0, 3) if rs.rand() < 0.5 else (S - 1) * dl // 2
         N, C, K = rs.randint(1, 12), rs.randint(1, 60), rs.randint(1, 80)
         H = rs.randint(1, 48)
