@@ -242,14 +242,22 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                 const dim3 grid(pl.grid);
 #define TCONV_GXM(BR, CBV, VECV, MULTI, NTH)                                                         \
     {                                                                                                \
-        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV, MULTI, NTH>;                                \
+        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV, MULTI, NTH, false>;                         \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
+            return cuda_fail(cudaGetLastError());                                                    \
+        kern<<<grid, pl.threads, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);   \
+    }
+#define TCONV_GXW(BR, CBV, VECV)                                                                     \
+    {                                                                                                \
+        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV, false, 256, true>;                          \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<grid, pl.threads, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);   \
     }
 #define TCONV_GX(BR, CBV, VECV)                                                                      \
     {                                                                                                \
-        if (pl.imgs > 1) TCONV_GXM(BR, CBV, VECV, true, 256)                                         \
+        if (g.wide) TCONV_GXW(BR, CBV, VECV)                                                         \
+        else if (pl.imgs > 1) TCONV_GXM(BR, CBV, VECV, true, 256)                                    \
         else if (pl.threads > 256) TCONV_GXM(BR, CBV, VECV, false, 1024)                             \
         else TCONV_GXM(BR, CBV, VECV, false, 256)                                                    \
     }
@@ -263,6 +271,7 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
 #undef TCONV_GX2
 #undef TCONV_GX
 #undef TCONV_GXM
+#undef TCONV_GXW
                 name = "bwd_code";
             } else {
                 const size_t total = (size_t)g.N * g.C * g.H * g.W;
@@ -274,7 +283,7 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
         if (gw || gw2 || galpha || gbeta) {
             CodeGwPlan gp;
             plan_code_gw(g, &gp);
-            if (tiled && !g.wide && gp.smem <= kBwdSmemLimit) {
+            if (tiled && gp.smem <= kBwdSmemLimit) {
                 // zero-padded copy of x for the branch values of grad_alpha / grad_beta, placed after
                 // the grad_bias partials in the workspace
                 const size_t bias_part = ((size_t)16 * g.K * sizeof(float) + 255) / 256 * 256;
@@ -290,15 +299,24 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                 }
 #define TCONV_GWK(BR, XSV, VECV, WARPV, GRID)                                                         \
     {                                                                                                \
-        auto kern = bwd_code_gw_kernel<T, BR, XSV, VECV, WARPV>;                                     \
+        auto kern = bwd_code_gw_kernel<T, BR, XSV, VECV, WARPV, false>;                              \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<(unsigned)(GRID), 256, gp.smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
                                                       (const T*)gy, codes, gw, gw2, galpha, gbeta, gp); \
     }
+#define TCONV_GWW(BR, XSV, VECV)                                                                     \
+    {                                                                                                \
+        auto kern = bwd_code_gw_kernel<T, BR, XSV, VECV, false, true>;                               \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
+            return cuda_fail(cudaGetLastError());                                                    \
+        kern<<<(unsigned)((size_t)g.K * g.C), 256, gp.smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
+                                                      (const T*)gy, codes, gw, gw2, galpha, gbeta, gp); \
+    }
 #define TCONV_GW(BR, XSV, VECV)                                                                      \
     {                                                                                                \
-        if (gp.warp) TCONV_GWK(BR, XSV, VECV, true, ((size_t)g.K * g.C + 7) / 8)                     \
+        if (g.wide) TCONV_GWW(BR, XSV, VECV)                                                         \
+        else if (gp.warp) TCONV_GWK(BR, XSV, VECV, true, ((size_t)g.K * g.C + 7) / 8)                \
         else TCONV_GWK(BR, XSV, VECV, false, (size_t)g.K * g.C)                                      \
     }
 #define TCONV_GWV(BR, XSV) { if (vecw) TCONV_GW(BR, XSV, true) else TCONV_GW(BR, XSV, false) }
@@ -308,6 +326,7 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
 #undef TCONV_GWV
 #undef TCONV_GW
 #undef TCONV_GWK
+#undef TCONV_GWW
                 g_launches += 1;
                 name = "bwd_code";
             } else {

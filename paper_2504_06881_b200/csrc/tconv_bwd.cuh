@@ -286,12 +286,48 @@ __device__ __forceinline__ unsigned load_c4(const uint8_t* p, int ow0, int OW) {
     }
 }
 
+// The 4 winner codes of a quad.  Narrow codes (R*S <= 16): one byte each, argmin tap in the low
+// nibble, argmax tap in the high nibble.  WIDE (R*S <= 256): 16 bits each, argmin tap in the low
+// byte, argmax tap in the high byte; `p` then points at the first of 4 adjacent 16-bit codes.
+template <bool WIDE> struct Codes4 { unsigned lo, hi; };
+template <bool WIDE, bool VEC>
+__device__ __forceinline__ Codes4<WIDE> load_codes4(const uint8_t* p, int ow0, int OW) {
+    Codes4<WIDE> r;
+    r.hi = 0u;
+    if constexpr (!WIDE) {
+        r.lo = load_c4<VEC>(p, ow0, OW);
+    } else if constexpr (VEC) {
+        const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+        r.lo = v.x; r.hi = v.y;
+    } else {
+        const uint16_t* q = reinterpret_cast<const uint16_t*>(p);
+        r.lo = 0u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (ow0 + j < OW) {
+                const unsigned cde = q[j];
+                if (j < 2) r.lo |= cde << (16 * j); else r.hi |= cde << (16 * (j - 2));
+            }
+    }
+    return r;
+}
+template <bool WIDE>
+__device__ __forceinline__ void taps_of(const Codes4<WIDE>& c4, int j, unsigned& tmin, unsigned& tmax) {
+    if constexpr (!WIDE) {
+        const unsigned code = (c4.lo >> (8 * j)) & 0xffu;
+        tmin = code & 15u; tmax = code >> 4;
+    } else {
+        const unsigned code = ((j < 2 ? c4.lo : c4.hi) >> (16 * (j & 1))) & 0xffffu;
+        tmin = code & 0xffu; tmax = code >> 8;
+    }
+}
+
 // BR: 0 = both branches (compound / parallel), 1 = min branch only, 2 = max branch only.
 // CB channels per CTA (the CTA's last channel block may hold fewer: those lanes idle).
 // VEC: OW is a multiple of 4 (aligned vector loads of grad_y and of the codes).
 // MULTI: the CTA owns pl.imgs whole images (small maps); else one band of rows of one image.
 // NTH: upper bound of the CTA size (256, or 1024 for tiles that leave room for one or two CTAs per SM).
-template <typename T, int BR, int CB, bool VEC, bool MULTI, int NTH>
+template <typename T, int BR, int CB, bool VEC, bool MULTI, int NTH, bool WIDE>
 __global__ void __launch_bounds__(NTH)
 bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
@@ -329,7 +365,8 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     }
     __syncthreads();
     const size_t plane = (size_t)g.OH * g.OW;
-    const size_t cstep = (size_t)g.C * plane;        // codes: one output channel k further
+    constexpr int CW = WIDE ? 2 : 1;                     // bytes per code
+    const size_t cstep = (size_t)g.C * plane * CW;    // codes: one output channel k further (bytes)
     const unsigned tstride = 4u * NQp * sizeof(float); // bytes between the accumulators of two taps
     for (int q = threadIdx.x; q < NQ; q += blockDim.x) {
         const int il = MULTI ? q / NQ1 : 0;
@@ -345,19 +382,19 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
 #pragma unroll
         for (int cb = 0; cb < CB; ++cb) {
             const int c = min(c0 + cb, g.C - 1);
-            cp[cb] = codes + ((size_t)n * g.K * g.C + c) * plane + pix;
+            cp[cb] = codes + (((size_t)n * g.K * g.C + c) * plane + pix) * CW;
             Ab[cb] = reinterpret_cast<char*>(A + (size_t)cb * g.RS * 4 * NQp + q);
         }
         // operands of output channel k + PF are requested while channel k is consumed
         constexpr int PF = 4;
         float gv[PF][4];
-        unsigned cw[PF][CB];
+        Codes4<WIDE> cw[PF][CB];
 #pragma unroll
         for (int u = 0; u < PF; ++u)
             if (u < g.K) {
                 load_g4<T, VEC>(gp + (size_t)u * plane, ow0, g.OW, gv[u]);
 #pragma unroll
-                for (int cb = 0; cb < CB; ++cb) cw[u][cb] = load_c4<VEC>(cp[cb] + (size_t)u * cstep, ow0, g.OW);
+                for (int cb = 0; cb < CB; ++cb) cw[u][cb] = load_codes4<WIDE, VEC>(cp[cb] + (size_t)u * cstep, ow0, g.OW);
             }
         gp += (size_t)PF * plane;          // the next channel to request
 #pragma unroll
@@ -377,13 +414,14 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
                     }
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const unsigned code = (cw[u][cb] >> (8 * j)) & 0xffu;
+                        unsigned tmin, tmax;
+                        taps_of<WIDE>(cw[u][cb], j, tmin, tmax);
                         if constexpr (BR == 0 || BR == 1) {
-                            float* dst = reinterpret_cast<float*>(Ab[cb] + (code & 15u) * tstride + j * NQp * sizeof(float));
+                            float* dst = reinterpret_cast<float*>(Ab[cb] + tmin * tstride + j * NQp * sizeof(float));
                             *dst = (BR == 0) ? __fmaf_rn(a, gv[u][j], *dst) : (*dst + gv[u][j]);
                         }
                         if constexpr (BR == 0 || BR == 2) {
-                            float* dst = reinterpret_cast<float*>(Ab[cb] + (code >> 4) * tstride + j * NQp * sizeof(float));
+                            float* dst = reinterpret_cast<float*>(Ab[cb] + tmax * tstride + j * NQp * sizeof(float));
                             *dst = (BR == 0) ? __fmaf_rn(b, gv[u][j], *dst) : (*dst + gv[u][j]);
                         }
                     }
@@ -392,7 +430,7 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
                     load_g4<T, VEC>(gp, ow0, g.OW, gv[u]);
 #pragma unroll
                     for (int cb = 0; cb < CB; ++cb) {
-                        cw[u][cb] = load_c4<VEC>(cp[cb], ow0, g.OW);
+                        cw[u][cb] = load_codes4<WIDE, VEC>(cp[cb], ow0, g.OW);
                         cp[cb] += cstep;
                     }
                     gp += plane;
@@ -466,7 +504,7 @@ __global__ void pad_input_kernel(Geo g, const T* __restrict__ x, T* __restrict__
 // WARP: one warp per (k, c) pair, eight pairs per CTA, the lanes walk the pair's (image, quad)
 // items and reduce with shuffles; for maps so small that a 256-thread CTA per pair would spend its
 // time zeroing, synchronising and reducing.  Else one CTA per pair.
-template <typename T, int BR, bool XS, bool VEC, bool WARP>
+template <typename T, int BR, bool XS, bool VEC, bool WARP, bool WIDE>
 __global__ void __launch_bounds__(256)
 bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
                    const float* __restrict__ alpha, const float* __restrict__ beta,
@@ -505,18 +543,20 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
     const int NQ = g.OH * QPR;
     const size_t plane = (size_t)g.OH * g.OW;
     const size_t gstep = (size_t)g.K * plane;            // grad_y: one image further
-    const size_t cstep = (size_t)g.K * g.C * plane;      // codes: one image further
+    constexpr int CW = WIDE ? 2 : 1;                      // bytes per code
+    const size_t cstep = (size_t)g.K * g.C * plane * CW; // codes: one image further (bytes)
     const size_t xstep = (size_t)g.C * pl.xs_elems;      // padded x: one image further
     float sa = 0.0f, sb = 0.0f;
     // one (image, quad) item: 4 gradients gv, 4 winner codes cw, padded-x pointer xp of the item
-    auto accumulate = [&](int oh, int ow0, const float* gv, unsigned cw, const T* xp) {
+    auto accumulate = [&](int oh, int ow0, const float* gv, const Codes4<WIDE>& cw, const T* xp) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             if (!VEC && ow0 + j >= g.OW) continue;
-            const unsigned code = (cw >> (8 * j)) & 0xffu;
+            unsigned tmin, tmax;
+            taps_of<WIDE>(cw, j, tmin, tmax);
             const float gvj = gv[j];
             if constexpr (BR == 0 || BR == 1) {
-                const unsigned t = code & 15u;
+                const unsigned t = tmin;
                 float* dst = reinterpret_cast<float*>(colb + t * 1024u);
                 *dst += gvj;
                 if (need_ab) {
@@ -532,7 +572,7 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
                 }
             }
             if constexpr (BR == 0 || BR == 2) {
-                const unsigned t = code >> 4;
+                const unsigned t = tmax;
                 float* dst = reinterpret_cast<float*>(colb + (g.RS + t) * 1024u);
                 *dst += gvj;
                 if (need_ab) {
@@ -556,20 +596,21 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
             const int ow0 = (q - oh * QPR) * 4;
             const size_t pix = (size_t)oh * g.OW + ow0;
             const T* gp = gy + (size_t)k * plane + pix;
-            const uint8_t* cp = codes + ((size_t)k * g.C + c) * plane + pix;
+            const uint8_t* cp = codes + (((size_t)k * g.C + c) * plane + pix) * CW;
             const T* xp = XS ? reinterpret_cast<const T*>(pl.xpad) + (size_t)c * pl.xs_elems +
                                    (size_t)oh * g.sh * pl.WP + ow0 * g.sw
                              : x + (size_t)c * g.H * g.W;
             float gv_cur[4], gv_nxt[4];
-            unsigned cw_cur, cw_nxt = 0;
+            Codes4<WIDE> cw_cur, cw_nxt;
+            cw_nxt.lo = cw_nxt.hi = 0u;
             load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
-            cw_cur = load_c4<VEC>(cp, ow0, g.OW);
+            cw_cur = load_codes4<WIDE, VEC>(cp, ow0, g.OW);
             for (int n = 0; n < g.N; ++n) {
                 if (n + 1 < g.N) {
                     gp += gstep;
                     cp += cstep;
                     load_g4<T, VEC>(gp, ow0, g.OW, gv_nxt);
-                    cw_nxt = load_c4<VEC>(cp, ow0, g.OW);
+                    cw_nxt = load_codes4<WIDE, VEC>(cp, ow0, g.OW);
                 }
                 accumulate(oh, ow0, gv_cur, cw_cur, xp);
                 xp += XS ? xstep : (size_t)g.C * g.H * g.W;
@@ -583,13 +624,14 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
         const int dn = nworkers / NQ, dq = nworkers - dn * NQ;
         int n = me / NQ, q = me - n * NQ;
         float gv_cur[4], gv_nxt[4];
-        unsigned cw_cur = 0, cw_nxt = 0;
+        Codes4<WIDE> cw_cur, cw_nxt;
+        cw_cur.lo = cw_cur.hi = cw_nxt.lo = cw_nxt.hi = 0u;
         auto item_ptrs = [&](int n_, int q_, int& oh, int& ow0, const T*& gp, const uint8_t*& cp, const T*& xp) {
             oh = q_ / QPR;
             ow0 = (q_ - oh * QPR) * 4;
             const size_t pix = (size_t)oh * g.OW + ow0;
             gp = gy + ((size_t)n_ * g.K + k) * plane + pix;
-            cp = codes + (((size_t)n_ * g.K + k) * g.C + c) * plane + pix;
+            cp = codes + ((((size_t)n_ * g.K + k) * g.C + c) * plane + pix) * CW;
             xp = XS ? reinterpret_cast<const T*>(pl.xpad) + ((size_t)n_ * g.C + c) * pl.xs_elems +
                           (size_t)oh * g.sh * pl.WP + ow0 * g.sw
                     : x + ((size_t)n_ * g.C + c) * g.H * g.W;
@@ -600,7 +642,7 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
         if (have) {
             item_ptrs(n, q, oh, ow0, gp, cp, xp);
             load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
-            cw_cur = load_c4<VEC>(cp, ow0, g.OW);
+            cw_cur = load_codes4<WIDE, VEC>(cp, ow0, g.OW);
         }
         while (have) {
             int n2 = n + dn, q2 = q + dq;
@@ -611,7 +653,7 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
             if (more) {
                 item_ptrs(n2, q2, oh2, ow2, gp2, cp2, xp2);
                 load_g4<T, VEC>(gp2, ow2, g.OW, gv_nxt);
-                cw_nxt = load_c4<VEC>(cp2, ow2, g.OW);
+                cw_nxt = load_codes4<WIDE, VEC>(cp2, ow2, g.OW);
             }
             accumulate(oh, ow0, gv_cur, cw_cur, xp);
             n = n2; q = q2; oh = oh2; ow0 = ow2; xp = xp2;
@@ -746,7 +788,6 @@ inline bool plan_idx_gw(const Geo& g, int* chunks, size_t* smem) {
 }
 
 inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
-    if (g.wide) return false;
     pl->QPR = (g.OW + 3) / 4;
     const int halo = (g.R - 1) * g.dh;
     for (int cb = kGxCB; cb >= 1; --cb) {
@@ -765,7 +806,7 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
             long im = 256 / q1;
             if (im > maxq / q1) im = maxq / q1;
             if (im > g.N) im = g.N;
-            if (im > 1) pl->imgs = (int)im;
+            if (im > 1 && !g.wide) pl->imgs = (int)im;   // wide codes: one image per CTA (fewer kernel variants)
         } else {
             // NR = ceil((THI + halo) / sh) + 1 at most
             thi = (int)((nr - 2) * g.sh) - halo;
@@ -788,6 +829,7 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
         int th = ((nq + passes - 1) / passes + 31) / 32 * 32;
         if (th < 256) th = 256;
         pl->threads = th < cap ? th : cap;
+        if (g.wide) pl->threads = 256;
         pl->ncblk = (g.C + cb - 1) / cb;
         const size_t nct = (size_t)((g.N + pl->imgs - 1) / pl->imgs) * pl->tiles_per_img * pl->ncblk;
         if (nct > 0x7fffffffu) return false;
