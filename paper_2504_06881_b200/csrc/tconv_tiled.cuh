@@ -420,7 +420,8 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
         if (WIN && CHAN == CH_SUM && out_row[q] >= 0) {
             const int n = out_row[q] / g.OH, oh = out_row[q] - n * g.OH;
             code_base[q] = reinterpret_cast<uint8_t*>(p.winners) +
-                           ((size_t)n * g.K + (size_t)kt * TILE_K) * g.C * plane + (size_t)oh * g.OW + qcol[q];
+                           (((size_t)n * g.K + (size_t)kt * TILE_K) * g.C * plane + (size_t)oh * g.OW + qcol[q]) *
+                               (RS > 16 ? 2 : 1);
         }
     }
     const int row_step = g.dh * p.XP;
@@ -470,7 +471,13 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                 // rank itself: 15 - tap for the min branch (low nibble of the code), 16 * (15 - tap)
                 // for the max branch (high nibble), both read back with one complement-and-mask.
                 // (a non-zero |d| * 2^125 is at least 256 > 240, the largest rank; |x + w| < 2^95 is assumed.)
-                constexpr float kS = 4294967296.0f;          // 2^32
+                // Windows above 16 taps use 16-bit codes: rank = 255 - tap (low byte) and
+                // 256 * (255 - tap) (high byte); the scale grows to 2^41 so that a non-zero
+                // |d| * 2^125 (at least 2^17) still exceeds every rank, |x + w| < 2^86 assumed.
+                constexpr bool WIDE = RS > 16;
+                constexpr int CW = WIDE ? 2 : 1;             // bytes per code
+                constexpr int RTOP = WIDE ? 255 : 15, RMUL = WIDE ? 256 : 16;
+                constexpr float kS = WIDE ? 2199023255552.0f : 4294967296.0f;   // 2^41 : 2^32
                 constexpr float kH = 4.253529586511731e37f;  // 2^125
                 constexpr float kB = 8388608.0f;             // 2^23
                 constexpr bool DO_MIN = TWO || TAP_MIN, DO_MAX = TWO || !TAP_MIN;
@@ -490,7 +497,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                     }
 #pragma unroll
                     for (int q = 0; q < Q; ++q) {
-                        unsigned packed[2] = {0u, 0u};
+                        unsigned packed[2] = {0u, 0u}, packed_hi[2] = {0u, 0u};   // 4 codes per channel (wide: two words)
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             float ta[RS][2], tb[PAR ? RS : 1][2];
@@ -528,7 +535,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                                 for (int tap = 0; tap < RS; ++tap) {
                                     float d0 = e0, d1 = e1;
                                     fma2s(kS, ta[tap][0], ta[tap][1], d0, d1);             // >= 0
-                                    key[tap][0] = key[tap][1] = kB + (float)(15 - tap);
+                                    key[tap][0] = key[tap][1] = kB + (float)(RTOP - tap);
                                     fma2s(-kH, d0, d1, key[tap][0], key[tap][1]);
                                 }
                                 bits_min[0] = __float_as_uint(fold_taps<RS>(key, 0, false));
@@ -541,7 +548,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                                 for (int tap = 0; tap < RS; ++tap) {
                                     float d0 = e0, d1 = e1;
                                     fma2s(kS, tm[tap][0], tm[tap][1], d0, d1);             // <= 0
-                                    key[tap][0] = key[tap][1] = kB + (float)(16 * (15 - tap));
+                                    key[tap][0] = key[tap][1] = kB + (float)(RMUL * (RTOP - tap));
                                     fma2s(kH, d0, d1, key[tap][0], key[tap][1]);
                                 }
                                 bits_max[0] = __float_as_uint(fold_taps<RS>(key, 0, false));
@@ -550,9 +557,12 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
 #pragma unroll
                             for (int h = 0; h < 2; ++h) {
                                 unsigned code;
-                                if constexpr (TWO) code = (~bits_min[h] & 0x0fu) | (~bits_max[h] & 0xf0u);
-                                else code = TAP_MIN ? (~bits_min[h] & 0x0fu) : (~bits_max[h] & 0xf0u);
-                                packed[h] |= code << (8 * j);
+                                constexpr unsigned MLO = WIDE ? 0x00ffu : 0x0fu, MHI = WIDE ? 0xff00u : 0xf0u;
+                                if constexpr (TWO) code = (~bits_min[h] & MLO) | (~bits_max[h] & MHI);
+                                else code = TAP_MIN ? (~bits_min[h] & MLO) : (~bits_max[h] & MHI);
+                                if constexpr (!WIDE) packed[h] |= code << (8 * j);
+                                else if (j < 2) packed[h] |= code << (16 * j);
+                                else packed_hi[h] |= code << (16 * (j - 2));
                             }
                         }
                         // one byte per (n, k, c, oh, ow): low nibble argmin tap, high nibble argmax tap
@@ -561,13 +571,20 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                             for (int h = 0; h < 2; ++h) {
                                 const int kl = kg * TK + 2 * kp + h;
                                 if (kt * TILE_K + kl >= g.K) continue;
-                                uint8_t* dst = code_base[q] + ((size_t)kl * g.C + c) * plane;
+                                uint8_t* dst = code_base[q] + ((size_t)kl * g.C + c) * plane * CW;
                                 if (qcol[q] + 3 < g.OW && ((g.OW & 3) == 0)) {
-                                    *reinterpret_cast<unsigned*>(dst) = packed[h];
+                                    if constexpr (WIDE) *reinterpret_cast<uint2*>(dst) = make_uint2(packed[h], packed_hi[h]);
+                                    else *reinterpret_cast<unsigned*>(dst) = packed[h];
                                 } else {
 #pragma unroll
                                     for (int j = 0; j < 4; ++j)
-                                        if (qcol[q] + j < g.OW) dst[j] = (uint8_t)(packed[h] >> (8 * j));
+                                        if (qcol[q] + j < g.OW) {
+                                            if constexpr (WIDE)
+                                                reinterpret_cast<uint16_t*>(dst)[j] =
+                                                    (uint16_t)((j < 2 ? packed[h] : packed_hi[h]) >> (16 * (j & 1)));
+                                            else
+                                                dst[j] = (uint8_t)(packed[h] >> (8 * j));
+                                        }
                                 }
                             }
                         }
@@ -995,9 +1012,7 @@ int launch_tiled_geom(FwdArgs& a) {
 template <int MODE, int CHAN>
 int launch_fwd_tiled_inst(FwdArgs& a) {
     if (a.dtype != TCONV_F32) return TCONV_ERR_UNSUPPORTED;  // bf16: separate kernel
-    // more than 16 taps: the nibble codes of the Sum forms do not fit (the winner-free forward and
-    // the Max / Min combines do)
-    if (a.g.wide && a.winners && a.g.chan == CH_SUM) return TCONV_ERR_UNSUPPORTED;
+    // (windows above 16 taps: the Sum forms emit 16-bit codes)
     if ((double)a.g.N * a.g.C * a.g.H * a.g.W >= 2.0e9) return TCONV_ERR_UNSUPPORTED;  // 32-bit offsets
     if (a.winners) return launch_tiled_geom<float, MODE, CHAN, true>(a);
     return launch_tiled_geom<float, MODE, CHAN, false>(a);
