@@ -118,35 +118,34 @@ bwd_gx_generic_kernel(Geo g, const float* __restrict__ alpha, const float* __res
     const int n = (int)(i / ((size_t)g.W * g.H * g.C));
     const size_t plane = (size_t)g.OH * g.OW;
     const bool twob = two_branch(g.mode);
+    // taps outermost: the output that reads this input through tap (r, s) is found once, then all
+    // output channels are visited (fixed order: taps ascending, k ascending inside a tap)
     float acc = 0.0f;
-    for (int k = 0; k < g.K; ++k) {
-        float a = 1.0f, b = 1.0f;
-        if (twob) {
-            if (alpha) a = alpha[(size_t)k * g.C + c];
-            if (beta) b = beta[(size_t)k * g.C + c];
-        }
-        const size_t obase = ((size_t)n * g.K + k) * plane;
-        const size_t cbase = (((size_t)n * g.K + k) * g.C + c) * plane;
-        for (int r = 0; r < g.R; ++r) {
-            const int nh = ih + g.ph - r * g.dh;
-            if (nh < 0 || nh % g.sh != 0) continue;
-            const int oh = nh / g.sh;
-            if (oh >= g.OH) continue;
-            for (int s = 0; s < g.S; ++s) {
-                const int nw = iw + g.pw - s * g.dw;
-                if (nw < 0 || nw % g.sw != 0) continue;
-                const int ow = nw / g.sw;
-                if (ow >= g.OW) continue;
-                const int tap = r * g.S + s;
-                const size_t op = (size_t)oh * g.OW + ow;
+    for (int r = 0; r < g.R; ++r) {
+        const int nh = ih + g.ph - r * g.dh;
+        if (nh < 0 || nh % g.sh != 0) continue;
+        const int oh = nh / g.sh;
+        if (oh >= g.OH) continue;
+        for (int s = 0; s < g.S; ++s) {
+            const int nw = iw + g.pw - s * g.dw;
+            if (nw < 0 || nw % g.sw != 0) continue;
+            const int ow = nw / g.sw;
+            if (ow >= g.OW) continue;
+            const int tap = r * g.S + s;
+            const size_t op = (size_t)oh * g.OW + ow;
+            for (int k = 0; k < g.K; ++k) {
+                const size_t obase = ((size_t)n * g.K + k) * plane;
                 if (g.chan != CH_SUM) {
                     if (((const int32_t*)winners)[obase + op] == c * g.RS + tap)
                         acc += to_f32(gy[obase + op]);
                 } else {
+                    const size_t cbase = (((size_t)n * g.K + k) * g.C + c) * plane;
                     int amn, amx;
                     read_code(g, winners, cbase + op, amn, amx);
                     const float gv = to_f32(gy[obase + op]);
                     if (twob) {
+                        const float a = alpha ? alpha[(size_t)k * g.C + c] : 1.0f;
+                        const float b = beta ? beta[(size_t)k * g.C + c] : 1.0f;
                         if (amn == tap) acc = __fmaf_rn(a, gv, acc);
                         if (amx == tap) acc = __fmaf_rn(b, gv, acc);
                     } else if ((g.mode == TCONV_MIN_PLUS ? amn : amx) == tap) {
