@@ -290,10 +290,11 @@ __device__ __forceinline__ unsigned load_c4(const uint8_t* p, int ow0, int OW) {
 // nibble, argmax tap in the high nibble.  WIDE (R*S <= 256): 16 bits each, argmin tap in the low
 // byte, argmax tap in the high byte; `p` then points at the first of 4 adjacent 16-bit codes.
 template <bool WIDE> struct Codes4 { unsigned lo, hi; };
+template <> struct Codes4<false> { unsigned lo; };
 template <bool WIDE, bool VEC>
 __device__ __forceinline__ Codes4<WIDE> load_codes4(const uint8_t* p, int ow0, int OW) {
     Codes4<WIDE> r;
-    r.hi = 0u;
+    if constexpr (WIDE) r.hi = 0u;
     if constexpr (!WIDE) {
         r.lo = load_c4<VEC>(p, ow0, OW);
     } else if constexpr (VEC) {
@@ -602,7 +603,8 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
                              : x + (size_t)c * g.H * g.W;
             float gv_cur[4], gv_nxt[4];
             Codes4<WIDE> cw_cur, cw_nxt;
-            cw_nxt.lo = cw_nxt.hi = 0u;
+            cw_nxt.lo = 0u;
+            if constexpr (WIDE) cw_nxt.hi = 0u;
             load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
             cw_cur = load_codes4<WIDE, VEC>(cp, ow0, g.OW);
             for (int n = 0; n < g.N; ++n) {
@@ -625,7 +627,8 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
         int n = me / NQ, q = me - n * NQ;
         float gv_cur[4], gv_nxt[4];
         Codes4<WIDE> cw_cur, cw_nxt;
-        cw_cur.lo = cw_cur.hi = cw_nxt.lo = cw_nxt.hi = 0u;
+        cw_cur.lo = cw_nxt.lo = 0u;
+        if constexpr (WIDE) cw_cur.hi = cw_nxt.hi = 0u;
         auto item_ptrs = [&](int n_, int q_, int& oh, int& ow0, const T*& gp, const uint8_t*& cp, const T*& xp) {
             oh = q_ / QPR;
             ow0 = (q_ - oh * QPR) * 4;
