@@ -65,12 +65,15 @@ class TropicalConvFn(torch.autograd.Function):
         if ev is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-        grads = tconv.backward(d, xc, wc, g, w2c, al, be, winners)
+        need = ["grad_w", "grad_w2", "grad_alpha", "grad_beta", "grad_bias"]
+        if ctx.needs_input_grad[0]:
+            need.append("grad_x")          # a first layer's input needs none: the kernel is skipped
+        grads = tconv.backward(d, xc, wc, g, w2c, al, be, winners, need=tuple(need))
         if ev is not None:
             e1.record()
             ev.append(("bwd", d, e0, e1))
         has_w2, has_a, has_b, has_bias = ctx.has
-        gx = grads["grad_x"].to(ctx.in_dtype)
+        gx = grads["grad_x"].to(ctx.in_dtype) if "grad_x" in grads else None
         return (gx, grads["grad_w"], grads.get("grad_w2") if has_w2 else None,
                 grads.get("grad_alpha") if has_a else None, grads.get("grad_beta") if has_b else None,
                 grads["grad_bias"] if has_bias else None, None)
