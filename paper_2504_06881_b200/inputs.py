@@ -110,3 +110,41 @@ def cfg3b(dtype="f32", mode="parallel", N=64):
 def cfg4(dtype="bf16", mode="compound", N=8, H=128, W=256, C=256, K=256):
     d = layer(N, C, H, W, K, 3, 3, stride=1, pad=2, dil=2, mode=mode, dtype=dtype)
     return d, dict(x=("relu_normal", 0.0, 1.0), w=("normal", 0.0, 0.05))
+
+
+# Three-dimensional layers (Section 3.2; the 3-D LeNet of the paper's appendix works on 28^3 and
+# 64^3 volumes with 5 x 5 x 5 windows).  Descriptor keys: N, C, D, H, W, K, T, R, S and the
+# triples stride / pad / dil in (depth, height, width) order.
+def layer3d(N, C, D, H, W, K, T=3, R=3, S=3, stride=1, pad=0, dil=1, mode="max_plus",
+            chan="default", dtype="f32") -> dict:
+    three = lambda v: (v, v, v) if isinstance(v, int) else tuple(v)
+    return dict(N=N, C=C, D=D, H=H, W=W, K=K, T=T, R=R, S=S, stride=three(stride), pad=three(pad),
+                dil=three(dil), mode=mode, chan=chan, dtype=dtype)
+
+
+def output_dhw(d: dict):
+    def ext(i, p, dl, k, s):
+        span = i + 2 * p - dl * (k - 1) - 1
+        return 0 if span < 0 else span // s + 1
+    return tuple(ext(d[a], d["pad"][j], d["dil"][j], d[b], d["stride"][j])
+                 for j, (a, b) in enumerate((("D", "T"), ("H", "R"), ("W", "S"))))
+
+
+def draw3d(d: dict, seed: int, x=("normal", 0.0, 1.0), w=("normal", 0.0, 0.1),
+           ab=("uniform", 0.0, 1.0), bias=("uniform", -0.1, 0.1), g=("normal", 0.0, 1.0)) -> dict:
+    """x[N,C,D,H,W], w / w2 [K,C,T,R,S], alpha / beta [K,C], bias[K], g[N,K,OD,OH,OW], drawn in
+    that order from one ``numpy.random.RandomState(seed)``."""
+    rs = np.random.RandomState(seed)
+    N, C, D, H, W, K, T, R, S = (d[k] for k in "NCDHWKTRS")
+    t = {}
+    t["x"] = _draw(rs, x, (N, C, D, H, W))
+    t["w"] = _draw(rs, w, (K, C, T, R, S))
+    t["w2"] = _draw(rs, w, (K, C, T, R, S))
+    t["alpha"] = _draw(rs, ab, (K, C))
+    t["beta"] = _draw(rs, ab, (K, C))
+    t["bias"] = _draw(rs, bias, (K,))
+    t["g"] = _draw(rs, g, (N, K) + output_dhw(d))
+    if d["dtype"] == "bf16":
+        for k in ("x", "w", "w2", "g"):
+            t[k] = to_bf16_values(t[k])
+    return t
