@@ -25,8 +25,8 @@ FWD_INSTANCES = [("fwd_inst_maxplus_sum", 0, 1), ("fwd_inst_maxplus_max", 0, 2),
 
 
 def _newest_source() -> float:
-    files = list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + [ROOT / "include" / "tconv.h",
-                                                                   Path(__file__)]
+    files = list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + \
+        list((ROOT / "include").glob("*.h")) + [Path(__file__)]
     return max(f.stat().st_mtime for f in files)
 
 
@@ -52,7 +52,8 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     if not force and LIB.exists() and LIB.stat().st_mtime >= _newest_source():
         return LIB
     OBJ.mkdir(exist_ok=True)
-    jobs = [(CSRC / "tconv_api.cu", OBJ / "tconv_api.o", [], verbose)]
+    jobs = [(CSRC / "tconv_api.cu", OBJ / "tconv_api.o", [], verbose),
+            (CSRC / "tconv3d_api.cu", OBJ / "tconv3d_api.o", [], verbose)]
     for name, mode, chan in FWD_INSTANCES:
         defs = [f"-DTCONV_INST_NAME={name}", f"-DTCONV_INST_MODE={mode}", f"-DTCONV_INST_CHAN={chan}"]
         jobs.append((CSRC / "tconv_fwd_inst.cu", OBJ / f"{name}.o", defs, verbose))

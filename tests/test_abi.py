@@ -12,13 +12,16 @@ ROOT = Path(__file__).resolve().parent.parent
 
 
 def test_every_declared_symbol_is_exported():
-    header = (ROOT / "include" / "tconv.h").read_text()
-    declared = set(re.findall(r"\b(tconv_[a-z0-9_]+)\s*\(", header))
-    assert declared, "no declarations found"
+    from paper_2504_06881_b200 import tconv3d
     lib = ctypes.CDLL(str(tconv.LIB_PATH))
-    for name in declared:
-        assert hasattr(lib, name), f"{name} declared in tconv.h but not exported"
-    assert declared == set(tconv.SYMBOLS)
+    headers = sorted((ROOT / "include").glob("*.h"))
+    assert [h.name for h in headers] == ["tconv.h", "tconv3d.h"]
+    for header, symbols in zip(headers, (tconv.SYMBOLS, tconv3d.SYMBOLS)):
+        declared = set(re.findall(r"\b(tconv(?:3d)?_[a-z0-9_]+)\s*\(", header.read_text()))
+        assert declared, "no declarations found"
+        for name in declared:
+            assert hasattr(lib, name), f"{name} declared in {header.name} but not exported"
+        assert declared == set(symbols), header.name
 
 
 def test_output_shape_and_sizes():
