@@ -44,7 +44,7 @@ int make_geo3(const tconv3d_desc_t* d, Geo3* g) {
     const double lim = 2147483647.0;
     const double vol = (double)g->OD * g->OH * g->OW;
     if ((double)d->N * d->C * d->D * d->H * d->W > lim || (double)d->N * d->K * vol * d->C > lim ||
-        (double)d->K * d->C * g->taps > lim || d->N > 65535)
+        (double)d->K * d->C * g->taps > lim || (double)d->N * d->K * vol > lim)
         return TCONV_ERR_TOO_LARGE;
     g->vol = (int)vol;
     g->mode = d->mode;
@@ -71,6 +71,22 @@ int gw_splits(const Geo3& g) {
     return (int)want;
 }
 
+// Splits of the same range for the grad_bias partial sums (K blocks otherwise).
+int bias_splits(const Geo3& g) {
+    const long long total = (long long)g.N * g.vol;
+    long long want = (2 * 148 + g.K - 1) / g.K;
+    const long long most = (total + 4095) / 4096;
+    if (want > most) want = most;
+    if (want < 1) want = 1;
+    if (want > 64) want = 64;
+    return (int)want;
+}
+
+size_t backward_scratch_floats(const Geo3& g) {
+    const size_t ns = (size_t)gw_splits(g);
+    return 2 * ns * g.K * g.C * g.taps + 2 * ns * g.K * g.C + (size_t)bias_splits(g) * g.K;
+}
+
 int check(cudaError_t e) { return e == cudaSuccess ? TCONV_OK : TCONV_ERR_CUDA; }
 
 template <typename T>
@@ -84,14 +100,24 @@ int forward3_t(const Geo3& g, const void* x, const void* w, const void* w2, cons
     if (cch < 1) cch = 1;
     if (cch > g.C) cch = g.C;
     const size_t smem = per_c * cch;
-    const dim3 grid((unsigned)((g.vol + kFwd3Threads - 1) / kFwd3Threads), (unsigned)((g.K + kt - 1) / kt),
-                    (unsigned)g.N);
-    if (kt == 4)
-        fwd3d_kernel<T, 4><<<grid, kFwd3Threads, smem, st>>>(g, cch, (const T*)x, (const T*)w, (const T*)w2,
-                                                            alpha, beta, bias, (T*)y, winners);
-    else
-        fwd3d_kernel<T, 2><<<grid, kFwd3Threads, smem, st>>>(g, cch, (const T*)x, (const T*)w, (const T*)w2,
-                                                            alpha, beta, bias, (T*)y, winners);
+    const long long flat = (long long)g.N * g.vol;
+    const dim3 grid((unsigned)((flat + kFwd3Threads - 1) / kFwd3Threads), (unsigned)((g.K + kt - 1) / kt));
+#define TCONV3_LAUNCH(KTV, WINV, SCV)                                                                     \
+    fwd3d_kernel<T, KTV, WINV, SCV><<<grid, kFwd3Threads, smem, st>>>(                                     \
+        g, cch, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, bias, (T*)y, winners)
+#define TCONV3_BY_S(KTV, WINV)                                   \
+    {                                                            \
+        if (g.S == 3) TCONV3_LAUNCH(KTV, WINV, 3);               \
+        else if (g.S == 5) TCONV3_LAUNCH(KTV, WINV, 5);          \
+        else TCONV3_LAUNCH(KTV, WINV, 0);                        \
+    }
+    if (kt == 4) {
+        if (winners) TCONV3_BY_S(4, true) else TCONV3_BY_S(4, false)
+    } else {
+        if (winners) TCONV3_BY_S(2, true) else TCONV3_BY_S(2, false)
+    }
+#undef TCONV3_BY_S
+#undef TCONV3_LAUNCH
     g3_launches += 1;
     return check(cudaGetLastError());
 }
@@ -103,15 +129,23 @@ int backward3_t(const Geo3& g, const void* x, const void* w, const void* w2, con
     const bool two = two_branch(g.mode);
     if (gx) {
         const size_t total = (size_t)g.N * g.C * g.D * g.H * g.W;
-        bwd3d_gx_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, alpha, beta, (const T*)gy,
-                                                                           winners, (T*)gx);
+        // channel slices only while the input has too few elements to fill the GPU with one thread
+        // each: every slice repeats the tap geometry of its element
+        const size_t want = ((size_t)148 * 2048 + total - 1) / total;
+        int slices = 1;
+        while (slices < kGx3Slices && (size_t)slices < want && 2 * slices <= g.K) slices *= 2;
+        const unsigned per_block = 32u * kGx3Slices / slices;
+        bwd3d_gx_kernel<T><<<(unsigned)((total + per_block - 1) / per_block), dim3(per_block, (unsigned)slices), 0, st>>>(
+            g, alpha, beta, (const T*)gy, winners, (T*)gx);
         g3_launches += 1;
     }
+    const int nsplit = gw_splits(g);
+    const size_t count = (size_t)g.K * g.C * g.taps;
+    float* pmin = (float*)ws;
+    float* pmax = pmin + (size_t)nsplit * count;
+    float* pab = pmax + (size_t)nsplit * count;          // [nsplit][K*C][2]
+    float* pbias = pab + (size_t)nsplit * g.K * g.C * 2;  // [bias splits][K]
     if (gw || gw2) {
-        const int nsplit = gw_splits(g);
-        const size_t count = (size_t)g.K * g.C * g.taps;
-        float* pmin = (float*)ws;
-        float* pmax = pmin + (size_t)nsplit * count;
         bwd3d_gw_kernel<T><<<dim3((unsigned)(g.K * g.C), (unsigned)nsplit), 256, 0, st>>>(
             g, nsplit, (const T*)gy, winners, pmin, pmax);
         bwd3d_gw_finish_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(g, nsplit, alpha, beta, pmin,
@@ -119,13 +153,18 @@ int backward3_t(const Geo3& g, const void* x, const void* w, const void* w2, con
         g3_launches += 2;
     }
     if (two && (galpha || gbeta)) {
-        bwd3d_gab_kernel<T><<<(unsigned)(g.K * g.C), 256, 0, st>>>(g, (const T*)x, (const T*)w, (const T*)w2,
-                                                                  (const T*)gy, winners, galpha, gbeta);
-        g3_launches += 1;
+        bwd3d_gab_kernel<T><<<dim3((unsigned)(g.K * g.C), (unsigned)nsplit), 256, 0, st>>>(
+            g, nsplit, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, winners, pab);
+        const int kc = g.K * g.C;
+        if (galpha) bwd3d_sum_splits_kernel<<<(kc + 255) / 256, 256, 0, st>>>(kc, nsplit, 2, 0, pab, galpha);
+        if (gbeta) bwd3d_sum_splits_kernel<<<(kc + 255) / 256, 256, 0, st>>>(kc, nsplit, 2, 1, pab, gbeta);
+        g3_launches += 1 + (galpha ? 1 : 0) + (gbeta ? 1 : 0);
     }
     if (gbias) {
-        bwd3d_bias_kernel<T><<<(unsigned)g.K, 256, 0, st>>>(g, (const T*)gy, gbias);
-        g3_launches += 1;
+        const int bs = bias_splits(g);
+        bwd3d_bias_kernel<T><<<dim3((unsigned)g.K, (unsigned)bs), 256, 0, st>>>(g, bs, (const T*)gy, pbias);
+        bwd3d_sum_splits_kernel<<<(g.K + 255) / 256, 256, 0, st>>>(g.K, bs, 1, 0, pbias, gbias);
+        g3_launches += 2;
     }
     return check(cudaGetLastError());
 }
@@ -158,7 +197,7 @@ size_t tconv3d_winner_bytes(const tconv3d_desc_t* desc) {
 size_t tconv3d_workspace_bytes(const tconv3d_desc_t* desc, int backward) {
     Geo3 g;
     if (make_geo3(desc, &g) != TCONV_OK || !backward) return 0;
-    return align_up(winner_bytes3(g), 256) + 2 * (size_t)gw_splits(g) * g.K * g.C * g.taps * sizeof(float) + 256;
+    return align_up(winner_bytes3(g), 256) + backward_scratch_floats(g) * sizeof(float) + 256;
 }
 
 int tconv3d_forward(const tconv3d_desc_t* desc, const void* x, const void* w, const void* w2,

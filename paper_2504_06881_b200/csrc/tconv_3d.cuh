@@ -18,9 +18,12 @@ struct Geo3 {
 
 constexpr int kFwd3Threads = 128;
 
-// Forward.  grid (ceil(vol / 128), ceil(K / KT), N).  Shared memory: weights of `cch` input
-// channels for this block's KT output channels, [cc][tap][KT] (twice in parallel mode), as T.
-template <typename T, int KT>
+// Forward.  grid (ceil(N * vol / 128), ceil(K / KT)): one thread per (n, output position) of the
+// flattened range, KT output channels each.  Shared memory: weights of `cch` input channels for
+// this block's KT output channels, [cc][tap][KT] (twice in parallel mode), as T.
+// WIN: track the winning taps (strict compares, taps ascending); without it the extrema are plain
+// min / max.  SC: the window's innermost extent S when it is 3 or 5 (unrolled), else 0.
+template <typename T, int KT, bool WIN, int SC>
 __global__ void __launch_bounds__(kFwd3Threads)
 fwd3d_kernel(Geo3 g, int cch, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
              const float* __restrict__ alpha, const float* __restrict__ beta,
@@ -30,12 +33,13 @@ fwd3d_kernel(Geo3 g, int cch, const T* __restrict__ x, const T* __restrict__ w, 
     const bool par = g.mode == TCONV_PARALLEL;
     const bool twob = two_branch(g.mode);
     T* wmax_s = par ? wmin_s + (size_t)cch * g.taps * KT : wmin_s;
-    const int pos = blockIdx.x * kFwd3Threads + threadIdx.x;
-    const bool live = pos < g.vol;
-    const int k0 = blockIdx.y * KT, n = blockIdx.z;
-    const int ow = live ? pos % g.OW : 0, oh = live ? (pos / g.OW) % g.OH : 0,
-              od = live ? pos / (g.OW * g.OH) : 0;
+    const long long flat = (long long)blockIdx.x * kFwd3Threads + threadIdx.x;
+    const bool live = flat < (long long)g.N * g.vol;
+    const int n = live ? (int)(flat / g.vol) : 0, pos = live ? (int)(flat % g.vol) : 0;
+    const int k0 = blockIdx.y * KT;
+    const int ow = pos % g.OW, oh = (pos / g.OW) % g.OH, od = pos / (g.OW * g.OH);
     const int d0 = od * g.sd - g.pd, h0 = oh * g.sh - g.ph, w0 = ow * g.sw - g.pw;
+    const int S = SC ? SC : g.S;
     float acc[KT], best[KT];
     int win[KT];
 #pragma unroll
@@ -75,16 +79,46 @@ fwd3d_kernel(Geo3 g, int cch, const T* __restrict__ x, const T* __restrict__ w, 
                     const int ih = h0 + r * g.dh;
                     const bool okh = okd && ih >= 0 && ih < g.H;
                     const T* xrow = xc + ((size_t)(okh ? id : 0) * g.H + (okh ? ih : 0)) * g.W;
-                    for (int s = 0; s < g.S; ++s, ++tap) {
-                        const int iw = w0 + s * g.dw;
-                        T xv = zero_of<T>();
-                        if (okh && iw >= 0 && iw < g.W) xv = xrow[iw];
+                    if constexpr (SC != 0) {
+                        T xv[SC];
 #pragma unroll
-                        for (int j = 0; j < KT; ++j) {
-                            const float tmn = tap_add(xv, wa[tap * KT + j]);
-                            const float tmx = par ? tap_add(xv, wb[tap * KT + j]) : tmn;
-                            if (tmn < mn[j]) { mn[j] = tmn; amn[j] = tap; }
-                            if (tmx > mx[j]) { mx[j] = tmx; amx[j] = tap; }
+                        for (int s = 0; s < SC; ++s) {
+                            const int iw = w0 + s * g.dw;
+                            xv[s] = (okh && iw >= 0 && iw < g.W) ? xrow[iw] : zero_of<T>();
+                        }
+#pragma unroll
+                        for (int s = 0; s < SC; ++s) {
+#pragma unroll
+                            for (int j = 0; j < KT; ++j) {
+                                const float tmn = tap_add(xv[s], wa[(tap + s) * KT + j]);
+                                const float tmx = par ? tap_add(xv[s], wb[(tap + s) * KT + j]) : tmn;
+                                if constexpr (WIN) {
+                                    if (tmn < mn[j]) { mn[j] = tmn; amn[j] = tap + s; }
+                                    if (tmx > mx[j]) { mx[j] = tmx; amx[j] = tap + s; }
+                                } else {
+                                    mn[j] = fminf(mn[j], tmn);
+                                    mx[j] = fmaxf(mx[j], tmx);
+                                }
+                            }
+                        }
+                        tap += SC;
+                    } else {
+                        for (int s = 0; s < S; ++s, ++tap) {
+                            const int iw = w0 + s * g.dw;
+                            T xv = zero_of<T>();
+                            if (okh && iw >= 0 && iw < g.W) xv = xrow[iw];
+#pragma unroll
+                            for (int j = 0; j < KT; ++j) {
+                                const float tmn = tap_add(xv, wa[tap * KT + j]);
+                                const float tmx = par ? tap_add(xv, wb[tap * KT + j]) : tmn;
+                                if constexpr (WIN) {
+                                    if (tmn < mn[j]) { mn[j] = tmn; amn[j] = tap; }
+                                    if (tmx > mx[j]) { mx[j] = tmx; amx[j] = tap; }
+                                } else {
+                                    mn[j] = fminf(mn[j], tmn);
+                                    mx[j] = fmaxf(mx[j], tmx);
+                                }
+                            }
                         }
                     }
                 }
@@ -107,7 +141,7 @@ fwd3d_kernel(Geo3 g, int cch, const T* __restrict__ x, const T* __restrict__ w, 
                     else { if (m < best[j]) { best[j] = m; win[j] = c * g.taps + am; } }
                     if (is_min) amx[j] = 0; else amn[j] = 0;
                 }
-                if (winners && g.chan == CH_SUM)
+                if (WIN && g.chan == CH_SUM)
                     ((uint16_t*)winners)[(((size_t)n * g.K + k) * g.C + c) * g.vol + pos] =
                         (uint16_t)(amn[j] | (amx[j] << 8));
             }
@@ -122,7 +156,7 @@ fwd3d_kernel(Geo3 g, int cch, const T* __restrict__ x, const T* __restrict__ w, 
         if (bias) out = __fadd_rn(out, bias[k]);
         const size_t o = ((size_t)n * g.K + k) * g.vol + pos;
         if (y) y[o] = from_f32<T>(out);
-        if (winners && g.chan != CH_SUM) ((int32_t*)winners)[o] = win[j];
+        if (WIN && g.chan != CH_SUM) ((int32_t*)winners)[o] = win[j];
     }
 }
 
@@ -142,48 +176,64 @@ __device__ __forceinline__ void winners3(const Geo3& g, const void* winners, int
     }
 }
 
-// grad_x in gather form: one thread per input element visits, taps ascending and output channels
-// ascending inside a tap, every output whose window reads it.
+// grad_x in gather form.  A block of 256 threads owns 256 / slices consecutive input elements
+// (threadIdx.x) and splits the output channels over blockDim.y = 1, 2, 4 or 8 slices (k = slice, slice + slices, ...): each thread visits,
+// taps ascending and its channels ascending inside a tap, the outputs whose window reads its
+// element; the slices' partial sums are then added in slice order.  (Small 3-D layers have few
+// input elements: the slices keep enough warps in flight to hide the dependent loads.)
+constexpr int kGx3Slices = 8;
+
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(32 * kGx3Slices)
 bwd3d_gx_kernel(Geo3 g, const float* __restrict__ alpha, const float* __restrict__ beta,
                 const T* __restrict__ gy, const void* __restrict__ winners, T* __restrict__ gx) {
+    __shared__ float part[32 * kGx3Slices];
     const size_t total = (size_t)g.N * g.C * g.D * g.H * g.W;
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    const int iw = (int)(i % g.W), ih = (int)((i / g.W) % g.H), id = (int)((i / ((size_t)g.W * g.H)) % g.D);
-    const int c = (int)((i / ((size_t)g.W * g.H * g.D)) % g.C), n = (int)(i / ((size_t)g.W * g.H * g.D * g.C));
+    const int slice = threadIdx.y, slices = blockDim.y;
+    const bool live = i < total;
     const bool twob = two_branch(g.mode);
     float acc = 0.0f;
-    for (int t = 0; t < g.T; ++t) {
-        const int nd = id + g.pd - t * g.dd;
-        if (nd < 0 || nd % g.sd != 0 || nd / g.sd >= g.OD) continue;
-        for (int r = 0; r < g.R; ++r) {
-            const int nh = ih + g.ph - r * g.dh;
-            if (nh < 0 || nh % g.sh != 0 || nh / g.sh >= g.OH) continue;
-            for (int s = 0; s < g.S; ++s) {
-                const int nw = iw + g.pw - s * g.dw;
-                if (nw < 0 || nw % g.sw != 0 || nw / g.sw >= g.OW) continue;
-                const int tap = (t * g.R + r) * g.S + s;
-                const int pos = ((nd / g.sd) * g.OH + nh / g.sh) * g.OW + nw / g.sw;
-                for (int k = 0; k < g.K; ++k) {
-                    int amn, amx;
-                    winners3(g, winners, n, k, c, pos, amn, amx);
-                    if (amn != tap && amx != tap) continue;
-                    const float gv = to_f32(gy[((size_t)n * g.K + k) * g.vol + pos]);
-                    if (twob) {
-                        const float a = alpha ? alpha[(size_t)k * g.C + c] : 1.0f;
-                        const float b = beta ? beta[(size_t)k * g.C + c] : 1.0f;
-                        if (amn == tap) acc = __fmaf_rn(a, gv, acc);
-                        if (amx == tap) acc = __fmaf_rn(b, gv, acc);
-                    } else {
-                        acc += gv;
+    if (live) {
+        const int iw = (int)(i % g.W), ih = (int)((i / g.W) % g.H), id = (int)((i / ((size_t)g.W * g.H)) % g.D);
+        const int c = (int)((i / ((size_t)g.W * g.H * g.D)) % g.C),
+                  n = (int)(i / ((size_t)g.W * g.H * g.D * g.C));
+        for (int t = 0; t < g.T; ++t) {
+            const int nd = id + g.pd - t * g.dd;
+            if (nd < 0 || nd % g.sd != 0 || nd / g.sd >= g.OD) continue;
+            for (int r = 0; r < g.R; ++r) {
+                const int nh = ih + g.ph - r * g.dh;
+                if (nh < 0 || nh % g.sh != 0 || nh / g.sh >= g.OH) continue;
+                for (int s = 0; s < g.S; ++s) {
+                    const int nw = iw + g.pw - s * g.dw;
+                    if (nw < 0 || nw % g.sw != 0 || nw / g.sw >= g.OW) continue;
+                    const int tap = (t * g.R + r) * g.S + s;
+                    const int pos = ((nd / g.sd) * g.OH + nh / g.sh) * g.OW + nw / g.sw;
+                    for (int k = slice; k < g.K; k += slices) {
+                        int amn, amx;
+                        winners3(g, winners, n, k, c, pos, amn, amx);
+                        if (amn != tap && amx != tap) continue;
+                        const float gv = to_f32(gy[((size_t)n * g.K + k) * g.vol + pos]);
+                        if (twob) {
+                            const float a = alpha ? alpha[(size_t)k * g.C + c] : 1.0f;
+                            const float b = beta ? beta[(size_t)k * g.C + c] : 1.0f;
+                            if (amn == tap) acc = __fmaf_rn(a, gv, acc);
+                            if (amx == tap) acc = __fmaf_rn(b, gv, acc);
+                        } else {
+                            acc += gv;
+                        }
                     }
                 }
             }
         }
     }
-    gx[i] = from_f32<T>(acc);
+    part[slice * blockDim.x + threadIdx.x] = acc;
+    __syncthreads();
+    if (slice == 0 && live) {
+        float total_acc = 0.0f;
+        for (int j = 0; j < slices; ++j) total_acc += part[j * blockDim.x + threadIdx.x];
+        gx[i] = from_f32<T>(total_acc);
+    }
 }
 
 constexpr int kGw3Stage = 1024;  // (winner, gradient) pairs staged per pass
@@ -259,20 +309,22 @@ bwd3d_gw_finish_kernel(Geo3 g, int nsplit, const float* __restrict__ alpha, cons
     }
 }
 
-// grad_alpha / grad_beta: one block per (k, c) sums grad_y * MinPlus3d resp. grad_y * MaxPlus3d,
-// the branch values rebuilt from the winning taps.
+// grad_alpha / grad_beta partial sums: block (k*C + c, split) sums grad_y * MinPlus3d resp.
+// grad_y * MaxPlus3d over its share of the (n, position) range, the branch values rebuilt from the
+// winning taps.  part[split][k*C + c][2].
 template <typename T>
 __global__ void __launch_bounds__(256)
-bwd3d_gab_kernel(Geo3 g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
-                 const T* __restrict__ gy, const void* __restrict__ winners, float* __restrict__ galpha,
-                 float* __restrict__ gbeta) {
+bwd3d_gab_kernel(Geo3 g, int nsplit, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
+                 const T* __restrict__ gy, const void* __restrict__ winners, float* __restrict__ part) {
     __shared__ float red[256];
-    const int c = blockIdx.x % g.C, k = blockIdx.x / g.C;
+    const int c = blockIdx.x % g.C, k = blockIdx.x / g.C, split = blockIdx.y;
     const long long total = (long long)g.N * g.vol;
+    const long long per = (total + nsplit - 1) / nsplit;
+    const long long j0 = split * per, j1 = min(total, j0 + per);
     const T* wmin = w + ((size_t)k * g.C + c) * g.taps;
     const T* wmax = (g.mode == TCONV_PARALLEL ? w2 : w) + ((size_t)k * g.C + c) * g.taps;
     float sa = 0.0f, sb = 0.0f;
-    for (long long j = threadIdx.x; j < total; j += blockDim.x) {
+    for (long long j = j0 + threadIdx.x; j < j1; j += blockDim.x) {
         const int n = (int)(j / g.vol), pos = (int)(j % g.vol);
         const int ow = pos % g.OW, oh = (pos / g.OW) % g.OH, od = pos / (g.OW * g.OH);
         int am[2];
@@ -295,23 +347,37 @@ bwd3d_gab_kernel(Geo3 g, const T* __restrict__ x, const T* __restrict__ w, const
     const float ta = block_sum(sa, red);
     const float tb = block_sum(sb, red);
     if (threadIdx.x == 0) {
-        if (galpha) galpha[(size_t)k * g.C + c] = ta;
-        if (gbeta) gbeta[(size_t)k * g.C + c] = tb;
+        float* o = part + ((size_t)split * g.K * g.C + blockIdx.x) * 2;
+        o[0] = ta;
+        o[1] = tb;
     }
 }
 
-// grad_bias: one block per k.
+// grad_bias partial sums: block (k, split); part[split][k].
 template <typename T>
 __global__ void __launch_bounds__(256)
-bwd3d_bias_kernel(Geo3 g, const T* __restrict__ gy, float* __restrict__ gbias) {
+bwd3d_bias_kernel(Geo3 g, int nsplit, const T* __restrict__ gy, float* __restrict__ part) {
     __shared__ float red[256];
-    const int k = blockIdx.x;
+    const int k = blockIdx.x, split = blockIdx.y;
     const long long total = (long long)g.N * g.vol;
+    const long long per = (total + nsplit - 1) / nsplit;
+    const long long j0 = split * per, j1 = min(total, j0 + per);
     float s = 0.0f;
-    for (long long j = threadIdx.x; j < total; j += blockDim.x)
+    for (long long j = j0 + threadIdx.x; j < j1; j += blockDim.x)
         s += to_f32(gy[((size_t)(j / g.vol) * g.K + k) * g.vol + (j % g.vol)]);
     const float t = block_sum(s, red);
-    if (threadIdx.x == 0) gbias[k] = t;
+    if (threadIdx.x == 0) part[(size_t)split * g.K + k] = t;
+}
+
+// Sums partials over the splits in order: out[i] = sum_split part[(split * count + i) * stride + off].
+__global__ void __launch_bounds__(256)
+bwd3d_sum_splits_kernel(int count, int nsplit, int stride, int off, const float* __restrict__ part,
+                        float* __restrict__ out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count) return;
+    float t = 0.0f;
+    for (int sp = 0; sp < nsplit; ++sp) t += part[((size_t)sp * count + i) * stride + off];
+    out[i] = t;
 }
 
 }  // namespace tconv

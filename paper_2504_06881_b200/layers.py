@@ -10,13 +10,13 @@ from __future__ import annotations
 from .nn import TropicalConv2d
 
 
-def _named(name, mode, chan="default", params="2p", doc=""):
+def _named(name, mode, chan="default", params="2p", doc="", base=TropicalConv2d):
     def __init__(self, in_channels, out_channels, kernel_size, stride=1, padding=0, dilation=1,
                  bias=True, dtype="f32", **kw):
-        TropicalConv2d.__init__(self, in_channels, out_channels, kernel_size, stride=stride,
-                                padding=padding, dilation=dilation, bias=bias, mode=mode, chan=chan,
-                                params=kw.pop("params", params), dtype=dtype, **kw)
-    return type(name, (TropicalConv2d,), {"__init__": __init__, "__doc__": doc})
+        base.__init__(self, in_channels, out_channels, kernel_size, stride=stride,
+                      padding=padding, dilation=dilation, bias=bias, mode=mode, chan=chan,
+                      params=kw.pop("params", params), dtype=dtype, **kw)
+    return type(name, (base,), {"__init__": __init__, "__doc__": doc})
 
 
 MaxPlusSumConv2d = _named("MaxPlusSumConv2d", "max_plus", "sum", doc="layer (i): sum over channels of the max-plus window")
@@ -35,6 +35,22 @@ ParallelMinMaxPlusSumConv2d2p = _named("ParallelMinMaxPlusSumConv2d2p", "paralle
 
 __all__ = [n for n in dir() if n.endswith(("Conv2d", "0p", "1p", "2p"))]
 
-from .nn import TropicalConv1d, TropicalDepthwiseConv2d  # noqa: E402  (1-D form; depthwise form of the MobileNetV2 variants)
+from .nn import TropicalConv1d, TropicalConv3d, TropicalDepthwiseConv2d  # noqa: E402  (1-D, 3-D and depthwise forms)
 
-__all__ += ["TropicalDepthwiseConv2d", "TropicalConv1d"]
+# the three-dimensional layers of Section 3.2 and the Conv3d forms of Sections 3.4 / 3.5: the same
+# names with Conv3d, ``nn.Conv3d``'s constructor arguments
+_SPECS = {"MaxPlusSum": ("max_plus", "sum", "2p"), "MinPlusSum": ("min_plus", "sum", "2p"),
+          "MinPlusMax": ("min_plus", "max", "2p"), "MinPlusMin": ("min_plus", "min", "2p"),
+          "MaxPlusMax": ("max_plus", "max", "2p"), "MaxPlusMin": ("max_plus", "min", "2p")}
+for _stem, (_mode, _chan, _params) in _SPECS.items():
+    globals()[_stem + "Conv3d"] = _named(_stem + "Conv3d", _mode, _chan, doc=f"{_stem}Conv2d in three dimensions",
+                                         base=TropicalConv3d)
+    __all__.append(_stem + "Conv3d")
+for _mode in ("compound", "parallel"):
+    for _params in ("0p", "1p", "2p"):
+        _name = f"{_mode.capitalize()}MinMaxPlusSumConv3d{_params}"
+        globals()[_name] = _named(_name, _mode, params=_params, doc=f"{_mode} mode in three dimensions, {_params}",
+                                  base=TropicalConv3d)
+        __all__.append(_name)
+
+__all__ += ["TropicalDepthwiseConv2d", "TropicalConv1d", "TropicalConv3d"]

@@ -90,17 +90,18 @@ class TropicalConv2d(nn.Module):
     dtype: arithmetic type of the kernels ("f32" or "bf16"); parameters stay fp32."""
 
     PARAMS = ("0p", "1p", "2p", "shared", "opposite", "fixed")
+    ND = 2          # spatial dimensions
+    FN = None       # autograd Function of the layer (set below the class)
 
     def __init__(self, in_channels, out_channels, kernel_size, stride=1, padding=0, dilation=1,
                  bias=True, mode="compound", chan="default", params="2p", dtype="f32", fixed=(0.5, 0.5)):
         super().__init__()
-        two = lambda v: (v, v) if isinstance(v, int) else tuple(v)
+        two = lambda v: (v,) * self.ND if isinstance(v, int) else tuple(v)
         self.kernel_size, self.stride, self.padding, self.dilation = map(two, (kernel_size, stride, padding, dilation))
         self.in_channels, self.out_channels = in_channels, out_channels
         self.mode, self.chan, self.params, self.dtype = mode, chan, params, dtype
-        R, S = self.kernel_size
-        self.weight = nn.Parameter(torch.empty(out_channels, in_channels, R, S))
-        self.weight2 = nn.Parameter(torch.empty(out_channels, in_channels, R, S)) if mode == "parallel" else None
+        self.weight = nn.Parameter(torch.empty(out_channels, in_channels, *self.kernel_size))
+        self.weight2 = nn.Parameter(torch.empty(out_channels, in_channels, *self.kernel_size)) if mode == "parallel" else None
         two_branch = mode in ("compound", "parallel")
         if params not in self.PARAMS:
             raise ValueError(f"params must be one of {self.PARAMS}")
@@ -114,7 +115,7 @@ class TropicalConv2d(nn.Module):
         self.reset_parameters()
 
     def reset_parameters(self):
-        fan_in = self.in_channels * self.kernel_size[0] * self.kernel_size[1]
+        fan_in = self.in_channels * math.prod(self.kernel_size)
         bound = 1.0 / math.sqrt(fan_in)
         for w in (self.weight, self.weight2):
             if w is not None:
@@ -142,7 +143,10 @@ class TropicalConv2d(nn.Module):
             elif self.params == "fixed":
                 alpha, beta = self.alpha_fixed, self.beta_fixed
         geom = (self.mode, self.chan, self.dtype, self.stride, self.padding, self.dilation)
-        return TropicalConvFn.apply(x, self.weight, self.weight2, alpha, beta, self.bias, geom)
+        return self.FN.apply(x, self.weight, self.weight2, alpha, beta, self.bias, geom)
+
+
+TropicalConv2d.FN = TropicalConvFn
 
 
 class TropicalBasicBlock(nn.Module):
@@ -301,3 +305,48 @@ class TropicalConv1d(nn.Module):
 
     def forward(self, x):                      # x: [N, C, L]
         return self.conv(x.unsqueeze(2)).squeeze(2)
+
+
+class TropicalConv3dFn(torch.autograd.Function):
+    """y = tconv3d_forward(...); backward = tconv3d_backward with the stored winners."""
+
+    @staticmethod
+    def forward(ctx, x, w, w2, alpha, beta, bias, geom):
+        from . import tconv3d
+        mode, chan, dtype, stride, pad, dil = geom
+        dt = tconv.TORCH_DTYPE[dtype]
+        N, C, D, H, W = x.shape
+        K, _, T, R, S = w.shape
+        d = dict(N=N, C=C, D=D, H=H, W=W, K=K, T=T, R=R, S=S, stride=tuple(stride), pad=tuple(pad),
+                 dil=tuple(dil), mode=mode, chan=chan, dtype=dtype)
+        cast = lambda t, ty: t.detach().to(ty).contiguous() if t is not None else None
+        xc, wc, w2c = cast(x, dt), cast(w, dt), cast(w2, dt)
+        al, be, bi = cast(alpha, torch.float32), cast(beta, torch.float32), cast(bias, torch.float32)
+        need_grad = any(t is not None and t.requires_grad for t in (x, w, w2, alpha, beta, bias))
+        y, winners = tconv3d.forward(d, xc, wc, w2c, al, be, bi, want_winners=need_grad)
+        ctx.d, ctx.in_dtype = d, x.dtype
+        ctx.save_for_backward(xc, wc, w2c, al, be, winners)
+        ctx.has = (w2 is not None, alpha is not None, beta is not None, bias is not None)
+        return y.to(x.dtype) if x.dtype != dt else y
+
+    @staticmethod
+    def backward(ctx, gy):
+        from . import tconv3d
+        xc, wc, w2c, al, be, winners = ctx.saved_tensors
+        d = ctx.d
+        g = gy.detach().to(tconv.TORCH_DTYPE[d["dtype"]]).contiguous()
+        grads = tconv3d.backward(d, xc, wc, g, w2c, al, be, winners, need_grad_x=ctx.needs_input_grad[0])
+        has_w2, has_a, has_b, has_bias = ctx.has
+        gx = grads["grad_x"].to(ctx.in_dtype) if "grad_x" in grads else None
+        return (gx, grads["grad_w"], grads.get("grad_w2") if has_w2 else None,
+                grads.get("grad_alpha") if has_a else None, grads.get("grad_beta") if has_b else None,
+                grads["grad_bias"] if has_bias else None, None)
+
+
+class TropicalConv3d(TropicalConv2d):
+    """Three-dimensional tropical convolution (Section 3.2 and the Conv3d forms of Sections 3.4 / 3.5)
+    with ``nn.Conv3d``'s constructor arguments; input [N, C, D, H, W]; mode / chan / params / dtype
+    as in TropicalConv2d.  Windows of up to 256 taps (the paper's 3-D LeNet uses 5 x 5 x 5)."""
+
+    ND = 3
+    FN = TropicalConv3dFn

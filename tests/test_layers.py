@@ -185,3 +185,60 @@ def test_conv1d_with_a_long_window_against_the_oracle(mode, chan):
     assert close(x.grad.unsqueeze(2), *gref["grad_x"]) and close(m.conv.weight.grad, *gref["grad_w"])
     if two:
         assert close(m.conv.alpha.grad, *gref["grad_alpha"]) and close(m.conv.beta.grad, *gref["grad_beta"])
+
+
+def test_conv3d_names_and_lenet3d_parameter_counts():
+    """3d:[5/6,2] -> pool -> 3d:[5/16] -> pool (Table 1, configuration 3d): the tropical layers of
+    the compound 2p variant hold the weights plus one (alpha, beta) pair per channel pair."""
+    c1 = layers.CompoundMinMaxPlusSumConv3d2p(1, 6, 5, stride=2)
+    c2 = layers.ParallelMinMaxPlusSumConv3d1p(6, 16, 5)
+    count = lambda m: sum(p.numel() for p in m.parameters())
+    assert count(c1) == 6 * 125 + 2 * 6 + 6
+    assert count(c2) == 2 * 16 * 6 * 125 + 16 * 6 + 16
+    assert (layers.MinPlusMaxConv3d(2, 3, 3).mode, layers.MinPlusMaxConv3d(2, 3, 3).chan) == ("min_plus", "max")
+    assert layers.MaxPlusSumConv3d(2, 3, (1, 2, 3)).weight.shape == (3, 2, 1, 2, 3)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("mode,params", [("compound", "2p"), ("compound", "1p"), ("parallel", "2p"), ("min_plus", "0p")])
+def test_conv3d_layer_against_the_oracle(mode, params):
+    from oracle import tconv3d_oracle as ora3
+    from paper_2504_06881_b200.nn import TropicalConv3d
+    N, C, K = 2, 3, 4
+    d = inputs.layer3d(N, C, 9, 8, 10, K, T=3, R=3, S=3, stride=(2, 1, 1), pad=1, mode=mode)
+    t = inputs.draw3d(d, 2400, ab=("uniform", -1.0, 1.0))
+    m = TropicalConv3d(C, K, 3, stride=(2, 1, 1), padding=1, mode=mode, params=params).cuda()
+    two, par = mode in ("compound", "parallel"), mode == "parallel"
+    with torch.no_grad():
+        m.weight.copy_(torch.from_numpy(t["w"]))
+        m.bias.copy_(torch.from_numpy(t["bias"]))
+        if par:
+            m.weight2.copy_(torch.from_numpy(t["w2"]))
+        if two:
+            m.alpha.copy_(torch.from_numpy(t["alpha"]))
+            if params == "2p":
+                m.beta.copy_(torch.from_numpy(t["beta"]))
+    beta = t["beta"] if params == "2p" else (1.0 - t["alpha"]).astype(np.float32)
+    kw = dict(w2=t["w2"] if par else None, alpha=t["alpha"] if two else None, beta=beta if two else None)
+    ref = ora3.forward(d, t["x"], t["w"], bias=t["bias"], **kw)
+    x = torch.from_numpy(t["x"]).cuda().requires_grad_(True)
+    y = m(x)
+    assert np.array_equal(y.detach().cpu().numpy().view(np.uint32), ref["y"].view(np.uint32))
+    y.backward(torch.from_numpy(t["g"]).cuda())
+    gref = ora3.backward(d, t["x"], t["w"], t["g"], **kw)
+
+    def close(got, want, scale):
+        return (np.abs(got.detach().cpu().numpy().astype(np.float64) - want) <= 1e-5 * scale + 1e-30).all()
+
+    assert close(x.grad, *gref["grad_x"]) and close(m.weight.grad, *gref["grad_w"])
+    assert close(m.bias.grad, *gref["grad_bias"])
+    if par:
+        assert close(m.weight2.grad, *gref["grad_w2"])
+    if two and params == "2p":
+        assert close(m.alpha.grad, *gref["grad_alpha"]) and close(m.beta.grad, *gref["grad_beta"])
+    if two and params == "1p":       # beta = 1 - alpha: the chain rule gives grad_alpha - grad_beta
+        want = gref["grad_alpha"][0] - gref["grad_beta"][0]
+        assert close(m.alpha.grad, want, gref["grad_alpha"][1] + gref["grad_beta"][1])
+    # a first layer: the input needs no gradient and none is computed
+    y2 = m(torch.from_numpy(t["x"]).cuda())
+    y2.sum().backward()
