@@ -565,6 +565,62 @@ def run_dw(args):
     print(json.dumps(out))
 
 
+def run_conv3d(args):
+    """The two tropical layers of the paper's 3-D LeNet (Table 1, configuration 3d: [5/6, 2] then
+    [5/16] on the pooled volume) at both input sizes of the appendix (28^3 with batch 32, 64^3 with
+    batch 2), mode --only (default compound), fp32 or bf16: forward, forward with winners and the
+    full backward per layer, in ms and Ttap/s.  The layers are a few tens of Mtap: the times are
+    close to launch latency, so no roofline fraction is claimed for them."""
+    import torch
+    from paper_2504_06881_b200 import inputs, tconv, tconv3d
+    torch.cuda.set_device(0)
+    mode = args.only or "compound"
+    dt = tconv.TORCH_DTYPE[args.dtype]
+    two, par = mode in ("compound", "parallel"), mode == "parallel"
+    layers = [("28^3 L1", inputs.layer3d(32, 1, 28, 28, 28, 6, T=5, R=5, S=5, stride=2, mode=mode, dtype=args.dtype)),
+              ("28^3 L2", inputs.layer3d(32, 6, 6, 6, 6, 16, T=5, R=5, S=5, mode=mode, dtype=args.dtype)),
+              ("64^3 L1", inputs.layer3d(2, 1, 64, 64, 64, 6, T=5, R=5, S=5, stride=2, mode=mode, dtype=args.dtype)),
+              ("64^3 L2", inputs.layer3d(2, 6, 15, 15, 15, 16, T=5, R=5, S=5, mode=mode, dtype=args.dtype))]
+    out = {"workload": f"3-D LeNet tropical layers, {mode} {args.dtype}", "layers": {}}
+    l0 = tconv3d.tconv3d_launch_count()
+    for name, d in layers:
+        t = inputs.draw3d(d, 1070)
+        dev = lambda a, ty=None: torch.from_numpy(a).cuda().to(ty) if ty else torch.from_numpy(a).cuda()
+        x, w, w2, g = (dev(t[k], dt) for k in ("x", "w", "w2", "g"))
+        al, be, bias = dev(t["alpha"]), dev(t["beta"]), dev(t["bias"])
+        y = torch.empty(t["g"].shape, device="cuda", dtype=dt)
+        win = tconv3d.winner_buffer(d, "cuda")
+        ws = torch.empty(tconv3d.tconv3d_workspace_bytes(d, True), dtype=torch.uint8, device="cuda")
+        gx, gw, gw2 = torch.empty_like(x), torch.empty_like(w, dtype=torch.float32), torch.empty_like(w, dtype=torch.float32)
+        ga, gb, gbi = torch.empty_like(al), torch.empty_like(be), torch.empty_like(bias)
+        fa = (d, x, w, w2 if par else None, al if two else None, be if two else None, bias, y)
+        calls = {"fwd": lambda: tconv3d.tconv3d_forward(*fa, None),
+                 "fwd_winners": lambda: tconv3d.tconv3d_forward(*fa, win),
+                 "bwd": lambda: tconv3d.tconv3d_backward(d, x, w, w2 if par else None, al if two else None,
+                                                         be if two else None, g, win, gx if d["C"] > 1 else None,
+                                                         gw, gw2 if par else None, ga if two else None,
+                                                         gb if two else None, gbi, ws)}
+        od = tconv3d.tconv3d_output_shape(d)
+        taps = d["N"] * d["K"] * od[0] * od[1] * od[2] * d["C"] * 125
+        row = {"Mtap": taps / 1e6}
+        for what, fn in calls.items():
+            assert fn() == 0
+            for _ in range(max(args.warmup, 3)):
+                fn()
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(max(args.steps, 5)):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            row[what + "_ms"] = float(np.median(ts))
+        row["fwd_Ttap_s"] = taps / row["fwd_ms"] / 1e9
+        out["layers"][name] = row
+    out["gpu_launches"] = tconv3d.tconv3d_launch_count() - l0
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -576,14 +632,16 @@ def main():
     ap.add_argument("--what", default="fwd", choices=["fwd", "fwd_winners", "bwd"])
     ap.add_argument("--images", type=int, default=128)
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5", "dw"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5", "dw", "conv3d"],
                     help="cfg5: report the hybrid ResNet-18 training step instead (use --only compound|parallel); "
-                         "dw: a depthwise (groups = C) layer against the HBM roofline")
+                         "dw: a depthwise (groups = C) layer against the HBM roofline; conv3d: the 3-D LeNet layers")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "cfg5":
         run_cfg5(args)
+    elif args.workload == "conv3d":
+        run_conv3d(args)
     elif args.workload == "dw":
         run_dw(args)
     elif args.only:
