@@ -42,3 +42,27 @@ def test_random_descriptors(seed):
             dd = inputs.layer(N, C, H, W, C, R, S, stride=st, pad=pad, dil=dl, mode=mode, dtype=dtype)
             tdw.check(dd, int(rs.randint(1 << 30)), ties=bool(rs.randint(2)))
         done += 1
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_three_dimensional_descriptors(seed):
+    import test_gpu_3d as t3
+    rs = np.random.RandomState(seed)
+    done = 0
+    while done < 40:
+        mode, chan = ALL[rs.randint(len(ALL))]
+        dtype = ["f32", "bf16"][rs.randint(2)]
+        T, R, S = (int(rs.randint(1, 6)) for _ in range(3))
+        stride = tuple(int(v) for v in rs.randint(1, 4, 3))
+        dil = tuple(int(v) for v in rs.randint(1, 3, 3))
+        pad = tuple(int(v) for v in rs.randint(0, 3, 3))
+        N, C, K = int(rs.randint(1, 5)), int(rs.randint(1, 20)), int(rs.randint(1, 20))
+        D, H, W = (int(rs.randint(1, 20)) for _ in range(3))
+        d = inputs.layer3d(N, C, D, H, W, K, T=T, R=R, S=S, stride=stride, pad=pad, dil=dil, mode=mode,
+                           chan=chan, dtype=dtype)
+        od = inputs.output_dhw(d)
+        if min(od) <= 0 or N * K * C * T * R * S * od[0] * od[1] * od[2] > 3e7:
+            continue
+        dist = None if rs.rand() < 0.6 else dict(x=("ints", -2, 2), w=("ints", -2, 2))
+        t3.check(d, int(rs.randint(1 << 30)), dists=dist)
+        done += 1
