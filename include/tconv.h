@@ -94,8 +94,11 @@ int tconv_output_shape(const tconv_desc_t *desc, int32_t *OH, int32_t *OW);
  * invalid.  Layout:
  *   Max / Min channel combine: int32 [N][K][OH][OW], value c*R*S + r*S + s;
  *   Sum channel combine (incl. compound, parallel): one code per
- *     (n, k, c, oh, ow), laid out [N][K][C][OH][OW]; uint8 with the argmin tap
- *     r*S+s in the low nibble and the argmax tap in the high nibble when
+ *     (n, k, c, oh, ow), laid out [N][K][C][OH][OWP] with the row pitch
+ *     OWP = OW rounded up to a multiple of 4 (the codes of a row's columns
+ *     OW..OWP-1 are padding: tconv_forward fills them with valid taps and
+ *     tconv_backward relies on that); uint8 with the argmin
+ *     tap r*S+s in the low nibble and the argmax tap in the high nibble when
  *     R*S <= 16, else uint16 with the argmin tap in the low byte and the argmax
  *     tap in the high byte (R*S <= 256).  A single-branch Sum layer fills only
  *     its own half; the other half is 0.

@@ -95,6 +95,7 @@ int make_geo(const tconv_desc_t* d, Geo* g) {
     g->OH = out_extent(d->H, d->pad_h, d->dil_h, d->R, d->stride_h);
     g->OW = out_extent(d->W, d->pad_w, d->dil_w, d->S, d->stride_w);
     g->RS = d->R * d->S;
+    g->OWP = (g->OW + 3) & ~3;
     g->mode = d->mode;
     g->chan = chan;
     g->wide = g->RS > 16;
@@ -108,9 +109,8 @@ int make_geo(const tconv_desc_t* d, Geo* g) {
 }
 
 size_t winner_bytes(const Geo& g) {
-    const size_t outs = (size_t)g.N * g.K * g.OH * g.OW;
-    if (g.chan != CH_SUM) return outs * sizeof(int32_t);
-    return outs * g.C * (g.wide ? 2 : 1);
+    if (g.chan != CH_SUM) return (size_t)g.N * g.K * g.OH * g.OW * sizeof(int32_t);
+    return (size_t)g.N * g.K * g.C * g.OH * g.OWP * (g.wide ? 2 : 1);
 }
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -151,6 +151,31 @@ int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const 
     g_launches += 1;
     return check_launch();
 }
+
+// grad_bias: partial sums over chunks of images at the front of the workspace, then their sum.
+template <typename T>
+void bias_gradient(const Geo& g, const void* gy, float* gbias, void* ws, size_t ws_bytes, bool tiled,
+                   cudaStream_t st) {
+    int chunks = g.N < 16 ? g.N : 16;
+    if (tiled && ws && ws_bytes >= (size_t)chunks * g.K * sizeof(float)) {
+        const int npc = (g.N + chunks - 1) / chunks;
+        chunks = (g.N + npc - 1) / npc;
+        bwd_bias_partial_kernel<T><<<dim3((unsigned)g.K, (unsigned)chunks), 256, 0, st>>>(
+            g, (const T*)gy, (float*)ws, npc);
+        bwd_reduce_partials_kernel<<<(unsigned)((g.K + 255) / 256), 256, 0, st>>>((const float*)ws, gbias,
+                                                                               (size_t)g.K, chunks);
+        g_launches += 2;
+    } else {
+        bwd_bias_kernel<T><<<(unsigned)g.K, 256, 0, st>>>(g, (const T*)gy, gbias);
+        g_launches += 1;
+    }
+}
+
+template <typename T>
+int backward_sum_t(const Geo& g0, const void* x, const void* w, const void* w2, const float* alpha,
+                   const float* beta, const void* gy0, const void* winners, void* gx, float* gw,
+                   float* gw2, float* galpha, float* gbeta, float* gbias, void* ws, size_t ws_bytes,
+                   cudaStream_t st);
 
 template <typename T>
 int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const float* alpha,
@@ -234,39 +259,74 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
             g_launches += 1;
         }
     } else {
+        return backward_sum_t<T>(g, x, w, w2, alpha, beta, gy, winners, gx, gw, gw2, galpha, gbeta, gbias, ws,
+                                 ws_bytes, st);
+    }
+    snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", name);
+    if (gbias && !bias_done) bias_gradient<T>(g, gy, gbias, ws, ws_bytes, tiled, st);
+    return check_launch();
+}
+
+// Backward of the Sum channel combine (layers (i), (ii), compound, parallel): per-channel winner codes.
+template <typename T>
+int backward_sum_t(const Geo& g0, const void* x, const void* w, const void* w2, const float* alpha,
+                   const float* beta, const void* gy0, const void* winners, void* gx, float* gw,
+                   float* gw2, float* galpha, float* gbeta, float* gbias, void* ws, size_t ws_bytes,
+                   cudaStream_t st) {
+    const bool twob = two_branch(g0.mode);
+    const bool tiled = !force_generic();
+    const char* name = "bwd_generic";
+    // output widths that are not a multiple of 4: the code-driven kernels see a layer of width OWP
+    // and a zero-padded copy of grad_y (last block of the workspace)
+    Geo g = g0;
+    const void* gy = gy0;
+    const size_t bias_part = ((size_t)16 * g0.K * sizeof(float) + 255) / 256 * 256;
+    if (tiled && (g0.OW & 3) != 0 && ws) {
+        const Geo gq = widened_geo(g0);
+        const size_t off = bias_part + padded_x_bytes(gq, (int)sizeof(T));
+        const size_t need = padded_gy_bytes(g0, (int)sizeof(T));
+        if (ws_bytes >= off + need) {
+            T* gpad = (T*)((char*)ws + off);
+            const size_t total = (size_t)g0.N * g0.K * g0.OH * g0.OWP;
+            pad_grad_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g0, (const T*)gy0, gpad);
+            g_launches += 1;
+            g = gq;
+            gy = gpad;
+        }
+    }
+    const bool quads = tiled && (g.OW & 3) == 0;   // the code-driven kernels read whole, aligned quads
+    {
         const uint8_t* codes = (const uint8_t*)winners;
         const int br = twob ? 0 : (g.mode == TCONV_MIN_PLUS ? 1 : 2);
         CodeGxPlan pl;
         if (gx) {
-            if (tiled && plan_code_gx(g, &pl)) {
+            if (quads && plan_code_gx(g, &pl)) {
                 const dim3 grid(pl.grid);
-#define TCONV_GXM(BR, CBV, VECV, MULTI, NTH)                                                         \
+#define TCONV_GXM(BR, CBV, MULTI, NTH)                                                               \
     {                                                                                                \
-        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV, MULTI, NTH, false>;                         \
+        auto kern = bwd_code_gx_kernel<T, BR, CBV, MULTI, NTH, false>;                               \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<grid, pl.threads, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);   \
     }
-#define TCONV_GXW(BR, CBV, VECV)                                                                     \
+#define TCONV_GXW(BR, CBV)                                                                           \
     {                                                                                                \
-        auto kern = bwd_code_gx_kernel<T, BR, CBV, VECV, false, 256, true>;                          \
+        auto kern = bwd_code_gx_kernel<T, BR, CBV, false, 256, true>;                                \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<grid, pl.threads, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);   \
     }
-#define TCONV_GX(BR, CBV, VECV)                                                                      \
+#define TCONV_GX(BR, CBV)                                                                            \
     {                                                                                                \
-        if (g.wide) TCONV_GXW(BR, CBV, VECV)                                                         \
-        else if (pl.imgs > 1) TCONV_GXM(BR, CBV, VECV, true, 256)                                    \
-        else if (pl.threads > 256) TCONV_GXM(BR, CBV, VECV, false, 1024)                             \
-        else TCONV_GXM(BR, CBV, VECV, false, 256)                                                    \
+        if (g.wide) TCONV_GXW(BR, CBV)                                                               \
+        else if (pl.imgs > 1) TCONV_GXM(BR, CBV, true, 256)                                          \
+        else if (pl.threads > 256) TCONV_GXM(BR, CBV, false, 1024)                                   \
+        else TCONV_GXM(BR, CBV, false, 256)                                                          \
     }
 #define TCONV_GX2(BR)                                                                                \
     {                                                                                                \
-        if (pl.CB == 2) { if (vec) TCONV_GX(BR, 2, true) else TCONV_GX(BR, 2, false) }               \
-        else { if (vec) TCONV_GX(BR, 1, true) else TCONV_GX(BR, 1, false) }                           \
+        if (pl.CB == 2) TCONV_GX(BR, 2) else TCONV_GX(BR, 1)                                         \
     }
-                const bool vec = (g.OW & 3) == 0;
                 if (br == 0) TCONV_GX2(0) else if (br == 1) TCONV_GX2(1) else TCONV_GX2(2)
 #undef TCONV_GX2
 #undef TCONV_GX
@@ -274,19 +334,18 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
 #undef TCONV_GXW
                 name = "bwd_code";
             } else {
-                const size_t total = (size_t)g.N * g.C * g.H * g.W;
+                const size_t total = (size_t)g0.N * g0.C * g0.H * g0.W;
                 bwd_gx_generic_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
-                    g, alpha, beta, (const T*)gy, winners, (T*)gx);
+                    g0, alpha, beta, (const T*)gy0, winners, (T*)gx);
             }
             g_launches += 1;
         }
         if (gw || gw2 || galpha || gbeta) {
             CodeGwPlan gp;
             plan_code_gw(g, &gp);
-            if (tiled && gp.smem <= kBwdSmemLimit) {
+            if (quads && gp.smem <= kBwdSmemLimit) {
                 // zero-padded copy of x for the branch values of grad_alpha / grad_beta, placed after
                 // the grad_bias partials in the workspace
-                const size_t bias_part = ((size_t)16 * g.K * sizeof(float) + 255) / 256 * 256;
                 const size_t pad_bytes = padded_x_bytes(g, (int)sizeof(T));
                 if (br == 0 && (galpha || gbeta) && ws && ws_bytes >= bias_part + pad_bytes &&
                     (double)g.N * g.C * gp.HP * gp.WP < 2.0e9) {
@@ -297,30 +356,29 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                     gp.xs_elems = gp.HP * gp.WP;
                     gp.xpad = xpad;
                 }
-#define TCONV_GWK(BR, XSV, VECV, WARPV, GRID)                                                         \
+#define TCONV_GWK(BR, XSV, WARPV, GRID)                                                               \
     {                                                                                                \
-        auto kern = bwd_code_gw_kernel<T, BR, XSV, VECV, WARPV, false>;                              \
+        auto kern = bwd_code_gw_kernel<T, BR, XSV, WARPV, false>;                                    \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<(unsigned)(GRID), 256, gp.smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
                                                       (const T*)gy, codes, gw, gw2, galpha, gbeta, gp); \
     }
-#define TCONV_GWW(BR, XSV, VECV)                                                                     \
+#define TCONV_GWW(BR, XSV)                                                                           \
     {                                                                                                \
-        auto kern = bwd_code_gw_kernel<T, BR, XSV, VECV, false, true>;                               \
+        auto kern = bwd_code_gw_kernel<T, BR, XSV, false, true>;                                     \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<(unsigned)((size_t)g.K * g.C), 256, gp.smem, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, \
                                                       (const T*)gy, codes, gw, gw2, galpha, gbeta, gp); \
     }
-#define TCONV_GW(BR, XSV, VECV)                                                                      \
+#define TCONV_GW(BR, XSV)                                                                            \
     {                                                                                                \
-        if (g.wide) TCONV_GWW(BR, XSV, VECV)                                                         \
-        else if (gp.warp) TCONV_GWK(BR, XSV, VECV, true, ((size_t)g.K * g.C + 7) / 8)                \
-        else TCONV_GWK(BR, XSV, VECV, false, (size_t)g.K * g.C)                                      \
+        if (g.wide) TCONV_GWW(BR, XSV)                                                               \
+        else if (gp.warp) TCONV_GWK(BR, XSV, true, ((size_t)g.K * g.C + 7) / 8)                      \
+        else TCONV_GWK(BR, XSV, false, (size_t)g.K * g.C)                                            \
     }
-#define TCONV_GWV(BR, XSV) { if (vecw) TCONV_GW(BR, XSV, true) else TCONV_GW(BR, XSV, false) }
-                const bool vecw = (g.OW & 3) == 0;
+#define TCONV_GWV(BR, XSV) TCONV_GW(BR, XSV)
                 if (br == 0) { if (gp.xs_elems) TCONV_GWV(0, true) else TCONV_GWV(0, false) }
                 else if (br == 1) TCONV_GWV(1, false) else TCONV_GWV(2, false)
 #undef TCONV_GWV
@@ -331,34 +389,20 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                 name = "bwd_code";
             } else {
                 if (gw || gw2) {
-                    bwd_gw_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C * g.RS), 256, 0, st>>>(
-                        g, alpha, beta, (const T*)gy, winners, gw, gw2);
+                    bwd_gw_generic_kernel<T><<<(unsigned)((size_t)g0.K * g0.C * g0.RS), 256, 0, st>>>(
+                        g0, alpha, beta, (const T*)gy0, winners, gw, gw2);
                     g_launches += 1;
                 }
                 if (twob && (galpha || gbeta)) {
-                    bwd_gab_generic_kernel<T><<<(unsigned)((size_t)g.K * g.C), 256, 0, st>>>(
-                        g, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, winners, galpha, gbeta);
+                    bwd_gab_generic_kernel<T><<<(unsigned)((size_t)g0.K * g0.C), 256, 0, st>>>(
+                        g0, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy0, winners, galpha, gbeta);
                     g_launches += 1;
                 }
             }
         }
     }
-    if (gbias && !bias_done) {
-        int chunks = g.N < 16 ? g.N : 16;
-        if (tiled && ws && ws_bytes >= (size_t)chunks * g.K * sizeof(float)) {
-            const int npc = (g.N + chunks - 1) / chunks;
-            chunks = (g.N + npc - 1) / npc;
-            bwd_bias_partial_kernel<T><<<dim3((unsigned)g.K, (unsigned)chunks), 256, 0, st>>>(
-                g, (const T*)gy, (float*)ws, npc);
-            bwd_reduce_partials_kernel<<<(unsigned)((g.K + 255) / 256), 256, 0, st>>>((const float*)ws, gbias,
-                                                                                   (size_t)g.K, chunks);
-            g_launches += 2;
-        } else {
-            bwd_bias_kernel<T><<<(unsigned)g.K, 256, 0, st>>>(g, (const T*)gy, gbias);
-            g_launches += 1;
-        }
-    }
     snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", name);
+    if (gbias) bias_gradient<T>(g0, gy0, gbias, ws, ws_bytes, tiled, st);
     return check_launch();
 }
 

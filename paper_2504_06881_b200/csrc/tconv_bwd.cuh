@@ -255,60 +255,33 @@ struct CodeGxPlan {
     size_t smem;
 };
 
-// Loads 4 horizontally adjacent gradients (VEC: one aligned vector load).
-template <typename T, bool VEC>
-__device__ __forceinline__ void load_g4(const T* p, int ow0, int OW, float* gv) {
-    if constexpr (VEC) {
-        if constexpr (sizeof(T) == 4) {
-            const float4 v = __ldg(reinterpret_cast<const float4*>(p));
-            gv[0] = v.x; gv[1] = v.y; gv[2] = v.z; gv[3] = v.w;
-        } else {
-            const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
-            gv[0] = __uint_as_float(v.x << 16); gv[1] = __uint_as_float(v.x & 0xffff0000u);
-            gv[2] = __uint_as_float(v.y << 16); gv[3] = __uint_as_float(v.y & 0xffff0000u);
-        }
+// Loads 4 horizontally adjacent gradients (one aligned vector load: the output width these kernels
+// see is a multiple of 4).
+template <typename T>
+__device__ __forceinline__ void load_g4(const T* p, float* gv) {
+    if constexpr (sizeof(T) == 4) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(p));
+        gv[0] = v.x; gv[1] = v.y; gv[2] = v.z; gv[3] = v.w;
     } else {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) gv[j] = (ow0 + j < OW) ? to_f32(p[j]) : 0.0f;
-    }
-}
-// Loads the 4 winner codes of a quad as one word (VEC: one aligned 32-bit load).
-template <bool VEC>
-__device__ __forceinline__ unsigned load_c4(const uint8_t* p, int ow0, int OW) {
-    if constexpr (VEC) {
-        return __ldg(reinterpret_cast<const unsigned*>(p));
-    } else {
-        unsigned cw = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (ow0 + j < OW) cw |= (unsigned)p[j] << (8 * j);
-        return cw;
+        const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+        gv[0] = __uint_as_float(v.x << 16); gv[1] = __uint_as_float(v.x & 0xffff0000u);
+        gv[2] = __uint_as_float(v.y << 16); gv[3] = __uint_as_float(v.y & 0xffff0000u);
     }
 }
 
-// The 4 winner codes of a quad.  Narrow codes (R*S <= 16): one byte each, argmin tap in the low
-// nibble, argmax tap in the high nibble.  WIDE (R*S <= 256): 16 bits each, argmin tap in the low
-// byte, argmax tap in the high byte; `p` then points at the first of 4 adjacent 16-bit codes.
+// The 4 winner codes of a quad, one aligned load.  Narrow codes (R*S <= 16): one byte each, argmin
+// tap in the low nibble, argmax tap in the high nibble.  WIDE (R*S <= 256): 16 bits each, argmin tap
+// in the low byte, argmax tap in the high byte; `p` then points at the first of 4 adjacent codes.
 template <bool WIDE> struct Codes4 { unsigned lo, hi; };
 template <> struct Codes4<false> { unsigned lo; };
-template <bool WIDE, bool VEC>
-__device__ __forceinline__ Codes4<WIDE> load_codes4(const uint8_t* p, int ow0, int OW) {
+template <bool WIDE>
+__device__ __forceinline__ Codes4<WIDE> load_codes4(const uint8_t* p) {
     Codes4<WIDE> r;
-    if constexpr (WIDE) r.hi = 0u;
     if constexpr (!WIDE) {
-        r.lo = load_c4<VEC>(p, ow0, OW);
-    } else if constexpr (VEC) {
+        r.lo = __ldg(reinterpret_cast<const unsigned*>(p));
+    } else {
         const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
         r.lo = v.x; r.hi = v.y;
-    } else {
-        const uint16_t* q = reinterpret_cast<const uint16_t*>(p);
-        r.lo = 0u;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (ow0 + j < OW) {
-                const unsigned cde = q[j];
-                if (j < 2) r.lo |= cde << (16 * j); else r.hi |= cde << (16 * (j - 2));
-            }
     }
     return r;
 }
@@ -325,10 +298,10 @@ __device__ __forceinline__ void taps_of(const Codes4<WIDE>& c4, int j, unsigned&
 
 // BR: 0 = both branches (compound / parallel), 1 = min branch only, 2 = max branch only.
 // CB channels per CTA (the CTA's last channel block may hold fewer: those lanes idle).
-// VEC: OW is a multiple of 4 (aligned vector loads of grad_y and of the codes).
+// The output width is a multiple of 4 (the caller pads grad_y otherwise): aligned vector loads.
 // MULTI: the CTA owns pl.imgs whole images (small maps); else one band of rows of one image.
 // NTH: upper bound of the CTA size (256, or 1024 for tiles that leave room for one or two CTAs per SM).
-template <typename T, int BR, int CB, bool VEC, bool MULTI, int NTH, bool WIDE>
+template <typename T, int BR, int CB, bool MULTI, int NTH, bool WIDE>
 __global__ void __launch_bounds__(NTH)
 bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
@@ -367,7 +340,7 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     __syncthreads();
     const size_t plane = (size_t)g.OH * g.OW;
     constexpr int CW = WIDE ? 2 : 1;                     // bytes per code
-    const size_t cstep = (size_t)g.C * plane * CW;    // codes: one output channel k further (bytes)
+    const size_t cstep = (size_t)g.C * plane * CW;   // codes: one output channel k further (bytes)
     const unsigned tstride = 4u * NQp * sizeof(float); // bytes between the accumulators of two taps
     for (int q = threadIdx.x; q < NQ; q += blockDim.x) {
         const int il = MULTI ? q / NQ1 : 0;
@@ -393,9 +366,9 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
 #pragma unroll
         for (int u = 0; u < PF; ++u)
             if (u < g.K) {
-                load_g4<T, VEC>(gp + (size_t)u * plane, ow0, g.OW, gv[u]);
+                load_g4<T>(gp + (size_t)u * plane, gv[u]);
 #pragma unroll
-                for (int cb = 0; cb < CB; ++cb) cw[u][cb] = load_codes4<WIDE, VEC>(cp[cb] + (size_t)u * cstep, ow0, g.OW);
+                for (int cb = 0; cb < CB; ++cb) cw[u][cb] = load_codes4<WIDE>(cp[cb] + (size_t)u * cstep);
             }
         gp += (size_t)PF * plane;          // the next channel to request
 #pragma unroll
@@ -428,10 +401,10 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
                     }
                 }
                 if (k + PF < g.K) {
-                    load_g4<T, VEC>(gp, ow0, g.OW, gv[u]);
+                    load_g4<T>(gp, gv[u]);
 #pragma unroll
                     for (int cb = 0; cb < CB; ++cb) {
-                        cw[u][cb] = load_codes4<WIDE, VEC>(cp[cb], ow0, g.OW);
+                        cw[u][cb] = load_codes4<WIDE>(cp[cb]);
                         cp[cb] += cstep;
                     }
                     gp += plane;
@@ -505,7 +478,7 @@ __global__ void pad_input_kernel(Geo g, const T* __restrict__ x, T* __restrict__
 // WARP: one warp per (k, c) pair, eight pairs per CTA, the lanes walk the pair's (image, quad)
 // items and reduce with shuffles; for maps so small that a 256-thread CTA per pair would spend its
 // time zeroing, synchronising and reducing.  Else one CTA per pair.
-template <typename T, int BR, bool XS, bool VEC, bool WARP, bool WIDE>
+template <typename T, int BR, bool XS, bool WARP, bool WIDE>
 __global__ void __launch_bounds__(256)
 bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
                    const float* __restrict__ alpha, const float* __restrict__ beta,
@@ -552,7 +525,6 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
     auto accumulate = [&](int oh, int ow0, const float* gv, const Codes4<WIDE>& cw, const T* xp) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (!VEC && ow0 + j >= g.OW) continue;
             unsigned tmin, tmax;
             taps_of<WIDE>(cw, j, tmin, tmax);
             const float gvj = gv[j];
@@ -605,14 +577,14 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
             Codes4<WIDE> cw_cur, cw_nxt;
             cw_nxt.lo = 0u;
             if constexpr (WIDE) cw_nxt.hi = 0u;
-            load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
-            cw_cur = load_codes4<WIDE, VEC>(cp, ow0, g.OW);
+            load_g4<T>(gp, gv_cur);
+            cw_cur = load_codes4<WIDE>(cp);
             for (int n = 0; n < g.N; ++n) {
                 if (n + 1 < g.N) {
                     gp += gstep;
                     cp += cstep;
-                    load_g4<T, VEC>(gp, ow0, g.OW, gv_nxt);
-                    cw_nxt = load_codes4<WIDE, VEC>(cp, ow0, g.OW);
+                    load_g4<T>(gp, gv_nxt);
+                    cw_nxt = load_codes4<WIDE>(cp);
                 }
                 accumulate(oh, ow0, gv_cur, cw_cur, xp);
                 xp += XS ? xstep : (size_t)g.C * g.H * g.W;
@@ -644,8 +616,8 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
         bool have = n < g.N;
         if (have) {
             item_ptrs(n, q, oh, ow0, gp, cp, xp);
-            load_g4<T, VEC>(gp, ow0, g.OW, gv_cur);
-            cw_cur = load_codes4<WIDE, VEC>(cp, ow0, g.OW);
+            load_g4<T>(gp, gv_cur);
+            cw_cur = load_codes4<WIDE>(cp);
         }
         while (have) {
             int n2 = n + dn, q2 = q + dq;
@@ -655,8 +627,8 @@ bwd_code_gw_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, cons
             const T* gp2 = nullptr; const uint8_t* cp2 = nullptr; const T* xp2 = nullptr;
             if (more) {
                 item_ptrs(n2, q2, oh2, ow2, gp2, cp2, xp2);
-                load_g4<T, VEC>(gp2, ow2, g.OW, gv_nxt);
-                cw_nxt = load_codes4<WIDE, VEC>(cp2, ow2, g.OW);
+                load_g4<T>(gp2, gv_nxt);
+                cw_nxt = load_codes4<WIDE>(cp2);
             }
             accumulate(oh, ow0, gv_cur, cw_cur, xp);
             n = n2; q = q2; oh = oh2; ow0 = ow2; xp = xp2;
@@ -751,11 +723,37 @@ inline size_t padded_x_bytes(const Geo& g, int esize) {
     return ((size_t)g.N * g.C * pl.HP * pl.WP * esize + 255) / 256 * 256;
 }
 
+// Sum forms whose output width is not a multiple of 4 run their code-driven kernels as a layer of
+// output width OWP on a copy of grad_y with zero-padded rows (every quad whole, every load an
+// aligned vector): the geometry those kernels see, and the bytes of the copy.
+inline Geo widened_geo(const Geo& g) {
+    Geo q = g;
+    q.OW = g.OWP;
+    return q;
+}
+inline size_t padded_gy_bytes(const Geo& g, int esize) {
+    if ((g.OW & 3) == 0) return 0;
+    return ((size_t)g.N * g.K * g.OH * g.OWP * esize + 255) / 256 * 256;
+}
+
 inline size_t bwd_ws_bytes(const Geo& g) {
     // partial histograms of the Max / Min combine: at most 16 chunks of [K][C*RS + 1] floats;
-    // Sum forms: 16 chunks of grad_bias partials
-    if (g.chan == CH_SUM) return (size_t)16 * g.K * sizeof(float) + 256 + padded_x_bytes(g, 4);
+    // Sum forms: 16 chunks of grad_bias partials, the padded copy of x, the padded copy of grad_y
+    if (g.chan == CH_SUM)
+        return (size_t)16 * g.K * sizeof(float) + 256 + padded_x_bytes(widened_geo(g), 4) + padded_gy_bytes(g, 4);
     return (size_t)16 * g.K * ((size_t)g.C * g.RS + 1) * sizeof(float) + 256;
+}
+
+// grad_y with rows padded by zeros to OWP elements: one thread per padded element.
+template <typename T>
+__global__ void __launch_bounds__(256)
+pad_grad_kernel(Geo g, const T* __restrict__ gy, T* __restrict__ out) {
+    const size_t total = (size_t)g.N * g.K * g.OH * g.OWP;
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int ow = (int)(i % g.OWP);
+    const size_t row = i / g.OWP;
+    out[i] = ow < g.OW ? gy[row * g.OW + ow] : zero_of<T>();
 }
 
 constexpr size_t kBwdSmemLimit = 160 * 1024;   // planning budget per CTA

@@ -16,6 +16,7 @@ struct Geo {
     int N, C, H, W, K, R, S;
     int sh, sw, ph, pw, dh, dw;
     int OH, OW, RS;
+    int OWP;         // OW rounded up to a multiple of 4: row pitch of the Sum-form winner codes
     int mode, chan;  // tconv_mode_t, resolved channel combine
     int wide;        // Sum-form winner codes are uint16 (R*S > 16) instead of uint8
 };

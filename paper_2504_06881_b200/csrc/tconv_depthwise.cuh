@@ -178,7 +178,6 @@ dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T*
 #endif
     constexpr int RT = TCONV_DW_RT;             // output rows per strip
     constexpr int L = 3 * SW + 3;               // input columns 4 outputs touch
-    constexpr int NROWS = (RT - 1) * SW + 3;    // input rows a strip touches
     constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
     constexpr bool PAR = (MODE == TCONV_PARALLEL);
     constexpr bool DO_MIN = TWO || MODE == TCONV_MIN_PLUS, DO_MAX = TWO || MODE == TCONV_MAX_PLUS;

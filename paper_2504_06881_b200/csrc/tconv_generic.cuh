@@ -54,7 +54,6 @@ fwd_generic_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w,
     float best = (g.chan == CH_MAX) ? -INFINITY : INFINITY;
     float acc = 0.0f;
     int win = -1;
-    const size_t plane = (size_t)g.OH * g.OW;
     for (int c = 0; c < g.C; ++c) {
         float mn, mx;
         int amn, amx;
@@ -78,9 +77,15 @@ fwd_generic_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w,
             if (g.mode == TCONV_MIN_PLUS) amx = 0; else amn = 0;
         }
         if (winners && g.chan == CH_SUM) {
-            const size_t ci = (((size_t)n * g.K + k) * g.C + c) * plane + (size_t)oh * g.OW + ow;
+            const size_t ci = (((size_t)n * g.K + k) * g.C + c) * ((size_t)g.OH * g.OWP) + (size_t)oh * g.OWP + ow;
             if (g.wide) ((uint16_t*)winners)[ci] = (uint16_t)(amn | (amx << 8));
             else ((uint8_t*)winners)[ci] = (uint8_t)(amn | (amx << 4));
+            // the row's padding codes (columns OW .. OWP-1) hold tap 0: the backward kernels read whole quads
+            if (ow == g.OW - 1)
+                for (int pcol = g.OW; pcol < g.OWP; ++pcol) {
+                    if (g.wide) ((uint16_t*)winners)[ci + (pcol - ow)] = 0;
+                    else ((uint8_t*)winners)[ci + (pcol - ow)] = 0;
+                }
         }
     }
     float out = (g.chan == CH_SUM) ? acc : best;
@@ -139,9 +144,9 @@ bwd_gx_generic_kernel(Geo g, const float* __restrict__ alpha, const float* __res
                     if (((const int32_t*)winners)[obase + op] == c * g.RS + tap)
                         acc += to_f32(gy[obase + op]);
                 } else {
-                    const size_t cbase = (((size_t)n * g.K + k) * g.C + c) * plane;
+                    const size_t cbase = (((size_t)n * g.K + k) * g.C + c) * ((size_t)g.OH * g.OWP);
                     int amn, amx;
-                    read_code(g, winners, cbase + op, amn, amx);
+                    read_code(g, winners, cbase + (size_t)oh * g.OWP + ow, amn, amx);
                     const float gv = to_f32(gy[obase + op]);
                     if (twob) {
                         const float a = alpha ? alpha[(size_t)k * g.C + c] : 1.0f;
@@ -181,7 +186,8 @@ bwd_gw_generic_kernel(Geo g, const float* __restrict__ alpha, const float* __res
             if (((const int32_t*)winners)[oi] == c * g.RS + tap) smax += to_f32(gy[oi]);
         } else {
             int amn, amx;
-            read_code(g, winners, (((size_t)n * g.K + k) * g.C + c) * plane + op, amn, amx);
+            read_code(g, winners, (((size_t)n * g.K + k) * g.C + c) * ((size_t)g.OH * g.OWP) +
+                                      (op / g.OW) * g.OWP + op % g.OW, amn, amx);
             const float gv = to_f32(gy[oi]);
             if (twob) {
                 if (amn == tap) smin += gv;
@@ -231,7 +237,8 @@ bwd_gab_generic_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w,
         const size_t op = j % plane;
         const int oh = (int)(op / g.OW), ow = (int)(op % g.OW);
         int amn, amx;
-        read_code(g, winners, (((size_t)n * g.K + k) * g.C + c) * plane + op, amn, amx);
+        read_code(g, winners, (((size_t)n * g.K + k) * g.C + c) * ((size_t)g.OH * g.OWP) + (size_t)oh * g.OWP + ow,
+                  amn, amx);
         const float gv = to_f32(gy[((size_t)n * g.K + k) * plane + op]);
         const T* xc = x + ((size_t)n * g.C + c) * g.H * g.W;
         {

@@ -412,6 +412,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
             }
 
     const size_t plane = (size_t)g.OH * g.OW;
+    const size_t cplane = (size_t)g.OH * g.OWP;   // winner codes: rows padded to whole quads
     // Sum forms with winners: where this thread's codes of (its first output channel, input channel 0) go
     uint8_t* code_base[Q];
 #pragma unroll
@@ -420,7 +421,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
         if (WIN && CHAN == CH_SUM && out_row[q] >= 0) {
             const int n = out_row[q] / g.OH, oh = out_row[q] - n * g.OH;
             code_base[q] = reinterpret_cast<uint8_t*>(p.winners) +
-                           (((size_t)n * g.K + (size_t)kt * TILE_K) * g.C * plane + (size_t)oh * g.OW + qcol[q]) *
+                           (((size_t)n * g.K + (size_t)kt * TILE_K) * g.C * cplane + (size_t)oh * g.OWP + qcol[q]) *
                                (RS > 16 ? 2 : 1);
         }
     }
@@ -571,20 +572,10 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                             for (int h = 0; h < 2; ++h) {
                                 const int kl = kg * TK + 2 * kp + h;
                                 if (kt * TILE_K + kl >= g.K) continue;
-                                uint8_t* dst = code_base[q] + ((size_t)kl * g.C + c) * plane * CW;
-                                if (qcol[q] + 3 < g.OW && ((g.OW & 3) == 0)) {
+                                uint8_t* dst = code_base[q] + ((size_t)kl * g.C + c) * cplane * CW;
+                                if (qcol[q] < g.OW) {   // the quad's 4 codes in one store (rows are padded)
                                     if constexpr (WIDE) *reinterpret_cast<uint2*>(dst) = make_uint2(packed[h], packed_hi[h]);
                                     else *reinterpret_cast<unsigned*>(dst) = packed[h];
-                                } else {
-#pragma unroll
-                                    for (int j = 0; j < 4; ++j)
-                                        if (qcol[q] + j < g.OW) {
-                                            if constexpr (WIDE)
-                                                reinterpret_cast<uint16_t*>(dst)[j] =
-                                                    (uint16_t)((j < 2 ? packed[h] : packed_hi[h]) >> (16 * (j & 1)));
-                                            else
-                                                dst[j] = (uint8_t)(packed[h] >> (8 * j));
-                                        }
                                 }
                             }
                         }

@@ -498,8 +498,8 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                         for (int k = 0; k < 8; ++k) {
                             const int kk = kt * TILE_K + kg * 8 + k;
                             if (kk >= g.K) continue;
-                            uint8_t* dst = codes + (((size_t)n * g.K + kk) * g.C + c) * plane +
-                                           (size_t)oh * g.OW + qcol[q];
+                            uint8_t* dst = codes + (((size_t)n * g.K + kk) * g.C + c) * ((size_t)g.OH * g.OWP) +
+                                           (size_t)oh * g.OWP + qcol[q];
                             unsigned c01, c23;
                             if constexpr (TWO) {
                                 c01 = amn[k][q][0] | (amx[k][q][0] << 4);
@@ -509,13 +509,8 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                                 c23 = TAP_MIN ? amx[k][q][1] : (amx[k][q][1] << 4);
                             }
                             const unsigned packed = __byte_perm(c01, c23, 0x6420);
-                            if (qcol[q] + 3 < g.OW && ((g.OW & 3) == 0)) {
-                                *reinterpret_cast<unsigned*>(dst) = packed;
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 4; ++j)
-                                    if (qcol[q] + j < g.OW) dst[j] = (uint8_t)(packed >> (8 * j));
-                            }
+                            // the quad's 4 codes in one store (code rows are padded to whole quads)
+                            if (qcol[q] < g.OW) *reinterpret_cast<unsigned*>(dst) = packed;
                         }
                     }
                 }

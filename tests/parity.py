@@ -39,9 +39,11 @@ def winners_as_numpy(d, winners):
     raw = winners.cpu().numpy()
     if chan != "sum":
         return raw.view(np.int32).reshape(N, K, OH, OW)
+    # Sum-form codes: rows padded to a multiple of 4 codes; the padding is not part of the result
+    OWP = (OW + 3) // 4 * 4
     if d["R"] * d["S"] <= 16:
-        return raw.reshape(N, K, C, OH, OW)
-    return raw.view(np.uint16).reshape(N, K, C, OH, OW)
+        return raw.reshape(N, K, C, OH, OWP)[..., :OW]
+    return raw.view(np.uint16).reshape(N, K, C, OH, OWP)[..., :OW]
 
 
 def oracle_wide_codes(d, t, la):

@@ -29,7 +29,9 @@ def test_output_shape_and_sizes():
     assert tconv.tconv_output_shape(d) == (32, 32)
     assert tconv.tconv_winner_bytes(d) == 2 * 16 * 3 * 32 * 32
     assert tconv.tconv_winner_bytes(dict(d, mode="max_plus")) == 4 * 2 * 16 * 32 * 32
-    assert tconv.tconv_winner_bytes(dict(d, R=5, S=5)) == 2 * 2 * 16 * 3 * 30 * 30
+    assert tconv.tconv_winner_bytes(dict(d, R=5, S=5)) == 2 * 2 * 16 * 3 * 30 * 32      # code rows padded to 4
+    assert tconv.tconv_winner_bytes(dict(d, W=9)) == 2 * 16 * 3 * 32 * 12
+    assert tconv.tconv_winner_bytes(dict(d, W=9, mode="max_plus")) == 4 * 2 * 16 * 32 * 9
     assert tconv.tconv_workspace_bytes(d, True) >= tconv.tconv_winner_bytes(d)
     d2 = inputs.layer(1, 1, 56, 56, 1, 3, 3, stride=2, pad=1, dil=1)
     assert tconv.tconv_output_shape(d2) == (28, 28)
