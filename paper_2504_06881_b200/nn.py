@@ -290,23 +290,6 @@ class TropicalDepthwiseConv2d(nn.Module):
         return TropicalDepthwiseFn.apply(x, self.weight, self.weight2, alpha, beta, self.bias, geom)
 
 
-class TropicalConv1d(nn.Module):
-    """1-D tropical convolution (Section 3.2): the 2-D operator on a signal of unit height, with a
-    1 x kernel_size window.  Same arguments as ``nn.Conv1d``; mode / chan / params / dtype as in
-    TropicalConv2d.  Windows of up to 256 taps (the paper's audio networks use 80) run through the
-    any-shape kernels of the library."""
-
-    def __init__(self, in_channels, out_channels, kernel_size, stride=1, padding=0, dilation=1,
-                 bias=True, mode="compound", chan="default", params="2p", dtype="f32", fixed=(0.5, 0.5)):
-        super().__init__()
-        self.conv = TropicalConv2d(in_channels, out_channels, (1, kernel_size), stride=(1, stride),
-                                   padding=(0, padding), dilation=(1, dilation), bias=bias, mode=mode,
-                                   chan=chan, params=params, dtype=dtype, fixed=fixed)
-
-    def forward(self, x):                      # x: [N, C, L]
-        return self.conv(x.unsqueeze(2)).squeeze(2)
-
-
 class TropicalConv3dFn(torch.autograd.Function):
     """y = tconv3d_forward(...); backward = tconv3d_backward with the stored winners."""
 
@@ -350,3 +333,29 @@ class TropicalConv3d(TropicalConv2d):
 
     ND = 3
     FN = TropicalConv3dFn
+
+
+class TropicalConv1d(nn.Module):
+    """1-D tropical convolution (Section 3.2) with ``nn.Conv1d``'s constructor arguments; mode / chan /
+    params / dtype as in TropicalConv2d.  The length-3, stride-1 layers run as 1 x 3 windows on a signal
+    of unit height through the tiled 2-D kernels; every other window (up to 256 taps; the paper's audio
+    networks open with length 80) runs as a 1 x 1 x k window through the any-shape kernels of the
+    three-dimensional entry points, which are the faster ones for long windows."""
+
+    def __init__(self, in_channels, out_channels, kernel_size, stride=1, padding=0, dilation=1,
+                 bias=True, mode="compound", chan="default", params="2p", dtype="f32", fixed=(0.5, 0.5)):
+        super().__init__()
+        self.tiled = (kernel_size == 3 and stride == 1 and dilation == 1)
+        if self.tiled:
+            self.conv = TropicalConv2d(in_channels, out_channels, (1, kernel_size), stride=(1, stride),
+                                       padding=(0, padding), dilation=(1, dilation), bias=bias, mode=mode,
+                                       chan=chan, params=params, dtype=dtype, fixed=fixed)
+        else:
+            self.conv = TropicalConv3d(in_channels, out_channels, (1, 1, kernel_size), stride=(1, 1, stride),
+                                       padding=(0, 0, padding), dilation=(1, 1, dilation), bias=bias, mode=mode,
+                                       chan=chan, params=params, dtype=dtype, fixed=fixed)
+
+    def forward(self, x):                      # x: [N, C, L]
+        if self.tiled:
+            return self.conv(x.unsqueeze(2)).squeeze(2)
+        return self.conv(x[:, :, None, None, :])[:, :, 0, 0, :]

@@ -152,21 +152,23 @@ def test_depthwise_layer_against_the_oracle(mode, params):
 @pytest.mark.gpu
 @pytest.mark.parametrize("mode,chan", [("compound", "default"), ("parallel", "default"), ("max_plus", "default"),
                                        ("min_plus", "sum")])
-def test_conv1d_with_a_long_window_against_the_oracle(mode, chan):
-    """Kernel length 80, stride 4 (the first layer of the paper's 1-D audio networks), as a
-    1 x 80 window on a signal of unit height."""
+@pytest.mark.parametrize("S,st,pad", [(80, 4, 38), (3, 1, 1)])
+def test_conv1d_against_the_oracle(mode, chan, S, st, pad):
+    """Kernel length 80, stride 4 (the first layer of the paper's 1-D audio networks) and the length-3
+    layers that follow it, against the 2-D oracle on a signal of unit height."""
     from oracle import tconv_oracle as ora
     from paper_2504_06881_b200.nn import TropicalConv1d
-    N, C, K, Ln, S, st = 2, 3, 5, 400, 80, 4
-    d = inputs.layer(N, C, 1, Ln, K, 1, S, stride=(1, st), pad=(0, 38), mode=mode, chan=chan)
+    N, C, K, Ln = 2, 3, 5, 400
+    d = inputs.layer(N, C, 1, Ln, K, 1, S, stride=(1, st), pad=(0, pad), mode=mode, chan=chan)
     t = inputs.draw(d, 2300)
-    m = TropicalConv1d(C, K, S, stride=st, padding=38, mode=mode, chan=chan).cuda()
+    m = TropicalConv1d(C, K, S, stride=st, padding=pad, mode=mode, chan=chan).cuda()
+    assert m.tiled == (S == 3)
     two, par = mode in ("compound", "parallel"), mode == "parallel"
     with torch.no_grad():
-        m.conv.weight.copy_(torch.from_numpy(t["w"]))
+        m.conv.weight.copy_(torch.from_numpy(t["w"]).reshape(m.conv.weight.shape))
         m.conv.bias.copy_(torch.from_numpy(t["bias"]))
         if par:
-            m.conv.weight2.copy_(torch.from_numpy(t["w2"]))
+            m.conv.weight2.copy_(torch.from_numpy(t["w2"]).reshape(m.conv.weight.shape))
         if two:
             m.conv.alpha.copy_(torch.from_numpy(t["alpha"]))
             m.conv.beta.copy_(torch.from_numpy(t["beta"]))
@@ -182,7 +184,7 @@ def test_conv1d_with_a_long_window_against_the_oracle(mode, chan):
     def close(got, want, scale):
         return (np.abs(got.detach().cpu().numpy().astype(np.float64) - want) <= 1e-5 * scale + 1e-30).all()
 
-    assert close(x.grad.unsqueeze(2), *gref["grad_x"]) and close(m.conv.weight.grad, *gref["grad_w"])
+    assert close(x.grad.unsqueeze(2), *gref["grad_x"]) and close(m.conv.weight.grad.reshape(K, C, 1, S), *gref["grad_w"])
     if two:
         assert close(m.conv.alpha.grad, *gref["grad_alpha"]) and close(m.conv.beta.grad, *gref["grad_beta"])
 
