@@ -104,3 +104,27 @@ def test_depthwise_descriptor_checks_on_the_host():
     assert tconv.tconv_dw_winner_bytes(dict(ok, R=5, S=5, pad_h=2, pad_w=2)) == 0   # a code nibble holds 16 taps
     assert tconv.tconv_dw_winner_bytes(dict(ok, N=0)) == 0
     assert tconv.tconv_dw_winner_bytes(inputs.layer(70_000, 1024, 64, 64, 1024, 3, 3, pad=1)) == 0   # > 2^31 - 1 elements
+
+
+def test_three_dimensional_descriptor_checks():
+    """Host-side calls of include/tconv3d.h (no GPU needed)."""
+    from paper_2504_06881_b200 import tconv3d
+    d = inputs.layer3d(1, 1, 4, 4, 4, 1, T=3, R=3, S=3)
+    assert tconv3d.tconv3d_output_shape(d) == (2, 2, 2)
+    assert tconv3d.tconv3d_output_shape(inputs.layer3d(2, 1, 28, 28, 28, 6, T=5, R=5, S=5, stride=2)) == (12, 12, 12)
+    assert tconv3d.tconv3d_output_shape(dict(d, D=9, H=8, W=7, stride=(2, 1, 3), pad=(1, 0, 2), dil=(2, 1, 1))) == (4, 6, 3)
+    assert tconv3d.tconv3d_winner_bytes(d) == 4 * 8                     # int32 per output
+    assert tconv3d.tconv3d_winner_bytes(dict(d, chan="sum")) == 2 * 8   # uint16 per (output, channel)
+    assert tconv3d.tconv3d_winner_bytes(dict(d, C=3, mode="compound")) == 2 * 3 * 8
+    assert tconv3d.tconv3d_winner_bytes(dict(d, T=9, R=9, S=9, pad=(4, 4, 4))) == 0      # > 256 taps
+    assert tconv3d.tconv3d_workspace_bytes(d, False) == 0
+    assert tconv3d.tconv3d_workspace_bytes(d, True) >= tconv3d.tconv3d_winner_bytes(d)
+    with pytest.raises(tconv.TconvError):
+        tconv3d.tconv3d_output_shape(dict(d, D=2))                       # window larger than the volume
+    with pytest.raises(tconv.TconvError) as e:
+        tconv3d.tconv3d_output_shape(dict(d, mode="compound", chan="max"))
+    assert e.value.status == -2
+    for key in ("N", "C", "D", "H", "W", "K", "T", "R", "S"):
+        assert tconv3d.tconv3d_winner_bytes(dict(d, **{key: 0})) == 0
+    assert tconv3d.tconv3d_winner_bytes(dict(d, stride=(0, 1, 1))) == 0
+    assert tconv3d.tconv3d_winner_bytes(inputs.layer3d(4096, 64, 64, 64, 64, 64, pad=1)) == 0   # > 2^31 - 1 elements

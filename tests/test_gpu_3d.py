@@ -89,15 +89,3 @@ def test_parameter_free_and_no_bias():
 def test_largest_window_and_unit_window():
     check(inputs.layer3d(1, 2, 8, 8, 9, 2, T=4, R=8, S=8, pad=(1, 3, 3), mode="compound"), 308)
     check(inputs.layer3d(2, 3, 3, 4, 5, 2, T=1, R=1, S=1, mode="parallel"), 309)
-
-
-def test_descriptor_checks():
-    d = inputs.layer3d(1, 1, 4, 4, 4, 1, T=3, R=3, S=3)
-    assert tconv3d.tconv3d_output_shape(d) == (2, 2, 2)
-    assert tconv3d.tconv3d_winner_bytes(d) == 4 * 8
-    assert tconv3d.tconv3d_winner_bytes(dict(d, chan="sum")) == 2 * 8
-    assert tconv3d.tconv3d_winner_bytes(dict(d, T=9, R=9, S=9, pad=(4, 4, 4))) == 0      # > 256 taps
-    with pytest.raises(tconv.TconvError):
-        tconv3d.tconv3d_output_shape(dict(d, D=2))
-    with pytest.raises(tconv.TconvError):
-        tconv3d.tconv3d_output_shape(dict(d, mode="compound", chan="max"))
