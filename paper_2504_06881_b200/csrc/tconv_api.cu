@@ -316,22 +316,28 @@ int backward_sum_t(const Geo& g0, const void* x, const void* w, const void* w2, 
             return cuda_fail(cudaGetLastError());                                                    \
         kern<<<grid, pl.threads, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);   \
     }
+#define TCONV_GXC(BR, CBV, NTH)                                                                      \
+    {                                                                                                \
+        auto kern = bwd_code_gx_kernel<T, BR, CBV, false, NTH, false, true>;                         \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess) \
+            return cuda_fail(cudaGetLastError());                                                    \
+        kern<<<grid, pl.threads, pl.smem, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, pl);   \
+    }
 #define TCONV_GX(BR, CBV)                                                                            \
     {                                                                                                \
-        if (g.wide) TCONV_GXW(BR, CBV)                                                               \
+        if (pl.ncol > 1 && !g.wide) { if (pl.threads > 256) TCONV_GXC(BR, CBV, 1024) else TCONV_GXC(BR, CBV, 256) } \
+        else if (g.wide) TCONV_GXW(BR, CBV)                                                          \
         else if (pl.imgs > 1) TCONV_GXM(BR, CBV, true, 256)                                          \
         else if (pl.threads > 256) TCONV_GXM(BR, CBV, false, 1024)                                   \
         else TCONV_GXM(BR, CBV, false, 256)                                                          \
     }
-#define TCONV_GX2(BR)                                                                                \
-    {                                                                                                \
-        if (pl.CB == 2) TCONV_GX(BR, 2) else TCONV_GX(BR, 1)                                         \
-    }
+#define TCONV_GX2(BR) TCONV_GX(BR, 1)
                 if (br == 0) TCONV_GX2(0) else if (br == 1) TCONV_GX2(1) else TCONV_GX2(2)
 #undef TCONV_GX2
 #undef TCONV_GX
 #undef TCONV_GXM
 #undef TCONV_GXW
+#undef TCONV_GXC
                 name = "bwd_code";
             } else {
                 const size_t total = (size_t)g0.N * g0.C * g0.H * g0.W;

@@ -242,7 +242,10 @@ __global__ void bwd_reduce_partials_kernel(const float* __restrict__ partial, fl
 }
 
 // ---------------------------------------------------------------------------------- codes: grad_x
-constexpr int kGxCB = 2;   // most channels a CTA of bwd_code_gx_kernel handles
+// Most channels a CTA of bwd_code_gx_kernel handles.  One: two channels share the gradient loads,
+// but the tile then takes twice the shared memory, and resident CTAs count for more (measured on
+// every layer of the benchmark configurations, 3 to 27 % in favour of one channel).
+constexpr int kGxCB = 1;
 
 struct CodeGxPlan {
     int imgs;                // images per CTA (> 1 only when a CTA owns whole images of a small map)
@@ -251,7 +254,8 @@ struct CodeGxPlan {
     int NRmax, QPR, NQpad;   // contributing output rows (max), quads per row, padded quad count
     int threads;             // CTA size: 256, or more where the tile leaves room for only 1-2 CTAs per SM
     int ncblk;               // channel blocks (the fastest-varying part of the CTA index)
-    unsigned grid;           // CTAs: image groups x row bands x channel blocks
+    int ncol, TWI, QPRt;     // column tiles of a wide map: tiles per row band, owned input columns, quads per tile row
+    unsigned grid;           // CTAs: image groups x row bands x column tiles x channel blocks
     size_t smem;
 };
 
@@ -301,7 +305,8 @@ __device__ __forceinline__ void taps_of(const Codes4<WIDE>& c4, int j, unsigned&
 // The output width is a multiple of 4 (the caller pads grad_y otherwise): aligned vector loads.
 // MULTI: the CTA owns pl.imgs whole images (small maps); else one band of rows of one image.
 // NTH: upper bound of the CTA size (256, or 1024 for tiles that leave room for one or two CTAs per SM).
-template <typename T, int BR, int CB, bool MULTI, int NTH, bool WIDE>
+// COLS: the band of rows is cut into pl.ncol column tiles (wide maps; never with MULTI).
+template <typename T, int BR, int CB, bool MULTI, int NTH, bool WIDE, bool COLS = false>
 __global__ void __launch_bounds__(NTH)
 bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
                    const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
@@ -310,7 +315,19 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     // a CTA owns either a band of input rows of one image or pl.imgs whole images of a small map;
     // its output quads are numbered image by image
     // channel blocks vary fastest over the grid: CTAs that run together share one band of grad_y
-    const int cblk = blockIdx.x % pl.ncblk, xt = blockIdx.x / pl.ncblk;
+    const int cblk = blockIdx.x % pl.ncblk;
+    int xt = blockIdx.x / pl.ncblk;
+    // column tile: owned input columns [iw0, iwn), first quad column qc0 of the outputs that read them
+    int iw0 = 0, iwn = g.W, qc0 = 0, qpr = pl.QPR;
+    if constexpr (COLS) {
+        const int ct = xt % pl.ncol;
+        xt /= pl.ncol;
+        iw0 = ct * pl.TWI;
+        iwn = min(g.W, iw0 + pl.TWI);
+        const int numw = iw0 + g.pw - (g.S - 1) * g.dw;
+        qc0 = (numw <= 0 ? 0 : (numw + g.sw - 1) / g.sw) >> 2;
+        qpr = pl.QPRt;
+    }
     const int tile_i = xt % pl.tiles_per_img;
     const int n_first = MULTI ? (xt / pl.tiles_per_img) * pl.imgs : xt / pl.tiles_per_img;
     const int nimg = MULTI ? min(pl.imgs, g.N - n_first) : 1;
@@ -322,7 +339,7 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
     const int oh_lo = num <= 0 ? 0 : (num + g.sh - 1) / g.sh;
     const int oh_hi = min(g.OH - 1, (ih0 + rows - 1 + g.ph) / g.sh);
     const int NR = oh_hi - oh_lo + 1;
-    const int NQ1 = NR * pl.QPR;          // quads of one image
+    const int NQ1 = NR * qpr;             // quads of one image (of its column tile)
     const int NQ = NQ1 * nimg;
     const int NQp = pl.NQpad;
     const int nacc = CB * g.RS * 4 * NQp;
@@ -346,8 +363,9 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
         const int il = MULTI ? q / NQ1 : 0;
         const int q1 = q - il * NQ1;
         const int n = n_first + il;
-        const int orow = q1 / pl.QPR;
-        const int ow0 = (q1 - orow * pl.QPR) * 4;
+        const int orow = q1 / qpr;
+        const int ow0 = (qc0 + q1 - orow * qpr) * 4;
+        if (COLS && ow0 >= g.OW) continue;     // the last column tile's rows may end early
         const size_t pix = (size_t)(oh_lo + orow) * g.OW + ow0;
         const T* gp = gy + (size_t)n * g.K * plane + pix;
         // a channel past C reads channel C-1 again; its alpha = beta = 0 (or it is skipped below)
@@ -423,7 +441,7 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
         T* gxc = gx + ((size_t)(n_first + il) * g.C + c0 + cb) * g.H * g.W;
         for (int row = warp; row < rows; row += nwarps) {
             const int ih = ih0 + row;
-            for (int iw = lane; iw < g.W; iw += 32) {
+            for (int iw = iw0 + lane; iw < iwn; iw += 32) {
                 float s = 0.0f;
                 for (int r = 0; r < g.R; ++r) {
                     int oh = ih + g.ph - r * g.dh;
@@ -432,7 +450,7 @@ bwd_code_gx_kernel(Geo g, const float* __restrict__ alpha, const float* __restri
                         oh /= g.sh;
                     }
                     if (oh < oh_lo || oh > oh_hi) continue;
-                    const float* Ar = Ac + (oh - oh_lo) * pl.QPR;
+                    const float* Ar = Ac + (oh - oh_lo) * qpr - qc0;
                     for (int sx = 0; sx < g.S; ++sx) {
                         int ow = iw + g.pw - sx * g.dw;
                         if (!unit_stride) {
@@ -788,8 +806,76 @@ inline bool plan_idx_gw(const Geo& g, int* chunks, size_t* smem) {
     return true;
 }
 
+// One column-tiled candidate: cb channels, ncol column tiles, budget bytes of accumulators.
+inline bool plan_code_gx_cols(const Geo& g, int cb, int ncol, size_t budget, CodeGxPlan* pl) {
+    const int halo = (g.R - 1) * g.dh;
+    pl->QPR = (g.OW + 3) / 4;
+    pl->imgs = 1;
+    pl->ncol = ncol;
+    pl->TWI = ((g.W + ncol - 1) / ncol + 3) / 4 * 4;
+    pl->ncol = (g.W + pl->TWI - 1) / pl->TWI;
+    const int span = (pl->TWI - 1 + (g.S - 1) * g.dw) / g.sw + 1;   // outputs that read one tile's columns
+    pl->QPRt = (span + 3) / 4 + 1;                                   // + 1: the first of them need not start a quad
+    if (pl->QPRt > pl->QPR) pl->QPRt = pl->QPR;
+    const size_t per_quad = (size_t)cb * g.RS * 4 * sizeof(float);
+    const long maxq = (long)(budget / per_quad) / 32 * 32;
+    long nr = maxq / pl->QPRt;
+    if (nr > g.OH) nr = g.OH;
+    int thi = nr >= g.OH ? g.H : (int)((nr - 2) * g.sh) - halo;
+    if (thi < 2 * halo || thi < 1) return false;
+    if (thi > g.H) thi = g.H;
+    pl->CB = cb;
+    pl->THI = thi;
+    pl->tiles_per_img = (g.H + thi - 1) / thi;
+    pl->NRmax = (int)nr;
+    pl->NQpad = (int)((nr * pl->QPRt + 31) / 32 * 32);
+    pl->smem = ((size_t)cb * g.RS * 4 * pl->NQpad + 2 * (size_t)g.K * kGxCB) * sizeof(float);
+    if (pl->smem > kBwdSmemLimit + 16 * 1024) return false;
+    const int per_sm = (int)((227 * 1024) / (pl->smem + 1024));
+    const int cap = per_sm >= 3 ? 256 : (per_sm == 2 ? 512 : 1024);
+    const int nq = (int)nr * pl->QPRt;
+    const int passes = (nq + cap - 1) / cap;
+    int th = ((nq + passes - 1) / passes + 31) / 32 * 32;
+    if (th < 256) th = 256;
+    pl->threads = th < cap ? th : cap;
+    if (g.wide) pl->threads = 256;
+    pl->ncblk = (g.C + cb - 1) / cb;
+    const size_t nct = (size_t)g.N * pl->tiles_per_img * pl->ncol * pl->ncblk;
+    if (nct > 0x7fffffffu) return false;
+    pl->grid = (unsigned)nct;
+    return true;
+}
+
 inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
     pl->QPR = (g.OW + 3) / 4;
+    pl->ncol = 1;
+    pl->TWI = g.W;
+    pl->QPRt = pl->QPR;
+    static const char* force = getenv("TCONV_GX_PLAN");   // debug switch: "cb,ncol,kilobytes"
+    if (force) {
+        int cb = 0, ncol = 0, kb = 0;
+        if (sscanf(force, "%d,%d,%d", &cb, &ncol, &kb) == 3 && cb >= 1 && cb <= kGxCB && ncol >= 1 && kb >= 16 &&
+            !g.wide && plan_code_gx_cols(g, cb, ncol, (size_t)kb * 1024, pl))
+            return true;
+        pl->ncol = 1; pl->TWI = g.W; pl->QPRt = pl->QPR;
+    }
+    // Maps with at least 128 quads (smaller ones share a CTA between several images, below): one
+    // channel per CTA and a small tile, so that five CTAs stay resident per SM and hide the latency
+    // of the code loads (measured on 32x32 to 128x256 maps: 5 to 35 % faster than two channels in
+    // 160 KB); maps from 128 columns on are also cut into column tiles of 64 input columns, which
+    // keeps the bands tall enough for their halo (128x256 at dilation 2: 20.1 -> 12.6 ms).
+    if (!g.wide && (long)g.OH * pl->QPR * 2 > 256) {
+        CodeGxPlan cand = *pl;
+        if (g.W >= 128 && plan_code_gx_cols(g, 1, (g.W + 63) / 64, 72 * 1024, &cand) && cand.ncol > 1) {
+            *pl = cand;
+            return true;
+        }
+        cand = *pl;
+        if (plan_code_gx_cols(g, 1, 1, 40 * 1024, &cand)) {
+            *pl = cand;
+            return true;
+        }
+    }
     const int halo = (g.R - 1) * g.dh;
     for (int cb = kGxCB; cb >= 1; --cb) {
         // rows of output quads that fit: CB * RS * 4 floats per quad
