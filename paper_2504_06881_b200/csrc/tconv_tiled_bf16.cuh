@@ -117,12 +117,26 @@ __global__ void repack_weights_bf16_kernel(int K, int C, int RS, int tile_k, int
     }
 }
 
-template <int MODE, int CHAN, bool WIN, bool XTMA, bool RAG, int R, int S, int SW, int DW, int Q, int KG, int PW>
+// KPT words of packed weights of one tap (one or two 16-byte loads)
+template <int KPT>
+__device__ __forceinline__ void loadw(const unsigned* p, unsigned* out) {
+    const uint4 a = *reinterpret_cast<const uint4*>(p);
+    out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+    if constexpr (KPT == 8) {
+        const uint4 b = *reinterpret_cast<const uint4*>(p + 4);
+        out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+    }
+}
+
+// KPT: output channels per thread, 8, or 4 for layers that would otherwise keep too few warps
+// resident (small maps with many channels at a small batch).
+template <int MODE, int CHAN, bool WIN, bool XTMA, bool RAG, int R, int S, int SW, int DW, int Q, int KG, int PW, int KPT = 8>
 __global__ void __launch_bounds__(KG * PW * 32)
 fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams p) {
     static_assert(S == 3, "the pixel-pair selection below is written for 3 taps per row");
+    static_assert(KPT == 8 || KPT == 4, "output channels per thread");
     constexpr int RS = R * S;
-    constexpr int TILE_K = KG * 8;
+    constexpr int TILE_K = KG * KPT;
     constexpr int NT = KG * PW * 32;
     constexpr int NWARPS = KG * PW;
     constexpr int L = 3 * SW + (S - 1) * DW + 1;   // input elements one quad touches per row
@@ -284,12 +298,12 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
     };
 
     // running state: fp32 sums (Sum forms) or packed running best (Max / Min combine)
-    float acc[SUMF ? 8 : 1][Q][4];
-    unsigned best[SUMF ? 1 : 8][Q][2];
-    unsigned cbest[(WIN && !SUMF) ? 8 : 1][Q][2];   // winning channel per pixel, two 16-bit fields
+    float acc[SUMF ? KPT : 1][Q][4];
+    unsigned best[SUMF ? 1 : KPT][Q][2];
+    unsigned cbest[(WIN && !SUMF) ? KPT : 1][Q][2];   // winning channel per pixel, two 16-bit fields
     constexpr unsigned kNegInf2 = 0xFF80FF80u, kPosInf2 = 0x7F807F80u;
 #pragma unroll
-    for (int k = 0; k < 8; ++k)
+    for (int k = 0; k < KPT; ++k)
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
             if constexpr (SUMF) {
@@ -320,10 +334,10 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
             if (ch + 1 < p.nchunks) cp_async_wait<1>(); else cp_async_wait<0>();
             __syncthreads();
         }
-        const unsigned* ws = st + w_off + kg * 8;
-        const unsigned* ws2 = st + w2_off + kg * 8;
-        const float* as = reinterpret_cast<const float*>(st + a_off) + kg * 8;
-        const float* bs = reinterpret_cast<const float*>(st + b_off) + kg * 8;
+        const unsigned* ws = st + w_off + kg * KPT;
+        const unsigned* ws2 = st + w2_off + kg * KPT;
+        const float* as = reinterpret_cast<const float*>(st + a_off) + kg * KPT;
+        const float* bs = reinterpret_cast<const float*>(st + b_off) + kg * KPT;
         const int nc = min(p.CC, g.C - ch * p.CC);
         for (int cc = 0; cc < nc; ++cc) {
             unsigned xw[Q][R][NW];
@@ -336,9 +350,9 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
             const unsigned* wc2 = ws2 + cc * (RS * TILE_K);
             const int c = ch * p.CC + cc;
 
-            unsigned mx[CARRIED ? 1 : 8][Q][2];
-            unsigned mn[TWO ? 8 : 1][Q][2];
-            unsigned amx[(WIN && SUMF) ? 8 : 1][Q][2], amn[(WIN && TWO) ? 8 : 1][Q][2];
+            unsigned mx[CARRIED ? 1 : KPT][Q][2];
+            unsigned mn[TWO ? KPT : 1][Q][2];
+            unsigned amx[(WIN && SUMF) ? KPT : 1][Q][2], amn[(WIN && TWO) ? KPT : 1][Q][2];
 
             if constexpr (WIN && SUMF) {
 #pragma unroll
@@ -346,17 +360,9 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                     constexpr unsigned one2 = 0x00010001u;
                     const unsigned tap2 = one2 * (unsigned)tap;
                     const int r = tap / S, sx = tap % S;
-                    unsigned wv[8], wv2[8];
-                    {
-                        const uint4 a = *reinterpret_cast<const uint4*>(wc + tap * TILE_K);
-                        const uint4 b = *reinterpret_cast<const uint4*>(wc + tap * TILE_K + 4);
-                        wv[0] = a.x; wv[1] = a.y; wv[2] = a.z; wv[3] = a.w; wv[4] = b.x; wv[5] = b.y; wv[6] = b.z; wv[7] = b.w;
-                    }
-                    if constexpr (PAR) {
-                        const uint4 a = *reinterpret_cast<const uint4*>(wc2 + tap * TILE_K);
-                        const uint4 b = *reinterpret_cast<const uint4*>(wc2 + tap * TILE_K + 4);
-                        wv2[0] = a.x; wv2[1] = a.y; wv2[2] = a.z; wv2[3] = a.w; wv2[4] = b.x; wv2[5] = b.y; wv2[6] = b.z; wv2[7] = b.w;
-                    }
+                    unsigned wv[KPT], wv2[KPT];
+                    loadw<KPT>(wc + tap * TILE_K, wv);
+                    if constexpr (PAR) loadw<KPT>(wc2 + tap * TILE_K, wv2);
 #pragma unroll
                     for (int q = 0; q < Q; ++q)
 #pragma unroll
@@ -367,7 +373,7 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                             else if (sx == 1) xp = pp == 0 ? pixel_pair<SW, EODD + 0 * SW + 1 * DW>(xw[q][r]) : pixel_pair<SW, EODD + 2 * SW + 1 * DW>(xw[q][r]);
                             else xp = pp == 0 ? pixel_pair<SW, EODD + 0 * SW + 2 * DW>(xw[q][r]) : pixel_pair<SW, EODD + 2 * SW + 2 * DW>(xw[q][r]);
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
+                            for (int k = 0; k < KPT; ++k) {
                                 const unsigned t = hadd2u(xp, wv[k]);
                                 const unsigned t2 = PAR ? hadd2u(xp, wv2[k]) : t;
                                 if constexpr (TWO) {
@@ -400,20 +406,12 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                 for (int gi = 0; gi < NG; ++gi) {
                     const int t0 = (gi == 0) ? 0 : FIRST + 2 * (gi - 1);
                     const int nt = (gi == 0) ? (FIRST < RS ? FIRST : RS) : ((RS - t0) < 2 ? (RS - t0) : 2);
-                    unsigned wv[3][8], wv2[PAR ? 3 : 1][8];
+                    unsigned wv[3][KPT], wv2[PAR ? 3 : 1][KPT];
 #pragma unroll
                     for (int u = 0; u < 3; ++u)
                         if (u < nt) {
-                            const uint4 a = *reinterpret_cast<const uint4*>(wc + (t0 + u) * TILE_K);
-                            const uint4 b = *reinterpret_cast<const uint4*>(wc + (t0 + u) * TILE_K + 4);
-                            wv[u][0] = a.x; wv[u][1] = a.y; wv[u][2] = a.z; wv[u][3] = a.w;
-                            wv[u][4] = b.x; wv[u][5] = b.y; wv[u][6] = b.z; wv[u][7] = b.w;
-                            if constexpr (PAR) {
-                                const uint4 c4 = *reinterpret_cast<const uint4*>(wc2 + (t0 + u) * TILE_K);
-                                const uint4 d4 = *reinterpret_cast<const uint4*>(wc2 + (t0 + u) * TILE_K + 4);
-                                wv2[u][0] = c4.x; wv2[u][1] = c4.y; wv2[u][2] = c4.z; wv2[u][3] = c4.w;
-                                wv2[u][4] = d4.x; wv2[u][5] = d4.y; wv2[u][6] = d4.z; wv2[u][7] = d4.w;
-                            }
+                            loadw<KPT>(wc + (t0 + u) * TILE_K, wv[u]);
+                            if constexpr (PAR) loadw<KPT>(wc2 + (t0 + u) * TILE_K, wv2[u]);
                         }
 #pragma unroll
                     for (int q = 0; q < Q; ++q)
@@ -430,7 +428,7 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                                     else xp[u] = pp == 0 ? pixel_pair<SW, EODD + 0 * SW + 2 * DW>(xw[q][r]) : pixel_pair<SW, EODD + 2 * SW + 2 * DW>(xw[q][r]);
                                 }
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
+                            for (int k = 0; k < KPT; ++k) {
                                 unsigned ta[3], tb[3];
 #pragma unroll
                                 for (int u = 0; u < 3; ++u)
@@ -463,13 +461,13 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
 
             // channel combine
             if constexpr (!CARRIED) {
-                float av[8], bv[8];
+                float av[KPT], bv[KPT];
                 if constexpr (TWO) {
-                    load8(as + cc * TILE_K, av);
-                    load8(bs + cc * TILE_K, bv);
+                    loadn<KPT>(as + cc * TILE_K, av);
+                    loadn<KPT>(bs + cc * TILE_K, bv);
                 }
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
+                for (int k = 0; k < KPT; ++k)
 #pragma unroll
                     for (int q = 0; q < Q; ++q)
 #pragma unroll
@@ -495,8 +493,8 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                         if (out_row[q] < 0) continue;
                         const int n = out_row[q] / g.OH, oh = out_row[q] - n * g.OH;
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const int kk = kt * TILE_K + kg * 8 + k;
+                        for (int k = 0; k < KPT; ++k) {
+                            const int kk = kt * TILE_K + kg * KPT + k;
                             if (kk >= g.K) continue;
                             uint8_t* dst = codes + (((size_t)n * g.K + kk) * g.C + c) * ((size_t)g.OH * g.OWP) +
                                            (size_t)oh * g.OWP + qcol[q];
@@ -526,8 +524,8 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
         if (out_row[q] < 0) continue;
         const int n = out_row[q] / g.OH, oh = out_row[q] - n * g.OH;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int kk = kt * TILE_K + kg * 8 + k;
+        for (int k = 0; k < KPT; ++k) {
+            const int kk = kt * TILE_K + kg * KPT + k;
             if (kk >= g.K) continue;
             const size_t o = ((size_t)n * g.K + kk) * plane + (size_t)oh * g.OW + qcol[q];
             float v[4];
@@ -588,7 +586,10 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
     }
 }
 
-template <int MODE, int CHAN, bool WIN, int R, int S, int SW, int DW, int Q, int KG, int PW>
+// PLAIN_ONLY: instantiate only the kernel without TMA and without ragged tiles (what small maps
+// use); a plan that wants either is left to the caller's next choice.
+template <int MODE, int CHAN, bool WIN, int R, int S, int SW, int DW, int Q, int KG, int PW, int KPT = 8,
+          bool PLAIN_ONLY = false>
 int launch_tiled_variant_bf16(FwdArgs& a) {
     constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
     constexpr bool PAR = (MODE == TCONV_PARALLEL);
@@ -596,7 +597,8 @@ int launch_tiled_variant_bf16(FwdArgs& a) {
     if (g.C > 65535) return TCONV_ERR_UNSUPPORTED;   // winner channel kept in 16 bits
     TiledPlan pl;
     pl.p.g = g;
-    if (!plan_tiles<R, S, SW, DW, Q, KG, PW>(g, PAR, TWO, 2, &pl)) return TCONV_ERR_UNSUPPORTED;
+    if (!plan_tiles<R, S, SW, DW, Q, KG, PW, KPT>(g, PAR, TWO, 2, &pl)) return TCONV_ERR_UNSUPPORTED;
+    if (PLAIN_ONLY && (pl.xtma || pl.p.ragged)) return TCONV_ERR_UNSUPPORTED;
     const size_t need = pl.ws_w * (PAR ? 2 : 1) + (TWO ? 2 * pl.ws_ab : 0);
     if (!a.ws || a.ws_bytes < need) return TCONV_ERR_WORKSPACE_TOO_SMALL;
     float* wt = reinterpret_cast<float*>(a.ws);
@@ -615,12 +617,15 @@ int launch_tiled_variant_bf16(FwdArgs& a) {
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
 #define TCONV_LAUNCH_BF16(XTMAV, RAGV)                                                                \
     {                                                                                                \
-        auto kern = fwd_tiled_bf16_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW>;    \
+        auto kern = fwd_tiled_bf16_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, KPT>; \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) \
             return TCONV_ERR_CUDA;                                                                   \
         kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);                                    \
     }
-    if (pl.xtma) {
+    if constexpr (PLAIN_ONLY) {
+        TCONV_LAUNCH_BF16(false, false)
+        a.name = WIN ? "fwd_tiled_bf16_k4_win" : "fwd_tiled_bf16_k4";
+    } else if (pl.xtma) {
         if (pl.p.ragged) TCONV_LAUNCH_BF16(true, true) else TCONV_LAUNCH_BF16(true, false)
         a.name = WIN ? "fwd_tiled_bf16_tma_win" : "fwd_tiled_bf16_tma";
     } else {
@@ -639,6 +644,21 @@ int launch_tiled_geom_bf16(FwdArgs& a) {
     constexpr int Q = CARRIED ? 2 : 1;
     const Geo& g = a.g;
     if (g.R == 3 && g.S == 3) {
+        // Small maps with many channels at a small batch leave few warps to an SM when every thread
+        // owns 8 output channels (7x7 x 512 at batch 64: 12 warps per SM, and the layer takes as long
+        // as one CTA): 4 channels per thread double the warps.  Measured on the 14x14 and 7x7 layers
+        // of the ResNet-18 shape at batch 64: 4 to 12 % faster with winners, 6 to 13 % slower
+        // without (there the second staging of the x tiles costs more), so only with winners.
+        static const int k4 = getenv("TCONV_BF16_K4") ? atoi(getenv("TCONV_BF16_K4")) : -1;   // debug switch: 0 off, 1 always
+        const long warps8 = (((long)g.N * g.OH * ((g.OW + 3) / 4) + 31) / 32) * ((g.K + 7) / 8);
+        const bool fine = k4 == 0 ? false : (k4 == 1 ? true : (WIN && warps8 < 148L * 32));
+        if constexpr (Q == 1) {
+            if (fine && g.dw == 1 && (g.sw == 1 || g.sw == 2)) {
+                const int rc = g.sw == 1 ? launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 1, 1, 1, 4, 1, 4, true>(a)
+                                         : launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 2, 1, 1, 4, 1, 4, true>(a);
+                if (rc != TCONV_ERR_UNSUPPORTED) return rc;
+            }
+        }
         if (g.sw == 1 && g.dw == 1) return launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 1, 1, Q, 4, 1>(a);
         if (g.sw == 2 && g.dw == 1) return launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 2, 1, Q, 4, 1>(a);
         if (g.sw == 1 && g.dw == 2) return launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 1, 2, Q, 4, 1>(a);
