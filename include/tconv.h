@@ -154,11 +154,10 @@ int tconv_backward(const tconv_desc_t *desc, const void *x, const void *w, const
  * Forward pass for callers that cannot allocate device memory.  (The paper has no
  * counterpart of this entry point; it exists for the library's users.)
  *
- * Some callers have no way to hand over a workspace: code that runs inside a region
- * where the CUDA allocator must not be touched (for example between the capture calls
- * of a stream, or in a real-time loop that was given a fixed memory budget), plug-ins
- * whose host application owns all device memory, and small C programs that link this
- * library without a tensor framework.  For them this variant of tconv_forward takes
+ * Some callers have no way to hand over a workspace: code that runs where the CUDA
+ * allocator must not be touched (a real-time loop that was given a fixed memory budget
+ * at start-up), plug-ins whose host application owns all device memory, and small C
+ * programs that link this library without a tensor framework.  For them this variant of tconv_forward takes
  * its scratch (the repacked weights, alpha and beta of the tiled kernels) from a fixed
  * array inside the library image instead of a caller workspace.  It calls no
  * cudaMalloc, cudaFree or other allocating routine.

@@ -129,9 +129,61 @@ def check_layer(d, dists=None, seed=0, use_bias=True, stored_winners=True, recom
     return rep
 
 
-def sampled_check(d, t, sample_n, sample_k):
-    """Full-size GPU run against the oracle on a sample: images sample_n x output channels
-    [sample_k[0], sample_k[1]).  t holds numpy tensors x, w, w2, alpha, beta, bias, g."""
+def _backward_by_k_slices(ds, xs, w, g, w2, al, be, step=2):
+    """The oracle's backward on a one-image problem, output channels cut into slices that run
+    as concurrent oracle calls (the C loops run outside the interpreter lock): grad_x and its
+    bound add up over the slices, the parameter gradients concatenate along k."""
+    from concurrent.futures import ThreadPoolExecutor
+    K = ds["K"]
+    cuts = [(a, min(K, a + step)) for a in range(0, K, step)]
+
+    def one(cut):
+        a, b = cut
+        sl = lambda v: None if v is None else np.ascontiguousarray(v[a:b])
+        return ora.backward(dict(ds, K=b - a), xs, sl(w), np.ascontiguousarray(g[:, a:b]), sl(w2), sl(al), sl(be))
+
+    with ThreadPoolExecutor(max_workers=max(1, min(len(cuts), ora.threads()))) as ex:
+        parts = list(ex.map(one, cuts))
+    out = {}
+    for name in parts[0]:
+        if name == "grad_x":
+            out[name] = tuple(sum(p[name][i] for p in parts) for i in (0, 1))
+        else:
+            out[name] = tuple(np.concatenate([p[name][i] for p in parts], 0) for i in (0, 1))
+    return out
+
+
+def _one_output_reference(d, t, n, k, oh, ow):
+    """The oracle on the receptive field of one output: the window's taps gathered into an
+    R x S patch per channel (zeros where the window leaves the image), run as a layer with a
+    single output.  Returns (y, winner index or per-channel codes)."""
+    C, R, S = d["C"], d["R"], d["S"]
+    patch = np.zeros((1, C, R, S), np.float32)
+    for r in range(R):
+        ih = oh * d["stride_h"] - d["pad_h"] + r * d["dil_h"]
+        if not 0 <= ih < d["H"]:
+            continue
+        for s in range(S):
+            iw = ow * d["stride_w"] - d["pad_w"] + s * d["dil_w"]
+            if 0 <= iw < d["W"]:
+                patch[0, :, r, s] = t["x"][n, :, ih, iw]
+    d1 = dict(d, N=1, K=1, H=R, W=S, stride_h=1, stride_w=1, pad_h=0, pad_w=0, dil_h=1, dil_w=1)
+    two = d["mode"] in ("compound", "parallel")
+    ref = ora.forward(d1, patch, np.ascontiguousarray(t["w"][k:k + 1]),
+                      np.ascontiguousarray(t["w2"][k:k + 1]) if d["mode"] == "parallel" else None,
+                      np.ascontiguousarray(t["alpha"][k:k + 1]) if two else None,
+                      np.ascontiguousarray(t["beta"][k:k + 1]) if two else None,
+                      np.ascontiguousarray(t["bias"][k:k + 1]))
+    win = ref["idx"][0, 0, 0, 0] if ref["idx"] is not None else ref["codes"][0, 0, :, 0, 0]
+    return ref["y"][0, 0, 0, 0], win
+
+
+def sampled_check(d, t, sample_n, sample_k, fwd_blocks=(), random_outputs=0, random_seed=0):
+    """Full-size GPU run against the oracle on a sample.  Forward, winners and backward:
+    images sample_n x output channels [sample_k[0], sample_k[1]) (the upstream gradient is zero
+    outside that block).  Forward and winners only: every (n, k0, k1) of fwd_blocks, and
+    random_outputs seeded random outputs (n, k, oh, ow), each against the oracle run on that
+    output's receptive field.  t holds numpy tensors x, w, w2, alpha, beta, bias, g."""
     dt = tconv.TORCH_DTYPE[d["dtype"]]
     two = d["mode"] in ("compound", "parallel")
     par = d["mode"] == "parallel"
@@ -153,20 +205,39 @@ def sampled_check(d, t, sample_n, sample_k):
     torch.cuda.synchronize()
     assert tconv.tconv_device_status() == 0
     assert "tiled" in kernel_fwd, kernel_fwd
-    wn = winners_as_numpy(d, win)
+    sum_form = ora.resolved_chan(d) == "sum"
+
+    def winners_of(n, ka, kb):
+        """winners of image n, output channels [ka, kb), as the oracle lays them out"""
+        OH, OW = inputs.output_hw(d)
+        if not sum_form:
+            return win.view(torch.int32).view(d["N"], d["K"], OH, OW)[n, ka:kb].cpu().numpy()
+        assert d["R"] * d["S"] <= 16, "one-byte codes"
+        OWP = (OW + 3) // 4 * 4
+        raw = win.view(d["N"], d["K"], d["C"], OH, OWP)[n, ka:kb, :, :, :OW]
+        return raw.cpu().numpy()
+
+    def forward_block(n, ka, kb):
+        dsb = dict(d, N=1, K=kb - ka)
+        slb = lambda a: np.ascontiguousarray(a[ka:kb])
+        ref = ora.forward(dsb, np.ascontiguousarray(t["x"][n:n + 1]), slb(t["w"]), slb(t["w2"]) if par else None,
+                          slb(t["alpha"]) if two else None, slb(t["beta"]) if two else None, slb(t["bias"]))
+        yg = y[n, ka:kb].float().cpu().numpy()
+        ok = same_bits(yg, ref["y"][0])
+        assert ok.all(), (d["mode"], n, ka, kb, f"{int((~ok).sum())} outputs differ, first at {np.argwhere(~ok)[0]}")
+        want = ref["idx"] if ref["idx"] is not None else ref["codes"]
+        got = winners_of(n, ka, kb)
+        assert np.array_equal(got, want[0]), (d["mode"], n, ka, kb, f"{int((got != want[0]).sum())} winners differ")
+
     ds = dict(d, N=1, K=k1 - k0)
     sl = lambda a: np.ascontiguousarray(a[k0:k1])
     al, be = (sl(t["alpha"]), sl(t["beta"])) if two else (None, None)
     acc = {}
     for n in sample_n:
+        forward_block(n, k0, k1)
         xs = np.ascontiguousarray(t["x"][n:n + 1])
-        ref = ora.forward(ds, xs, sl(t["w"]), sl(t["w2"]) if par else None, al, be, sl(t["bias"]))
-        yg = y[n, k0:k1].float().cpu().numpy()
-        assert same_bits(yg, ref["y"][0]).all(), (d["mode"], n, "forward differs")
-        want = ref["idx"] if ref["idx"] is not None else ref["codes"]
-        assert np.array_equal(wn[n, k0:k1], want[0]), (d["mode"], n, "winners differ")
-        rb = ora.backward(ds, xs, sl(t["w"]), np.ascontiguousarray(gm[n:n + 1, k0:k1]),
-                          sl(t["w2"]) if par else None, al, be)
+        rb = _backward_by_k_slices(ds, xs, sl(t["w"]), np.ascontiguousarray(gm[n:n + 1, k0:k1]),
+                                   sl(t["w2"]) if par else None, al, be)
         compare_grads(d, {"grad_x": grads["grad_x"][n:n + 1]}, {"grad_x": rb["grad_x"]})
         for name, (gv, ga) in rb.items():
             if name == "grad_x":
@@ -182,7 +253,24 @@ def sampled_check(d, t, sample_n, sample_k):
         rest = torch.cat([got[:k0], got[k1:]])
         assert torch.count_nonzero(rest) == 0, name
     others = [n for n in range(d["N"]) if n not in sample_n]
-    assert torch.count_nonzero(grads["grad_x"][others[:4]]) == 0
+    if others:
+        assert torch.count_nonzero(grads["grad_x"][others[:4]]) == 0
+    for (n, ka, kb) in fwd_blocks:
+        forward_block(n, ka, kb)
+    if random_outputs:
+        rs = np.random.RandomState(random_seed)
+        OH, OW = inputs.output_hw(d)
+        pts = np.stack([rs.randint(0, d["N"], random_outputs), rs.randint(0, d["K"], random_outputs),
+                        rs.randint(0, OH, random_outputs), rs.randint(0, OW, random_outputs)], 1)
+        ii = [torch.from_numpy(pts[:, j]).cuda() for j in range(4)]
+        yg = y[ii[0], ii[1], ii[2], ii[3]].float().cpu().numpy()
+        if sum_form:
+            OWP = (OW + 3) // 4 * 4
+            wg = win.view(d["N"], d["K"], d["C"], OH, OWP)[ii[0], ii[1], :, ii[2], ii[3]].cpu().numpy()
+        else:
+            wg = win.view(torch.int32).view(d["N"], d["K"], OH, OW)[ii[0], ii[1], ii[2], ii[3]].cpu().numpy()
+        for j, (n, k, oh, ow) in enumerate(pts):
+            yr, wr = _one_output_reference(d, t, int(n), int(k), int(oh), int(ow))
+            assert same_bits(yg[j], yr).all(), (d["mode"], "random output", tuple(pts[j]), yg[j], yr)
+            assert np.array_equal(wg[j], wr), (d["mode"], "random output winners", tuple(pts[j]))
     return kernel_fwd
-
-

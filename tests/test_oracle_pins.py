@@ -476,6 +476,83 @@ def test_bf16_tap_rounding_and_final_rounding():
     assert np.all((ys.view(np.uint32) & 0xFFFF) == 0)
 
 
+def _bf16_unfold_forward(d, t):
+    """The unfold formulation in bf16, from library routines only: torch bf16 addition for the
+    tap sums (one rounding each), numpy min / max / argmin / argmax (first occurrence) over the
+    window axis, the channel combine in fp32 in ascending channel order (fused multiply-adds
+    emulated in float64: the product of a bf16 value and a float32 is exact there), the bias
+    added in fp32 and one conversion of the result to bf16 by torch.  Returns y (bf16 values as
+    float32), idx, codes."""
+    N, C, K, R, S = d["N"], d["C"], d["K"], d["R"], d["S"]
+    OH, OW = unfold_ref.out_hw(d)
+    mode, chan = d["mode"], d["chan"]
+    if chan == "default":
+        chan = {"max_plus": "max", "min_plus": "min"}.get(mode, "sum")
+    p = torch.from_numpy(unfold_ref.unfold(dict(d, dtype="f32"), t["x"])).to(torch.bfloat16)   # exact: bf16 values
+
+    def taps(w):
+        wr = torch.from_numpy(w).to(torch.bfloat16).reshape(1, K, C, R * S, 1, 1)
+        return (p[:, None] + wr).float().numpy()              # [N,K,C,RS,OH,OW], one bf16 rounding per sum
+
+    t1 = taps(t["w"])
+    t2 = taps(t["w2"]) if mode == "parallel" else t1
+    mn, amn = t1.min(axis=3), t1.argmin(axis=3)
+    mx, amx = t2.max(axis=3), t2.argmax(axis=3)
+    idx = codes = None
+    if mode in ("compound", "parallel"):
+        acc = np.zeros((N, K, OH, OW), np.float32)
+        for c in range(C):
+            a = np.broadcast_to(t["alpha"][None, :, c, None, None], acc.shape)
+            b = np.broadcast_to(t["beta"][None, :, c, None, None], acc.shape)
+            acc = unfold_ref.fmaf32(a, mn[:, :, c], acc)
+            acc = unfold_ref.fmaf32(b, mx[:, :, c], acc)
+        codes = (amn | (amx << 4)).astype(np.uint8)
+    else:
+        m, am = (mn, amn) if mode == "min_plus" else (mx, amx)
+        if chan == "sum":
+            acc = np.zeros((N, K, OH, OW), np.float32)
+            for c in range(C):
+                acc = acc + m[:, :, c]                          # float32 adds, channel order
+            codes = (am if mode == "min_plus" else (am << 4)).astype(np.uint8)
+        else:
+            cs = m.argmax(axis=2) if chan == "max" else m.argmin(axis=2)
+            acc = np.take_along_axis(m, cs[:, :, None], axis=2)[:, :, 0]
+            tap = np.take_along_axis(am, cs[:, :, None], axis=2)[:, :, 0]
+            idx = (cs * (R * S) + tap).astype(np.int32)
+    acc = acc.astype(np.float32) + t["bias"].astype(np.float32)[None, :, None, None]
+    y = torch.from_numpy(np.ascontiguousarray(acc, np.float32)).to(torch.bfloat16).float().numpy()
+    return y, idx, codes
+
+
+@pytest.mark.parametrize("mode,chan", ALL_MODES)
+def test_p1_bf16_matches_unfold_formulation(mode, chan):
+    """bf16 layers: output bits and winners equal the unfold formulation built from torch's
+    bf16 addition and numpy's reductions, on random inputs (rounded tap sums collide often in
+    bf16, so ties already occur) and on small integers (ties everywhere)."""
+    cases = [dict(), dict(x=("ints", -3, 3), w=("ints", -2, 2), ab=("dyadic", 1, 1), bias=("dyadic", 4, 1))]
+    for ci, dist in enumerate(cases):
+        for gi, (s, p, dl) in enumerate([(1, 1, 1), (2, 0, 1), (1, 2, 2), (2, 1, 2)]):
+            d = inputs.layer(2, 5, 9, 8, 4, 3, 3, stride=s, pad=p, dil=dl, mode=mode, chan=chan, dtype="bf16")
+            if min(inputs.output_hw(d)) <= 0:
+                continue
+            t = inputs.draw(d, 150 + 10 * ci + gi, **dist)
+            o = run_fwd(d, t)
+            y, idx, codes = _bf16_unfold_forward(d, t)
+            assert same_bits(o["y"], y), (mode, chan, dist, s, p, dl)
+            if idx is not None:
+                assert np.array_equal(o["idx"], idx)
+            else:
+                mask = 0xFF if mode in ("compound", "parallel") else (0x0F if mode == "min_plus" else 0xF0)
+                assert np.array_equal(o["codes"] & mask, codes & mask)
+            if ci == 0 and gi == 0:
+                # the random case must really contain bf16 ties (else the winner check is idle)
+                t1 = torch.from_numpy(unfold_ref.unfold(dict(d, dtype="f32"), t["x"])).to(torch.bfloat16)[:, None] \
+                    + torch.from_numpy(t["w"]).to(torch.bfloat16).reshape(1, d["K"], d["C"], 9, 1, 1)
+                t1 = t1.float().numpy()
+                ext = t1.min(axis=3, keepdims=True) if mode != "max_plus" else t1.max(axis=3, keepdims=True)
+                assert ((t1 == ext).sum(axis=3) > 1).any()
+
+
 def test_output_shape_follows_pytorch_convention():
     for (H, W, R, S, s, p, dl) in itertools.product((7, 10), (8,), (1, 3), (2, 3), (1, 2, 3), (0, 1, 2), (1, 2)):
         d = inputs.layer(1, 1, H, W, 1, R, S, stride=s, pad=p, dil=dl)
