@@ -44,6 +44,11 @@ PROBES = {"max_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
           "min_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
           "compound": ("f32_add_minmax2", "f32_add_minmax3", "f32_add2_minmax3"),
           "parallel": ("f32_2add_minmax2", "f32_2add_minmax3", "f32_2add2_minmax3")}
+# the same for the bf16 kernels: tap sums by add, by fma(x, 1, w), or the two alternating
+PROBES_BF16 = {"max_plus": ("bf16x2_add_max", "bf16x2_fma_max", "bf16x2_mix_max"),
+               "min_plus": ("bf16x2_add_max", "bf16x2_fma_max", "bf16x2_mix_max"),
+               "compound": ("bf16x2_add_minmax", "bf16x2_fma_minmax", "bf16x2_mix_minmax"),
+               "parallel": ("bf16x2_2add_minmax", "bf16x2_2fma_minmax", "bf16x2_2mix_minmax")}
 # register-only probes of the winner-emitting Sum-form inner loop (sums, extrema, FMA keys, key fold)
 WIN_PROBES = {"compound": "f32_win_compound", "parallel": "f32_win_parallel"}
 
@@ -166,14 +171,18 @@ def run_reference(args):
 class Layer:
     """Device-resident tensors of one layer plus its outputs, allocated once."""
 
-    def __init__(self, mode, chan, seed, torch, tconv, inputs, dev, n_images=128, dtype="f32"):
-        self.d, dist = inputs.cfg2(mode, chan, N=n_images)
+    def __init__(self, mode, chan, seed, torch, tconv, inputs, dev, n_images=128, dtype="f32", desc=None,
+                 e2e=True):
+        self.d, dist = desc if desc is not None else inputs.cfg2(mode, chan, N=n_images)
         self.d = dict(self.d, dtype=dtype)
         d = self.d
+        mode = d["mode"]
         t = inputs.draw(d, seed, **dist)
         dt = tconv.TORCH_DTYPE[dtype]
-        self.host = {k: torch.from_numpy(v).to(dt if k in ("x", "w", "w2", "g") else torch.float32).pin_memory()
+        self.host = {k: torch.from_numpy(v).to(dt if k in ("x", "w", "w2", "g") else torch.float32)
                      for k, v in t.items()}
+        if e2e:
+            self.host = {k: v.pin_memory() for k, v in self.host.items()}
         self.two = mode in ("compound", "parallel")
         self.par = mode == "parallel"
         self.dev = {k: v.to(dev, non_blocking=True) for k, v in self.host.items()}
@@ -192,12 +201,14 @@ class Layer:
         self.ops = 2 * tconv.tconv_paper_ops(d)
         self.taps = N * K * OH * OW * C * 9
         self.tconv = tconv
+        self.ev_done = self.ev_out = None   # last kernels / last device-to-host copies of the e2e leg
+        if not e2e:
+            return
         # pinned host landing buffers of the end-to-end leg
         self.h_y = torch.empty((N, K, OH, OW), dtype=dt).pin_memory()
         self.h_gx = torch.empty((N, C, H, W), dtype=dt).pin_memory()
         self.h_small = {k: torch.empty_like(getattr(self, k), device="cpu").pin_memory()
                         for k in ("gw", "gw2", "ga", "gb", "gbias") if getattr(self, k) is not None}
-        self.ev_done = self.ev_out = None   # last kernels / last device-to-host copies of the e2e leg
 
     def fwd(self, with_winners=True):
         v = self.dev
@@ -256,7 +267,11 @@ class Layer:
 
 
 def measure_alu_peak(torch, tconv):
-    """Best measured taps/s over the candidate instruction mixes, per mode."""
+    """Best measured taps/s over the candidate instruction mixes, per mode, for fp32 and for bf16.
+    Every mix runs in two forms: with a few extra adds per iteration that advance its operands
+    (8 % of a max-plus probe's instructions, left uncorrected) and with the operands advanced by
+    feeding tap sums back (no extra instruction); the better of the two counts.  Returns (peaks
+    fp32, peaks bf16, rates)."""
     sink = torch.zeros(4, device="cuda")
     names, i = {}, 0
     while tconv.tconv_alu_probe_name(i) is not None:
@@ -274,7 +289,45 @@ def measure_alu_peak(torch, tconv):
             r = taps / (e0.elapsed_time(e1) * 1e-3)
             best = r if best is None else max(best, r)
         rate[name] = best
-    return {m: max(rate[p] for p in ps) for m, ps in PROBES.items()}, rate
+    # every mix in both forms: operands advanced by extra adds, or by feeding tap sums back ("_fb")
+    both = lambda ps: [rate[p] for p in ps] + [rate[p + "_fb"] for p in ps]
+    peaks = {m: max(both(ps)) for m, ps in PROBES.items()}
+    peaks16 = {m: max(both(ps)) for m, ps in PROBES_BF16.items()}
+    return peaks, peaks16, rate
+
+
+# headline layers of the benchmark spec's target outside the bench step: (name, inputs.<cfg>, dtype)
+HEADLINE = [("cfg3a parallel f32", "cfg3a", "f32"), ("cfg3a parallel bf16", "cfg3a", "bf16"),
+            ("cfg3b parallel f32", "cfg3b", "f32"), ("cfg3b parallel bf16", "cfg3b", "bf16"),
+            ("cfg4 compound bf16", "cfg4", "bf16")]
+
+
+def time_headline_layers(torch, tconv, inputs, dev, peaks, peaks16):
+    """Winner-free forward (ms, Ttap/s, fraction of the mode's measured add+max/min peak), forward
+    with winners and full backward of the other headline layers, 5 repeats each (median)."""
+    out = {}
+    for name, cfg, dtype in HEADLINE:
+        d, dist = getattr(inputs, cfg)(dtype)
+        L = Layer(None, None, 1030, torch, tconv, inputs, dev, dtype=dtype, desc=(d, dist), e2e=False)
+        rec = {}
+        for what, fn in (("fwd", lambda: L.fwd(False)), ("fwd_winners", L.fwd), ("bwd", L.bwd)):
+            fn()
+            ts = []
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record(); torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            rec[what + "_ms"] = float(np.median(ts))
+            rec[what + "_kernel"] = tconv.tconv_last_kernel()
+        pk = (peaks if dtype == "f32" else peaks16)[d["mode"]]
+        rec["taps"] = L.taps
+        rec["fwd_Ttap_s"] = L.taps / (rec["fwd_ms"] * 1e-3) / 1e12
+        rec["fwd_frac_of_alu_peak"] = L.taps / (rec["fwd_ms"] * 1e-3) / pk
+        rec["alu_peak_Ttap_s"] = pk / 1e12
+        out[name] = rec
+        del L
+        torch.cuda.empty_cache()
+    return out
 
 
 def max_over_ranks(torch, dist, values, device, world):
@@ -375,7 +428,8 @@ def run_gpu(args):
             rec[what] = float(np.median(ts))
             rec[what + "_kernel"] = tconv.tconv_last_kernel()
         per[L.d["mode"]] = rec
-    peaks, probe_rates = measure_alu_peak(torch, tconv)
+    peaks, peaks16, probe_rates = measure_alu_peak(torch, tconv)
+    headline = time_headline_layers(torch, tconv, inputs, dev, peaks, peaks16) if (rank == 0 and not args.no_headline) else None
 
     ms, ms_e2e = max_over_ranks(torch, dist, [ms, ms_e2e], dev, world)
     if rank != 0:
@@ -393,20 +447,18 @@ def run_gpu(args):
                              key=lambda mw: per[mw[0]][mw[1]])
     L = next(x for x in layers if x.d["mode"] == dom_mode)
     achieved = L.taps / (per[dom_mode][dom_what] * 1e-3) / 1e12
-    win_mix = dom_what == "fwd_winners" and dom_mode in WIN_PROBES
-    peak = probe_rates[WIN_PROBES[dom_mode]] if win_mix else peaks[dom_mode]
     roofline = {"bound": "alu", "kernel": per[dom_mode][dom_what + "_kernel"], "call": f"{dom_mode} {dom_what}",
-                "achieved": achieved, "peak": peak / 1e12, "unit": "Ttap/s",
-                "frac": achieved / (peak / 1e12),
+                "achieved": achieved, "peak": peaks[dom_mode] / 1e12, "unit": "Ttap/s",
+                "frac": achieved / (peaks[dom_mode] / 1e12),
                 "traffic": DRAM_BYTES_FULL.get((dom_mode, dom_what)),
                 "traffic_note": "DRAM bytes per launch, one-pass ncu capture at this size (profiles/dram_traffic_cfg2_n128.md)",
-                "peak_source": ("measured in this run: register-only probe of the winner-emitting inner loop of "
-                                "the mode (tap sums, extrema, two fused multiply-adds per tap and branch for "
-                                "the winner keys, key fold)" if win_mix else
-                                "measured in this run: best register-only add+max/min probe of the mode "
-                                "(taps/s of the winner-free instruction mix; a backward kernel does other "
-                                "work per tap than that mix)"),
-                "frac_of_winner_free_peak": achieved / (peaks[dom_mode] / 1e12)}
+                "peak_source": ("measured in this run: best register-only add+max/min probe of the mode (taps/s "
+                                "of the winner-free instruction mix, 1 add + 1-2 compares per tap); winner emission "
+                                "and the backward do other work per tap than that mix and are held to the same "
+                                "denominator")}
+    if dom_what == "fwd_winners" and dom_mode in WIN_PROBES:
+        # secondary: against a register-only replay of the kernel's own winner-emitting loop
+        roofline["frac_of_own_mix"] = achieved / (probe_rates[WIN_PROBES[dom_mode]] / 1e12)
     fwd_frac = {m: {"ms": per[m]["fwd"], "Ttap_s": L2.taps / (per[m]["fwd"] * 1e-3) / 1e12,
                     "frac_of_alu_peak": L2.taps / (per[m]["fwd"] * 1e-3) / peaks[m],
                     "kernel": per[m]["fwd_kernel"]}
@@ -431,8 +483,13 @@ def run_gpu(args):
                     "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu,
-            "per_mode_ms": per, "forward_vs_alu_peak": fwd_frac,
-            "alu_probe_Ttap_s": {k: v / 1e12 for k, v in probe_rates.items()}}
+            "per_mode_ms": per, "forward_vs_alu_peak": fwd_frac, "headline_layers": headline,
+            "alu_peak_Ttap_s": {"f32": {m: v / 1e12 for m, v in peaks.items()},
+                                "bf16": {m: v / 1e12 for m, v in peaks16.items()}},
+            "alu_probe_Ttap_s": {k: v / 1e12 for k, v in probe_rates.items()},
+            "alu_probe_note": ("register-only loops; plain names advance their operands with extra adds (5 per 64 "
+                               "taps, uncorrected), _fb names feed tap sums back (no extra instruction); a mode's "
+                               "peak is the best of all its mixes in both forms")}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -632,6 +689,8 @@ def main():
     ap.add_argument("--what", default="fwd", choices=["fwd", "fwd_winners", "bwd"])
     ap.add_argument("--images", type=int, default=128)
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
+    ap.add_argument("--no-headline", action="store_true",
+                    help="skip the headline_layers section (cfg 3a / 3b / 4 timed after the step)")
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5", "dw", "conv3d"],
                     help="cfg5: report the hybrid ResNet-18 training step instead (use --only compound|parallel); "
                          "dw: a depthwise (groups = C) layer against the HBM roofline; conv3d: the 3-D LeNet layers")

@@ -1,11 +1,14 @@
 // Register-only throughput probes of the add + max/min instruction mixes the
 // tropical kernels can be built from.  Each thread keeps a TK x TP block of
 // running extrema and folds taps x[j] + w[i] into them, exactly the inner loop of
-// the forward pass minus its memory traffic.  The x operands are advanced by a
-// real add in every iteration (TP + 1 extra adds per TK * TP * 2 taps): an empty
-// asm barrier is not enough, because the assembler, which never sees it, would
-// hoist the loop-invariant tap sums out of the loop and the probe would measure
-// min/max alone.
+// the forward pass minus its memory traffic.  The x operands must change from one
+// iteration to the next (an empty asm barrier is not enough: the assembler, which
+// never sees it, would hoist the loop-invariant tap sums out of the loop and the
+// probe would measure min/max alone).  Two ways, both built (template flag FEED),
+// and the caller takes the better rate: advancing adds (TP + 1 extra adds per
+// TK * TP * 2 taps, left uncorrected), or feedback: TP + 1 of the tap sums an
+// iteration forms anyway become the next iteration's x operands, so that every
+// instruction of the loop body is a tap sum or a min / max.
 #pragma once
 #include "tconv_common.cuh"
 
@@ -44,6 +47,9 @@ __device__ __forceinline__ void add2f(float x, float wlo, float whi, float& lo, 
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(tt));
 }
 
+#define TCONV_OPAQUE_F(v) asm volatile("" : "+f"(v))
+#define TCONV_OPAQUE_R(v) asm volatile("" : "+r"(v))
+
 enum {
     PROBE_F32_ADD_MAX2 = 0,      // max-plus / min-plus: add, 2-input max
     PROBE_F32_ADD_MAX3,          // two adds feed one 3-input max
@@ -63,6 +69,12 @@ enum {
     PROBE_F32_WIN_SINGLE,        // Sum form with winners, one branch: sums, extremum, FMA keys, key fold
     PROBE_F32_WIN_COMPOUND,      // the same for compound (shared sums, two branches)
     PROBE_F32_WIN_PARALLEL,      // the same for parallel (two sets of sums)
+    PROBE_BF16X2_FMA_MAX,        // bf16 pairs, every tap sum as fma(x, 1, w) (same rounding, the other pipe)
+    PROBE_BF16X2_FMA_MINMAX,
+    PROBE_BF16X2_2FMA_MINMAX,
+    PROBE_BF16X2_MIX_MAX,        // bf16 pairs, tap sums alternate between add and fma(x, 1, w)
+    PROBE_BF16X2_MIX_MINMAX,
+    PROBE_BF16X2_2MIX_MINMAX,
     PROBE_COUNT
 };
 
@@ -71,14 +83,18 @@ static const char* const kProbeNames[PROBE_COUNT] = {
     "f32_add_minmax3",    "f32_add2_minmax3",  "f32_2add_minmax2", "f32_2add_minmax3",
     "f32_2add2_minmax3",  "bf16x2_add_max",    "bf16x2_add_minmax", "bf16x2_2add_minmax",
     "f32_add_only",       "f32_max2_only",     "f32_max3_only",   "f32_win_single",
-    "f32_win_compound",   "f32_win_parallel"};
+    "f32_win_compound",   "f32_win_parallel",  "bf16x2_fma_max",  "bf16x2_fma_minmax",
+    "bf16x2_2fma_minmax", "bf16x2_mix_max",    "bf16x2_mix_minmax", "bf16x2_2mix_minmax"};
+
+__host__ __device__ constexpr bool probe_is_bf16(int v) {
+    return (v >= PROBE_BF16X2_ADD_MAX && v <= PROBE_BF16X2_2ADD_MINMAX) ||
+           (v >= PROBE_BF16X2_FMA_MAX && v <= PROBE_BF16X2_2MIX_MINMAX);
+}
 
 // Taps folded per thread per loop iteration, by variant (must match the kernel).
 __host__ inline int probe_taps_per_iter(int v) {
+    if (probe_is_bf16(v)) return 4 * 8 * 2 * 2;               // 4 channel pairs x 8 pixels x 2 lanes x 2 taps
     switch (v) {
-        case PROBE_BF16X2_ADD_MAX:
-        case PROBE_BF16X2_ADD_MINMAX:
-        case PROBE_BF16X2_2ADD_MINMAX: return 4 * 8 * 2 * 2;  // 4 channel pairs x 8 pixels x 2 lanes x 2 taps
         case PROBE_F32_WIN_SINGLE:
         case PROBE_F32_WIN_COMPOUND:
         case PROBE_F32_WIN_PARALLEL: return 4 * 4 * 9;        // 4 channels x 4 pixels x a 3x3 window
@@ -86,18 +102,23 @@ __host__ inline int probe_taps_per_iter(int v) {
     }
 }
 
-#define TCONV_OPAQUE_F(v) asm volatile("" : "+f"(v))
-#define TCONV_OPAQUE_R(v) asm volatile("" : "+r"(v))
-
-template <int V>
+template <int V, bool FEED>
 __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, float* sink) {
     constexpr int TK = 8, TP = 4;
-    if constexpr (V >= PROBE_BF16X2_ADD_MAX && V <= PROBE_BF16X2_2ADD_MINMAX) {
-        // packed bf16 pairs: a register holds two output channels
+    if constexpr (probe_is_bf16(V)) {
+        // packed bf16 pairs: a register holds two tap sums.  Three ways to form a tap sum with one
+        // bf16 rounding: add.bf16x2, fma.bf16x2(x, 1, w) (the multiply by one is exact, so the
+        // result is the same; it issues to the fused-multiply-add pipe), or the two alternating;
+        // min / max are nested in pairs so that the assembler may fuse them into 3-input forms.
         constexpr int KP = 4, PX = 8;
+        constexpr int KIND = (V >= PROBE_BF16X2_MIX_MAX) ? 2 : (V >= PROBE_BF16X2_FMA_MAX) ? 1 : 0;   // 0 add, 1 fma, 2 mix
+        constexpr int BASE = KIND == 2 ? PROBE_BF16X2_MIX_MAX : KIND == 1 ? PROBE_BF16X2_FMA_MAX : PROBE_BF16X2_ADD_MAX;
+        constexpr int SHAPE = V - BASE;                                // 0 max, 1 min + max, 2 parallel
         __nv_bfloat162 x[PX + 1], wa[KP], wb[KP], va[KP], vb[KP];
         __nv_bfloat162 mn[KP][PX], mx[KP][PX];
         const __nv_bfloat162 dx2 = __float2bfloat162_rn(seed * 0.0078125f);
+        __nv_bfloat162 one2 = __float2bfloat162_rn(1.0f);
+        TCONV_OPAQUE_R(*reinterpret_cast<unsigned*>(&one2));
         for (int j = 0; j <= PX; ++j) x[j] = __float2bfloat162_rn(seed * (float)(j + threadIdx.x));
         for (int i = 0; i < KP; ++i) {
             wa[i] = __float2bfloat162_rn(seed * (float)(i + 3));
@@ -106,9 +127,16 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
             vb[i] = __float2bfloat162_rn(seed * (float)(i + 9));
             for (int j = 0; j < PX; ++j) { mn[i][j] = x[j]; mx[i][j] = x[j]; }
         }
+        auto tap = [&](const __nv_bfloat162& xv, const __nv_bfloat162& wv, bool second) {
+            if (KIND == 1 || (KIND == 2 && second)) return __hfma2(xv, one2, wv);
+            return __hadd2(xv, wv);
+        };
         for (int it = 0; it < iters; ++it) {
+            __nv_bfloat162 xn[PX + 1];                                  // next iteration's operands
+            if constexpr (!FEED) {
 #pragma unroll
-            for (int j = 0; j <= PX; ++j) x[j] = __hadd2(x[j], dx2);   // operands change every iteration
+                for (int j = 0; j <= PX; ++j) xn[j] = __hadd2(x[j], dx2);
+            }
 #pragma unroll
             for (int i = 0; i < KP; ++i) {
                 TCONV_OPAQUE_R(*reinterpret_cast<unsigned*>(&wa[i]));
@@ -120,20 +148,25 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
             for (int i = 0; i < KP; ++i)
 #pragma unroll
                 for (int j = 0; j < PX; ++j) {
-                    const __nv_bfloat162 t0 = __hadd2(x[j], wa[i]);
-                    const __nv_bfloat162 t1 = __hadd2(x[j + 1], wb[i]);
-                    if constexpr (V == PROBE_BF16X2_ADD_MAX) {
+                    const __nv_bfloat162 t0 = tap(x[j], wa[i], false);
+                    const __nv_bfloat162 t1 = tap(x[j + 1], wb[i], true);
+                    if constexpr (FEED) {
+                        if (i == 0) { xn[j] = t0; if (j == PX - 1) xn[PX] = t1; }
+                    }
+                    if constexpr (SHAPE == 0) {
                         mx[i][j] = __hmax2(__hmax2(mx[i][j], t0), t1);
-                    } else if constexpr (V == PROBE_BF16X2_ADD_MINMAX) {
+                    } else if constexpr (SHAPE == 1) {
                         mx[i][j] = __hmax2(__hmax2(mx[i][j], t0), t1);
                         mn[i][j] = __hmin2(__hmin2(mn[i][j], t0), t1);
                     } else {
-                        const __nv_bfloat162 u0 = __hadd2(x[j], va[i]);
-                        const __nv_bfloat162 u1 = __hadd2(x[j + 1], vb[i]);
+                        const __nv_bfloat162 u0 = tap(x[j], va[i], true);
+                        const __nv_bfloat162 u1 = tap(x[j + 1], vb[i], false);
                         mx[i][j] = __hmax2(__hmax2(mx[i][j], u0), u1);
                         mn[i][j] = __hmin2(__hmin2(mn[i][j], t0), t1);
                     }
                 }
+#pragma unroll
+            for (int j = 0; j <= PX; ++j) x[j] = xn[j];
         }
         __nv_bfloat162 r = mx[0][0];
         for (int i = 0; i < KP; ++i)
@@ -241,8 +274,12 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
             for (int j = 0; j < TP; ++j) { mn[i][j] = x[j]; mx[i][j] = x[j]; }
         }
         for (int it = 0; it < iters; ++it) {
+            constexpr bool no_adds = (V == PROBE_F32_MAX2_ONLY || V == PROBE_F32_MAX3_ONLY);
+            float xn[TP + 1];                                            // next iteration's operands
+            if constexpr (no_adds || !FEED) {
 #pragma unroll
-            for (int j = 0; j <= TP; ++j) x[j] = __fadd_rn(x[j], dx);    // operands change every iteration
+                for (int j = 0; j <= TP; ++j) xn[j] = __fadd_rn(x[j], dx);
+            }
 #pragma unroll
             for (int i = 0; i < TK; ++i) {
                 TCONV_OPAQUE_F(w0[i]); TCONV_OPAQUE_F(w1[i]);
@@ -279,6 +316,9 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
                     } else {
                         ua0 = ta0; ub0 = tb0; ua1 = ta1; ub1 = tb1;
                     }
+                    if constexpr (!no_adds && FEED) {
+                        if (i == 0) { xn[j] = ta0; if (j == TP - 1) xn[TP] = ta1; }
+                    }
                     if constexpr (V == PROBE_F32_ADD_ONLY) {
                         mx[i][j] += ta0 + ta1;          // 4 adds per 2 taps: an upper bound
                         mx[i + 1][j] += tb0 + tb1;      // on what the FP32 pipe sustains
@@ -301,6 +341,8 @@ __global__ void __launch_bounds__(256) alu_probe_kernel(int iters, float seed, f
                         mn[i + 1][j] = min3f(mn[i + 1][j], tb0, tb1);
                     }
                 }
+#pragma unroll
+            for (int j = 0; j <= TP; ++j) x[j] = xn[j];
         }
         float r = 0.0f;
         for (int i = 0; i < TK; ++i)

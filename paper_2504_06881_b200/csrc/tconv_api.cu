@@ -735,7 +735,10 @@ int tconv_dw_backward(const tconv_desc_t* desc, const void* x, const void* w, co
 }
 
 int tconv_alu_probe(int variant, int iters, void* sink, double* taps_per_launch, void* stream) {
-    if (variant < 0 || variant >= PROBE_COUNT || iters <= 0 || !sink) return TCONV_ERR_INVALID_ARG;
+    // variants PROBE_COUNT .. 2 * PROBE_COUNT - 1: the same mixes with operand feedback
+    if (variant < 0 || variant >= 2 * PROBE_COUNT || iters <= 0 || !sink) return TCONV_ERR_INVALID_ARG;
+    const bool feed = variant >= PROBE_COUNT;
+    const int mix = feed ? variant - PROBE_COUNT : variant;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -744,33 +747,33 @@ int tconv_alu_probe(int variant, int iters, void* sink, double* taps_per_launch,
     const unsigned blocks = (unsigned)sms * 8u;
     cudaStream_t st = (cudaStream_t)stream;
     const float seed = 1.0009765625f;
-    // debug switch: dynamic shared memory per block, to limit the resident blocks per SM
-    static const size_t probe_smem = [] {
-        const char* e = getenv("TCONV_PROBE_SMEM");
-        return e ? (size_t)atol(e) : (size_t)0;
-    }();
 #define TCONV_PROBE_CASE(V)                                                                          \
     case V:                                                                                          \
-        if (probe_smem) cudaFuncSetAttribute(alu_probe_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)probe_smem); \
-        alu_probe_kernel<V><<<blocks, 256, probe_smem, st>>>(iters, seed, (float*)sink);             \
+        if (feed) alu_probe_kernel<V, true><<<blocks, 256, 0, st>>>(iters, seed, (float*)sink);      \
+        else alu_probe_kernel<V, false><<<blocks, 256, 0, st>>>(iters, seed, (float*)sink);          \
         break;
-    switch (variant) {
+    switch (mix) {
         TCONV_PROBE_CASE(0) TCONV_PROBE_CASE(1) TCONV_PROBE_CASE(2) TCONV_PROBE_CASE(3)
         TCONV_PROBE_CASE(4) TCONV_PROBE_CASE(5) TCONV_PROBE_CASE(6) TCONV_PROBE_CASE(7)
         TCONV_PROBE_CASE(8) TCONV_PROBE_CASE(9) TCONV_PROBE_CASE(10) TCONV_PROBE_CASE(11)
         TCONV_PROBE_CASE(12) TCONV_PROBE_CASE(13) TCONV_PROBE_CASE(14) TCONV_PROBE_CASE(15)
-        TCONV_PROBE_CASE(16) TCONV_PROBE_CASE(17)
+        TCONV_PROBE_CASE(16) TCONV_PROBE_CASE(17) TCONV_PROBE_CASE(18) TCONV_PROBE_CASE(19)
+        TCONV_PROBE_CASE(20) TCONV_PROBE_CASE(21) TCONV_PROBE_CASE(22) TCONV_PROBE_CASE(23)
     }
 #undef TCONV_PROBE_CASE
+    static_assert(PROBE_COUNT == 24, "one case per probe variant");
     g_launches += 1;
     if (taps_per_launch)
-        *taps_per_launch = (double)blocks * 256.0 * iters * probe_taps_per_iter(variant);
+        *taps_per_launch = (double)blocks * 256.0 * iters * probe_taps_per_iter(mix);
     return check_launch();
 }
 
 const char* tconv_alu_probe_name(int variant) {
-    if (variant < 0 || variant >= PROBE_COUNT) return nullptr;
-    return kProbeNames[variant];
+    static char names[2 * PROBE_COUNT][40];
+    if (variant < 0 || variant >= 2 * PROBE_COUNT) return nullptr;
+    if (variant < PROBE_COUNT) return kProbeNames[variant];
+    snprintf(names[variant], sizeof(names[variant]), "%s_fb", kProbeNames[variant - PROBE_COUNT]);
+    return names[variant];
 }
 
 const char* tconv_status_string(int status) {
