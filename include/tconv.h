@@ -7,10 +7,10 @@
  *     R x S window of x[n, c, ih, iw] + w[k, c, r, s];
  *   - the six TCNN layers (i)-(vi), Section 3.1: Sum, Max or Min of the base
  *     operator over the input channels c;
- *   - the compound layer, Section 3.4:
+ *   - the compound layer, section "Compound tropical convolution layers":
  *       y = sum_c ( alpha[k,c] * MinPlus2d(x, w) + beta[k,c] * MaxPlus2d(x, w) ),
  *     both branches sharing one addition per tap;
- *   - the parallel layer, Section 3.5: the same with w in the min branch and
+ *   - the parallel layer, section "Parallel tropical convolution layers": the same with w in the min branch and
  *     w2 in the max branch;
  *   - backward: the upstream gradient is routed wholly to the winning tap(s).
  *
@@ -32,7 +32,11 @@
  *
  * Every function that returns int returns TCONV_OK (0) or a negative
  * tconv_status_t; nothing throws, aborts or prints.  Non-finite inputs are
- * outside the contract.  There is no CPU implementation behind this interface.
+ * outside the contract.  Winner codes of the fp32 Sum forms (incl. compound and
+ * parallel) are recovered from scaled differences of tap sums: they are exact for
+ * |x + w| < 2^95 (windows of up to 16 taps) and |x + w| < 2^86 (larger windows);
+ * beyond that the outputs y are still exact but winners may be wrong.  There is no
+ * CPU implementation behind this interface.
  */
 #ifndef TCONV_H
 #define TCONV_H
@@ -47,8 +51,8 @@ extern "C" {
 typedef enum {
     TCONV_MAX_PLUS = 0, /* MaxPlus2d base operator (Section 3.1)            */
     TCONV_MIN_PLUS = 1, /* MinPlus2d base operator (Section 3.1)            */
-    TCONV_COMPOUND = 2, /* compound layer, Section 3.4 (Sum over channels)  */
-    TCONV_PARALLEL = 3  /* parallel layer, Section 3.5 (Sum over channels)  */
+    TCONV_COMPOUND = 2, /* compound layer (CompoundMinMaxPlusSumConv2d2p), Sum over channels */
+    TCONV_PARALLEL = 3  /* parallel layer (ParallelMinMaxPlusSumConv2d2p), Sum over channels */
 } tconv_mode_t;
 
 typedef enum {
@@ -113,7 +117,8 @@ size_t tconv_winner_bytes(const tconv_desc_t *desc);
 size_t tconv_workspace_bytes(const tconv_desc_t *desc, int backward);
 
 /*
- * Forward pass of one layer (Sections 3.1, 3.4, 3.5).
+ * Forward pass of one layer (sections "Tropical algebra and tropical convolution", "Compound tropical convolution layers",
+ * "Parallel tropical convolution layers").
  *   x, w        inputs and weights (dtype of the descriptor).
  *   w2          max-branch weights, parallel mode only; NULL otherwise.
  *   alpha, beta fp32 [K][C], compound / parallel only; NULL means all ones

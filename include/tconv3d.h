@@ -4,9 +4,9 @@
  * The operations are the three-dimensional extension of the paper's Section 3.2 (base operators
  * MinPlus3d / MaxPlus3d: min / max over the T x R x S window of x + w, and the six Conv3d
  * layers (i)-(vi) that take Sum, Max or Min of a base operator over the input channels) and the
- * Conv3d forms of the compound layer (Section 3.4: sum over c of alpha * MinPlus3d + beta *
+ * Conv3d forms of the compound layer (section "Compound tropical convolution layers": sum over c of alpha * MinPlus3d + beta *
  * MaxPlus3d of one weight, the two branches sharing each addition) and of the parallel layer
- * (Section 3.5: weight w in the min branch, w2 in the max branch).
+ * (section "Parallel tropical convolution layers": weight w in the min branch, w2 in the max branch).
  *
  * Conventions (the same as tconv.h, which provides the enums and status codes used here):
  *   - every pointer is a DEVICE pointer unless stated; descriptors and sizes live on the host;

@@ -7,9 +7,9 @@
  *   - base operators MinPlus3d / MaxPlus3d (Section 3.2): min / max over the three-dimensional
  *     window of X[position + offset, c_in] + W[offset, c_in, c_out];
  *   - the six Conv3d layers (i)-(vi) of Section 3.2: Sum, Max or Min of a base operator over c_in;
- *   - CompoundMinPlusSumConv3d2p (Section 3.4): sum over c_in of alpha * MinPlus3d + beta *
+ *   - CompoundMinPlusSumConv3d2p (section "Compound tropical convolution layers"): sum over c_in of alpha * MinPlus3d + beta *
  *     MaxPlus3d of the same weight (one shared addition per tap);
- *   - ParallelMinPlusSumConv3d2p (Section 3.5): the same with W1 in the min branch and W2 in
+ *   - ParallelMinPlusSumConv3d2p (section "Parallel tropical convolution layers"): the same with W1 in the min branch and W2 in
  *     the max branch.
  *
  * Readings (the same as for the two-dimensional oracle): zero padding takes part in min/max as

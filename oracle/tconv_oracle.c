@@ -7,10 +7,12 @@
  *     Kh x Kw window of X[h+i, w+j, c_in] + W[i, j, c_in, c_out];
  *   - the six TCNN layers (i)-(vi) of Section 3.1: Sum, Max or Min of the base
  *     operator over c_in;
- *   - the compound layer (Section 3.4, CompoundMinPlusSumConv2d2p):
+ *   - the compound layer (section "Compound tropical convolution layers",
+ *     CompoundMinPlusSumConv2d2p):
  *       Y = sum_c ( alpha[c,k] * MinPlus2d(X,W) + beta[c,k] * MaxPlus2d(X,W) ),
- *     where both branches share the same addition (remark closing Section 3.4);
- *   - the parallel layer (Section 3.5, ParallelMinPlusSumConv2d2p): the same
+ *     where both branches share the same addition (remark closing that section);
+ *   - the parallel layer (section "Parallel tropical convolution layers",
+ *     ParallelMinPlusSumConv2d2p): the same
  *     with W1 in the min branch and W2 in the max branch;
  *   - the operation counts of Section 4.1 (instrumented counters).
  *
@@ -22,6 +24,12 @@
  * last; alpha/beta stored [K][C]; the backward pass routes the upstream
  * gradient wholly to the winner.  Parity unpinned by the paper: padding value,
  * gradient tie rule, alpha/beta memory layout, bias placement.
+ *
+ * Second padding reading (pad_mode = 1, "neutral"): a padded tap holds the
+ * identity of the branch's semiring (+inf for min-plus, -inf for max-plus; the
+ * section "Tropical algebra and tropical convolution" gives these identities),
+ * i.e. it never takes part in the min / max: the tap is skipped.  A window that
+ * lies wholly in the padding yields the identity itself.
  *
  * Tensors are dense: x[N][C][H][W], w/w2[K][C][R][S], y/g[N][K][OH][OW],
  * alpha/beta[K][C], bias[K].  All values travel as float; in bf16 mode the
@@ -47,6 +55,7 @@ typedef struct {
     int32_t N, C, H, W, K, R, S;
     int32_t stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
     int32_t mode, chan, dtype;
+    int32_t pad_mode; /* 0: zero padding takes part as x = 0; 1: padded taps are skipped */
 } ora_desc;
 
 /* Section 4.1 tallies: additions, comparisons, multiplications. */
@@ -146,6 +155,8 @@ static ora_window base_ops(const ora_desc *d, const float *x, const float *wmin,
             float xv = 0.0f; /* zero padding */
             if (ih >= 0 && ih < d->H && iw >= 0 && iw < d->W)
                 xv = x[(((size_t)n * d->C + c) * d->H + ih) * d->W + iw];
+            else if (d->pad_mode == 1)
+                continue; /* neutral padding: the tap holds the semiring identity */
             size_t wi = (((size_t)k * d->C + c) * d->R + r) * d->S + s;
             float tmn = tap_add(xv, wmin[wi], d->dtype);
             float tmx = tmn;
@@ -207,7 +218,7 @@ int ora_forward(const ora_desc *d, const float *x, const float *w, const float *
                         ora_window o = base_ops(d, x, wmin, wmax, n, k, c, oh, ow, cnt,
                                                 want_min, want_max);
                         if (two_branch) {
-                            /* Section 3.4 / 3.5: alpha * MinPlus2d + beta * MaxPlus2d,
+                            /* compound / parallel layer definitions: alpha * MinPlus2d + beta * MaxPlus2d,
                              * min branch first, each a fused multiply-add in fp32 */
                             float a = alpha ? alpha[(size_t)k * d->C + c] : 1.0f;
                             float b = beta ? beta[(size_t)k * d->C + c] : 1.0f;

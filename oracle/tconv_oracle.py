@@ -22,12 +22,13 @@ _LIB = _HERE / "libtconv_oracle.so"
 MODES = {"max_plus": 0, "min_plus": 1, "compound": 2, "parallel": 3}
 CHANS = {"default": 0, "sum": 1, "max": 2, "min": 3}
 DTYPES = {"f32": 0, "bf16": 1}
+PAD_MODES = {"zero": 0, "neutral": 1}
 
 
 class _Desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "N", "C", "H", "W", "K", "R", "S", "stride_h", "stride_w", "pad_h", "pad_w",
-        "dil_h", "dil_w", "mode", "chan", "dtype")]
+        "dil_h", "dil_w", "mode", "chan", "dtype", "pad_mode")]
 
 
 class _Counts(ctypes.Structure):
@@ -74,7 +75,8 @@ def make_desc(N, C, H, W, K, R, S, stride=(1, 1), pad=(0, 0), dil=(1, 1),
 def _cdesc(d: dict) -> _Desc:
     return _Desc(d["N"], d["C"], d["H"], d["W"], d["K"], d["R"], d["S"], d["stride_h"],
                  d["stride_w"], d["pad_h"], d["pad_w"], d["dil_h"], d["dil_w"],
-                 MODES[d["mode"]], CHANS[d["chan"]], DTYPES[d["dtype"]])
+                 MODES[d["mode"]], CHANS[d["chan"]], DTYPES[d["dtype"]],
+                 PAD_MODES[d.get("pad_mode", "zero")])
 
 
 def output_shape(d: dict):

@@ -1,8 +1,10 @@
-"""The paper's layer names over ``TropicalConv2d`` (Section 3.1 layers (i)-(vi), Sections 3.4 / 3.5,
-Appendix "Compatibility with PyTorch"): every class takes ``nn.Conv2d``'s constructor arguments.
+"""The paper's layer names over ``TropicalConv2d`` (layers (i)-(vi) of the section "Tropical algebra
+and tropical convolution", the sections "Compound tropical convolution layers" and "Parallel
+tropical convolution layers", appendix "Compatibility with PyTorch"): every class takes
+``nn.Conv2d``'s constructor arguments.
 
-Base operator + channel combine:  MinPlusSumConv2d (ii), MaxPlusSumConv2d (i), MinPlusMaxConv2d
-(iii), MaxPlusMinConv2d (vi), MinPlusMinConv2d (iv), MaxPlusMaxConv2d (v).
+Base operator + channel combine, in the paper's numbering:  MinPlusSumConv2d (i), MaxPlusSumConv2d
+(ii), MinPlusMaxConv2d (iii), MinPlusMinConv2d (iv), MaxPlusMaxConv2d (v), MaxPlusMinConv2d (vi).
 Compound / parallel with 0, 1 (beta = 1 - alpha) or 2 learnable scalar sets per (c_out, c_in).
 """
 from __future__ import annotations
@@ -19,8 +21,8 @@ def _named(name, mode, chan="default", params="2p", doc="", base=TropicalConv2d)
     return type(name, (base,), {"__init__": __init__, "__doc__": doc})
 
 
-MaxPlusSumConv2d = _named("MaxPlusSumConv2d", "max_plus", "sum", doc="layer (i): sum over channels of the max-plus window")
-MinPlusSumConv2d = _named("MinPlusSumConv2d", "min_plus", "sum", doc="layer (ii): sum over channels of the min-plus window")
+MaxPlusSumConv2d = _named("MaxPlusSumConv2d", "max_plus", "sum", doc="layer (ii): sum over channels of the max-plus window")
+MinPlusSumConv2d = _named("MinPlusSumConv2d", "min_plus", "sum", doc="layer (i): sum over channels of the min-plus window")
 MinPlusMaxConv2d = _named("MinPlusMaxConv2d", "min_plus", "max", doc="layer (iii): max over channels of the min-plus window")
 MinPlusMinConv2d = _named("MinPlusMinConv2d", "min_plus", "min", doc="layer (iv): min over channels and window")
 MaxPlusMaxConv2d = _named("MaxPlusMaxConv2d", "max_plus", "max", doc="layer (v): max over channels and window")

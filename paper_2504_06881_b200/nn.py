@@ -83,7 +83,7 @@ class TropicalConv2d(nn.Module):
     """Tropical convolution layer with ``nn.Conv2d``'s constructor arguments.
 
     mode: "max_plus" | "min_plus" | "compound" | "parallel"; chan: "default" | "sum" | "max" | "min".
-    params (compound / parallel; the specialisations of Section 3.6): "2p" learnable alpha and beta
+    params (compound / parallel; the paper's section "Specializations of compound/parallel tropical convolutions"): "2p" learnable alpha and beta
     per (c_out, c_in); "1p" complementary weights beta = 1 - alpha; "shared" beta = alpha;
     "opposite" beta = -alpha; "0p" alpha = beta = 1 (no scalars); "fixed" the constants
     ``fixed=(alpha, beta)``, e.g. (0.5, 0.5) or (1, -1), held as buffers.

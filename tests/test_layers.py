@@ -1,5 +1,6 @@
 """The named layer set (Section 3.1 layers (i)-(vi), compound / parallel with 0p / 1p / 2p scalars,
-the alpha / beta specialisations of Section 3.6)."""
+the alpha / beta specialisations of the paper's section
+"Specializations of compound/parallel tropical convolutions")."""
 from pathlib import Path
 
 import numpy as np

@@ -231,7 +231,8 @@ def test_p8_degenerate_cases():
 # ---------------------------------------------------------------- P9
 @pytest.mark.parametrize("a,b", [(1.0, 1.0), (0.5, 0.5), (1.0, -1.0)])
 def test_p9_compound_is_combination_of_separate_outputs(a, b):
-    """Uniform alpha = a, beta = b (the fixed specialisations of Section 3.3):
+    """Uniform alpha = a, beta = b (the fixed specialisations of the section
+    "Specializations of compound/parallel tropical convolutions"):
     compound = a*MinPlusSum + b*MaxPlusSum, exactly on the dyadic grid."""
     d = inputs.layer(2, 4, 6, 6, 3, 3, 3, stride=1, pad=1, mode="compound")
     t = inputs.draw(d, 91, **DYADIC)
@@ -560,3 +561,108 @@ def test_output_shape_follows_pytorch_convention():
             continue
         ref = F.conv2d(torch.zeros(1, 1, H, W), torch.zeros(1, 1, R, S), stride=s, padding=p, dilation=dl)
         assert tuple(ref.shape[2:]) == ora.output_shape(d) == inputs.output_hw(d)
+
+
+# ---------------------------------------------------------------- neutral (identity) padding
+NEUTRAL_GEOMS = [(1, 1, 1), (2, 1, 1), (1, 2, 1), (1, 2, 2), (2, 1, 2), (1, 4, 2)]
+
+
+@pytest.mark.parametrize("mode,chan", ALL_MODES)
+def test_neutral_padding_matches_unfold_with_identity_fill(mode, chan):
+    """pad_mode "neutral": the padding holds the semiring identity (+inf in the min branch, -inf in
+    the max branch), so padded taps never win.  Output bits and winners equal the numpy unfold
+    formulation whose padding is filled with those infinities."""
+    for gi, (s, p, dl) in enumerate(NEUTRAL_GEOMS):
+        d = dict(inputs.layer(2, 3, 8, 7, 4, 3, 3, stride=s, pad=p, dil=dl, mode=mode, chan=chan),
+                 pad_mode="neutral")
+        t = inputs.draw(d, 300 + gi)
+        o = run_fwd(d, t)
+        two = mode in ("compound", "parallel")
+        y, idx, codes = unfold_ref.forward(d, t["x"], t["w"], t["w2"], t["alpha"] if two else None,
+                                           t["beta"] if two else None, t["bias"])
+        assert np.isfinite(o["y"]).all()
+        assert same_bits(o["y"], y), (mode, chan, s, p, dl)
+        if idx is not None:
+            assert np.array_equal(o["idx"], idx)
+        else:
+            mask = 0xFF if two else (0x0F if mode == "min_plus" else 0xF0)
+            assert np.array_equal(o["codes"] & mask, codes & mask)
+        # the Sum forms differ from the zero-padding reading somewhere on the border (a padded tap
+        # x = 0 wins some per-channel extremum there)
+        if chan == "sum" and gi == 0:
+            assert not same_bits(o["y"], run_fwd(dict(d, pad_mode="zero"), t)["y"])
+
+
+@pytest.mark.parametrize("stride,pad,R", [(1, 1, 3), (2, 1, 3), (1, 1, 2), (3, 1, 3)])
+def test_neutral_padding_zero_weight_is_padded_max_pooling(stride, pad, R):
+    """w = 0 with neutral padding: MaxPlus-Max is the max over channels of torch's max_pool2d with
+    the same padding (which pads with -inf); MinPlus-Min via -x."""
+    d = dict(inputs.layer(2, 3, 11, 12, 2, R, R, stride=stride, pad=pad, mode="max_plus"), pad_mode="neutral")
+    t = inputs.draw(d, 310)
+    w0 = np.zeros_like(t["w"])
+    y = ora.forward(d, t["x"], w0)["y"]
+    pooled = F.max_pool2d(torch.from_numpy(t["x"]), R, stride=stride, padding=pad).numpy()
+    assert same_bits(y, pooled.max(axis=1, keepdims=True).repeat(2, axis=1))
+    ymin = ora.forward(dict(d, mode="min_plus"), t["x"], w0)["y"]
+    pooled = -F.max_pool2d(torch.from_numpy(-t["x"]), R, stride=stride, padding=pad).numpy()
+    assert same_bits(ymin, pooled.min(axis=1, keepdims=True).repeat(2, axis=1))
+
+
+def test_neutral_padding_constant_input_sees_only_the_valid_taps():
+    """x = 0 with neutral padding: every output is the extremum of the weights of the taps that
+    lie inside the image (brute force over the window), so border outputs differ from interior
+    ones only through which taps are valid."""
+    d = dict(inputs.layer(1, 2, 5, 6, 3, 3, 3, stride=1, pad=1, mode="max_plus"), pad_mode="neutral")
+    t = inputs.draw(d, 311)
+    y = ora.forward(d, np.zeros_like(t["x"]), t["w"])["y"]
+    OH, OW = inputs.output_hw(d)
+    for k in range(3):
+        for oh in range(OH):
+            for ow in range(OW):
+                vals = [t["w"][k, c, r, s] for c in range(2) for r in range(3) for s in range(3)
+                        if 0 <= oh - 1 + r < 5 and 0 <= ow - 1 + s < 6]
+                assert y[0, k, oh, ow] == max(vals)
+
+
+@pytest.mark.parametrize("mode,chan", ALL_MODES)
+def test_neutral_padding_backward_loses_nothing_to_the_padding(mode, chan):
+    """With neutral padding every winner lies inside the image, so the whole upstream gradient
+    reaches grad_x even with pad > 0 (with zero padding the part won by padded taps does not):
+    sum(grad_x) = sum_k coefficient * grad_bias[k], exactly on dyadic inputs."""
+    d = dict(inputs.layer(2, 3, 6, 7, 4, 3, 3, stride=1, pad=1, mode=mode, chan=chan), pad_mode="neutral")
+    t = inputs.draw(d, 312, **DYADIC)
+    two = mode in ("compound", "parallel")
+    gr = ora.backward(d, t["x"], t["w"], t["g"], t["w2"] if mode == "parallel" else None,
+                      t["alpha"] if two else None, t["beta"] if two else None)
+    gb = gr["grad_bias"][0]
+    if two:
+        want = ((t["alpha"] + t["beta"]).astype(np.float64).sum(axis=1) * gb).sum()
+    elif chan == "sum":
+        want = d["C"] * gb.sum()
+    else:
+        want = gb.sum()
+    assert gr["grad_x"][0].sum() == want
+    # the zero-padding reading routes part of the gradient into the padding on these inputs
+    gz = ora.backward(dict(d, pad_mode="zero"), t["x"], t["w"], t["g"], t["w2"] if mode == "parallel" else None,
+                      t["alpha"] if two else None, t["beta"] if two else None)
+    assert not np.array_equal(gz["grad_x"][0], gr["grad_x"][0])
+
+
+def test_neutral_padding_backward_is_the_directional_derivative():
+    """Piecewise linearity with neutral padding: for tie-free inputs and a step that changes no
+    winner, the forward difference equals <grad, direction> (float64 arithmetic on the oracle's
+    float32 outputs, dyadic grid so that every operation is exact)."""
+    d = dict(inputs.layer(1, 2, 5, 5, 2, 3, 3, stride=1, pad=1, mode="compound"), pad_mode="neutral")
+    rs = np.random.RandomState(313)
+    x = (rs.permutation(50).reshape(1, 2, 5, 5) * 0.25).astype(np.float32)          # distinct, dyadic
+    w = (rs.permutation(36).reshape(2, 2, 3, 3) * 16.0).astype(np.float32)          # gaps of 16 > range of x
+    al = np.array([[0.5, 1.0], [2.0, -1.0]], np.float32); be = np.array([[1.0, 0.5], [-0.5, 2.0]], np.float32)
+    g = rs.randint(-3, 4, (1, 2, 5, 5)).astype(np.float32)
+    gr = ora.backward(d, x, w, g, None, al, be)
+    u = rs.randint(-2, 3, x.shape).astype(np.float32) * 2.0 ** -6
+    y0 = ora.forward(d, x, w, None, al, be)["y"].astype(np.float64)
+    y1 = ora.forward(d, x + u, w, None, al, be)["y"].astype(np.float64)
+    assert np.array_equal(ora.forward(d, x, w, None, al, be)["codes"], ora.forward(d, x + u, w, None, al, be)["codes"])
+    lhs = ((y1 - y0) * g).sum()
+    rhs = (gr["grad_x"][0] * u).sum()
+    assert lhs == rhs

@@ -18,11 +18,11 @@ def out_hw(d):
             ext(d["W"], d["pad_w"], d["dil_w"], d["S"], d["stride_w"]))
 
 
-def unfold(d, x):
-    """patches[N, C, R*S, OH, OW] with zero padding."""
+def unfold(d, x, fill=0.0):
+    """patches[N, C, R*S, OH, OW]; the padding holds `fill` (zero padding by default)."""
     OH, OW = out_hw(d)
     N, C, H, W, R, S = d["N"], d["C"], d["H"], d["W"], d["R"], d["S"]
-    xp = np.zeros((N, C, H + 2 * d["pad_h"], W + 2 * d["pad_w"]), x.dtype)
+    xp = np.full((N, C, H + 2 * d["pad_h"], W + 2 * d["pad_w"]), fill, x.dtype)
     xp[:, :, d["pad_h"]:d["pad_h"] + H, d["pad_w"]:d["pad_w"] + W] = x
     p = np.empty((N, C, R * S, OH, OW), x.dtype)
     for r in range(R):
@@ -46,13 +46,18 @@ def forward(d, x, w, w2=None, alpha=None, beta=None, bias=None):
     mode, chan = d["mode"], d["chan"]
     if chan == "default":
         chan = {"max_plus": "max", "min_plus": "min"}.get(mode, "sum")
-    p = unfold(d, x.astype(np.float32))                      # [N,C,RS,OH,OW]
+    neutral = d.get("pad_mode", "zero") == "neutral"
     wr = w.astype(np.float32).reshape(K, C, R * S)
-    t1 = p[:, None] + wr[None, :, :, :, None, None]          # [N,K,C,RS,OH,OW], float32 adds
-    if mode == "parallel":
-        t2 = p[:, None] + w2.astype(np.float32).reshape(K, C, R * S)[None, :, :, :, None, None]
+    wr2 = w2.astype(np.float32).reshape(K, C, R * S) if mode == "parallel" else wr
+    if not neutral:
+        p = unfold(d, x.astype(np.float32))                  # [N,C,RS,OH,OW]
+        t1 = p[:, None] + wr[None, :, :, :, None, None]      # [N,K,C,RS,OH,OW], float32 adds
+        t2 = p[:, None] + wr2[None, :, :, :, None, None] if mode == "parallel" else t1
     else:
-        t2 = t1
+        # neutral padding: the padding holds the identity of each branch's semiring, so a padded
+        # tap sum is +inf in the min branch and -inf in the max branch and never wins
+        t1 = unfold(d, x.astype(np.float32), np.inf)[:, None] + wr[None, :, :, :, None, None]
+        t2 = unfold(d, x.astype(np.float32), -np.inf)[:, None] + wr2[None, :, :, :, None, None]
     mn, amn = t1.min(axis=3), t1.argmin(axis=3)              # [N,K,C,OH,OW]
     mx, amx = t2.max(axis=3), t2.argmax(axis=3)
     idx = codes = None
