@@ -18,7 +18,10 @@
  *   - geometry follows the PyTorch convolution convention (cross-correlation,
  *     OH = floor((H + 2*pad_h - dil_h*(R-1) - 1) / stride_h) + 1, input row
  *     ih = oh*stride_h - pad_h + r*dil_h);
- *   - padding is zero padding: a padded tap takes part in min / max as x = 0;
+ *   - padding is zero padding by default: a padded tap takes part in min / max as x = 0;
+ *     with pad_mode = TCONV_PAD_NEUTRAL a padded tap holds the identity of its branch's
+ *     semiring (+inf under min, -inf under max: section "Tropical algebra and tropical
+ *     convolution"), i.e. it never wins;
  *   - ties go to the lowest flattened (c, r, s); channels are combined in
  *     ascending order, in fp32, compound/parallel as
  *       acc = fmaf(alpha, min_c, acc); acc = fmaf(beta, max_c, acc);
@@ -69,6 +72,19 @@ typedef enum {
 } tconv_dtype_t;
 
 typedef enum {
+    TCONV_PAD_ZERO = 0,   /* padded taps take part in min / max as x = 0 */
+    TCONV_PAD_NEUTRAL = 1 /* padded taps are skipped (semiring identity); every window must keep at
+                             least one tap inside the image, else TCONV_ERR_UNSUPPORTED; dense 2-D
+                             entry points only */
+} tconv_pad_mode_t;
+
+typedef enum {
+    TCONV_X_SAME = 0, /* x has the descriptor's dtype */
+    TCONV_X_F32 = 1   /* dtype = TCONV_BF16 only: x is float and is rounded to bf16 (nearest even)
+                         while it is staged, bit-identical to converting x first; grad_x stays bf16 */
+} tconv_x_dtype_t;
+
+typedef enum {
     TCONV_OK = 0,
     TCONV_ERR_INVALID_ARG = -1,         /* NULL descriptor / required pointer, non-positive size    */
     TCONV_ERR_UNSUPPORTED = -2,         /* e.g. compound with a Max/Min channel combine, R*S > 256 */
@@ -88,6 +104,8 @@ typedef struct {
     int32_t mode;  /* tconv_mode_t  */
     int32_t chan;  /* tconv_chan_t  */
     int32_t dtype; /* tconv_dtype_t */
+    int32_t pad_mode; /* tconv_pad_mode_t */
+    int32_t x_dtype;  /* tconv_x_dtype_t  */
 } tconv_desc_t;
 
 /* Output extent of the layer (PyTorch convention, Section 5).  Host call. */

@@ -84,6 +84,9 @@ int make_geo(const tconv_desc_t* d, Geo* g) {
     if (d->mode < TCONV_MAX_PLUS || d->mode > TCONV_PARALLEL) return TCONV_ERR_INVALID_ARG;
     if (d->chan < TCONV_CHAN_DEFAULT || d->chan > TCONV_CHAN_MIN) return TCONV_ERR_INVALID_ARG;
     if (d->dtype != TCONV_F32 && d->dtype != TCONV_BF16) return TCONV_ERR_INVALID_ARG;
+    if (d->pad_mode != TCONV_PAD_ZERO && d->pad_mode != TCONV_PAD_NEUTRAL) return TCONV_ERR_INVALID_ARG;
+    if (d->x_dtype != TCONV_X_SAME && d->x_dtype != TCONV_X_F32) return TCONV_ERR_INVALID_ARG;
+    if (d->x_dtype == TCONV_X_F32 && d->dtype != TCONV_BF16) return TCONV_ERR_INVALID_ARG;
     int chan = d->chan;
     if (chan == TCONV_CHAN_DEFAULT)
         chan = d->mode == TCONV_MAX_PLUS ? CH_MAX : d->mode == TCONV_MIN_PLUS ? CH_MIN : CH_SUM;
@@ -99,7 +102,25 @@ int make_geo(const tconv_desc_t* d, Geo* g) {
     g->mode = d->mode;
     g->chan = chan;
     g->wide = g->RS > 16;
+    g->neutral = d->pad_mode == TCONV_PAD_NEUTRAL;
+    g->xf32 = d->x_dtype == TCONV_X_F32;
     if (g->OH <= 0 || g->OW <= 0) return TCONV_ERR_INVALID_ARG;
+    if (g->neutral) {
+        // every window must keep a tap inside the image (else its result would be an infinity)
+        auto covered = [](int out, int in, int stride, int pad, int dil, int taps) {
+            for (int o = 0; o < out; ++o) {
+                bool any = false;
+                for (int t = 0; t < taps && !any; ++t) {
+                    const long i = (long)o * stride - pad + (long)t * dil;
+                    any = (i >= 0 && i < in);
+                }
+                if (!any) return false;
+            }
+            return true;
+        };
+        if (!covered(g->OH, g->H, g->sh, g->ph, g->dh, g->R) || !covered(g->OW, g->W, g->sw, g->pw, g->dw, g->S))
+            return TCONV_ERR_UNSUPPORTED;
+    }
     // one-dimensional launches index blocks with 31 bits
     const double outputs = (double)g->N * g->K * g->OH * g->OW;
     const double inputs = (double)g->N * g->C * g->H * g->W;
@@ -143,6 +164,7 @@ int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const 
         }
         if (rc != TCONV_ERR_UNSUPPORTED) return rc;
     }
+    if (g.xf32) return TCONV_ERR_UNSUPPORTED;   // float x for a bf16 layer: tiled kernels only
     const size_t total = (size_t)g.N * g.K * g.OH * g.OW;
     const unsigned blocks = (unsigned)((total + 255) / 256);
     fwd_generic_kernel<T><<<blocks, 256, 0, st>>>(g, (const T*)x, (const T*)w, (const T*)w2, alpha,
@@ -357,10 +379,13 @@ int backward_sum_t(const Geo& g0, const void* x, const void* w, const void* w2, 
                     (double)g.N * g.C * gp.HP * gp.WP < 2.0e9) {
                     T* xpad = (T*)((char*)ws + bias_part);
                     const size_t total = (size_t)g.N * g.C * gp.HP * gp.WP;
-                    pad_input_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, (const T*)x, xpad, gp.HP, gp.WP);
+                    if (g.xf32) pad_input_kernel<float, T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, (const float*)x, xpad, gp.HP, gp.WP);
+                    else pad_input_kernel<T, T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, (const T*)x, xpad, gp.HP, gp.WP);
                     g_launches += 1;
                     gp.xs_elems = gp.HP * gp.WP;
                     gp.xpad = xpad;
+                } else if (g.xf32 && br == 0 && (galpha || gbeta)) {
+                    return TCONV_ERR_UNSUPPORTED;   // float x is only read through the padded (converted) copy
                 }
 #define TCONV_GWK(BR, XSV, WARPV, GRID)                                                               \
     {                                                                                                \
@@ -399,6 +424,7 @@ int backward_sum_t(const Geo& g0, const void* x, const void* w, const void* w2, 
                         g0, alpha, beta, (const T*)gy0, winners, gw, gw2);
                     g_launches += 1;
                 }
+                if (twob && (galpha || gbeta) && g0.xf32) return TCONV_ERR_UNSUPPORTED;
                 if (twob && (galpha || gbeta)) {
                     bwd_gab_generic_kernel<T><<<(unsigned)((size_t)g0.K * g0.C), 256, 0, st>>>(
                         g0, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy0, winners, galpha, gbeta);
@@ -423,7 +449,7 @@ int make_dw_geo(const tconv_desc_t* d, Geo* g) {
     const int rc = make_geo(d, g);
     if (rc != TCONV_OK) return rc;
     if (g->K != g->C) return TCONV_ERR_INVALID_ARG;
-    if (g->RS > 16) return TCONV_ERR_UNSUPPORTED;
+    if (g->RS > 16 || g->neutral || g->xf32) return TCONV_ERR_UNSUPPORTED;
     g->chan = CH_SUM;
     const double lim = 2147483647.0;
     if ((double)g->N * g->C * g->OH * ((g->OW + 3) / 4) > lim || (double)g->N * g->C * g->H * g->W > lim ||

@@ -481,8 +481,9 @@ struct CodeGwPlan {
 };
 
 // xpad[n][c][HP][WP] = x with ph rows / pw columns of zeros in front (and zeros behind)
-template <typename T>
-__global__ void pad_input_kernel(Geo g, const T* __restrict__ x, T* __restrict__ xpad, int HP, int WP) {
+// TS: element type of x itself (float for a bf16 layer fed with float x: rounded here)
+template <typename TS, typename T>
+__global__ void pad_input_kernel(Geo g, const TS* __restrict__ x, T* __restrict__ xpad, int HP, int WP) {
     const size_t total = (size_t)g.N * g.C * HP * WP;
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total) return;
@@ -490,7 +491,7 @@ __global__ void pad_input_kernel(Geo g, const T* __restrict__ x, T* __restrict__
     const int pr = (int)((i / WP) % HP);
     const size_t nc = i / ((size_t)WP * HP);
     const int ih = pr - g.ph, iw = pc - g.pw;
-    xpad[i] = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? x[(nc * g.H + ih) * g.W + iw] : zero_of<T>();
+    xpad[i] = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? from_f32<T>(to_f32(x[(nc * g.H + ih) * g.W + iw])) : zero_of<T>();
 }
 
 // WARP: one warp per (k, c) pair, eight pairs per CTA, the lanes walk the pair's (image, quad)

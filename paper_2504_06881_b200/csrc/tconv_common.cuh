@@ -19,7 +19,16 @@ struct Geo {
     int OWP;         // OW rounded up to a multiple of 4: row pitch of the Sum-form winner codes
     int mode, chan;  // tconv_mode_t, resolved channel combine
     int wide;        // Sum-form winner codes are uint16 (R*S > 16) instead of uint8
+    int neutral;     // padded taps hold NaN, which min / max skip (neutral padding), instead of zero
+    int xf32;        // bf16 layer whose x is float: rounded to bf16 while it is staged
 };
+
+// Value a padded tap reads: zero, or a quiet NaN under neutral padding (min.f32 / max.f32 and their
+// bf16x2 forms return the other operand when one is NaN, so the tap never takes part).
+__device__ __forceinline__ float pad_value(const Geo& g, float) { return g.neutral ? __int_as_float(0x7fc00000) : 0.0f; }
+__device__ __forceinline__ __nv_bfloat16 pad_value(const Geo& g, __nv_bfloat16) {
+    return __ushort_as_bfloat16((unsigned short)(g.neutral ? 0x7fc0 : 0));
+}
 
 __host__ __device__ inline bool two_branch(int mode) {
     return mode == TCONV_COMPOUND || mode == TCONV_PARALLEL;

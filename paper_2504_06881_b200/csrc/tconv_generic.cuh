@@ -26,6 +26,7 @@ __device__ __forceinline__ void window_generic(const Geo& g, const T* __restrict
             const int iw = ow * g.sw - g.pw + s * g.dw;
             T xv = zero_of<T>();
             if (row_ok && iw >= 0 && iw < g.W) xv = xc[(size_t)ih * g.W + iw];
+            else if (g.neutral) continue;    // neutral padding: the tap is skipped
             const int tap = r * g.S + s;
             const float tmn = tap_add(xv, wmin[tap]);
             const float tmx = shared_add ? tmn : tap_add(xv, wmax[tap]);

@@ -377,7 +377,8 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                     for (int col = lane; col < p.XW; col += 32) {
                         const int iw = iw0 + col;
                         const bool ok = rok && iw >= 0 && iw < g.W;
-                        cp_async4(dst_row + col, ok ? src_row + iw : xg, ok);
+                        if (!ok && g.neutral) dst_row[col] = pad_value(g, 0.0f);   // plain store, visible after the barrier
+                        else cp_async4(dst_row + col, ok ? src_row + iw : xg, ok);
                     }
                 }
             }
@@ -730,7 +731,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
                     for (int tap = RS - 1; tap >= 0; --tap) {
                         const int ih = oh * g.sh - g.ph + (tap / S) * g.dh;
                         const int iw = ow * SW - g.pw + (tap % S) * DW;
-                        const float xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xc[(size_t)ih * g.W + iw] : 0.0f;
+                        const float xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) ? xc[(size_t)ih * g.W + iw] : pad_value(g, 0.0f);
                         if (__fadd_rn(xv, wk[tap]) == acc[k][q][j]) tapw = tap;
                     }
                     idx[o + j] = c * RS + tapw;
@@ -796,7 +797,8 @@ inline bool plan_tiles_opt(const Geo& g, bool par, bool two, int esize, bool all
     const int tiles_img = (g.OH + th_img - 1) / th_img;
     const bool rows_fit = p.ragged ? (g.OH * p.QPR >= NQ)
                                    : ((double)g.OH / (tiles_img * th_img) >= 0.75 && th_img * p.QPR * 4 >= NQ * 3);
-    pl->xtma = ((g.W * esize) % 16 == 0) && (g.pw == (S - 1) * DW / 2) && rows_fit;
+    // (a bf16 layer fed with float x converts while staging element by element: no tensor copy)
+    pl->xtma = !g.xf32 && ((g.W * esize) % 16 == 0) && (g.pw == (S - 1) * DW / 2) && rows_fit;
     p.XW = (p.TW - 1) * SW + (S - 1) * DW + 1;   // == (QPR-1)*4*SW + L
     if (pl->xtma && p.ragged) {
         p.TH = rows_max;
@@ -891,7 +893,7 @@ inline encode_tiled_fn get_encode_tiled() {
     return fn;
 }
 
-// x viewed as [N*C][H][W]; box = [CC][NSLOTS][XP]; out-of-range elements read as zero.
+// x viewed as [N*C][H][W]; box = [CC][NSLOTS][XP]; out-of-range elements read as the padding value.
 inline bool make_x_map(const Geo& g, const void* x, int esize, const TiledParams& p, CUtensorMap* map) {
     encode_tiled_fn enc = get_encode_tiled();
     if (!enc) return false;
@@ -900,9 +902,10 @@ inline bool make_x_map(const Geo& g, const void* x, int esize, const TiledParams
     const cuuint32_t box[3] = {(cuuint32_t)p.XP, (cuuint32_t)p.NSLOTS, (cuuint32_t)p.CC};
     const cuuint32_t estr[3] = {1, 1, 1};
     const CUtensorMapDataType dt = esize == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    // out-of-range elements: zeros (zero padding) or NaN (neutral padding: min / max skip a NaN)
     return enc(map, dt, 3, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+               g.neutral ? CU_TENSOR_MAP_FLOAT_OOB_FILL_NAN_REQUEST_ZERO_FMA : CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Arguments of one forward launch (host side).

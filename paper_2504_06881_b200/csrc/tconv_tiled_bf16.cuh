@@ -117,6 +117,13 @@ __global__ void repack_weights_bf16_kernel(int K, int C, int RS, int tile_k, int
     }
 }
 
+// Element i of x as bf16 bits: x holds bf16, or float values that are rounded to nearest even here
+// (the same rounding a conversion of the whole tensor would apply).
+__device__ __forceinline__ unsigned short load_x(const unsigned short* x, size_t i, int xf32) {
+    if (!xf32) return x[i];
+    return __bfloat16_as_ushort(__float2bfloat16_rn(reinterpret_cast<const float*>(x)[i]));
+}
+
 // KPT words of packed weights of one tap (one or two 16-byte loads)
 template <int KPT>
 __device__ __forceinline__ void loadw(const unsigned* p, unsigned* out) {
@@ -271,12 +278,14 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
             // and the loads of the chunk's channels are issued together before any is stored
             unsigned short* xs = reinterpret_cast<unsigned short*>(st);
             const int per_c = p.NSLOTS * p.XP;
+            const unsigned short pad_bits = (unsigned short)(g.neutral ? 0x7fc0 : 0);   // padding: zero, or NaN (skipped by min / max)
             for (int i = tid; i < per_c; i += NT) {
                 const int so = src_tab[i];
                 unsigned short v[8];
 #pragma unroll
                 for (int cc = 0; cc < 8; ++cc)
-                    v[cc] = (so >= 0 && cc < p.CC && c0 + cc < g.C) ? xg[(size_t)(c0 + cc) * chw + so] : (unsigned short)0;
+                    v[cc] = (cc < p.CC && c0 + cc < g.C) ? (so >= 0 ? load_x(xg, (size_t)(c0 + cc) * chw + so, g.xf32) : pad_bits)
+                                                          : (unsigned short)0;
 #pragma unroll
                 for (int cc = 0; cc < 8; ++cc)
                     if (cc < p.CC) xs[cc * per_c + i] = v[cc];
@@ -377,9 +386,12 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                                 const unsigned t = hadd2u(xp, wv[k]);
                                 const unsigned t2 = PAR ? hadd2u(xp, wv2[k]) : t;
                                 if constexpr (TWO) {
-                                    if (tap == 0) {
+                                    if (tap == 0 && !g.neutral) {
                                         mn[k][q][pp] = t; amn[k][q][pp] = 0u; mx[k][q][pp] = t2; amx[k][q][pp] = 0u;
                                     } else {
+                                        if (tap == 0) {   // neutral padding: tap 0 may be a NaN; start from the identities
+                                            mn[k][q][pp] = kPosInf2; mx[k][q][pp] = kNegInf2; amn[k][q][pp] = amx[k][q][pp] = 0u;
+                                        }
                                         const unsigned ml = hbetter_mask(t, mn[k][q][pp], true);
                                         mn[k][q][pp] = hext2u(mn[k][q][pp], t, true);
                                         amn[k][q][pp] = (tap2 & ml) | (amn[k][q][pp] & ~ml);
@@ -388,9 +400,10 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                                         amx[k][q][pp] = (tap2 & mg) | (amx[k][q][pp] & ~mg);
                                     }
                                 } else {
-                                    if (tap == 0) {
+                                    if (tap == 0 && !g.neutral) {
                                         mx[k][q][pp] = t; amx[k][q][pp] = 0u;
                                     } else {
+                                        if (tap == 0) { mx[k][q][pp] = TAP_MIN ? kPosInf2 : kNegInf2; amx[k][q][pp] = 0u; }
                                         const unsigned mg = hbetter_mask(t, mx[k][q][pp], TAP_MIN);
                                         mx[k][q][pp] = hext2u(mx[k][q][pp], t, TAP_MIN);
                                         amx[k][q][pp] = (tap2 & mg) | (amx[k][q][pp] & ~mg);
@@ -558,7 +571,6 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
             }
             if constexpr (WIN && !SUMF) {
                 int32_t* idx = reinterpret_cast<int32_t*>(p.winners);
-                const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(p.x);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int ow = qcol[q] + j;
@@ -567,7 +579,7 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                     const int c = (j & 1) ? (int)(cpair >> 16) : (int)(cpair & 0xffffu);
                     const unsigned bpair = best[k][q][j >> 1];
                     const float bestv = (j & 1) ? bf_hi(bpair) : bf_lo(bpair);
-                    const __nv_bfloat16* xc = xb + ((size_t)n * g.C + c) * chw;
+                    const size_t xc = ((size_t)n * g.C + c) * chw;
                     // the window's weights in their original layout: 9 adjacent values
                     const __nv_bfloat16* wk = reinterpret_cast<const __nv_bfloat16*>(p.w) + ((size_t)kk * g.C + c) * RS;
                     int tapw = 0;
@@ -576,7 +588,8 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
                         const int ih = oh * g.sh - g.ph + (tap / S) * g.dh;
                         const int iw = ow * SW - g.pw + (tap % S) * DW;
                         const __nv_bfloat16 xv = (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W)
-                                                     ? xc[(size_t)ih * g.W + iw] : __float2bfloat16_rn(0.0f);
+                                                     ? __ushort_as_bfloat16(load_x(xg, xc + (size_t)ih * g.W + iw, g.xf32))
+                                                     : pad_value(g, __nv_bfloat16());
                         if (tap_add(xv, wk[tap]) == bestv) tapw = tap;
                     }
                     idx[o + j] = c * RS + tapw;

@@ -18,6 +18,8 @@ LIB_PATH = _PKG / "libtconv.so"
 MODES = {"max_plus": 0, "min_plus": 1, "compound": 2, "parallel": 3}
 CHANS = {"default": 0, "sum": 1, "max": 2, "min": 3}
 DTYPES = {"f32": 0, "bf16": 1}
+PAD_MODES = {"zero": 0, "neutral": 1}
+X_DTYPES = {"same": 0, "f32": 1}
 TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
 
 # every symbol include/tconv.h declares
@@ -40,7 +42,7 @@ class Desc(ctypes.Structure):
     """tconv_desc_t."""
     _fields_ = [(n, ctypes.c_int32) for n in (
         "N", "C", "H", "W", "K", "R", "S", "stride_h", "stride_w", "pad_h", "pad_w",
-        "dil_h", "dil_w", "mode", "chan", "dtype")]
+        "dil_h", "dil_w", "mode", "chan", "dtype", "pad_mode", "x_dtype")]
 
 
 def _load() -> ctypes.CDLL:
@@ -94,7 +96,8 @@ def make_desc(d: dict) -> Desc:
     """C descriptor from a plain dict (keys = field names; mode/chan/dtype by name)."""
     return Desc(d["N"], d["C"], d["H"], d["W"], d["K"], d["R"], d["S"], d["stride_h"],
                 d["stride_w"], d["pad_h"], d["pad_w"], d["dil_h"], d["dil_w"],
-                MODES[d["mode"]], CHANS[d["chan"]], DTYPES[d["dtype"]])
+                MODES[d["mode"]], CHANS[d["chan"]], DTYPES[d["dtype"]],
+                PAD_MODES[d.get("pad_mode", "zero")], X_DTYPES[d.get("x_dtype", "same")])
 
 
 def _p(t):
@@ -222,6 +225,21 @@ def _check(t, shape, dtype, name):
                          f"{dtype}, got {tuple(t.shape)} {t.dtype} on {t.device}")
 
 
+def _x_dtype(d: dict):
+    """torch dtype of x: the layer's, or float32 for a bf16 layer that converts x while staging."""
+    return torch.float32 if d.get("x_dtype", "same") == "f32" else TORCH_DTYPE[d["dtype"]]
+
+
+def _on_stream(stream, *tensors):
+    """Tensors allocated here (on the current stream) and used by kernels on `stream`: tell the
+    caching allocator, so that their memory is not reused while those kernels still run."""
+    if stream is None or stream == torch.cuda.current_stream():
+        return
+    for t in tensors:
+        if t is not None:
+            t.record_stream(stream)
+
+
 def winner_buffer(d: dict, device) -> torch.Tensor:
     return torch.empty(tconv_winner_bytes(d), dtype=torch.uint8, device=device)
 
@@ -231,7 +249,7 @@ def forward(d: dict, x, w, w2=None, alpha=None, beta=None, bias=None, want_winne
     """Allocate y (and the winner buffer) and run tconv_forward.  Returns (y, winners)."""
     N, C, H, W, K, R, S = (d[k] for k in "NCHWKRS")
     dt = TORCH_DTYPE[d["dtype"]]
-    _check(x, (N, C, H, W), dt, "x"); _check(w, (K, C, R, S), dt, "w"); _check(w2, (K, C, R, S), dt, "w2")
+    _check(x, (N, C, H, W), _x_dtype(d), "x"); _check(w, (K, C, R, S), dt, "w"); _check(w2, (K, C, R, S), dt, "w2")
     _check(alpha, (K, C), torch.float32, "alpha"); _check(beta, (K, C), torch.float32, "beta")
     _check(bias, (K,), torch.float32, "bias")
     OH, OW = tconv_output_shape(d)
@@ -239,6 +257,7 @@ def forward(d: dict, x, w, w2=None, alpha=None, beta=None, bias=None, want_winne
     winners = winner_buffer(d, x.device) if want_winners else None
     nws = tconv_workspace_bytes(d, False)
     ws = torch.empty(nws, dtype=torch.uint8, device=x.device) if nws else None
+    _on_stream(stream, y, winners, ws)
     rc = tconv_forward(d, x, w, w2, alpha, beta, bias, y, winners, ws, stream)
     if rc != 0:
         raise TconvError(rc, "tconv_forward")
@@ -251,7 +270,7 @@ def backward(d: dict, x, w, grad_y, w2=None, alpha=None, beta=None, winners=None
     N, C, H, W, K, R, S = (d[k] for k in "NCHWKRS")
     dt = TORCH_DTYPE[d["dtype"]]
     OH, OW = tconv_output_shape(d)
-    _check(x, (N, C, H, W), dt, "x"); _check(w, (K, C, R, S), dt, "w"); _check(w2, (K, C, R, S), dt, "w2")
+    _check(x, (N, C, H, W), _x_dtype(d), "x"); _check(w, (K, C, R, S), dt, "w"); _check(w2, (K, C, R, S), dt, "w2")
     _check(grad_y, (N, K, OH, OW), dt, "grad_y")
     two = d["mode"] in ("compound", "parallel")
     dev = x.device
@@ -274,6 +293,7 @@ def backward(d: dict, x, w, grad_y, w2=None, alpha=None, beta=None, winners=None
         # the figure includes room for recomputed winners, not needed when they are passed
         nws -= (tconv_winner_bytes(d) + 255) // 256 * 256
     ws = torch.empty(nws, dtype=torch.uint8, device=dev) if nws > 0 else None
+    _on_stream(stream, ws, *out.values())
     rc = tconv_backward(d, x, w, w2, alpha, beta, grad_y, winners, out.get("grad_x"),
                         out.get("grad_w"), out.get("grad_w2"), out.get("grad_alpha"),
                         out.get("grad_beta"), out.get("grad_bias"), ws, stream)
@@ -292,6 +312,7 @@ def dw_forward(d: dict, x, w, w2=None, alpha=None, beta=None, bias=None, want_wi
     OH, OW = tconv_output_shape(d)
     y = torch.empty((N, C, OH, OW), dtype=dt, device=x.device)
     winners = torch.empty((N, C, OH, OW), dtype=torch.uint8, device=x.device) if want_winners else None
+    _on_stream(stream, y, winners)
     rc = tconv_dw_forward(d, x, w, w2, alpha, beta, bias, y, winners, stream)
     if rc != 0:
         raise TconvError(rc, "tconv_dw_forward")
@@ -316,6 +337,7 @@ def dw_backward(d: dict, x, w, grad_y, w2=None, alpha=None, beta=None, winners=N
         out["grad_alpha"] = torch.empty((C,), dtype=f32, device=dev)
         out["grad_beta"] = torch.empty((C,), dtype=f32, device=dev)
     ws = torch.empty(tconv_dw_workspace_bytes(d, True), dtype=torch.uint8, device=dev)
+    _on_stream(stream, ws, *out.values())
     rc = tconv_dw_backward(d, x, w, w2, alpha, beta, grad_y, winners, out["grad_x"], out["grad_w"],
                            out.get("grad_w2"), out.get("grad_alpha"), out.get("grad_beta"),
                            out["grad_bias"], ws, stream)
