@@ -154,6 +154,24 @@ int tconv_forward(const tconv_desc_t *desc, const void *x, const void *w, const 
                   void *winners, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Forward pass that also returns the per-channel statistics of its output,
+ *   sum_y[k]  = sum over (n, oh, ow) of y[n][k][oh][ow],
+ *   sum_y2[k] = sum over (n, oh, ow) of y[n][k][oh][ow]^2      (fp32 [K] each),
+ * i.e. what the batch normalisation that follows every tropical layer in the paper's
+ * residual blocks (section "ResNet Models": Conv-BN-Tropical-BN and Tropical-BN-Tropical-BN)
+ * needs for its mean and variance, without reading y again.  The sums are taken over the
+ * stored values (bf16 layers: after rounding) in the kernel's epilogue: per pixel tile with a
+ * fixed shuffle tree, then over the tiles in a fixed order (deterministic, no atomics).  Other
+ * arguments and results as tconv_forward; workspace_bytes must be at least
+ * tconv_stats_workspace_bytes(desc).
+ */
+size_t tconv_stats_workspace_bytes(const tconv_desc_t *desc);
+int tconv_forward_stats(const tconv_desc_t *desc, const void *x, const void *w, const void *w2,
+                        const float *alpha, const float *beta, const float *bias, void *y,
+                        void *winners, float *sum_y, float *sum_y2, void *workspace,
+                        size_t workspace_bytes, void *stream);
+
+/*
  * Backward pass: routes grad_y to the winner(s) of every output.
  *   winners     the buffer tconv_forward filled for the same inputs, or NULL to
  *               have the winners recomputed (into the workspace).

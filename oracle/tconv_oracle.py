@@ -147,6 +147,16 @@ def forward(d: dict, x, w, w2=None, alpha=None, beta=None, bias=None,
     return out
 
 
+def channel_stats(y):
+    """Per-channel sums of an output y[N][K][OH][OW] and of its squares, in float64, with the sums
+    of absolute values beside them (the scale of a summation error bound): what the batch
+    normalisation after a tropical layer (the paper's section "ResNet Models") takes its mean and
+    variance from.  Returns {"sum_y": (s, abs), "sum_y2": (s, abs)}."""
+    y = np.asarray(y, np.float64)
+    return {"sum_y": (y.sum(axis=(0, 2, 3)), np.abs(y).sum(axis=(0, 2, 3))),
+            "sum_y2": ((y * y).sum(axis=(0, 2, 3)), (y * y).sum(axis=(0, 2, 3)))}
+
+
 def backward(d: dict, x, w, g, w2=None, alpha=None, beta=None):
     """Run the oracle backward.  Returns a dict name -> (grad, abs_sum), both
     float64: ``grad_x``, ``grad_w``, ``grad_w2`` (parallel only), ``grad_alpha``,

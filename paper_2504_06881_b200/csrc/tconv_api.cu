@@ -146,12 +146,25 @@ bool force_generic() {
     return v;
 }
 
+// Upper bound of the scratch the channel statistics need: one {sum, sum of squares} pair per
+// (pixel tile of the tiled kernels, output channel).  A tile holds at least one row of at most 8
+// quads (32 output columns), so there are at most N * OH * ceil(quads per row / 8) of them.
+size_t stats_scratch_bytes(const Geo& g) {
+    const size_t tiles = (size_t)g.N * g.OH * (((g.OW + 3) / 4 + 7) / 8) + 16;
+    const size_t kp = ((size_t)g.K + 63) / 64 * 64;
+    return align_up(tiles * kp * 2 * sizeof(float), 256);
+}
+
+// stats_ws: NULL, or scratch of stats_scratch_bytes() for the per-tile channel statistics, which are
+// then summed into sum_y / sum_y2.
 template <typename T>
 int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const float* alpha,
               const float* beta, const float* bias, void* y, void* winners, void* ws,
-              size_t ws_bytes, cudaStream_t st) {
+              size_t ws_bytes, cudaStream_t st, float* stats_ws = nullptr, float* sum_y = nullptr,
+              float* sum_y2 = nullptr) {
     if (!force_generic()) {
         FwdArgs a;
+        a.stats = stats_ws; a.stats_bytes = stats_ws ? stats_scratch_bytes(g) : 0; a.stats_tiles = 0; a.stats_k = 0;
         a.g = g; a.dtype = sizeof(T) == 4 ? TCONV_F32 : TCONV_BF16;
         a.x = x; a.w = w; a.w2 = w2; a.alpha = alpha; a.beta = beta; a.bias = bias;
         a.y = y; a.winners = winners; a.ws = ws; a.ws_bytes = ws_bytes;
@@ -160,6 +173,11 @@ int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const 
         if (rc == TCONV_OK) {
             snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", a.name);
             g_launches += 2;  // weight repack + tiled kernel
+            if (stats_ws) {
+                stats_finish_kernel<<<(unsigned)((g.K * 32 + 255) / 256), 256, 0, st>>>(stats_ws, a.stats_tiles, a.stats_k,
+                                                                                   g.K, sum_y, sum_y2);
+                g_launches += 1;
+            }
             return check_launch();
         }
         if (rc != TCONV_ERR_UNSUPPORTED) return rc;
@@ -171,6 +189,14 @@ int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const 
                                                   beta, bias, (T*)y, winners);
     snprintf(g_last_kernel, sizeof(g_last_kernel), "fwd_generic");
     g_launches += 1;
+    if (stats_ws && y) {
+        // statistics from the stored output
+        const int chunks = g.N < 16 ? g.N : 16, npc = (g.N + chunks - 1) / chunks;
+        const int rows = (g.N + npc - 1) / npc;
+        stats_direct_kernel<T><<<dim3((unsigned)g.K, (unsigned)rows), 256, 0, st>>>(g, (const T*)y, stats_ws, npc);
+        stats_finish_kernel<<<(unsigned)((g.K * 32 + 255) / 256), 256, 0, st>>>(stats_ws, rows, g.K, g.K, sum_y, sum_y2);
+        g_launches += 2;
+    }
     return check_launch();
 }
 
@@ -655,6 +681,36 @@ int tconv_forward(const tconv_desc_t* desc, const void* x, const void* w, const 
                                 workspace_bytes, st);
     return forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, bias, y, winners, workspace,
                                     workspace_bytes, st);
+}
+
+size_t tconv_stats_workspace_bytes(const tconv_desc_t* desc) {
+    Geo g;
+    if (make_geo(desc, &g) != TCONV_OK) return 0;
+    return tconv_workspace_bytes(desc, 0) + stats_scratch_bytes(g);
+}
+
+int tconv_forward_stats(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,
+                        const float* alpha, const float* beta, const float* bias, void* y, void* winners,
+                        float* sum_y, float* sum_y2, void* workspace, size_t workspace_bytes, void* stream) {
+    Geo g;
+    int rc = make_geo(desc, &g);
+    if (rc != TCONV_OK) return rc;
+    if (!x || !w || !y || !sum_y || !sum_y2 || !workspace) return TCONV_ERR_INVALID_ARG;
+    if (g.mode == TCONV_PARALLEL && !w2) return TCONV_ERR_INVALID_ARG;
+    if (misaligned(x) || misaligned(w) || misaligned(w2) || misaligned(alpha) || misaligned(beta) ||
+        misaligned(bias) || misaligned(y) || misaligned(winners) || misaligned(workspace) || misaligned(sum_y) ||
+        misaligned(sum_y2))
+        return TCONV_ERR_MISALIGNED;
+    const size_t fwd = tconv_workspace_bytes(desc, 0);
+    if (workspace_bytes < fwd + stats_scratch_bytes(g)) return TCONV_ERR_WORKSPACE_TOO_SMALL;
+    if (!two_branch(g.mode)) { alpha = nullptr; beta = nullptr; }
+    cudaStream_t st = (cudaStream_t)stream;
+    g_last_error[0] = 0;
+    float* stats_ws = (float*)((char*)workspace + fwd);
+    if (desc->dtype == TCONV_F32)
+        return forward_t<float>(g, x, w, w2, alpha, beta, bias, y, winners, workspace, fwd, st, stats_ws, sum_y, sum_y2);
+    return forward_t<__nv_bfloat16>(g, x, w, w2, alpha, beta, bias, y, winners, workspace, fwd, st, stats_ws, sum_y,
+                                    sum_y2);
 }
 
 int tconv_backward(const tconv_desc_t* desc, const void* x, const void* w, const void* w2,

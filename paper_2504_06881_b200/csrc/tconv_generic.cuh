@@ -282,4 +282,50 @@ bwd_bias_kernel(Geo g, const T* __restrict__ gy, float* __restrict__ gbias) {
     if (threadIdx.x == 0) gbias[k] = t;
 }
 
+// ---------------------------------------------------------------------------------- channel statistics
+// sum_y[k], sum_y2[k] = sums over the partial rows (fixed order) of {sum y, sum y^2}: one warp per
+// output channel, lane l adds rows l, l + 32, ... in order, then a fixed shuffle tree.
+__global__ void __launch_bounds__(256)
+stats_finish_kernel(const float* __restrict__ partial, int rows, int pitch, int K, float* __restrict__ sum_y,
+                    float* __restrict__ sum_y2) {
+    const int k = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    if (k >= K) return;
+    float s1 = 0.0f, s2 = 0.0f;
+    for (int r = lane; r < rows; r += 32) {
+        const float2 v = *reinterpret_cast<const float2*>(partial + ((size_t)r * pitch + k) * 2);
+        s1 += v.x; s2 += v.y;
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        s1 += __shfl_xor_sync(0xffffffffu, s1, d);
+        s2 += __shfl_xor_sync(0xffffffffu, s2, d);
+    }
+    if (lane == 0) {
+        if (sum_y) sum_y[k] = s1;
+        if (sum_y2) sum_y2[k] = s2;
+    }
+}
+
+// Statistics of a stored output (layers the tiled kernels do not serve): grid (K, chunks of images),
+// partial[chunk][k] = {sum y, sum y^2} over the chunk.
+template <typename T>
+__global__ void __launch_bounds__(256)
+stats_direct_kernel(Geo g, const T* __restrict__ y, float* __restrict__ partial, int n_per_chunk) {
+    __shared__ float red[256];
+    const int k = blockIdx.x, chunk = blockIdx.y;
+    const size_t plane = (size_t)g.OH * g.OW;
+    const int n_lo = chunk * n_per_chunk, n_hi = min(g.N, n_lo + n_per_chunk);
+    float s1 = 0.0f, s2 = 0.0f;
+    for (int n = n_lo; n < n_hi; ++n) {
+        const T* src = y + ((size_t)n * g.K + k) * plane;
+        for (size_t j = threadIdx.x; j < plane; j += blockDim.x) {
+            const float v = to_f32(src[j]);
+            s1 += v; s2 = __fmaf_rn(v, v, s2);
+        }
+    }
+    const float t1 = block_sum(s1, red);
+    const float t2 = block_sum(s2, red);
+    if (threadIdx.x == 0) *reinterpret_cast<float2*>(partial + ((size_t)chunk * g.K + k) * 2) = make_float2(t1, t2);
+}
+
 }  // namespace tconv

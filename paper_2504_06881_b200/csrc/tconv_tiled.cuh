@@ -200,6 +200,8 @@ struct TiledParams {
     const float* bias;
     void* y;
     void* winners;
+    float* stats;      // NULL, or per-tile partial sums {sum y, sum y^2} per output channel: [tile][stats_k][2]
+    int stats_k;       // channel pitch of the partials (K rounded up to the k tile)
     int* status;       // device status word: set non-zero when a bounded wait gives up
     int TW, QPR, TH;   // tile: output columns, quads per row, output rows
     int n_col_tiles, n_row_tiles;
@@ -692,6 +694,32 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
 
     // epilogue: bias, store, winner index of the Max / Min channel combines
     float* yg = reinterpret_cast<float*>(p.y);
+    if (p.stats) {
+        // per-channel sums of the outputs and of their squares over this tile (the statistics a
+        // following batch normalisation needs): per thread over its pixels, then a fixed shuffle
+        // tree over the warp, which owns all pixels of the tile for its TK channels
+        static_assert(PW == 1, "one warp per channel group owns the whole pixel tile");
+#pragma unroll
+        for (int k = 0; k < TK; ++k) {
+            const int kk = kt * TILE_K + kg * TK + k;
+            const float bk = (p.bias && kk < g.K) ? p.bias[kk] : 0.0f;
+            float s1 = 0.0f, s2 = 0.0f;
+#pragma unroll
+            for (int q = 0; q < Q; ++q)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float v = p.bias ? __fadd_rn(acc[k][q][j], bk) : acc[k][q][j];
+                    if (out_row[q] >= 0 && qcol[q] + j < g.OW) { s1 += v; s2 = __fmaf_rn(v, v, s2); }
+                }
+#pragma unroll
+            for (int dlt = 16; dlt > 0; dlt >>= 1) {
+                s1 += __shfl_xor_sync(0xffffffffu, s1, dlt);
+                s2 += __shfl_xor_sync(0xffffffffu, s2, dlt);
+            }
+            if (lane == 0 && kk < g.K)
+                *reinterpret_cast<float2*>(p.stats + ((size_t)blockIdx.x * p.stats_k + kk) * 2) = make_float2(s1, s2);
+        }
+    }
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
         if (out_row[q] < 0) continue;
@@ -912,6 +940,10 @@ inline bool make_x_map(const Geo& g, const void* x, int esize, const TiledParams
 struct FwdArgs {
     Geo g;
     int dtype;
+    float* stats;      // NULL, or where the tiled kernel leaves its per-tile channel statistics
+    size_t stats_bytes;
+    int stats_tiles;   // out: tiles the kernel wrote (0: the kernel that ran wrote none)
+    int stats_k;       // out: channel pitch of the partials
     const void *x, *w, *w2;
     const float *alpha, *beta, *bias;
     void* y;
@@ -946,6 +978,11 @@ int launch_tiled_variant(FwdArgs& a) {
         g.K, g.C, g.RS, pl.tile_k, pl.p.Cpad, nkt, (const T*)a.w, (const T*)a.w2, a.alpha, a.beta, wt, wt2, at, bt);
     pl.p.x = a.x; pl.p.w = a.w; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
+    pl.p.stats = nullptr; pl.p.stats_k = nkt * pl.tile_k;
+    if (a.stats) {
+        if ((size_t)pl.grid.x * pl.p.stats_k * 2 * sizeof(float) > a.stats_bytes) return TCONV_ERR_WORKSPACE_TOO_SMALL;
+        pl.p.stats = a.stats; a.stats_tiles = (int)pl.grid.x; a.stats_k = pl.p.stats_k;
+    }
 #define TCONV_LAUNCH_F32(XTMAV, RAGV)                                                                 \
     {                                                                                                \
         auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, TK>; \

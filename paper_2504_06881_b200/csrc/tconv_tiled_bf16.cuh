@@ -532,6 +532,34 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
 
     // epilogue
     unsigned short* yg = reinterpret_cast<unsigned short*>(p.y);
+    if (p.stats) {
+        // per-channel sums of the stored (bf16-rounded) outputs and of their squares over this tile
+        static_assert(PW == 1, "one warp per channel group owns the whole pixel tile");
+#pragma unroll
+        for (int k = 0; k < KPT; ++k) {
+            const int kk = kt * TILE_K + kg * KPT + k;
+            const float bk = (p.bias && kk < g.K) ? p.bias[kk] : 0.0f;
+            float s1 = 0.0f, s2 = 0.0f;
+#pragma unroll
+            for (int q = 0; q < Q; ++q)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float v;
+                    if constexpr (SUMF) v = acc[k][q][j];
+                    else v = (j & 1) ? bf_hi(best[k][q][j >> 1]) : bf_lo(best[k][q][j >> 1]);
+                    if (p.bias) v = __fadd_rn(v, bk);
+                    v = __bfloat162float(__float2bfloat16_rn(v));
+                    if (out_row[q] >= 0 && qcol[q] + j < g.OW) { s1 += v; s2 = __fmaf_rn(v, v, s2); }
+                }
+#pragma unroll
+            for (int dlt = 16; dlt > 0; dlt >>= 1) {
+                s1 += __shfl_xor_sync(0xffffffffu, s1, dlt);
+                s2 += __shfl_xor_sync(0xffffffffu, s2, dlt);
+            }
+            if (lane == 0 && kk < g.K)
+                *reinterpret_cast<float2*>(p.stats + ((size_t)blockIdx.x * p.stats_k + kk) * 2) = make_float2(s1, s2);
+        }
+    }
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
         if (out_row[q] < 0) continue;
@@ -628,6 +656,11 @@ int launch_tiled_variant_bf16(FwdArgs& a) {
         a.alpha, a.beta, (unsigned*)wt, (unsigned*)wt2, at, bt);
     pl.p.x = a.x; pl.p.w = a.w; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
+    pl.p.stats = nullptr; pl.p.stats_k = nkt * pl.tile_k;
+    if (a.stats) {
+        if ((size_t)pl.grid.x * pl.p.stats_k * 2 * sizeof(float) > a.stats_bytes) return TCONV_ERR_WORKSPACE_TOO_SMALL;
+        pl.p.stats = a.stats; a.stats_tiles = (int)pl.grid.x; a.stats_k = pl.p.stats_k;
+    }
 #define TCONV_LAUNCH_BF16(XTMAV, RAGV)                                                                \
     {                                                                                                \
         auto kern = fwd_tiled_bf16_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, KPT>; \

@@ -24,7 +24,7 @@ TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
 
 # every symbol include/tconv.h declares
 SYMBOLS = ("tconv_output_shape", "tconv_winner_bytes", "tconv_workspace_bytes", "tconv_forward",
-           "tconv_backward", "tconv_forward_noalloc", "tconv_forward_noalloc_max_scratch", "tconv_paper_ops", "tconv_alu_probe", "tconv_alu_probe_name",
+           "tconv_backward", "tconv_forward_stats", "tconv_stats_workspace_bytes", "tconv_forward_noalloc", "tconv_forward_noalloc_max_scratch", "tconv_paper_ops", "tconv_alu_probe", "tconv_alu_probe_name",
            "tconv_device_status", "tconv_status_string", "tconv_last_error", "tconv_last_kernel",
            "tconv_launch_count", "tconv_dw_winner_bytes", "tconv_dw_workspace_bytes", "tconv_dw_forward",
            "tconv_dw_backward")
@@ -62,6 +62,10 @@ def _load() -> ctypes.CDLL:
     lib.tconv_forward.restype = ctypes.c_int
     lib.tconv_backward.argtypes = [dp, vp, vp, vp, fp, fp, vp, vp, vp, fp, fp, fp, fp, fp, vp, sz, vp]
     lib.tconv_backward.restype = ctypes.c_int
+    lib.tconv_forward_stats.argtypes = [dp, vp, vp, vp, fp, fp, fp, vp, vp, fp, fp, vp, sz, vp]
+    lib.tconv_forward_stats.restype = ctypes.c_int
+    lib.tconv_stats_workspace_bytes.argtypes = [dp]
+    lib.tconv_stats_workspace_bytes.restype = sz
     lib.tconv_forward_noalloc.argtypes = [dp, vp, vp, vp, fp, fp, fp, vp, vp, vp]
     lib.tconv_forward_noalloc.restype = ctypes.c_int
     lib.tconv_forward_noalloc_max_scratch.restype = sz
@@ -177,6 +181,17 @@ def tconv_dw_backward(d: dict, x, w, w2, alpha, beta, grad_y, winners, grad_x, g
                                   _stream(stream))
 
 
+def tconv_stats_workspace_bytes(d: dict) -> int:
+    return int(_lib.tconv_stats_workspace_bytes(ctypes.byref(make_desc(d))))
+
+
+def tconv_forward_stats(d, x, w, w2, alpha, beta, bias, y, winners, sum_y, sum_y2, workspace, stream=None) -> int:
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    return _lib.tconv_forward_stats(ctypes.byref(make_desc(d)), _p(x), _p(w), _p(w2), _p(alpha), _p(beta),
+                                    _p(bias), _p(y), _p(winners), _p(sum_y), _p(sum_y2), _p(workspace), nbytes,
+                                    _stream(stream))
+
+
 def tconv_forward_noalloc_max_scratch() -> int:
     return int(_lib.tconv_forward_noalloc_max_scratch())
 
@@ -262,6 +277,27 @@ def forward(d: dict, x, w, w2=None, alpha=None, beta=None, bias=None, want_winne
     if rc != 0:
         raise TconvError(rc, "tconv_forward")
     return y, winners
+
+
+def forward_stats(d: dict, x, w, w2=None, alpha=None, beta=None, bias=None, want_winners=False, stream=None):
+    """forward() that also returns the per-channel sums of y and of y^2 (fp32 [K] each), taken in
+    the kernel's epilogue.  Returns (y, winners, sum_y, sum_y2)."""
+    N, C, H, W, K, R, S = (d[k] for k in "NCHWKRS")
+    dt = TORCH_DTYPE[d["dtype"]]
+    _check(x, (N, C, H, W), _x_dtype(d), "x"); _check(w, (K, C, R, S), dt, "w"); _check(w2, (K, C, R, S), dt, "w2")
+    _check(alpha, (K, C), torch.float32, "alpha"); _check(beta, (K, C), torch.float32, "beta")
+    _check(bias, (K,), torch.float32, "bias")
+    OH, OW = tconv_output_shape(d)
+    y = torch.empty((N, K, OH, OW), dtype=dt, device=x.device)
+    winners = winner_buffer(d, x.device) if want_winners else None
+    sum_y = torch.empty((K,), dtype=torch.float32, device=x.device)
+    sum_y2 = torch.empty((K,), dtype=torch.float32, device=x.device)
+    ws = torch.empty(tconv_stats_workspace_bytes(d), dtype=torch.uint8, device=x.device)
+    _on_stream(stream, y, winners, sum_y, sum_y2, ws)
+    rc = tconv_forward_stats(d, x, w, w2, alpha, beta, bias, y, winners, sum_y, sum_y2, ws, stream)
+    if rc != 0:
+        raise TconvError(rc, "tconv_forward_stats")
+    return y, winners, sum_y, sum_y2
 
 
 def backward(d: dict, x, w, grad_y, w2=None, alpha=None, beta=None, winners=None, stream=None,

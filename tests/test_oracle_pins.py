@@ -666,3 +666,20 @@ def test_neutral_padding_backward_is_the_directional_derivative():
     lhs = ((y1 - y0) * g).sum()
     rhs = (gr["grad_x"][0] * u).sum()
     assert lhs == rhs
+
+
+# ---------------------------------------------------------------- channel statistics
+def test_channel_stats_give_numpy_mean_and_variance():
+    """The sums the oracle reports reproduce numpy's per-channel mean and (biased) variance, and a
+    constant map gives the closed forms count * c and count * c^2."""
+    rs = np.random.RandomState(320)
+    y = rs.standard_normal((3, 5, 7, 6)).astype(np.float32)
+    st = ora.channel_stats(y)
+    cnt = 3 * 7 * 6
+    mean = st["sum_y"][0] / cnt
+    var = st["sum_y2"][0] / cnt - mean ** 2
+    assert np.allclose(mean, y.astype(np.float64).mean(axis=(0, 2, 3)), rtol=0, atol=1e-12)
+    assert np.allclose(var, y.astype(np.float64).var(axis=(0, 2, 3)), rtol=0, atol=1e-12)
+    c = np.full((2, 4, 3, 3), 1.5, np.float32)
+    st = ora.channel_stats(c)
+    assert np.array_equal(st["sum_y"][0], np.full(4, 18 * 1.5)) and np.array_equal(st["sum_y2"][0], np.full(4, 18 * 2.25))
