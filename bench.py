@@ -529,7 +529,8 @@ def run_cfg5(args):
     torch.manual_seed(1050)
     rs = np.random.RandomState(1050)
     N = 64
-    net = HybridResNet18(mode=args.only or "compound", dtype="bf16").cuda()
+    net = HybridResNet18(mode=args.only or "compound", dtype="bf16", fused_bn=args.fused_bn).cuda()
+    TropicalConvFn.fuse_cast = bool(args.fuse_cast)
     x = torch.from_numpy(rs.standard_normal((N, 3, 224, 224)).astype(np.float32)).cuda()
     labels = torch.from_numpy(rs.randint(0, 1000, N)).cuda()
     opt = torch.optim.SGD(net.parameters(), lr=0.01, momentum=0.9)
@@ -560,7 +561,8 @@ def run_cfg5(args):
     taps = sum(d["N"] * d["K"] * d["C"] * 9 * tconv.tconv_output_shape(d)[0] * tconv.tconv_output_shape(d)[1]
                for k, d, a, b in ev if k == "fwd") / args.steps
     print(json.dumps({"workload": "cfg5: ResNet-18-shaped hybrid net, N=64, 224x224, stages 2-4 tropical (bf16 kernels)",
-                      "mode": args.only or "compound", "step_ms": ms, "tropical_fwd_ms": t_fwd,
+                      "mode": args.only or "compound", "fused_bn": bool(args.fused_bn),
+                      "float_x_read_by_the_kernels": bool(args.fuse_cast), "step_ms": ms, "tropical_fwd_ms": t_fwd,
                       "tropical_bwd_ms": t_bwd, "tropical_layers": len([1 for e in ev if e[0] == "fwd"]) // args.steps,
                       "tropical_taps_fwd": taps, "tropical_Gop_s_fwd_bwd": ops / ((t_fwd + t_bwd) * 1e-3) / 1e9,
                       "loss": float(loss.detach())}))
@@ -689,6 +691,10 @@ def main():
     ap.add_argument("--what", default="fwd", choices=["fwd", "fwd_winners", "bwd"])
     ap.add_argument("--images", type=int, default=128)
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
+    ap.add_argument("--fused-bn", action="store_true",
+                    help="cfg5: batch-normalisation statistics from the tropical kernels' epilogue")
+    ap.add_argument("--fuse-cast", action="store_true",
+                    help="cfg5: the bf16 kernels read the float activations directly (x_dtype) instead of a converted copy")
     ap.add_argument("--no-headline", action="store_true",
                     help="skip the headline_layers section (cfg 3a / 3b / 4 timed after the step)")
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5", "dw", "conv3d"],

@@ -25,6 +25,10 @@ class TropicalConvFn(torch.autograd.Function):
     call is bracketed by a pair of CUDA events appended to it (for the benchmark's per-layer times)."""
 
     events = None
+    # True: bf16 layers read a float x directly (x_dtype) instead of a converted copy.  Off by default:
+    # the conversion while staging rules out the copy-engine path, which costs more than the cast
+    # kernel saves on the ResNet-18 shape (tropical forward 21.5 -> 23.9 ms per step).
+    fuse_cast = False
 
     @staticmethod
     def forward(ctx, x, w, w2, alpha, beta, bias, geom):
@@ -34,7 +38,12 @@ class TropicalConvFn(torch.autograd.Function):
         K, _, R, S = w.shape
         d = dict(N=N, C=C, H=H, W=W, K=K, R=R, S=S, stride_h=stride[0], stride_w=stride[1],
                  pad_h=pad[0], pad_w=pad[1], dil_h=dil[0], dil_w=dil[1], mode=mode, chan=chan, dtype=dtype)
-        xc = x.detach().to(dt).contiguous()
+        # a float x for a bf16 layer is rounded by the kernel while it stages x (no cast kernel, no
+        # bf16 copy); layers the tiled kernels do not serve fall back to the explicit cast
+        fused_cast = TropicalConvFn.fuse_cast and dtype == "bf16" and x.dtype == torch.float32
+        xc = x.detach().contiguous() if fused_cast else x.detach().to(dt).contiguous()
+        if fused_cast:
+            d["x_dtype"] = "f32"
         wc = w.detach().to(dt).contiguous()
         w2c = w2.detach().to(dt).contiguous() if w2 is not None else None
         al = alpha.detach().float().contiguous() if alpha is not None else None
@@ -45,7 +54,14 @@ class TropicalConvFn(torch.autograd.Function):
         if ev is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-        y, winners = tconv.forward(d, xc, wc, w2c, al, be, bi, want_winners=need_grad)
+        try:
+            y, winners = tconv.forward(d, xc, wc, w2c, al, be, bi, want_winners=need_grad)
+        except tconv.TconvError as err:
+            if not fused_cast or err.status != -2:
+                raise
+            d.pop("x_dtype")
+            xc = x.detach().to(dt).contiguous()
+            y, winners = tconv.forward(d, xc, wc, w2c, al, be, bi, want_winners=need_grad)
         if ev is not None:
             e1.record()
             ev.append(("fwd", d, e0, e1))
@@ -68,7 +84,13 @@ class TropicalConvFn(torch.autograd.Function):
         need = ["grad_w", "grad_w2", "grad_alpha", "grad_beta", "grad_bias"]
         if ctx.needs_input_grad[0]:
             need.append("grad_x")          # a first layer's input needs none: the kernel is skipped
-        grads = tconv.backward(d, xc, wc, g, w2c, al, be, winners, need=tuple(need))
+        try:
+            grads = tconv.backward(d, xc, wc, g, w2c, al, be, winners, need=tuple(need))
+        except tconv.TconvError as err:
+            if d.get("x_dtype") != "f32" or err.status != -2:
+                raise
+            d = {k: v for k, v in d.items() if k != "x_dtype"}      # a path that reads x itself: convert first
+            grads = tconv.backward(d, xc.to(dt), wc, g, w2c, al, be, winners, need=tuple(need))
         if ev is not None:
             e1.record()
             ev.append(("bwd", d, e0, e1))
@@ -77,6 +99,115 @@ class TropicalConvFn(torch.autograd.Function):
         return (gx, grads["grad_w"], grads.get("grad_w2") if has_w2 else None,
                 grads.get("grad_alpha") if has_a else None, grads.get("grad_beta") if has_b else None,
                 grads["grad_bias"] if has_bias else None, None)
+
+
+class TropicalConvBNFn(torch.autograd.Function):
+    """Tropical layer followed by training-mode batch normalisation, the pair the paper's residual
+    blocks are made of (section "ResNet Models").  The layer's kernel leaves the per-channel sums of
+    y and y^2 (tconv_forward_stats), so the normalisation reads y once (scale and shift) instead of
+    twice (statistics, then scale and shift).  Backward: the usual batch-normalisation gradient
+    (channel reductions of grad and grad * y, then one elementwise pass), then tconv_backward."""
+
+    @staticmethod
+    def forward(ctx, x, w, w2, alpha, beta, gamma, bn_bias, geom, eps):
+        mode, chan, dtype, stride, pad, dil = geom
+        dt = tconv.TORCH_DTYPE[dtype]
+        N, C, H, W = x.shape
+        K, _, R, S = w.shape
+        d = dict(N=N, C=C, H=H, W=W, K=K, R=R, S=S, stride_h=stride[0], stride_w=stride[1],
+                 pad_h=pad[0], pad_w=pad[1], dil_h=dil[0], dil_w=dil[1], mode=mode, chan=chan, dtype=dtype)
+        fused_cast = TropicalConvFn.fuse_cast and dtype == "bf16" and x.dtype == torch.float32
+        xc = x.detach().contiguous() if fused_cast else x.detach().to(dt).contiguous()
+        if fused_cast:
+            d["x_dtype"] = "f32"
+        wc = w.detach().to(dt).contiguous()
+        w2c = w2.detach().to(dt).contiguous() if w2 is not None else None
+        al = alpha.detach().float().contiguous() if alpha is not None else None
+        be = beta.detach().float().contiguous() if beta is not None else None
+        ev = TropicalConvFn.events
+        if ev is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        try:
+            y, winners, s1, s2 = tconv.forward_stats(d, xc, wc, w2c, al, be, None, want_winners=True)
+        except tconv.TconvError as err:
+            if not fused_cast or err.status != -2:
+                raise
+            d.pop("x_dtype")
+            xc = x.detach().to(dt).contiguous()
+            y, winners, s1, s2 = tconv.forward_stats(d, xc, wc, w2c, al, be, None, want_winners=True)
+        if ev is not None:
+            e1.record()
+            ev.append(("fwd", d, e0, e1))
+        cnt = float(y.shape[0] * y.shape[2] * y.shape[3])
+        mean = s1 / cnt
+        var = (s2 / cnt - mean * mean).clamp_min_(0.0)          # biased variance of the batch
+        invstd = torch.rsqrt(var + eps)
+        scale = gamma.detach().float() * invstd
+        shift = bn_bias.detach().float() - mean * scale
+        out = torch.addcmul(shift.view(1, -1, 1, 1), y, scale.view(1, -1, 1, 1))    # one pass over y, fp32 result
+        ctx.d, ctx.in_dtype, ctx.cnt = d, x.dtype, cnt
+        ctx.save_for_backward(xc, wc, w2c, al, be, winners, y, mean, invstd, gamma.detach().float())
+        ctx.has = (w2 is not None, alpha is not None, beta is not None)
+        ctx.mark_non_differentiable(mean, var)
+        return out.to(x.dtype), mean, var
+
+    @staticmethod
+    def backward(ctx, go, _gm, _gv):
+        xc, wc, w2c, al, be, winners, y, mean, invstd, gamma = ctx.saved_tensors
+        d, cnt = ctx.d, ctx.cnt
+        dt = tconv.TORCH_DTYPE[d["dtype"]]
+        go = go.float()
+        yf = y.float()
+        sum_go = go.sum(dim=(0, 2, 3))
+        sum_go_y = (go * yf).sum(dim=(0, 2, 3))
+        sum_go_xmu = sum_go_y - mean * sum_go
+        g_gamma = sum_go_xmu * invstd
+        g_bias = sum_go
+        # dy = gamma * invstd * (go - sum_go / cnt - (y - mean) * invstd^2 * sum_go_xmu / cnt)
+        k1 = (gamma * invstd).view(1, -1, 1, 1)
+        k2 = (invstd * invstd * sum_go_xmu / cnt).view(1, -1, 1, 1)
+        k3 = (sum_go / cnt - mean * invstd * invstd * sum_go_xmu / cnt).view(1, -1, 1, 1)
+        gy = (k1 * (go - yf * k2 - k3)).to(dt).contiguous()
+        ev = TropicalConvFn.events
+        if ev is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        need = ["grad_w", "grad_w2", "grad_alpha", "grad_beta"]
+        if ctx.needs_input_grad[0]:
+            need.append("grad_x")
+        try:
+            grads = tconv.backward(d, xc, wc, gy, w2c, al, be, winners, need=tuple(need))
+        except tconv.TconvError as err:
+            if d.get("x_dtype") != "f32" or err.status != -2:
+                raise
+            d = {k: v for k, v in d.items() if k != "x_dtype"}
+            grads = tconv.backward(d, xc.to(dt), wc, gy, w2c, al, be, winners, need=tuple(need))
+        if ev is not None:
+            e1.record()
+            ev.append(("bwd", d, e0, e1))
+        has_w2, has_a, has_b = ctx.has
+        gx = grads["grad_x"].to(ctx.in_dtype) if "grad_x" in grads else None
+        return (gx, grads["grad_w"], grads.get("grad_w2") if has_w2 else None,
+                grads.get("grad_alpha") if has_a else None, grads.get("grad_beta") if has_b else None,
+                g_gamma, g_bias, None, None)
+
+
+def tropical_conv_bn(conv: "TropicalConv2d", bn: nn.BatchNorm2d, x):
+    """conv followed by bn; in training mode with the layer's fused channel statistics."""
+    if not (bn.training and x.is_cuda and conv.bias is None and bn.affine and bn.track_running_stats
+            and conv.params in ("2p", "0p") and type(conv) is TropicalConv2d):
+        return bn(conv(x))
+    geom = (conv.mode, conv.chan, conv.dtype, conv.stride, conv.padding, conv.dilation)
+    out, mean, var = TropicalConvBNFn.apply(x, conv.weight, conv.weight2, conv.alpha, conv.beta, bn.weight, bn.bias,
+                                            geom, bn.eps)
+    with torch.no_grad():
+        cnt = out.shape[0] * out.shape[2] * out.shape[3]
+        m = bn.momentum if bn.momentum is not None else 0.1
+        bn.running_mean.mul_(1 - m).add_(mean, alpha=m)
+        bn.running_var.mul_(1 - m).add_(var * (cnt / max(cnt - 1, 1)), alpha=m)
+        bn.num_batches_tracked += 1
+    return out
 
 
 class TropicalConv2d(nn.Module):
@@ -153,8 +284,9 @@ class TropicalBasicBlock(nn.Module):
     """The paper's TCNN basic block 2: Tropical - BN - Tropical - BN, intermediate ReLU removed,
     identity (or 1x1 standard-convolution) shortcut, ReLU after the sum."""
 
-    def __init__(self, cin, cout, stride, mode, dtype):
+    def __init__(self, cin, cout, stride, mode, dtype, fused_bn=False):
         super().__init__()
+        self.fused_bn = fused_bn    # batch-normalisation statistics from the tropical kernels' epilogue
         self.conv1 = TropicalConv2d(cin, cout, 3, stride=stride, padding=1, bias=False, mode=mode, dtype=dtype)
         self.bn1 = nn.BatchNorm2d(cout)
         self.conv2 = TropicalConv2d(cout, cout, 3, stride=1, padding=1, bias=False, mode=mode, dtype=dtype)
@@ -164,7 +296,10 @@ class TropicalBasicBlock(nn.Module):
             self.down = nn.Sequential(nn.Conv2d(cin, cout, 1, stride=stride, bias=False), nn.BatchNorm2d(cout))
 
     def forward(self, x):
-        out = self.bn2(self.conv2(self.bn1(self.conv1(x))))
+        if self.fused_bn:
+            out = tropical_conv_bn(self.conv2, self.bn2, tropical_conv_bn(self.conv1, self.bn1, x))
+        else:
+            out = self.bn2(self.conv2(self.bn1(self.conv1(x))))
         return torch.relu(out + (x if self.down is None else self.down(x)))
 
 
@@ -184,14 +319,14 @@ class HybridResNet18(nn.Module):
     """ResNet-18 shape; every 3x3 convolution of stages 2-4 is a tropical layer of the given mode
     (stem, stage 1 and the 1x1 downsamples are standard convolutions)."""
 
-    def __init__(self, mode="compound", dtype="bf16", num_classes=1000):
+    def __init__(self, mode="compound", dtype="bf16", num_classes=1000, fused_bn=False):
         super().__init__()
         self.stem = nn.Sequential(nn.Conv2d(3, 64, 7, stride=2, padding=3, bias=False), nn.BatchNorm2d(64),
                                   nn.ReLU(inplace=True), nn.MaxPool2d(3, stride=2, padding=1))
         self.layer1 = nn.Sequential(StandardBasicBlock(64, 64, 1), StandardBasicBlock(64, 64, 1))
-        self.layer2 = nn.Sequential(TropicalBasicBlock(64, 128, 2, mode, dtype), TropicalBasicBlock(128, 128, 1, mode, dtype))
-        self.layer3 = nn.Sequential(TropicalBasicBlock(128, 256, 2, mode, dtype), TropicalBasicBlock(256, 256, 1, mode, dtype))
-        self.layer4 = nn.Sequential(TropicalBasicBlock(256, 512, 2, mode, dtype), TropicalBasicBlock(512, 512, 1, mode, dtype))
+        self.layer2 = nn.Sequential(TropicalBasicBlock(64, 128, 2, mode, dtype, fused_bn), TropicalBasicBlock(128, 128, 1, mode, dtype, fused_bn))
+        self.layer3 = nn.Sequential(TropicalBasicBlock(128, 256, 2, mode, dtype, fused_bn), TropicalBasicBlock(256, 256, 1, mode, dtype, fused_bn))
+        self.layer4 = nn.Sequential(TropicalBasicBlock(256, 512, 2, mode, dtype, fused_bn), TropicalBasicBlock(512, 512, 1, mode, dtype, fused_bn))
         self.head = nn.Sequential(nn.AdaptiveAvgPool2d(1), nn.Flatten(), nn.Linear(512, num_classes))
 
     def forward(self, x):
