@@ -36,7 +36,6 @@ def _nvcc_base(verbose: bool):
            "-Xcompiler", "-fPIC", "-I", str(ROOT / "include"), "-I", str(CSRC)]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("TCONV_NVCC_EXTRA", "").split()   # experiment switches (-D...)
     return cmd
 
 

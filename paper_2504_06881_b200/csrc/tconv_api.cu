@@ -500,7 +500,7 @@ int dw_forward_t(const Geo& g, const void* x, const void* w, const void* w2, con
     const int QPR = (g.OW + 3) / 4;
     if (g.R == 3 && g.S == 3 && g.dh == 1 && g.dw == 1 && g.sh == g.sw && (g.sw == 1 || g.sw == 2)) {
         // 3x3 windows: strips of 4 columns x 6 rows with a register window of three input rows
-        const int strips = (g.OH + TCONV_DW_RT - 1) / TCONV_DW_RT;
+        const int strips = (g.OH + kDwRT - 1) / kDwRT;
         const size_t total3 = (size_t)g.N * g.C * strips * QPR;
         const unsigned blocks3 = (unsigned)((total3 + 255) / 256);
         const bool vec = (g.pw == 1 && (g.W & 3) == 0);
@@ -600,7 +600,7 @@ int dw_backward_t(const Geo& g, const void* x, const void* w, const void* w2, co
                         nch <= g.N && g.OH * g.OW >= 100;   // tiny planes: too few strips per image
         if (k3) {
             // 3x3 windows: strips over a register window, the chunks are ranges of images
-            const int QPR3 = (g.OW + 3) / 4, strips3 = (g.OH + TCONV_DW_RT - 1) / TCONV_DW_RT;
+            const int QPR3 = (g.OW + 3) / 4, strips3 = (g.OH + kDwRT - 1) / kDwRT;
             const bool vec3 = (g.pw == 1 && (g.W & 3) == 0);
 #define TCONV_DW_P3(BR, PARV, SWV, VECV)                                                              \
     {                                                                                                \

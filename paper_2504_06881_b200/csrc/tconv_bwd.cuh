@@ -852,14 +852,6 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
     pl->ncol = 1;
     pl->TWI = g.W;
     pl->QPRt = pl->QPR;
-    static const char* force = getenv("TCONV_GX_PLAN");   // debug switch: "cb,ncol,kilobytes"
-    if (force) {
-        int cb = 0, ncol = 0, kb = 0;
-        if (sscanf(force, "%d,%d,%d", &cb, &ncol, &kb) == 3 && cb >= 1 && cb <= kGxCB && ncol >= 1 && kb >= 16 &&
-            !g.wide && plan_code_gx_cols(g, cb, ncol, (size_t)kb * 1024, pl))
-            return true;
-        pl->ncol = 1; pl->TWI = g.W; pl->QPRt = pl->QPR;
-    }
     // Maps with at least 128 quads (smaller ones share a CTA between several images, below): one
     // channel per CTA and a small tile, so that five CTAs stay resident per SM and hide the latency
     // of the code loads (measured on 32x32 to 128x256 maps: 5 to 35 % faster than two channels in

@@ -167,16 +167,15 @@ __device__ __forceinline__ void dw_load_row(const T* rp, bool row_ok, unsigned m
 // columns x RT output rows of one (n, c) plane and slides a window of three input rows held in
 // registers down the strip: every input row of the strip is loaded once per thread.  The nine
 // weights of the channel sit in registers.
+constexpr int kDwRT = 6;   // output rows per strip of the 3x3 depthwise kernels
+
 template <typename T, int MODE, bool WIN, int SW, bool VEC>
 __global__ void __launch_bounds__(256)
 dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
                const float* __restrict__ alpha, const float* __restrict__ beta,
                const float* __restrict__ bias, T* __restrict__ y, uint8_t* __restrict__ codes,
                int QPR, int strips, unsigned total) {
-#ifndef TCONV_DW_RT
-#define TCONV_DW_RT 6
-#endif
-    constexpr int RT = TCONV_DW_RT;             // output rows per strip
+    constexpr int RT = kDwRT;             // output rows per strip
     constexpr int L = 3 * SW + 3;               // input columns 4 outputs touch
     constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
     constexpr bool PAR = (MODE == TCONV_PARALLEL);
@@ -531,7 +530,7 @@ __global__ void __launch_bounds__(256)
 dw_bwd_params3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
                       const T* __restrict__ gy, const uint8_t* __restrict__ codes,
                       float* __restrict__ partial, int nchunks, int need_ab, int QPR, int strips) {
-    constexpr int RT = TCONV_DW_RT;
+    constexpr int RT = kDwRT;
     constexpr int L = 3 * SW + 3;
     extern __shared__ float col[];   // [kDwAcc][256]
     const int c = blockIdx.x, chunk = blockIdx.y, tid = threadIdx.x;

@@ -83,10 +83,13 @@ __device__ __forceinline__ void mbar_init(void* bar, unsigned count) {
 __device__ __forceinline__ void mbar_expect_tx(void* bar, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Bounded wait: gives up after a fixed number of polls and reports failure.
-__device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity) {
+// Bounded wait: gives up after `limit` polls and reports failure.  A poll that finds the phase
+// incomplete blocks for a hardware time slice (measured: 4 us), so 2^16 polls bound a wait at a
+// quarter of a second, five orders of magnitude above the microseconds a copy takes.
+constexpr int kPollLimit = 1 << 16;
+__device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity, int limit = kPollLimit) {
     const unsigned addr = smem_u32(bar);
-    for (int i = 0; i < (1 << 20); ++i) {
+    for (int i = 0; i < limit; ++i) {
         unsigned ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -203,6 +206,8 @@ struct TiledParams {
     float* stats;      // NULL, or per-tile partial sums {sum y, sum y^2} per output channel: [tile][stats_k][2]
     int stats_k;       // channel pitch of the partials (K rounded up to the k tile)
     int* status;       // device status word: set non-zero when a bounded wait gives up
+    int poll_limit;    // polls a wait may take (kPollLimit; lower under the failure-test switch)
+    int debug_drop;    // failure-test switch: the copies of the first chunk are never issued
     int TW, QPR, TH;   // tile: output columns, quads per row, output rows
     int n_col_tiles, n_row_tiles;
     int tiles_per_img; // > 0: row tiles stay inside one image; 0: rows run over the flattened (n, oh) space
@@ -231,21 +236,15 @@ template <int S, int DW, int ESIZE = 4> struct TmaShift {
 // Q quads of 4 pixels per thread, KG groups of 8 output channels and PW pixel warps per CTA.
 // Resident CTAs per SM the register allocation aims at: the winner-free kernels are bound by
 // the ALU / FMA pipes and want four or more warps per scheduler to hide their latencies.
-#ifndef TCONV_MINB_SINGLE
-#define TCONV_MINB_SINGLE 4
-#endif
-#ifndef TCONV_MINB_WINSUM
-#define TCONV_MINB_WINSUM 3
-#endif
-#ifndef TCONV_Q_CARRIED
-#define TCONV_Q_CARRIED 2
-#endif
+constexpr int kMinBlocksSingle = 4;   // single-branch kernels
+constexpr int kMinBlocksWinSum = 3;   // Sum forms that emit winners (168 registers)
+constexpr int kQuadsCarried = 2;      // quads per thread of the carried max-plus / min-plus chain
 template <int MODE, int CHAN, bool WIN, bool XTMA, bool RAG, int R, int S, int SW, int DW, int Q, int KG, int PW, int TK>
 __global__ void __launch_bounds__(KG * PW * 32,
-                                  (WIN && CHAN == CH_SUM) ? TCONV_MINB_WINSUM
+                                  (WIN && CHAN == CH_SUM) ? kMinBlocksWinSum
                                   : WIN ? 1
                                   : (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL) ? (TK == 4 ? 4 : 1)
-                                  : TCONV_MINB_SINGLE)
+                                  : kMinBlocksSingle)
 fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams p) {
     static_assert(TK == 2 || TK == 4 || TK == 8, "output channels per thread");
     constexpr int RS = R * S;
@@ -353,7 +352,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
         float* st = stage0 + s * p.stage_floats;
         const int c0 = ch * p.CC;
         if constexpr (XTMA) {
-            if (tid == 0) {
+            if (tid == 0 && !(p.debug_drop && ch == 0)) {
                 const unsigned bytes = (unsigned)((p.xbox * (two_imgs ? 2 : 1) + p.w_stage * (PAR ? 2 : 1) + 2 * p.ab_stage) * sizeof(float));
                 mbar_expect_tx(&bars[s], bytes);
                 tma_load_3d(st, &xmap, iw0 - SHIFT, oh_first * g.sh - g.ph, n0 * g.C + c0, &bars[s]);
@@ -436,12 +435,12 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
         float* st = stage0 + s * p.stage_floats;
         if (ch + 1 < p.nchunks) issue_chunk(ch + 1, s ^ 1);
         if constexpr (XTMA) {
-            if (!mbar_wait(&bars[s], (ch >> 1) & 1)) {
+            if (!mbar_wait(&bars[s], (ch >> 1) & 1, p.poll_limit)) {
                 // the copy did not land in time: flag it, give the copies in flight one more
                 // bounded chance to finish, and leave
                 if (p.status) *p.status = 1;
-                mbar_wait(&bars[s], (ch >> 1) & 1);
-                if (ch + 1 < p.nchunks) mbar_wait(&bars[s ^ 1], ((ch + 1) >> 1) & 1);
+                mbar_wait(&bars[s], (ch >> 1) & 1, p.poll_limit);
+                if (ch + 1 < p.nchunks) mbar_wait(&bars[s ^ 1], ((ch + 1) >> 1) & 1, p.poll_limit);
                 return;
             }
         } else {
@@ -771,6 +770,19 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
 
 // ----------------------------------------------------------------------------------
 // host side: tile selection and launch
+
+// Failure-test switch (environment, read once): TCONV_DEBUG_DROP_COPY=<polls> makes the copy-engine
+// kernels skip the copies of their first chunk and lowers the poll limit of their waits to <polls>,
+// so that a test can watch a bounded wait run out with nothing in flight.  0 / unset: off.
+inline int failure_test_polls() {
+    static const int v = [] {
+        const char* e = getenv("TCONV_DEBUG_DROP_COPY");
+        const long n = e ? atol(e) : 0;
+        return (int)(n < 0 ? 0 : (n > kPollLimit ? kPollLimit : n));
+    }();
+    return v;
+}
+
 struct TiledPlan {
     TiledParams p;
     dim3 grid;
@@ -884,9 +896,6 @@ inline bool plan_tiles_opt(const Geo& g, bool par, bool two, int esize, bool all
 // the order ragged / whole rows, 8 / 4 channels per chunk; else whole rows with 8 channels.
 template <int R, int S, int SW, int DW, int Q, int KG, int PW, int TK = 8>
 inline bool plan_tiles(const Geo& g, bool par, bool two, int esize, TiledPlan* pl) {
-    static const char* force = getenv("TCONV_PLAN");   // debug switch: "r8", "r6", "r4", "n8", "n6", "n4"
-    if (force && (force[0] == 'r' || force[0] == 'n') && (force[1] == '8' || force[1] == '6' || force[1] == '4'))
-        return plan_tiles_opt<R, S, SW, DW, Q, KG, PW, TK>(g, par, two, esize, force[0] == 'r', force[1] - '0', pl);
     // 8 channels per chunk when four CTAs stay resident, else 4 channels when three do (measured
     // on the stride-2 56 -> 28 layer: 8.06 against 7.86 Ttap/s for whole-row tiles at four CTAs)
     // (two-branch kernels with 8 channels per thread hold two CTAs per SM by their registers: their
@@ -983,6 +992,8 @@ int launch_tiled_variant(FwdArgs& a) {
         if ((size_t)pl.grid.x * pl.p.stats_k * 2 * sizeof(float) > a.stats_bytes) return TCONV_ERR_WORKSPACE_TOO_SMALL;
         pl.p.stats = a.stats; a.stats_tiles = (int)pl.grid.x; a.stats_k = pl.p.stats_k;
     }
+    pl.p.debug_drop = failure_test_polls() > 0;
+    pl.p.poll_limit = pl.p.debug_drop ? failure_test_polls() : kPollLimit;
 #define TCONV_LAUNCH_F32(XTMAV, RAGV)                                                                 \
     {                                                                                                \
         auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, TK>; \
@@ -1010,17 +1021,11 @@ int launch_tiled_geom(FwdArgs& a) {
     // extremum of layers (iv), (v) without winners), else one
     constexpr bool CARRIED = !TWO && !WIN && ((MODE == TCONV_MAX_PLUS && CHAN == CH_MAX) ||
                                               (MODE == TCONV_MIN_PLUS && CHAN == CH_MIN));
-    constexpr int Q = CARRIED ? TCONV_Q_CARRIED : 1;
+    constexpr int Q = CARRIED ? kQuadsCarried : 1;
     // Sum forms that emit winners work on one pair of output channels at a time: 4 channels per
     // thread (2 or 8 measured no faster); two-branch kernels keep three values per output: 4 channels per thread leave room for
     // four resident CTAs per SM (measured 3-6 % faster than 8 channels per thread)
-#ifndef TCONV_TK_TWO
-#define TCONV_TK_TWO 4
-#endif
-#ifndef TCONV_TK_WINSUM
-#define TCONV_TK_WINSUM 4
-#endif
-    constexpr int TK = (WIN && CHAN == CH_SUM) ? TCONV_TK_WINSUM : (TWO ? TCONV_TK_TWO : 8);
+    constexpr int TK = (WIN && CHAN == CH_SUM) ? 4 : (TWO ? 4 : 8);
     const Geo& g = a.g;
     if (g.R == 3 && g.S == 3) {
         if (g.sw == 1 && g.dw == 1) return launch_tiled_variant<T, MODE, CHAN, WIN, 3, 3, 1, 1, Q, 4, 1, TK>(a);

@@ -259,7 +259,7 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
         unsigned* st = stage0 + s * p.stage_floats;
         const int c0 = ch * p.CC;
         if constexpr (XTMA) {
-            if (tid == 0) {
+            if (tid == 0 && !(p.debug_drop && ch == 0)) {
                 const unsigned bytes = (unsigned)(p.xbox * 2 * (two_imgs ? 2 : 1) +
                                                   (p.w_stage * (PAR ? 2 : 1) + 2 * p.ab_stage) * 4);
                 mbar_expect_tx(&bars[s], bytes);
@@ -333,10 +333,10 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
         unsigned* st = stage0 + s * p.stage_floats;
         if (ch + 1 < p.nchunks) issue_chunk(ch + 1, s ^ 1);
         if constexpr (XTMA) {
-            if (!mbar_wait(&bars[s], (ch >> 1) & 1)) {
+            if (!mbar_wait(&bars[s], (ch >> 1) & 1, p.poll_limit)) {
                 if (p.status) *p.status = 1;
-                mbar_wait(&bars[s], (ch >> 1) & 1);
-                if (ch + 1 < p.nchunks) mbar_wait(&bars[s ^ 1], ((ch + 1) >> 1) & 1);
+                mbar_wait(&bars[s], (ch >> 1) & 1, p.poll_limit);
+                if (ch + 1 < p.nchunks) mbar_wait(&bars[s ^ 1], ((ch + 1) >> 1) & 1, p.poll_limit);
                 return;
             }
         } else {
@@ -661,6 +661,8 @@ int launch_tiled_variant_bf16(FwdArgs& a) {
         if ((size_t)pl.grid.x * pl.p.stats_k * 2 * sizeof(float) > a.stats_bytes) return TCONV_ERR_WORKSPACE_TOO_SMALL;
         pl.p.stats = a.stats; a.stats_tiles = (int)pl.grid.x; a.stats_k = pl.p.stats_k;
     }
+    pl.p.debug_drop = failure_test_polls() > 0;
+    pl.p.poll_limit = pl.p.debug_drop ? failure_test_polls() : kPollLimit;
 #define TCONV_LAUNCH_BF16(XTMAV, RAGV)                                                                \
     {                                                                                                \
         auto kern = fwd_tiled_bf16_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, KPT>; \
@@ -695,9 +697,8 @@ int launch_tiled_geom_bf16(FwdArgs& a) {
         // as one CTA): 4 channels per thread double the warps.  Measured on the 14x14 and 7x7 layers
         // of the ResNet-18 shape at batch 64: 4 to 12 % faster with winners, 6 to 13 % slower
         // without (there the second staging of the x tiles costs more), so only with winners.
-        static const int k4 = getenv("TCONV_BF16_K4") ? atoi(getenv("TCONV_BF16_K4")) : -1;   // debug switch: 0 off, 1 always
         const long warps8 = (((long)g.N * g.OH * ((g.OW + 3) / 4) + 31) / 32) * ((g.K + 7) / 8);
-        const bool fine = k4 == 0 ? false : (k4 == 1 ? true : (WIN && warps8 < 148L * 32));
+        const bool fine = WIN && warps8 < 148L * 32;
         if constexpr (Q == 1) {
             if (fine && g.dw == 1 && (g.sw == 1 || g.sw == 2)) {
                 const int rc = g.sw == 1 ? launch_tiled_variant_bf16<MODE, CHAN, WIN, 3, 3, 1, 1, 1, 4, 1, 4, true>(a)
