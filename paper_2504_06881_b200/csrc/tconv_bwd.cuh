@@ -201,14 +201,31 @@ bwd_idx_gw_kernel(Geo g, const T* __restrict__ gy, const int32_t* __restrict__ i
     const int n_lo = chunk * n_per_chunk, n_hi = min(g.N, n_lo + n_per_chunk);
     const unsigned lt = lanemask_lt();
     float bsum = 0.0f;
-    for (int n = n_lo; n < n_hi; ++n) {
-        const size_t base = ((size_t)n * g.K + k) * plane;
-        for (int p0 = 0; p0 < plane; p0 += 256) {
-            const int p = p0 + threadIdx.x;
-            const bool valid = p < plane;
-            // an out-of-range lane takes a bin of its own so that it matches nobody
-            const int id = valid ? idx[base + p] : -1 - (int)threadIdx.x;
-            const float gv = valid ? to_f32(gy[base + p]) : 0.0f;
+    // items of the chunk in a fixed order: (image, block of 256 pixels); the winners and gradients of
+    // the next PF items are requested before the current ones are binned
+    constexpr int PF = 4;
+    const int blocks_per_img = (plane + 255) / 256;
+    const int items = (n_hi - n_lo) * blocks_per_img;
+    auto fetch = [&](int it, int& id, float& gv) {
+        const int nn = it / blocks_per_img, p = (it - nn * blocks_per_img) * 256 + (int)threadIdx.x;
+        const bool valid = it < items && p < plane;
+        const size_t at = ((size_t)(n_lo + nn) * g.K + k) * plane + p;
+        // an out-of-range lane takes a bin of its own so that it matches nobody
+        id = valid ? __ldg(idx + at) : -1 - (int)threadIdx.x;
+        gv = valid ? to_f32(__ldg(gy + at)) : 0.0f;
+    };
+    int idq[PF];
+    float gq[PF];
+#pragma unroll
+    for (int u = 0; u < PF; ++u) fetch(u, idq[u], gq[u]);
+    for (int it0 = 0; it0 < items; it0 += PF) {
+#pragma unroll
+        for (int u = 0; u < PF; ++u) {
+            if (it0 + u >= items) break;
+            const int id = idq[u];
+            const float gv = gq[u];
+            fetch(it0 + u + PF, idq[u], gq[u]);
+            const bool valid = id >= 0;
             bsum += gv;
             const unsigned same = __match_any_sync(0xffffffffu, id);
             const int rank = __popc(same & lt);

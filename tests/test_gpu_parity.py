@@ -141,15 +141,21 @@ def test_single_pixel_and_single_channel_edges():
         parity.check_layer(dict(d, dtype="bf16"), None, 702)
 
 
-def test_backward_is_deterministic():
-    d = inputs.layer(4, 16, 20, 20, 24, 3, 3, pad=1, mode="parallel")
-    t = inputs.draw(d, 801)
+@pytest.mark.parametrize("mode,dist", [("parallel", None), ("max_plus", None), ("min_plus", None),
+                                       ("max_plus", dict(x=("ints", -1, 1), w=("ints", -1, 1)))])
+def test_backward_is_deterministic(mode, dist):
+    """Three runs give the same bits: the Sum forms (private columns, fixed trees) and the Max / Min
+    channel combines (row phases, ordered sub-steps, warp-private histograms), random and tie-heavy
+    winners, several row bands and column blocks."""
+    d = inputs.layer(4, 16, 40, 44, 24, 3, 3, pad=1, mode=mode)
+    t = inputs.draw(d, 801, **(dist or {}))
     from paper_2504_06881_b200 import tconv
     g = parity.to_dev(t, d)
+    la = parity.layer_args(d, g)
     runs = []
     for _ in range(3):
-        _, win = tconv.forward(d, g["x"], g["w"], g["w2"], g["alpha"], g["beta"], g["bias"], want_winners=True)
-        out = tconv.backward(d, g["x"], g["w"], g["g"], g["w2"], g["alpha"], g["beta"], win)
+        _, win = tconv.forward(d, g["x"], g["w"], la["w2"], la["alpha"], la["beta"], g["bias"], want_winners=True)
+        out = tconv.backward(d, g["x"], g["w"], g["g"], la["w2"], la["alpha"], la["beta"], win)
         torch.cuda.synchronize()
         runs.append({k: v.clone() for k, v in out.items()})
     for k in runs[0]:
