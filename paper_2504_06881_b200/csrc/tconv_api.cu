@@ -155,6 +155,16 @@ size_t stats_scratch_bytes(const Geo& g) {
     return align_up(tiles * kp * 2 * sizeof(float), 256);
 }
 
+// Channel statistics from a stored output (calls without winners, layers of the any-shape kernels).
+template <typename T>
+void stats_from_output(const Geo& g, const void* y, float* stats_ws, float* sum_y, float* sum_y2, cudaStream_t st) {
+    const int chunks = g.N < 16 ? g.N : 16, npc = (g.N + chunks - 1) / chunks;
+    const int rows = (g.N + npc - 1) / npc;
+    stats_direct_kernel<T><<<dim3((unsigned)g.K, (unsigned)rows), 256, 0, st>>>(g, (const T*)y, stats_ws, npc);
+    stats_finish_kernel<<<(unsigned)((g.K * 32 + 255) / 256), 256, 0, st>>>(stats_ws, rows, g.K, g.K, sum_y, sum_y2);
+    g_launches += 2;
+}
+
 // stats_ws: NULL, or scratch of stats_scratch_bytes() for the per-tile channel statistics, which are
 // then summed into sum_y / sum_y2.
 template <typename T>
@@ -173,10 +183,12 @@ int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const 
         if (rc == TCONV_OK) {
             snprintf(g_last_kernel, sizeof(g_last_kernel), "%s", a.name);
             g_launches += 2;  // weight repack + tiled kernel
-            if (stats_ws) {
+            if (stats_ws && a.stats_tiles > 0) {
                 stats_finish_kernel<<<(unsigned)((g.K * 32 + 255) / 256), 256, 0, st>>>(stats_ws, a.stats_tiles, a.stats_k,
                                                                                    g.K, sum_y, sum_y2);
                 g_launches += 1;
+            } else if (stats_ws) {
+                stats_from_output<T>(g, y, stats_ws, sum_y, sum_y2, st);
             }
             return check_launch();
         }
@@ -189,14 +201,7 @@ int forward_t(const Geo& g, const void* x, const void* w, const void* w2, const 
                                                   beta, bias, (T*)y, winners);
     snprintf(g_last_kernel, sizeof(g_last_kernel), "fwd_generic");
     g_launches += 1;
-    if (stats_ws && y) {
-        // statistics from the stored output
-        const int chunks = g.N < 16 ? g.N : 16, npc = (g.N + chunks - 1) / chunks;
-        const int rows = (g.N + npc - 1) / npc;
-        stats_direct_kernel<T><<<dim3((unsigned)g.K, (unsigned)rows), 256, 0, st>>>(g, (const T*)y, stats_ws, npc);
-        stats_finish_kernel<<<(unsigned)((g.K * 32 + 255) / 256), 256, 0, st>>>(stats_ws, rows, g.K, g.K, sum_y, sum_y2);
-        g_launches += 2;
-    }
+    if (stats_ws && y) stats_from_output<T>(g, y, stats_ws, sum_y, sum_y2, st);
     return check_launch();
 }
 

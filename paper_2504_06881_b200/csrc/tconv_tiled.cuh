@@ -83,13 +83,14 @@ __device__ __forceinline__ void mbar_init(void* bar, unsigned count) {
 __device__ __forceinline__ void mbar_expect_tx(void* bar, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Bounded wait: gives up after `limit` polls and reports failure.  A poll that finds the phase
+// Bounded wait: gives up after kPollLimit polls and reports failure.  A poll that finds the phase
 // incomplete blocks for a hardware time slice (measured: 4 us), so 2^16 polls bound a wait at a
-// quarter of a second, five orders of magnitude above the microseconds a copy takes.
+// quarter of a second, five orders of magnitude above the microseconds a copy takes.  (The limit is
+// a compile-time constant on purpose: a run-time limit costs the main loops a register.)
 constexpr int kPollLimit = 1 << 16;
-__device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity, int limit = kPollLimit) {
+__device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity) {
     const unsigned addr = smem_u32(bar);
-    for (int i = 0; i < limit; ++i) {
+    for (int i = 0; i < kPollLimit; ++i) {
         unsigned ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -203,11 +204,7 @@ struct TiledParams {
     const float* bias;
     void* y;
     void* winners;
-    float* stats;      // NULL, or per-tile partial sums {sum y, sum y^2} per output channel: [tile][stats_k][2]
-    int stats_k;       // channel pitch of the partials (K rounded up to the k tile)
     int* status;       // device status word: set non-zero when a bounded wait gives up
-    int poll_limit;    // polls a wait may take (kPollLimit; lower under the failure-test switch)
-    int debug_drop;    // failure-test switch: the copies of the first chunk are never issued
     int TW, QPR, TH;   // tile: output columns, quads per row, output rows
     int n_col_tiles, n_row_tiles;
     int tiles_per_img; // > 0: row tiles stay inside one image; 0: rows run over the flattened (n, oh) space
@@ -222,6 +219,11 @@ struct TiledParams {
     int GAP;           // extra input-row slots between two images of one tile (flattened tiles)
     int CC, Cpad, nchunks;
     int stage_floats, x_stage, w_stage, ab_stage;  // shared-memory layout of one stage (4-byte words)
+    // (later additions stay at the end: the register allocation of the kernels that sit at their
+    // register cap proved sensitive to the offsets of the fields above)
+    int stats_k;       // channel pitch of the statistics partials (K rounded up to the k tile)
+    int debug_drop;    // failure-test switch: the copies of the first chunk are never issued
+    float* stats;      // NULL, or per-tile partial sums {sum y, sum y^2} per output channel: [tile][stats_k][2]
 };
 
 // Column shift of the TMA path: the tile's first input column ow0*SW - pw is rounded
@@ -239,7 +241,8 @@ template <int S, int DW, int ESIZE = 4> struct TmaShift {
 constexpr int kMinBlocksSingle = 4;   // single-branch kernels
 constexpr int kMinBlocksWinSum = 3;   // Sum forms that emit winners (168 registers)
 constexpr int kQuadsCarried = 2;      // quads per thread of the carried max-plus / min-plus chain
-template <int MODE, int CHAN, bool WIN, bool XTMA, bool RAG, int R, int S, int SW, int DW, int Q, int KG, int PW, int TK>
+// STATS (winner-emitting kernels only): also leave the per-tile channel statistics.
+template <int MODE, int CHAN, bool WIN, bool XTMA, bool RAG, int R, int S, int SW, int DW, int Q, int KG, int PW, int TK, bool STATS = false>
 __global__ void __launch_bounds__(KG * PW * 32,
                                   (WIN && CHAN == CH_SUM) ? kMinBlocksWinSum
                                   : WIN ? 1
@@ -435,12 +438,12 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
         float* st = stage0 + s * p.stage_floats;
         if (ch + 1 < p.nchunks) issue_chunk(ch + 1, s ^ 1);
         if constexpr (XTMA) {
-            if (!mbar_wait(&bars[s], (ch >> 1) & 1, p.poll_limit)) {
+            if (!mbar_wait(&bars[s], (ch >> 1) & 1)) {
                 // the copy did not land in time: flag it, give the copies in flight one more
                 // bounded chance to finish, and leave
                 if (p.status) *p.status = 1;
-                mbar_wait(&bars[s], (ch >> 1) & 1, p.poll_limit);
-                if (ch + 1 < p.nchunks) mbar_wait(&bars[s ^ 1], ((ch + 1) >> 1) & 1, p.poll_limit);
+                mbar_wait(&bars[s], (ch >> 1) & 1);
+                if (ch + 1 < p.nchunks) mbar_wait(&bars[s ^ 1], ((ch + 1) >> 1) & 1);
                 return;
             }
         } else {
@@ -693,7 +696,7 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
 
     // epilogue: bias, store, winner index of the Max / Min channel combines
     float* yg = reinterpret_cast<float*>(p.y);
-    if (p.stats) {
+    if constexpr (STATS) {
         // per-channel sums of the outputs and of their squares over this tile (the statistics a
         // following batch normalisation needs): per thread over its pixels, then a fixed shuffle
         // tree over the warp, which owns all pixels of the tile for its TK channels
@@ -771,14 +774,13 @@ fwd_tiled_f32_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams
 // ----------------------------------------------------------------------------------
 // host side: tile selection and launch
 
-// Failure-test switch (environment, read once): TCONV_DEBUG_DROP_COPY=<polls> makes the copy-engine
-// kernels skip the copies of their first chunk and lowers the poll limit of their waits to <polls>,
-// so that a test can watch a bounded wait run out with nothing in flight.  0 / unset: off.
-inline int failure_test_polls() {
-    static const int v = [] {
+// Failure-test switch (environment, read once): TCONV_DEBUG_DROP_COPY=1 makes the copy-engine
+// kernels skip the copies of their first chunk, so that a test can watch a bounded wait run out with
+// nothing in flight.  Unset / 0: off.
+inline bool failure_test_switch() {
+    static const bool v = [] {
         const char* e = getenv("TCONV_DEBUG_DROP_COPY");
-        const long n = e ? atol(e) : 0;
-        return (int)(n < 0 ? 0 : (n > kPollLimit ? kPollLimit : n));
+        return e && e[0] == '1';
     }();
     return v;
 }
@@ -987,19 +989,25 @@ int launch_tiled_variant(FwdArgs& a) {
         g.K, g.C, g.RS, pl.tile_k, pl.p.Cpad, nkt, (const T*)a.w, (const T*)a.w2, a.alpha, a.beta, wt, wt2, at, bt);
     pl.p.x = a.x; pl.p.w = a.w; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
+    // channel statistics in the epilogue: winner-emitting kernels (the training forward); a call
+    // without winners takes them from the stored output afterwards (stats_tiles stays 0)
     pl.p.stats = nullptr; pl.p.stats_k = nkt * pl.tile_k;
-    if (a.stats) {
+    if (a.stats && WIN) {
         if ((size_t)pl.grid.x * pl.p.stats_k * 2 * sizeof(float) > a.stats_bytes) return TCONV_ERR_WORKSPACE_TOO_SMALL;
         pl.p.stats = a.stats; a.stats_tiles = (int)pl.grid.x; a.stats_k = pl.p.stats_k;
     }
-    pl.p.debug_drop = failure_test_polls() > 0;
-    pl.p.poll_limit = pl.p.debug_drop ? failure_test_polls() : kPollLimit;
-#define TCONV_LAUNCH_F32(XTMAV, RAGV)                                                                 \
+    pl.p.debug_drop = failure_test_switch();
+#define TCONV_LAUNCH_F32_S(XTMAV, RAGV, STATSV)                                                       \
     {                                                                                                \
-        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, TK>; \
+        auto kern = fwd_tiled_f32_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, TK, STATSV>; \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) \
             return TCONV_ERR_CUDA;                                                                   \
         kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);                                    \
+    }
+#define TCONV_LAUNCH_F32(XTMAV, RAGV)                                                                 \
+    {                                                                                                \
+        if constexpr (WIN) { if (pl.p.stats) TCONV_LAUNCH_F32_S(XTMAV, RAGV, true) else TCONV_LAUNCH_F32_S(XTMAV, RAGV, false) } \
+        else TCONV_LAUNCH_F32_S(XTMAV, RAGV, false)                                                  \
     }
     if (pl.xtma) {
         if (pl.p.ragged) TCONV_LAUNCH_F32(true, true) else TCONV_LAUNCH_F32(true, false)
@@ -1009,6 +1017,7 @@ int launch_tiled_variant(FwdArgs& a) {
         a.name = WIN ? "fwd_tiled_f32_win" : "fwd_tiled_f32";
     }
 #undef TCONV_LAUNCH_F32
+#undef TCONV_LAUNCH_F32_S
     return TCONV_OK;
 }
 

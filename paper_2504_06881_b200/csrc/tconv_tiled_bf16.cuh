@@ -137,7 +137,8 @@ __device__ __forceinline__ void loadw(const unsigned* p, unsigned* out) {
 
 // KPT: output channels per thread, 8, or 4 for layers that would otherwise keep too few warps
 // resident (small maps with many channels at a small batch).
-template <int MODE, int CHAN, bool WIN, bool XTMA, bool RAG, int R, int S, int SW, int DW, int Q, int KG, int PW, int KPT = 8>
+template <int MODE, int CHAN, bool WIN, bool XTMA, bool RAG, int R, int S, int SW, int DW, int Q, int KG, int PW, int KPT = 8,
+          bool STATS = false>
 __global__ void __launch_bounds__(KG * PW * 32)
 fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParams p) {
     static_assert(S == 3, "the pixel-pair selection below is written for 3 taps per row");
@@ -333,10 +334,10 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
         unsigned* st = stage0 + s * p.stage_floats;
         if (ch + 1 < p.nchunks) issue_chunk(ch + 1, s ^ 1);
         if constexpr (XTMA) {
-            if (!mbar_wait(&bars[s], (ch >> 1) & 1, p.poll_limit)) {
+            if (!mbar_wait(&bars[s], (ch >> 1) & 1)) {
                 if (p.status) *p.status = 1;
-                mbar_wait(&bars[s], (ch >> 1) & 1, p.poll_limit);
-                if (ch + 1 < p.nchunks) mbar_wait(&bars[s ^ 1], ((ch + 1) >> 1) & 1, p.poll_limit);
+                mbar_wait(&bars[s], (ch >> 1) & 1);
+                if (ch + 1 < p.nchunks) mbar_wait(&bars[s ^ 1], ((ch + 1) >> 1) & 1);
                 return;
             }
         } else {
@@ -532,7 +533,7 @@ fwd_tiled_bf16_kernel(const __grid_constant__ CUtensorMap xmap, const TiledParam
 
     // epilogue
     unsigned short* yg = reinterpret_cast<unsigned short*>(p.y);
-    if (p.stats) {
+    if constexpr (STATS) {
         // per-channel sums of the stored (bf16-rounded) outputs and of their squares over this tile
         static_assert(PW == 1, "one warp per channel group owns the whole pixel tile");
 #pragma unroll
@@ -657,18 +658,22 @@ int launch_tiled_variant_bf16(FwdArgs& a) {
     pl.p.x = a.x; pl.p.w = a.w; pl.p.wt = wt; pl.p.wt2 = wt2; pl.p.at = at; pl.p.bt = bt;
     pl.p.bias = a.bias; pl.p.y = a.y; pl.p.winners = a.winners; pl.p.status = a.status;
     pl.p.stats = nullptr; pl.p.stats_k = nkt * pl.tile_k;
-    if (a.stats) {
+    if (a.stats && WIN) {
         if ((size_t)pl.grid.x * pl.p.stats_k * 2 * sizeof(float) > a.stats_bytes) return TCONV_ERR_WORKSPACE_TOO_SMALL;
         pl.p.stats = a.stats; a.stats_tiles = (int)pl.grid.x; a.stats_k = pl.p.stats_k;
     }
-    pl.p.debug_drop = failure_test_polls() > 0;
-    pl.p.poll_limit = pl.p.debug_drop ? failure_test_polls() : kPollLimit;
-#define TCONV_LAUNCH_BF16(XTMAV, RAGV)                                                                \
+    pl.p.debug_drop = failure_test_switch();
+#define TCONV_LAUNCH_BF16_S(XTMAV, RAGV, STATSV)                                                      \
     {                                                                                                \
-        auto kern = fwd_tiled_bf16_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, KPT>; \
+        auto kern = fwd_tiled_bf16_kernel<MODE, CHAN, WIN, XTMAV, RAGV, R, S, SW, DW, Q, KG, PW, KPT, STATSV>; \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) \
             return TCONV_ERR_CUDA;                                                                   \
         kern<<<pl.grid, pl.threads, pl.smem, a.st>>>(xmap, pl.p);                                    \
+    }
+#define TCONV_LAUNCH_BF16(XTMAV, RAGV)                                                                \
+    {                                                                                                \
+        if constexpr (WIN) { if (pl.p.stats) TCONV_LAUNCH_BF16_S(XTMAV, RAGV, true) else TCONV_LAUNCH_BF16_S(XTMAV, RAGV, false) } \
+        else TCONV_LAUNCH_BF16_S(XTMAV, RAGV, false)                                                 \
     }
     if constexpr (PLAIN_ONLY) {
         TCONV_LAUNCH_BF16(false, false)
@@ -681,6 +686,7 @@ int launch_tiled_variant_bf16(FwdArgs& a) {
         a.name = WIN ? "fwd_tiled_bf16_win" : "fwd_tiled_bf16";
     }
 #undef TCONV_LAUNCH_BF16
+#undef TCONV_LAUNCH_BF16_S
     return TCONV_OK;
 }
 

@@ -34,27 +34,20 @@ print(json.dumps({"kernel": kernel, "seconds": dt, "first": first, "second": sec
 """
 
 
-def _run(polls):
-    env = dict(os.environ, TCONV_DEBUG_DROP_COPY=str(polls))
+def _run(switch):
+    env = dict(os.environ, TCONV_DEBUG_DROP_COPY=str(switch))
     out = subprocess.run([sys.executable, "-c", CHILD % str(ROOT)], env=env, capture_output=True, text=True, timeout=300)
     assert out.returncode == 0, out.stderr[-2000:]
     return json.loads(out.stdout.strip().splitlines()[-1])
 
 
 def test_bounded_wait_runs_out_and_reports_a_timeout():
-    r = _run(4096)
+    """The kernel waits twice on the dropped chunk (2^16 polls each, measured 4 us per poll) and
+    returns: the give-up takes about half a second, the host reads the timeout once."""
+    r = _run(1)
     assert "tma" in r["kernel"]
     assert r["first"] == -6 and r["second"] == 0 and r["usable"]
-    assert r["seconds"] < 5.0
-
-
-def test_give_up_time_at_the_production_poll_limit():
-    """The same with the production limit (2^16 polls per wait; the kernel waits twice on the
-    dropped chunk before it returns; measured 4 us per poll): the give-up stays around half a
-    second."""
-    r = _run(1 << 16)
-    assert r["first"] == -6 and r["second"] == 0 and r["usable"]
-    print("give-up time at 2^16 polls:", r["seconds"], "s")
+    print("give-up time:", r["seconds"], "s")
     assert r["seconds"] < 5.0
 
 
