@@ -680,6 +680,83 @@ def run_conv3d(args):
     print(json.dumps(out))
 
 
+def run_conv1d(args):
+    """The opening layer of the paper's audio networks (appendix "One-dimensional data
+    classification": one input channel, 128 output channels, window 80, stride 4, signals of 16000
+    samples; batch --images, default 32) and a mid-network layer with a window of 3 (128 -> 128
+    channels, length 1000), mode --only (default compound), fp32 or bf16: forward, forward with
+    winners and the full backward, in ms and Ttap/s, and the forward's fraction of the mode's
+    measured add+max/min peak."""
+    import torch
+    from paper_2504_06881_b200 import inputs, tconv, tconv3d
+    from paper_2504_06881_b200.nn import TropicalConv1d
+    torch.cuda.set_device(0)
+    mode = args.only or "compound"
+    dt = tconv.TORCH_DTYPE[args.dtype]
+    two, par = mode in ("compound", "parallel"), mode == "parallel"
+    peaks, peaks16, _ = measure_alu_peak(torch, tconv)
+    peak = (peaks16 if args.dtype == "bf16" else peaks)[mode]
+    n = args.images if args.images != 128 else 32
+    d = inputs.layer3d(n, 1, 1, 1, 16000, 128, T=1, R=1, S=80, stride=(1, 1, 4), mode=mode, dtype=args.dtype)
+    out = {"workload": f"1-D audio layers, {mode} {args.dtype}, batch {n}", "peak_Ttap_s": peak / 1e12, "layers": {}}
+    l0 = tconv3d.tconv3d_launch_count()
+    t = inputs.draw3d(d, 1080)
+    dev = lambda a, ty=None: torch.from_numpy(a).cuda().to(ty) if ty else torch.from_numpy(a).cuda()
+    x, w, w2, g = (dev(t[k], dt) for k in ("x", "w", "w2", "g"))
+    al, be, bias = dev(t["alpha"]), dev(t["beta"]), dev(t["bias"])
+    y = torch.empty(t["g"].shape, device="cuda", dtype=dt)
+    win = tconv3d.winner_buffer(d, "cuda")
+    ws = torch.empty(tconv3d.tconv3d_workspace_bytes(d, True), dtype=torch.uint8, device="cuda")
+    gx, gw, gw2 = torch.empty_like(x), torch.empty_like(w, dtype=torch.float32), torch.empty_like(w, dtype=torch.float32)
+    ga, gb, gbi = torch.empty_like(al), torch.empty_like(be), torch.empty_like(bias)
+    fa = (d, x, w, w2 if par else None, al if two else None, be if two else None, bias, y)
+    calls = {"fwd": lambda: tconv3d.tconv3d_forward(*fa, None),
+             "fwd_winners": lambda: tconv3d.tconv3d_forward(*fa, win),
+             "bwd": lambda: tconv3d.tconv3d_backward(d, x, w, w2 if par else None, al if two else None,
+                                                     be if two else None, g, win, gx, gw, gw2 if par else None,
+                                                     ga if two else None, gb if two else None, gbi, ws)}
+    od = tconv3d.tconv3d_output_shape(d)
+    taps = d["N"] * d["K"] * od[2] * d["C"] * 80
+    row = {"Mtap": taps / 1e6}
+    for what, fn in calls.items():
+        assert fn() == 0
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(max(args.steps, 5)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        row[what + "_ms"] = float(np.median(ts))
+    row["fwd_Ttap_s"] = taps / row["fwd_ms"] / 1e9
+    row["fwd_frac_of_alu_peak"] = taps / row["fwd_ms"] / 1e-3 / peak
+    out["layers"]["k80 s4 1->128 L16000"] = row
+    launches = tconv3d.tconv3d_launch_count() - l0
+    # a mid-network layer (window 3, stride 1) through the module: the tiled 2-D kernels
+    m = TropicalConv1d(128, 128, 3, padding=1, mode=mode, dtype=args.dtype).cuda()
+    xm = torch.randn(n, 128, 1000, device="cuda", requires_grad=True)
+    gm = torch.randn(n, 128, 1000, device="cuda")
+    def step():
+        xm.grad = None
+        m(xm).backward(gm)
+    l1 = tconv.tconv_launch_count()
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); step(); e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    out["layers"]["k3 s1 128->128 L1000 (module, fwd+bwd)"] = {"Mtap": n * 128 * 128 * 1000 * 3 / 1e6,
+                                                              "fwd_bwd_ms": float(np.median(ts))}
+    out["gpu_launches"] = launches + tconv.tconv_launch_count() - l1
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -697,9 +774,9 @@ def main():
                     help="cfg5: the bf16 kernels read the float activations directly (x_dtype) instead of a converted copy")
     ap.add_argument("--no-headline", action="store_true",
                     help="skip the headline_layers section (cfg 3a / 3b / 4 timed after the step)")
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5", "dw", "conv3d"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5", "dw", "conv3d", "conv1d"],
                     help="cfg5: report the hybrid ResNet-18 training step instead (use --only compound|parallel); "
-                         "dw: a depthwise (groups = C) layer against the HBM roofline; conv3d: the 3-D LeNet layers")
+                         "dw: a depthwise (groups = C) layer against the HBM roofline; conv3d: the 3-D LeNet layers; conv1d: the 1-D audio layers")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -707,6 +784,8 @@ def main():
         run_cfg5(args)
     elif args.workload == "conv3d":
         run_conv3d(args)
+    elif args.workload == "conv1d":
+        run_conv1d(args)
     elif args.workload == "dw":
         run_dw(args)
     elif args.only:

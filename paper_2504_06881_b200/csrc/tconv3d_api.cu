@@ -1,7 +1,10 @@
 // C ABI of the three-dimensional layers: host-side checks, launch plans, kernel launches.
 #include <cstdio>
 
+#include <cstdlib>
+
 #include "tconv3d.h"
+#include "tconv_1d.cuh"
 #include "tconv_3d.cuh"
 
 namespace tconv {
@@ -82,16 +85,122 @@ int bias_splits(const Geo3& g) {
     return (int)want;
 }
 
+// TCONV_FORCE_GENERIC=1 keeps every call on the any-shape kernels (read once per process).
+bool force_generic3() {
+    static const int v = [] {
+        const char* e = getenv("TCONV_FORCE_GENERIC");
+        return (e && e[0] == '1') ? 1 : 0;
+    }();
+    return v != 0;
+}
+
+// One-dimensional layers (unit depth and height, 1 x 1 x S window) with windows of four taps or
+// more at stride 1, 2 or 4 run on the kernels of tconv_1d.cuh.
+bool is_1d(const Geo3& g) {
+    return g.D == 1 && g.H == 1 && g.T == 1 && g.R == 1 && g.pd == 0 && g.ph == 0 && g.dw == 1 &&
+           (g.sw == 1 || g.sw == 2 || g.sw == 4) && g.S >= 4 && g.N <= 65535 && !force_generic3();
+}
+
+constexpr size_t kSmem1d = 96 * 1024;  // most dynamic shared memory a backward 1-D block asks for
+
+// Launch plan of the 1-D backward kernels.  ok = 0: the layer stays on the any-shape kernels (a
+// Max / Min channel combine over several channels, whose winners name one channel per output).
+struct Plan1 {
+    int ok;
+    int pt, tb, span, tiles, ks;  // grad_x: positions per thread, threads, array length, tiles, channel slices
+    int ptb, nsplit;              // parameter gradients: threads, splits of the (n, position) range
+    size_t gx_smem, p_smem, part_floats, scratch_floats;
+};
+
+Plan1 plan_1d(const Geo3& g) {
+    Plan1 p = {};
+    if (!is_1d(g) || !(g.chan == CH_SUM || g.C == 1)) return p;
+    const int st = g.sw, S = g.S, OL = g.OW;
+    p.pt = (S + st - 1) / st - 1;
+    if (p.pt < 8) p.pt = 8;
+    p.tb = kGx1Threads;
+    for (;;) {
+        p.span = p.tb * p.pt * st - st + S;
+        p.gx_smem = 2 * (size_t)p.span * sizeof(float);
+        if (p.gx_smem <= kSmem1d || p.tb == 32) break;
+        p.tb /= 2;
+    }
+    if (p.gx_smem > kSmem1d) return p;
+    p.tiles = (OL + p.tb * p.pt - 1) / (p.tb * p.pt);
+    const long long blocks = (long long)p.tiles * g.C * g.N;
+    long long ks = (4 * 148 + blocks - 1) / blocks;
+    if (ks > 8) ks = 8;
+    if (ks > g.K) ks = g.K;
+    if ((long long)g.C * ks > 65535) return p;
+    p.ks = (int)ks;
+    p.part_floats = (size_t)p.ks * g.N * g.C * p.tiles * p.span;
+    const int branches = two_branch(g.mode) ? 2 : 1;
+    p.ptb = 128;
+    for (;;) {
+        p.p_smem = ((size_t)branches * S * p.ptb + 2 * S + p.ptb) * sizeof(float);
+        if (p.p_smem <= kSmem1d || p.ptb == 32) break;
+        p.ptb /= 2;
+    }
+    if (p.p_smem > kSmem1d) return p;
+    const long long kc = (long long)g.K * g.C, total = (long long)g.N * OL;
+    long long want = (4 * 148 + kc - 1) / kc;
+    const long long most = (total + 2047) / 2048;
+    if (want > most) want = most;
+    if (want < 1) want = 1;
+    if (want > 64) want = 64;
+    p.nsplit = (int)want;
+    p.scratch_floats = 2 * (size_t)p.nsplit * kc * S + 2 * (size_t)p.nsplit * kc + (size_t)p.nsplit * g.K +
+                       p.part_floats;
+    p.ok = 1;
+    return p;
+}
+
 size_t backward_scratch_floats(const Geo3& g) {
     const size_t ns = (size_t)gw_splits(g);
-    return 2 * ns * g.K * g.C * g.taps + 2 * ns * g.K * g.C + (size_t)bias_splits(g) * g.K;
+    const size_t generic = 2 * ns * g.K * g.C * g.taps + 2 * ns * g.K * g.C + (size_t)bias_splits(g) * g.K;
+    const Plan1 p = plan_1d(g);
+    return (p.ok && p.scratch_floats > generic) ? p.scratch_floats : generic;
 }
 
 int check(cudaError_t e) { return e == cudaSuccess ? TCONV_OK : TCONV_ERR_CUDA; }
 
 template <typename T>
+int forward1d_t(const Geo3& g, const void* x, const void* w, const void* w2, const float* alpha,
+                const float* beta, const float* bias, void* y, void* winners, cudaStream_t st) {
+    const int q4 = (((g.S + g.sw - 1) / g.sw) + 3) & ~3;
+    const int br = g.mode == TCONV_MIN_PLUS ? 0 : (g.mode == TCONV_MAX_PLUS ? 1 : (g.mode == TCONV_COMPOUND ? 2 : 3));
+    const int kb = 4 * f1_kt(br, winners != nullptr);
+    const size_t smem = ((size_t)g.sw * f1_xw(q4) + (size_t)q4 * g.sw * kb * (br == 3 ? 2 : 1)) * sizeof(T);
+    const dim3 grid((unsigned)((g.OW + kF1Pos - 1) / kF1Pos), (unsigned)((g.K + kb - 1) / kb), (unsigned)g.N);
+#define TCONV1_LAUNCH(STV, BRV, WINV)                                                     \
+    fwd1d_kernel<T, STV, BRV, WINV><<<grid, kF1Threads, smem, st>>>(                       \
+        g, q4, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, bias, (T*)y, winners)
+#define TCONV1_BY_WIN(STV, BRV)                                  \
+    {                                                            \
+        if (winners) TCONV1_LAUNCH(STV, BRV, true);              \
+        else TCONV1_LAUNCH(STV, BRV, false);                     \
+    }
+#define TCONV1_BY_BR(STV)                                        \
+    {                                                            \
+        if (br == 0) TCONV1_BY_WIN(STV, 0)                       \
+        else if (br == 1) TCONV1_BY_WIN(STV, 1)                  \
+        else if (br == 2) TCONV1_BY_WIN(STV, 2)                  \
+        else TCONV1_BY_WIN(STV, 3)                               \
+    }
+    if (g.sw == 1) TCONV1_BY_BR(1)
+    else if (g.sw == 2) TCONV1_BY_BR(2)
+    else TCONV1_BY_BR(4)
+#undef TCONV1_BY_BR
+#undef TCONV1_BY_WIN
+#undef TCONV1_LAUNCH
+    g3_launches += 1;
+    return check(cudaGetLastError());
+}
+
+template <typename T>
 int forward3_t(const Geo3& g, const void* x, const void* w, const void* w2, const float* alpha,
                const float* beta, const float* bias, void* y, void* winners, cudaStream_t st) {
+    if (is_1d(g)) return forward1d_t<T>(g, x, w, w2, alpha, beta, bias, y, winners, st);
     const bool par = g.mode == TCONV_PARALLEL;
     // two output channels per thread when K is small and not a multiple of four, else four
     const int kt = (g.K % 4 == 0 || g.K > 8) ? 4 : 2;
@@ -122,10 +231,68 @@ int forward3_t(const Geo3& g, const void* x, const void* w, const void* w2, cons
     return check(cudaGetLastError());
 }
 
+// Backward of a 1-D layer on the kernels of tconv_1d.cuh.  Scratch: part_min, part_max
+// [nsplit][K*C][S], part_ab [nsplit][K*C][2], part_bias [nsplit][K], then the grad_x partial sums.
+template <typename T>
+int backward1d_t(const Geo3& g, const Plan1& p, const void* x, const void* w, const void* w2,
+                 const float* alpha, const float* beta, const void* gy, const void* winners, void* gx,
+                 float* gw, float* gw2, float* galpha, float* gbeta, float* gbias, char* ws, cudaStream_t st) {
+    static const cudaError_t attr = [] {
+        cudaError_t e = cudaFuncSetAttribute(bwd1d_gx_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem1d);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(bwd1d_params_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem1d);
+        return e;
+    }();
+    if (attr != cudaSuccess) return TCONV_ERR_CUDA;
+    const size_t kc = (size_t)g.K * g.C, count = kc * g.S;
+    float* pmin = (float*)ws;
+    float* pmax = pmin + (size_t)p.nsplit * count;
+    float* pab = pmax + (size_t)p.nsplit * count;
+    float* pbias = pab + (size_t)p.nsplit * kc * 2;
+    float* part = pbias + (size_t)p.nsplit * g.K;
+    if (gx) {
+        bwd1d_gx_kernel<T><<<dim3((unsigned)p.tiles, (unsigned)(g.C * p.ks), (unsigned)g.N), p.tb, p.gx_smem, st>>>(
+            g, p.pt, p.ks, p.span, alpha, beta, (const T*)gy, winners, part);
+        const size_t total = (size_t)g.N * g.C * g.W;
+        bwd1d_gx_finish_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+            g, p.tiles, p.ks, p.span, p.tb * p.pt * g.sw, part, (T*)gx);
+        g3_launches += 2;
+    }
+    const bool two = two_branch(g.mode);
+    if (gw || gw2 || gbias || (two && (galpha || gbeta))) {
+        bwd1d_params_kernel<T><<<dim3((unsigned)kc, (unsigned)p.nsplit), p.ptb, p.p_smem, st>>>(
+            g, p.nsplit, (const T*)x, (const T*)w, (const T*)w2, (const T*)gy, winners, pmin, pmax, pab, pbias);
+        g3_launches += 1;
+        if (gw || gw2) {
+            bwd3d_gw_finish_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(g, p.nsplit, alpha, beta, pmin,
+                                                                                   pmax, gw, gw2);
+            g3_launches += 1;
+        }
+        if (two && galpha) {
+            bwd3d_sum_splits_kernel<<<(unsigned)((kc + 255) / 256), 256, 0, st>>>((int)kc, p.nsplit, 2, 0, pab, galpha);
+            g3_launches += 1;
+        }
+        if (two && gbeta) {
+            bwd3d_sum_splits_kernel<<<(unsigned)((kc + 255) / 256), 256, 0, st>>>((int)kc, p.nsplit, 2, 1, pab, gbeta);
+            g3_launches += 1;
+        }
+        if (gbias) {
+            bwd3d_sum_splits_kernel<<<(g.K + 255) / 256, 256, 0, st>>>(g.K, p.nsplit, 1, 0, pbias, gbias);
+            g3_launches += 1;
+        }
+    }
+    return check(cudaGetLastError());
+}
+
 template <typename T>
 int backward3_t(const Geo3& g, const void* x, const void* w, const void* w2, const float* alpha,
                 const float* beta, const void* gy, const void* winners, void* gx, float* gw, float* gw2,
                 float* galpha, float* gbeta, float* gbias, char* ws, cudaStream_t st) {
+    {
+        const Plan1 p1 = plan_1d(g);
+        if (p1.ok)
+            return backward1d_t<T>(g, p1, x, w, w2, alpha, beta, gy, winners, gx, gw, gw2, galpha, gbeta, gbias, ws, st);
+    }
     const bool two = two_branch(g.mode);
     if (gx) {
         const size_t total = (size_t)g.N * g.C * g.D * g.H * g.W;

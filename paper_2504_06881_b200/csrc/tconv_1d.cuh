@@ -1,0 +1,389 @@
+// One-dimensional tropical convolution with long windows (Section 3.2; the paper's audio networks
+// open with a window of 80 samples at stride 4 on signals of 16000 samples, one input channel).
+// The layers arrive through the three-dimensional entry points as 1 x 1 x S windows on signals of
+// unit depth and height, and use the winner layouts of those entry points.
+//
+// Forward: the signal segment of a block sits in shared memory split by phase (index modulo the
+// stride), so that the taps s = q * stride + p of neighbouring output positions read neighbouring
+// words; a lane owns four consecutive positions and a few output channels, and walks the window
+// with a register window of eight samples per phase.  Taps beyond S hold NaN weights, which
+// min / max skip.  Backward: grad_x by scattering into block-private shared-memory arrays (threads
+// of even and odd index own one array each, a thread's positions cannot reach past its neighbour's),
+// the parameter gradients by private per-thread columns per tap; every sum has a fixed order.
+#pragma once
+#include "tconv_3d.cuh"
+
+namespace tconv {
+
+constexpr int kF1Threads = 128;  // four warps: one tile of positions, four groups of output channels
+constexpr int kF1Pos = 128;      // output positions per block: four per lane
+constexpr int kGx1Threads = 64;  // most threads of a grad_x block
+
+template <typename T, int N>
+struct alignas(sizeof(T) * N > 16 ? 16 : sizeof(T) * N) Vec {
+    T v[N];
+};
+
+__device__ __forceinline__ float fmin3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+template <typename T> __device__ __forceinline__ T nan_of();
+template <> __device__ __forceinline__ float nan_of<float>() { return __int_as_float(0x7fc00000); }
+template <> __device__ __forceinline__ __nv_bfloat16 nan_of<__nv_bfloat16>() {
+    return __ushort_as_bfloat16((unsigned short)0x7fc0);
+}
+
+// Branches of a layer: 0 min only, 1 max only, 2 both on one weight (compound), 3 both on two
+// weights (parallel).
+__host__ __device__ constexpr bool has_min(int br) { return br != 1; }
+__host__ __device__ constexpr bool has_max(int br) { return br != 0; }
+// Output channels per thread: eight while one extremum per output is live, else four.
+__host__ __device__ constexpr int f1_kt(int br, bool win) { return (br >= 2 || win) ? 4 : 8; }
+
+// Row pitch of the staged signal segment: the window of the last lane ends at 4 * 31 + q4 + 3.
+__host__ __device__ constexpr int f1_xw(int q4) { return (kF1Pos + q4 + 4 + 7) & ~7; }
+
+// Forward.  grid (ceil(OL / 128), ceil(K / (4 * KT)), N), 128 threads.  Shared memory: the block's
+// signal segment of one input channel by phase, xs[ST][xw] with xs[p][i] = x[(P0 + i) * ST + p - pad]
+// (zero outside the signal), xw = 128 + q4 + 4 rounded up to a multiple of eight, and the weights of that channel for the block's
+// 4 * KT output channels, ws[s][4 * KT] for s < q4 * ST (NaN for s >= S), twice in parallel mode.
+// q4 = ceil(S / ST) rounded up to a multiple of four.  WIN: taps are visited in ascending order
+// with strict compares, so that the lowest tap wins a tie.
+template <typename T, int ST, int BR, bool WIN>
+__global__ void __launch_bounds__(kF1Threads)
+fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
+             const float* __restrict__ alpha, const float* __restrict__ beta,
+             const float* __restrict__ bias, T* __restrict__ y, void* __restrict__ winners) {
+    constexpr int KT = f1_kt(BR, WIN);
+    constexpr int KB = 4 * KT;
+    constexpr bool MIN = has_min(BR), MAX = has_max(BR);
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int xw = f1_xw(q4);
+    T* xs = reinterpret_cast<T*>(smem_raw);
+    T* ws = xs + ST * xw;
+    T* ws2 = ws + q4 * ST * KB;
+    const int tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
+    const int P0 = blockIdx.x * kF1Pos, n = blockIdx.z;
+    const int kb0 = blockIdx.y * KB, k0 = kb0 + wv * KT;
+    const int L = g.W, OL = g.OW, S = g.S;
+    float out[KT][4];
+    int win[KT][4];
+#pragma unroll
+    for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            out[kk][j] = (g.chan == CH_SUM) ? 0.0f : (g.chan == CH_MAX ? -INFINITY : INFINITY);
+            win[kk][j] = -1;
+        }
+    for (int c = 0; c < g.C; ++c) {
+        __syncthreads();
+        {   // stage the signal segment by phase and the weights by tap
+            const T* xc = x + ((size_t)n * g.C + c) * L;
+            const long long base = (long long)P0 * ST - g.pw;
+            for (int j = tid; j < xw * ST; j += kF1Threads) {
+                const long long gi = base + j;
+                xs[(j % ST) * xw + j / ST] = (gi >= 0 && gi < L) ? xc[gi] : zero_of<T>();
+            }
+            const int span = q4 * ST;
+            for (int i = tid; i < KB * span; i += kF1Threads) {
+                const int kk = i / span, s = i - kk * span, k = kb0 + kk;
+                T a = zero_of<T>(), b = zero_of<T>();
+                if (s >= S) a = b = nan_of<T>();
+                else if (k < g.K) {
+                    const size_t wi = ((size_t)k * g.C + c) * S + s;
+                    a = w[wi];
+                    if (BR == 3) b = w2[wi];
+                }
+                ws[s * KB + kk] = a;
+                if (BR == 3) ws2[s * KB + kk] = b;
+            }
+        }
+        __syncthreads();
+        float mn[KT][4], mx[KT][4];
+        int amn[KT][4], amx[KT][4];
+#pragma unroll
+        for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                mn[kk][j] = INFINITY; mx[kk][j] = -INFINITY; amn[kk][j] = 0; amx[kk][j] = 0;
+            }
+        if constexpr (!WIN) {
+#pragma unroll
+            for (int p = 0; p < ST; ++p) {
+                const T* xp = xs + p * xw + 4 * lane;
+                for (int q0 = 0; q0 < q4; q0 += 4) {
+                    T r[8];
+                    *reinterpret_cast<Vec<T, 4>*>(r) = *reinterpret_cast<const Vec<T, 4>*>(xp + q0);
+                    *reinterpret_cast<Vec<T, 4>*>(r + 4) = *reinterpret_cast<const Vec<T, 4>*>(xp + q0 + 4);
+#pragma unroll
+                    for (int dq = 0; dq < 4; dq += 2) {
+                        const int s0 = (q0 + dq) * ST + p, s1 = s0 + ST;
+                        const Vec<T, KT> wa0 = *reinterpret_cast<const Vec<T, KT>*>(ws + s0 * KB + wv * KT);
+                        const Vec<T, KT> wa1 = *reinterpret_cast<const Vec<T, KT>*>(ws + s1 * KB + wv * KT);
+                        Vec<T, KT> wb0 = wa0, wb1 = wa1;
+                        if constexpr (BR == 3) {
+                            wb0 = *reinterpret_cast<const Vec<T, KT>*>(ws2 + s0 * KB + wv * KT);
+                            wb1 = *reinterpret_cast<const Vec<T, KT>*>(ws2 + s1 * KB + wv * KT);
+                        }
+#pragma unroll
+                        for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float t0 = tap_add(r[dq + j], wa0.v[kk]);
+                                const float t1 = tap_add(r[dq + 1 + j], wa1.v[kk]);
+                                if constexpr (MIN) mn[kk][j] = fmin3(mn[kk][j], t0, t1);
+                                if constexpr (BR == 3) {
+                                    const float u0 = tap_add(r[dq + j], wb0.v[kk]);
+                                    const float u1 = tap_add(r[dq + 1 + j], wb1.v[kk]);
+                                    mx[kk][j] = fmax3(mx[kk][j], u0, u1);
+                                } else if constexpr (MAX) {
+                                    mx[kk][j] = fmax3(mx[kk][j], t0, t1);
+                                }
+                            }
+                    }
+                }
+            }
+        } else {
+            const T* xl = xs + 4 * lane;
+            for (int q0 = 0; q0 < q4; q0 += 4) {
+                T r[ST][8];
+#pragma unroll
+                for (int p = 0; p < ST; ++p) {
+                    *reinterpret_cast<Vec<T, 4>*>(r[p]) = *reinterpret_cast<const Vec<T, 4>*>(xl + p * xw + q0);
+                    *reinterpret_cast<Vec<T, 4>*>(r[p] + 4) =
+                        *reinterpret_cast<const Vec<T, 4>*>(xl + p * xw + q0 + 4);
+                }
+#pragma unroll
+                for (int dq = 0; dq < 4; ++dq)
+#pragma unroll
+                    for (int p = 0; p < ST; ++p) {
+                        const int s = (q0 + dq) * ST + p;
+                        const Vec<T, KT> wa = *reinterpret_cast<const Vec<T, KT>*>(ws + s * KB + wv * KT);
+                        Vec<T, KT> wb = wa;
+                        if constexpr (BR == 3) wb = *reinterpret_cast<const Vec<T, KT>*>(ws2 + s * KB + wv * KT);
+#pragma unroll
+                        for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float t = tap_add(r[p][dq + j], wa.v[kk]);
+                                const float u = (BR == 3) ? tap_add(r[p][dq + j], wb.v[kk]) : t;
+                                if constexpr (MIN)
+                                    if (t < mn[kk][j]) { mn[kk][j] = t; amn[kk][j] = s; }
+                                if constexpr (MAX)
+                                    if (u > mx[kk][j]) { mx[kk][j] = u; amx[kk][j] = s; }
+                            }
+                    }
+            }
+        }
+        // channel combine, channels ascending
+#pragma unroll
+        for (int kk = 0; kk < KT; ++kk) {
+            const int k = k0 + kk;
+            if (k >= g.K) continue;
+            float a = 1.0f, b = 1.0f;
+            if (BR >= 2) {
+                if (alpha) a = alpha[(size_t)k * g.C + c];
+                if (beta) b = beta[(size_t)k * g.C + c];
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if constexpr (BR >= 2) {
+                    out[kk][j] = __fmaf_rn(a, mn[kk][j], out[kk][j]);
+                    out[kk][j] = __fmaf_rn(b, mx[kk][j], out[kk][j]);
+                } else {
+                    const float m = MIN ? mn[kk][j] : mx[kk][j];
+                    const int am = MIN ? amn[kk][j] : amx[kk][j];
+                    if (g.chan == CH_SUM) out[kk][j] = __fadd_rn(out[kk][j], m);
+                    else if (g.chan == CH_MAX) { if (m > out[kk][j]) { out[kk][j] = m; win[kk][j] = c * S + am; } }
+                    else { if (m < out[kk][j]) { out[kk][j] = m; win[kk][j] = c * S + am; } }
+                }
+                if (WIN && g.chan == CH_SUM) {
+                    const int pos = P0 + 4 * lane + j;
+                    if (pos < OL)
+                        ((uint16_t*)winners)[(((size_t)n * g.K + k) * g.C + c) * OL + pos] =
+                            (uint16_t)((MIN ? amn[kk][j] : 0) | ((MAX ? amx[kk][j] : 0) << 8));
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int kk = 0; kk < KT; ++kk) {
+        const int k = k0 + kk;
+        if (k >= g.K) continue;
+        const float bv = bias ? bias[k] : 0.0f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int pos = P0 + 4 * lane + j;
+            if (pos >= OL) continue;
+            float v = out[kk][j];
+            if (bias) v = __fadd_rn(v, bv);
+            const size_t o = ((size_t)n * g.K + k) * OL + pos;
+            if (y) y[o] = from_f32<T>(v);
+            if (WIN && g.chan != CH_SUM) ((int32_t*)winners)[o] = win[kk][j];
+        }
+    }
+}
+
+// grad_x partial sums by scattering.  grid (tiles, C * ks, N), blockDim.x = tb threads; a thread owns
+// pt consecutive output positions (pt * stride >= S - stride, so its windows end before the
+// positions of the thread after the next begin) and adds, channels of its slice ascending and
+// positions ascending, every gradient to the winner's element of the shared-memory array of its
+// parity.  The block's two arrays cover span = tb * pt * stride - stride + S elements from padded
+// index tile * tb * pt * stride; their sum goes to part[slice][n][c][tile][span].
+template <typename T>
+__global__ void __launch_bounds__(kGx1Threads)
+bwd1d_gx_kernel(Geo3 g, int pt, int ks, int span, const float* __restrict__ alpha,
+                const float* __restrict__ beta, const T* __restrict__ gy,
+                const void* __restrict__ winners, float* __restrict__ part) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* even = reinterpret_cast<float*>(smem_raw);
+    float* odd = even + span;
+    const int tid = threadIdx.x, tb = blockDim.x;
+    const int tile = blockIdx.x, c = blockIdx.y / ks, slice = blockIdx.y % ks, n = blockIdx.z;
+    const int OL = g.OW, st = g.sw;
+    const bool twob = two_branch(g.mode);
+    for (int i = tid; i < 2 * span; i += tb) even[i] = 0.0f;
+    __syncthreads();
+    float* mine = (tid & 1) ? odd : even;
+    const int lp0 = tid * pt, p0 = tile * tb * pt + lp0;
+    const int cnt = min(pt, OL - p0);
+    const int kper = (g.K + ks - 1) / ks;
+    const int kend = min(g.K, (slice + 1) * kper);
+    for (int k = slice * kper; k < kend; ++k) {
+        float a = 1.0f, b = 1.0f;
+        if (twob) {
+            if (alpha) a = alpha[(size_t)k * g.C + c];
+            if (beta) b = beta[(size_t)k * g.C + c];
+        }
+        const T* grow = gy + ((size_t)n * g.K + k) * OL + p0;
+        for (int i = 0; i < cnt; ++i) {
+            int amn, amx;
+            winners3(g, winners, n, k, c, p0 + i, amn, amx);
+            if (amn < 0 && amx < 0) continue;
+            const float gv = to_f32(grow[i]);
+            float* at = mine + (lp0 + i) * st;
+            if (amn >= 0) at[amn] = twob ? __fmaf_rn(a, gv, at[amn]) : at[amn] + gv;
+            if (amx >= 0) at[amx] = twob ? __fmaf_rn(b, gv, at[amx]) : at[amx] + gv;
+        }
+    }
+    __syncthreads();
+    float* o = part + ((((size_t)slice * g.N + n) * g.C + c) * gridDim.x + tile) * span;
+    for (int i = tid; i < span; i += tb) o[i] = even[i] + odd[i];
+}
+
+// grad_x from the partial sums: one thread per input element; the tiles that cover it (at most
+// two) in ascending order, slices ascending inside a tile.
+template <typename T>
+__global__ void __launch_bounds__(256)
+bwd1d_gx_finish_kernel(Geo3 g, int tiles, int ks, int span, int tile_x, const float* __restrict__ part,
+                       T* __restrict__ gx) {
+    const size_t total = (size_t)g.N * g.C * g.W;
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const int i = (int)(e % g.W);
+    const size_t nc = e / g.W;
+    const int n = (int)(nc / g.C), c = (int)(nc % g.C);
+    const int u = i + g.pw;  // padded index: position * stride + tap
+    const int b = u / tile_x;
+    float acc = 0.0f;
+    for (int t = b - 1; t <= b; ++t) {
+        if (t < 0 || t >= tiles) continue;
+        const int li = u - t * tile_x;
+        if (li >= span) continue;
+        for (int sl = 0; sl < ks; ++sl)
+            acc += part[((((size_t)sl * g.N + n) * g.C + c) * tiles + t) * span + li];
+    }
+    gx[e] = from_f32<T>(acc);
+}
+
+// Parameter-gradient partial sums of one (k, c) over a share of the (n, position) range: grid
+// (K * C, nsplit), blockDim.x = tb (a power of two).  Shared memory: per present branch a private
+// column per thread and tap, col[tap][tb], then the branch weights and tb floats for the block
+// sums.  Outputs: part_min / part_max [split][k*C+c][tap] (sums of grad_y over the outputs a tap
+// won), part_ab [split][k*C+c][2] (sums of grad_y * branch value, two-branch layers) and, from the
+// blocks of channel 0, part_bias [split][k].
+template <typename T>
+__global__ void __launch_bounds__(128)
+bwd1d_params_kernel(Geo3 g, int nsplit, const T* __restrict__ x, const T* __restrict__ w,
+                    const T* __restrict__ w2, const T* __restrict__ gy, const void* __restrict__ winners,
+                    float* __restrict__ part_min, float* __restrict__ part_max,
+                    float* __restrict__ part_ab, float* __restrict__ part_bias) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tid = threadIdx.x, tb = blockDim.x;
+    const int S = g.S, OL = g.OW, L = g.W;
+    const int kc = blockIdx.x, k = kc / g.C, c = kc % g.C, split = blockIdx.y;
+    const bool twob = two_branch(g.mode);
+    const bool use_min = g.mode != TCONV_MAX_PLUS, use_max = g.mode != TCONV_MIN_PLUS;
+    float* cmin = reinterpret_cast<float*>(smem_raw);
+    float* cmax = cmin + (use_min ? S * tb : 0);
+    float* wmin_s = cmax + (use_max ? S * tb : 0);
+    float* wmax_s = wmin_s + S;
+    float* red = wmax_s + S;
+    for (int i = tid; i < ((use_min ? 1 : 0) + (use_max ? 1 : 0)) * S * tb; i += tb) cmin[i] = 0.0f;
+    for (int s = tid; s < S; s += tb) {
+        const size_t wi = ((size_t)k * g.C + c) * S + s;
+        wmin_s[s] = to_f32(w[wi]);
+        wmax_s[s] = to_f32(g.mode == TCONV_PARALLEL ? w2[wi] : w[wi]);
+    }
+    __syncthreads();
+    const long long total = (long long)g.N * OL;
+    const long long per = (total + nsplit - 1) / nsplit;
+    const long long j0 = split * per, j1 = min(total, j0 + per);
+    float sa = 0.0f, sb = 0.0f, sg = 0.0f;
+    for (long long j = j0 + tid; j < j1; j += tb) {
+        const int n = (int)(j / OL), pos = (int)(j - (long long)n * OL);
+        int amn, amx;
+        winners3(g, winners, n, k, c, pos, amn, amx);
+        const float gv = to_f32(gy[((size_t)n * g.K + k) * OL + pos]);
+        sg += gv;
+        const T* xc = x + ((size_t)n * g.C + c) * L;
+        const int i0 = pos * g.sw - g.pw;
+        if (amn >= 0) {
+            cmin[amn * tb + tid] += gv;
+            if (twob) {
+                const int i = i0 + amn;
+                const T xv = (i >= 0 && i < L) ? xc[i] : zero_of<T>();
+                sa = __fmaf_rn(gv, tap_add(xv, from_f32<T>(wmin_s[amn])), sa);
+            }
+        }
+        if (amx >= 0) {
+            cmax[amx * tb + tid] += gv;
+            if (twob) {
+                const int i = i0 + amx;
+                const T xv = (i >= 0 && i < L) ? xc[i] : zero_of<T>();
+                sb = __fmaf_rn(gv, tap_add(xv, from_f32<T>(wmax_s[amx])), sb);
+            }
+        }
+    }
+    __syncthreads();
+    for (int s = tid; s < S; s += tb) {
+        float tmin = 0.0f, tmax = 0.0f;
+        for (int i = 0; i < tb; ++i) {
+            const int col = (i + tid) & (tb - 1);  // rotated start: the threads of a warp read different banks
+            if (use_min) tmin += cmin[s * tb + col];
+            if (use_max) tmax += cmax[s * tb + col];
+        }
+        const size_t o = ((size_t)split * g.K * g.C + kc) * S + s;
+        part_min[o] = tmin;
+        part_max[o] = tmax;
+    }
+    const float ta = block_sum(sa, red);
+    const float tb_sum = block_sum(sb, red);
+    const float tg = block_sum(sg, red);
+    if (tid == 0) {
+        float* o = part_ab + ((size_t)split * g.K * g.C + kc) * 2;
+        o[0] = ta;
+        o[1] = tb_sum;
+        if (c == 0) part_bias[(size_t)split * g.K + k] = tg;
+    }
+}
+
+}  // namespace tconv
