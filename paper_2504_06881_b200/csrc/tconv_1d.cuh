@@ -249,7 +249,8 @@ bwd1d_gx_kernel(Geo3 g, int pt, int ks, int span, const float* __restrict__ alph
     const int tid = threadIdx.x, tb = blockDim.x;
     const int tile = blockIdx.x, c = blockIdx.y / ks, slice = blockIdx.y % ks, n = blockIdx.z;
     const int OL = g.OW, st = g.sw;
-    const bool twob = two_branch(g.mode);
+    const bool twob = two_branch(g.mode), codes = g.chan == CH_SUM;
+    const bool use_min = g.mode != TCONV_MAX_PLUS, use_max = g.mode != TCONV_MIN_PLUS;
     for (int i = tid; i < 2 * span; i += tb) even[i] = 0.0f;
     __syncthreads();
     float* mine = (tid & 1) ? odd : even;
@@ -264,14 +265,34 @@ bwd1d_gx_kernel(Geo3 g, int pt, int ks, int span, const float* __restrict__ alph
             if (beta) b = beta[(size_t)k * g.C + c];
         }
         const T* grow = gy + ((size_t)n * g.K + k) * OL + p0;
-        for (int i = 0; i < cnt; ++i) {
-            int amn, amx;
-            winners3(g, winners, n, k, c, p0 + i, amn, amx);
-            if (amn < 0 && amx < 0) continue;
-            const float gv = to_f32(grow[i]);
-            float* at = mine + (lp0 + i) * st;
-            if (amn >= 0) at[amn] = twob ? __fmaf_rn(a, gv, at[amn]) : at[amn] + gv;
-            if (amx >= 0) at[amx] = twob ? __fmaf_rn(b, gv, at[amx]) : at[amx] + gv;
+        const uint16_t* crow = (const uint16_t*)winners + (((size_t)n * g.K + k) * g.C + c) * OL + p0;
+        const int32_t* irow = (const int32_t*)winners + ((size_t)n * g.K + k) * OL + p0;
+        // eight positions at a time: their winners and gradients are requested together
+        for (int i0 = 0; i0 < cnt; i0 += 8) {
+            int amn[8], amx[8];
+            float gv[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = min(i0 + u, cnt - 1);
+                if (codes) {
+                    const unsigned v = crow[i];
+                    amn[u] = use_min ? (int)(v & 0xFFu) : -1;
+                    amx[u] = use_max ? (int)(v >> 8) : -1;
+                } else {
+                    const int v = irow[i] - c * g.S;
+                    const int tap = (v >= 0 && v < g.S) ? v : -1;
+                    amn[u] = use_min ? tap : -1;
+                    amx[u] = use_min ? -1 : tap;
+                }
+                gv[u] = to_f32(grow[i]);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (i0 + u >= cnt) break;
+                float* at = mine + (lp0 + i0 + u) * st;
+                if (amn[u] >= 0) at[amn[u]] = twob ? __fmaf_rn(a, gv[u], at[amn[u]]) : at[amn[u]] + gv[u];
+                if (amx[u] >= 0) at[amx[u]] = twob ? __fmaf_rn(b, gv[u], at[amx[u]]) : at[amx[u]] + gv[u];
+            }
         }
     }
     __syncthreads();
@@ -338,29 +359,95 @@ bwd1d_params_kernel(Geo3 g, int nsplit, const T* __restrict__ x, const T* __rest
     const long long per = (total + nsplit - 1) / nsplit;
     const long long j0 = split * per, j1 = min(total, j0 + per);
     float sa = 0.0f, sb = 0.0f, sg = 0.0f;
-    for (long long j = j0 + tid; j < j1; j += tb) {
-        const int n = (int)(j / OL), pos = (int)(j - (long long)n * OL);
-        int amn, amx;
-        winners3(g, winners, n, k, c, pos, amn, amx);
-        const float gv = to_f32(gy[((size_t)n * g.K + k) * OL + pos]);
-        sg += gv;
-        const T* xc = x + ((size_t)n * g.C + c) * L;
-        const int i0 = pos * g.sw - g.pw;
-        if (amn >= 0) {
-            cmin[amn * tb + tid] += gv;
-            if (twob) {
-                const int i = i0 + amn;
-                const T xv = (i >= 0 && i < L) ? xc[i] : zero_of<T>();
-                sa = __fmaf_rn(gv, tap_add(xv, from_f32<T>(wmin_s[amn])), sa);
+    // Items (n, position) of this thread: j0 + tid, + tb, ...; eight at a time.  The winners and
+    // gradients of the next eight are requested before the current eight are worked on; of the
+    // current eight first the branch inputs are gathered, then the columns are updated in item order.
+    const bool codes = g.chan == CH_SUM;
+    const size_t crow = (size_t)g.K * g.C * OL, cbase = ((size_t)k * g.C + c) * OL;  // uint16 [n][k][c][pos]
+    const size_t grow = (size_t)g.K * OL, gbase = (size_t)k * OL;                    // grad_y, int32 winners [n][k][pos]
+    const size_t xrow = (size_t)g.C * L, xbase = (size_t)c * L;
+    const uint16_t* w16 = (const uint16_t*)winners;
+    const int32_t* w32 = (const int32_t*)winners;
+    struct Batch {
+        unsigned raw[8];
+        float gv[8];
+        int n[8], pos[8];
+    };
+    long long j_cur = j0 + tid;
+    int n_cur = (int)(j_cur / OL), pos_cur = (int)(j_cur - (long long)n_cur * OL);
+    auto fetch = [&](Batch& bt) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            bt.n[u] = -1;
+            bt.pos[u] = 0;
+            bt.raw[u] = 0;
+            bt.gv[u] = 0.0f;
+            if (j_cur < j1) {
+                bt.n[u] = n_cur;
+                bt.pos[u] = pos_cur;
+                bt.raw[u] = codes ? (unsigned)w16[n_cur * crow + cbase + pos_cur]
+                                  : (unsigned)w32[n_cur * grow + gbase + pos_cur];
+                bt.gv[u] = to_f32(gy[n_cur * grow + gbase + pos_cur]);
+            }
+            j_cur += tb;
+            pos_cur += tb;
+            if (pos_cur >= OL) {
+                const int q = pos_cur / OL;
+                n_cur += q;
+                pos_cur -= q * OL;
             }
         }
-        if (amx >= 0) {
-            cmax[amx * tb + tid] += gv;
-            if (twob) {
-                const int i = i0 + amx;
-                const T xv = (i >= 0 && i < L) ? xc[i] : zero_of<T>();
-                sb = __fmaf_rn(gv, tap_add(xv, from_f32<T>(wmax_s[amx])), sb);
+    };
+    auto work = [&](const Batch& bt) {
+        int amn[8], amx[8];
+        float vmin[8], vmax[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (codes) {
+                amn[u] = use_min ? (int)(bt.raw[u] & 0xFFu) : -1;
+                amx[u] = use_max ? (int)(bt.raw[u] >> 8) : -1;
+            } else {
+                const int v = (int)bt.raw[u] - c * S;
+                const int tap = (v >= 0 && v < S) ? v : -1;
+                amn[u] = use_min ? tap : -1;
+                amx[u] = use_min ? -1 : tap;
             }
+            if (bt.n[u] < 0) amn[u] = amx[u] = -1;
+        }
+        if (twob) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const T* xc = x + max(bt.n[u], 0) * xrow + xbase;
+                const int i0 = bt.pos[u] * g.sw - g.pw;
+                const int ia = i0 + max(amn[u], 0), ib = i0 + max(amx[u], 0);
+                const T xa = (ia >= 0 && ia < L) ? xc[ia] : zero_of<T>();
+                const T xb = (ib >= 0 && ib < L) ? xc[ib] : zero_of<T>();
+                vmin[u] = tap_add(xa, from_f32<T>(wmin_s[max(amn[u], 0)]));
+                vmax[u] = tap_add(xb, from_f32<T>(wmax_s[max(amx[u], 0)]));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            sg += bt.gv[u];
+            if (amn[u] >= 0) {
+                cmin[amn[u] * tb + tid] += bt.gv[u];
+                if (twob) sa = __fmaf_rn(bt.gv[u], vmin[u], sa);
+            }
+            if (amx[u] >= 0) {
+                cmax[amx[u] * tb + tid] += bt.gv[u];
+                if (twob) sb = __fmaf_rn(bt.gv[u], vmax[u], sb);
+            }
+        }
+    };
+    {
+        const int batches = (int)((j1 - j0 + 8LL * tb - 1) / (8LL * tb));
+        Batch ba, bb;
+        fetch(ba);
+        for (int it = 0; it < batches; it += 2) {
+            fetch(bb);
+            work(ba);
+            fetch(ba);
+            work(bb);
         }
     }
     __syncthreads();
