@@ -876,7 +876,11 @@ inline bool plan_code_gx(const Geo& g, CodeGxPlan* pl) {
     // keeps the bands tall enough for their halo (128x256 at dilation 2: 20.1 -> 12.6 ms).
     if (!g.wide && (long)g.OH * pl->QPR * 2 > 256) {
         CodeGxPlan cand = *pl;
-        if (g.W >= 128 && plan_code_gx_cols(g, 1, (g.W + 63) / 64, 72 * 1024, &cand) && cand.ncol > 1) {
+        // ... but no narrower than a CTA's 256 threads have quads for (signals of unit height)
+        long ncol = (g.W + 63) / 64;
+        const long most = (long)g.OH * pl->QPR / 256;
+        if (ncol > most) ncol = most < 1 ? 1 : most;
+        if (g.W >= 128 && plan_code_gx_cols(g, 1, (int)ncol, 72 * 1024, &cand) && cand.ncol > 1) {
             *pl = cand;
             return true;
         }

@@ -474,8 +474,9 @@ class TropicalConv1d(nn.Module):
     """1-D tropical convolution (Section 3.2) with ``nn.Conv1d``'s constructor arguments; mode / chan /
     params / dtype as in TropicalConv2d.  The length-3, stride-1 layers run as 1 x 3 windows on a signal
     of unit height through the tiled 2-D kernels; every other window (up to 256 taps; the paper's audio
-    networks open with length 80) runs as a 1 x 1 x k window through the any-shape kernels of the
-    three-dimensional entry points, which are the faster ones for long windows."""
+    networks open with length 80 at stride 4) goes as a 1 x 1 x k window through the three-dimensional
+    entry points, which run windows of four taps or more at stride 1, 2 or 4 (no dilation) on their
+    one-dimensional kernels and the rest on the any-shape kernels."""
 
     def __init__(self, in_channels, out_channels, kernel_size, stride=1, padding=0, dilation=1,
                  bias=True, mode="compound", chan="default", params="2p", dtype="f32", fixed=(0.5, 0.5)):
