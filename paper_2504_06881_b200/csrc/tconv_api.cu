@@ -509,9 +509,16 @@ int dw_forward_t(const Geo& g, const void* x, const void* w, const void* w2, con
         const size_t total3 = (size_t)g.N * g.C * strips * QPR;
         const unsigned blocks3 = (unsigned)((total3 + 255) / 256);
         const bool vec = (g.pw == 1 && (g.W & 3) == 0);
+        // bf16 at stride 1: the same strips on packed pairs of outputs
+        constexpr bool kBf16 = sizeof(T) == 2;
 #define TCONV_DW3(MODE, WINV, SWV, VECV)                                                              \
-    dw_fwd3_kernel<T, MODE, WINV, SWV, VECV><<<blocks3, 256, 0, st>>>(                               \
-        g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, bias, (T*)y, (uint8_t*)winners, QPR, strips, (unsigned)total3);
+    if constexpr (kBf16 && SWV == 1)                                                                  \
+        dw_fwd3_bf16_kernel<MODE, WINV, VECV><<<blocks3, 256, 0, st>>>(                               \
+            g, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w, (const __nv_bfloat16*)w2, alpha, beta, bias, \
+            (__nv_bfloat16*)y, (uint8_t*)winners, QPR, strips, (unsigned)total3);                      \
+    else                                                                                              \
+        dw_fwd3_kernel<T, MODE, WINV, SWV, VECV><<<blocks3, 256, 0, st>>>(                            \
+            g, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, bias, (T*)y, (uint8_t*)winners, QPR, strips, (unsigned)total3);
 #define TCONV_DW3_V(MODE, WINV, SWV) { if (vec) TCONV_DW3(MODE, WINV, SWV, true) else TCONV_DW3(MODE, WINV, SWV, false) }
 #define TCONV_DW3_S(MODE, WINV) { if (g.sw == 1) TCONV_DW3_V(MODE, WINV, 1) else TCONV_DW3_V(MODE, WINV, 2) }
 #define TCONV_DW3_W(MODE) { if (winners) TCONV_DW3_S(MODE, true) else TCONV_DW3_S(MODE, false) }

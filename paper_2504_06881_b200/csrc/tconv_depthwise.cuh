@@ -168,6 +168,7 @@ __device__ __forceinline__ void dw_load_row(const T* rp, bool row_ok, unsigned m
 // registers down the strip: every input row of the strip is loaded once per thread.  The nine
 // weights of the channel sit in registers.
 constexpr int kDwRT = 6;   // output rows per strip of the 3x3 depthwise kernels
+constexpr int kDwAhead = 3;   // output rows by which the forward strip kernels request their input rows ahead
 
 template <typename T, int MODE, bool WIN, int SW, bool VEC>
 __global__ void __launch_bounds__(256)
@@ -199,20 +200,26 @@ dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T*
     const float bk = bias ? bias[c] : 0.0f;
     const int ih0 = oh0 * SW - g.ph, c0 = ow0 * SW - g.pw;
     const bool full = (ow0 + 3 < g.OW) && ((g.OW & 3) == 0);
-    T win[3][L];   // input row rho of the strip lives in win[rho % 3]
+    // input row rho of the strip lives in win[rho % WR]; the rows that output row k + AH needs
+    // first are requested before output row k is computed
+    constexpr int AH = SW == 1 ? kDwAhead : 1;   // stride 2: a row is nine registers, one row ahead
+    constexpr int WR = 3 + AH * SW;
+    T win[WR][L];
     const unsigned cmask = dw_col_mask(c0, L, g.W);
     const T* rp0 = xp + (ptrdiff_t)ih0 * g.W + c0;   // column c0 of the strip's first input row
     auto load = [&](int rho) {
         const int ih = ih0 + rho;
-        dw_load_row<T, L, VEC>(rp0 + rho * g.W, ih >= 0 && ih < g.H, cmask, win[rho % 3]);
+        dw_load_row<T, L, VEC>(rp0 + rho * g.W, ih >= 0 && ih < g.H, cmask, win[rho % WR]);
     };
-    load(0);
-    load(1);
+#pragma unroll
+    for (int rho = 0; rho <= (AH - 1) * SW + 2; ++rho) load(rho);
 #pragma unroll
     for (int k = 0; k < RT; ++k) {
         if (oh0 + k >= g.OH) break;
+        if (k + AH < RT) {
 #pragma unroll
-        for (int rho = (k == 0 ? 2 : (k - 1) * SW + 3); rho <= k * SW + 2; ++rho) load(rho);
+            for (int rho = (k + AH - 1) * SW + 3; rho <= (k + AH) * SW + 2; ++rho) load(rho);
+        }
         // per pixel: nine tap sums, their extrema with 3-input min / max and, for the winner codes,
         // the first tap that attains each extremum, recovered on the FMA pipe: d = (t - m) * 2^32 is
         // zero exactly for winning taps, key = |d| * (-2^125) + (2^23 + rank) is 2^23 + rank for them
@@ -226,7 +233,7 @@ dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T*
             float ta[9], tb[PAR ? 9 : 1];
 #pragma unroll
             for (int tap = 0; tap < 9; ++tap) {
-                const T xv = win[(k * SW + tap / 3) % 3][j * SW + tap % 3];
+                const T xv = win[(k * SW + tap / 3) % WR][j * SW + tap % 3];
                 ta[tap] = tap_add(xv, wa[tap]);
                 if constexpr (PAR) tb[tap] = tap_add(xv, wb[tap]);
             }
@@ -282,6 +289,195 @@ dw_fwd3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, const T*
         }
         if constexpr (WIN) {
             const unsigned packed = code4[0] | (code4[1] << 8) | (code4[2] << 16) | (code4[3] << 24);
+            if (full) {
+                *reinterpret_cast<unsigned*>(codes + o) = packed;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (ow0 + j < g.OW) codes[o + j] = (uint8_t)(packed >> (8 * j));
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------- forward, 3x3, bf16 pairs
+// bf16, stride 1: the strip kernel above on packed pairs.  A 32-bit register holds the inputs of
+// two horizontally adjacent outputs; an input row of the strip is kept as the five pairs (e0,e1),
+// (e1,e2), ..., (e4,e5) of its six columns, so that tap column s of output pair p is pair 2p + s.
+// One add.bf16x2 forms two tap sums (each one rounded bf16 add), min / max.bf16x2 fold them (exact),
+// the two-branch combine runs in fp32.  Winner codes: taps descending, a per-half equality mask
+// against the extremum selects the tap, so the lowest equal tap stays.
+__device__ __forceinline__ unsigned dw_hadd2(unsigned a, unsigned b) {
+    unsigned d;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ unsigned dw_hmin2(unsigned a, unsigned b) {
+    unsigned d;
+    asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ unsigned dw_hmax2(unsigned a, unsigned b) {
+    unsigned d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ unsigned dw_fold9_h2(const unsigned* v, bool is_min) {
+    unsigned m = v[0];
+#pragma unroll
+    for (int i = 1; i < 9; ++i) m = is_min ? dw_hmin2(m, v[i]) : dw_hmax2(m, v[i]);
+    return m;
+}
+__device__ __forceinline__ unsigned dw_heq2_mask(unsigned a, unsigned b) {
+    return __heq2_mask(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+}
+
+template <int MODE, bool WIN, bool VEC>
+__global__ void __launch_bounds__(256)
+dw_fwd3_bf16_kernel(Geo g, const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
+                    const __nv_bfloat16* __restrict__ w2, const float* __restrict__ alpha,
+                    const float* __restrict__ beta, const float* __restrict__ bias,
+                    __nv_bfloat16* __restrict__ y, uint8_t* __restrict__ codes, int QPR, int strips,
+                    unsigned total) {
+    using T = __nv_bfloat16;
+    constexpr int RT = kDwRT, L = 6;
+    constexpr bool TWO = (MODE == TCONV_COMPOUND || MODE == TCONV_PARALLEL);
+    constexpr bool PAR = (MODE == TCONV_PARALLEL);
+    constexpr bool DO_MIN = TWO || MODE == TCONV_MIN_PLUS, DO_MAX = TWO || MODE == TCONV_MAX_PLUS;
+    const unsigned q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= total) return;
+    const unsigned t = q / (unsigned)QPR;
+    const int qx = (int)(q - t * (unsigned)QPR);
+    const size_t nc = t / (unsigned)strips;
+    const int oh0 = (int)(t - (unsigned)nc * (unsigned)strips) * RT;
+    const int c = (int)((unsigned)nc % (unsigned)g.C);
+    const int ow0 = qx * 4;
+    const T* xp = x + nc * (size_t)g.H * g.W;
+    unsigned wa[9], wb[9];   // {w, w}
+#pragma unroll
+    for (int i = 0; i < 9; ++i) {
+        wa[i] = 0x00010001u * (unsigned)__bfloat16_as_ushort(__ldg(w + (size_t)c * 9 + i));
+        wb[i] = PAR ? 0x00010001u * (unsigned)__bfloat16_as_ushort(__ldg(w2 + (size_t)c * 9 + i)) : wa[i];
+    }
+    const float a = (TWO && alpha) ? alpha[c] : 1.0f, b = (TWO && beta) ? beta[c] : 1.0f;
+    const float bk = bias ? bias[c] : 0.0f;
+    const int ih0 = oh0 - g.ph, c0 = ow0 - g.pw;
+    const bool full = (ow0 + 3 < g.OW) && ((g.OW & 3) == 0);
+    // Rows are requested kDwAhead output rows ahead into a ring of raw loads (first column, the four
+    // aligned columns as two words, last column) and turned into the five pairs when they enter the
+    // window of three rows, win[rho % 3].
+    constexpr int RW = kDwAhead + 1;
+    static_assert(kDwAhead >= 2, "row k + 2 must have been requested before output row k");
+    unsigned raw[RW][4];
+    unsigned win[3][5];
+    const unsigned cmask = dw_col_mask(c0, L, g.W);
+    const T* rp0 = xp + (ptrdiff_t)ih0 * g.W + c0;
+    auto issue = [&](int rho) {
+        const int ih = ih0 + rho;
+        const unsigned mask = (ih >= 0 && ih < g.H) ? cmask : 0u;
+        const unsigned short* rp = reinterpret_cast<const unsigned short*>(rp0 + rho * g.W);
+        unsigned* r = raw[rho % RW];
+        if constexpr (VEC) {
+            r[0] = (mask & 1u) ? (unsigned)__ldg(rp) : 0u;
+            if ((mask >> 1) & 1u) {
+                const uint2 v = __ldg(reinterpret_cast<const uint2*>(rp + 1));
+                r[1] = v.x;
+                r[2] = v.y;
+            } else {
+                r[1] = r[2] = 0u;
+            }
+            r[3] = ((mask >> 5) & 1u) ? (unsigned)__ldg(rp + 5) : 0u;
+        } else {
+            unsigned e[L];
+#pragma unroll
+            for (int i = 0; i < L; ++i) e[i] = ((mask >> i) & 1u) ? (unsigned)__ldg(rp + i) : 0u;
+            r[0] = e[0];
+            r[1] = e[1] | (e[2] << 16);
+            r[2] = e[3] | (e[4] << 16);
+            r[3] = e[5];
+        }
+    };
+    auto pack = [&](int rho) {
+        const unsigned* r = raw[rho % RW];
+        unsigned* d = win[rho % 3];
+        d[0] = __byte_perm(r[0], r[1], 0x5410);
+        d[1] = r[1];
+        d[2] = __byte_perm(r[1], r[2], 0x5432);
+        d[3] = r[2];
+        d[4] = __byte_perm(r[2], r[3], 0x5432);
+    };
+#pragma unroll
+    for (int rho = 0; rho <= kDwAhead; ++rho) issue(rho);
+    pack(0);
+    pack(1);
+#pragma unroll
+    for (int k = 0; k < RT; ++k) {
+        if (oh0 + k >= g.OH) break;
+        pack(k + 2);
+        if (k + kDwAhead <= RT) issue(k + kDwAhead + 1);
+        float mn[4], mx[4];
+        unsigned code2[2] = {0u, 0u};
+#pragma unroll
+        for (int pr = 0; pr < 2; ++pr) {
+            unsigned ta[9], tb[PAR ? 9 : 1];
+#pragma unroll
+            for (int tap = 0; tap < 9; ++tap) {
+                const unsigned xv = win[(k + tap / 3) % 3][2 * pr + tap % 3];
+                ta[tap] = dw_hadd2(xv, wa[tap]);
+                if constexpr (PAR) tb[tap] = dw_hadd2(xv, wb[tap]);
+            }
+            const unsigned* tm = PAR ? tb : ta;
+            unsigned m2 = 0u, M2 = 0u;
+            if constexpr (DO_MIN) {
+                m2 = dw_fold9_h2(ta, true);
+                mn[2 * pr] = __uint_as_float(m2 << 16);
+                mn[2 * pr + 1] = __uint_as_float(m2 & 0xffff0000u);
+            }
+            if constexpr (DO_MAX) {
+                M2 = dw_fold9_h2(tm, false);
+                mx[2 * pr] = __uint_as_float(M2 << 16);
+                mx[2 * pr + 1] = __uint_as_float(M2 & 0xffff0000u);
+            }
+            if constexpr (WIN) {
+                unsigned smn = 0u, smx = 0u;
+#pragma unroll
+                for (int tap = 8; tap >= 0; --tap) {
+                    if constexpr (DO_MIN) {
+                        const unsigned eq = dw_heq2_mask(ta[tap], m2);
+                        smn = (eq & (0x00010001u * (unsigned)tap)) | (~eq & smn);
+                    }
+                    if constexpr (DO_MAX) {
+                        const unsigned eq = dw_heq2_mask(tm[tap], M2);
+                        smx = (eq & (0x00010001u * (unsigned)tap)) | (~eq & smx);
+                    }
+                }
+                code2[pr] = smn | (smx << 4);
+            }
+        }
+        const size_t o = (nc * g.OH + oh0 + k) * (size_t)g.OW + ow0;
+        if (y) {
+            float v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float acc;
+                if constexpr (TWO) acc = __fmaf_rn(b, mx[j], __fmaf_rn(a, mn[j], 0.0f));
+                else acc = __fadd_rn(0.0f, DO_MIN ? mn[j] : mx[j]);
+                v[j] = bias ? __fadd_rn(acc, bk) : acc;
+            }
+            if (full) {
+                const __nv_bfloat162 p01 = __floats2bfloat162_rn(v[0], v[1]);
+                const __nv_bfloat162 p23 = __floats2bfloat162_rn(v[2], v[3]);
+                *reinterpret_cast<uint2*>(y + o) = make_uint2(*reinterpret_cast<const unsigned*>(&p01),
+                                                              *reinterpret_cast<const unsigned*>(&p23));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (ow0 + j < g.OW) y[o + j] = __float2bfloat16_rn(v[j]);
+            }
+        }
+        if constexpr (WIN) {
+            // bytes 0 and 2 of each pair's code word are the codes of its two outputs
+            const unsigned packed = __byte_perm(code2[0], code2[1], 0x6420);
             if (full) {
                 *reinterpret_cast<unsigned*>(codes + o) = packed;
             } else {
