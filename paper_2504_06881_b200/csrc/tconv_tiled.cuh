@@ -933,7 +933,39 @@ inline encode_tiled_fn get_encode_tiled() {
 }
 
 // x viewed as [N*C][H][W]; box = [CC][NSLOTS][XP]; out-of-range elements read as the padding value.
+// The encoded map is a pure function of the arguments below, so the last few are kept per host
+// thread (a training loop calls each layer with the same buffers step after step).
+struct XMapKey {
+    const void* x;
+    long long nc;
+    int W, H, esize, XP, NSLOTS, CC, neutral;
+};
+constexpr int kXMapCache = 16;
+
+inline bool encode_x_map(const Geo& g, const void* x, int esize, const TiledParams& p, CUtensorMap* map);
+
 inline bool make_x_map(const Geo& g, const void* x, int esize, const TiledParams& p, CUtensorMap* map) {
+    static thread_local XMapKey keys[kXMapCache];
+    static thread_local CUtensorMap maps[kXMapCache];
+    static thread_local int used = 0, next = 0;
+    XMapKey k;
+    memset(&k, 0, sizeof(k));
+    k.x = x; k.nc = (long long)g.N * g.C; k.W = g.W; k.H = g.H; k.esize = esize;
+    k.XP = p.XP; k.NSLOTS = p.NSLOTS; k.CC = p.CC; k.neutral = g.neutral;
+    for (int i = 0; i < used; ++i)
+        if (memcmp(&keys[i], &k, sizeof(k)) == 0) {
+            *map = maps[i];
+            return true;
+        }
+    if (!encode_x_map(g, x, esize, p, map)) return false;
+    keys[next] = k;
+    maps[next] = *map;
+    next = (next + 1) % kXMapCache;
+    if (used < kXMapCache) ++used;
+    return true;
+}
+
+inline bool encode_x_map(const Geo& g, const void* x, int esize, const TiledParams& p, CUtensorMap* map) {
     encode_tiled_fn enc = get_encode_tiled();
     if (!enc) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N * g.C};
