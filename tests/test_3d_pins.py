@@ -225,3 +225,47 @@ def test_gradient_conservation_without_padding():
     per_k = t["g"].astype(np.float64).sum(axis=(0, 2, 3, 4))
     want = ((t["alpha"].astype(np.float64) + t["beta"]) * per_k[:, None]).sum()
     assert abs(bc["grad_x"][0].sum() - want) < 1e-8 and abs(bc["grad_w"][0].sum() - want) < 1e-8
+
+
+@pytest.mark.parametrize("mode,chan", MODES)
+def test_one_dimensional_layers_with_long_windows(mode, chan):
+    """Unit depth and height with a 1 x 1 x 80 window at stride 4 (the opening layer of the paper's
+    audio networks) against a formulation written out in one dimension with numpy's strided
+    windows, and against the (pinned) two-dimensional oracle on a signal of unit height."""
+    d = inputs.layer3d(2, 3, 1, 1, 413, 4, T=1, R=1, S=80, stride=(1, 1, 4), pad=(0, 0, 9), mode=mode, chan=chan)
+    t = inputs.draw3d(d, 4242, x=("ints", -3, 3), w=("ints", -2, 2)) if chan in ("min", "max") else inputs.draw3d(d, 4242)
+    out = ora3.forward(d, t["x"], t["w"], bias=t["bias"], **_args(d, t))
+    N, C, K, S, L = d["N"], d["C"], d["K"], 80, 413
+    xp = np.zeros((N, C, L + 18), np.float32)
+    xp[:, :, 9:9 + L] = t["x"][:, :, 0, 0]
+    win = np.lib.stride_tricks.sliding_window_view(xp, S, axis=2)[:, :, ::4]          # [N, C, OL, S]
+    t1 = win[:, None] + t["w"].reshape(1, K, C, 1, S)                                 # [N, K, C, OL, S]
+    t2 = win[:, None] + t["w2"].reshape(1, K, C, 1, S) if mode == "parallel" else t1
+    mn, mx = t1.min(-1), t2.max(-1)
+    if mode in ("compound", "parallel"):
+        y = np.zeros(mn[:, :, 0].shape, np.float32)
+        for c in range(C):
+            y = _fmaf32(t["beta"][:, c].reshape(1, K, 1), mx[:, :, c], _fmaf32(t["alpha"][:, c].reshape(1, K, 1), mn[:, :, c], y))
+        assert np.array_equal(out["codes"][:, :, :, 0, 0], (t1.argmin(-1) | (t2.argmax(-1) << 8)).astype(np.uint16))
+    else:
+        m = mn if mode == "min_plus" else mx
+        rc = ora3.resolved_chan(d)
+        if rc == "sum":
+            y = np.zeros(m[:, :, 0].shape, np.float32)
+            for c in range(C):
+                y = (y + m[:, :, c]).astype(np.float32)
+        else:
+            y = m.max(2) if rc == "max" else m.min(2)
+    y = (y + t["bias"].reshape(1, K, 1)).astype(np.float32)
+    assert np.array_equal(out["y"][:, :, 0, 0], y)
+    # the same layer as a 1 x 80 window on a signal of unit height, through the two-dimensional oracle
+    d2 = inputs.layer(2, 3, 1, 413, 4, 1, 80, stride=(1, 4), pad=(0, 9), mode=mode, chan=chan)
+    two, par = mode in ("compound", "parallel"), mode == "parallel"
+    ref = ora2.forward(d2, t["x"][:, :, 0], t["w"][:, :, 0], t["w2"][:, :, 0] if par else None,
+                       t["alpha"] if two else None, t["beta"] if two else None, t["bias"])
+    assert np.array_equal(out["y"][:, :, 0], ref["y"])
+    g3 = ora3.backward(d, t["x"], t["w"], t["g"], **_args(d, t))
+    g2 = ora2.backward(d2, t["x"][:, :, 0], t["w"][:, :, 0], t["g"][:, :, 0], t["w2"][:, :, 0] if par else None,
+                       t["alpha"] if two else None, t["beta"] if two else None)
+    for k in g2:
+        assert np.allclose(np.asarray(g3[k]).reshape(np.asarray(g2[k]).shape), g2[k], rtol=1e-6, atol=1e-6), k
