@@ -586,6 +586,15 @@ int dw_backward_t(const Geo& g, const void* x, const void* w, const void* w2, co
 #undef TCONV_DW_GX3_V
 #undef TCONV_DW_GX3
         g_launches += 1;
+    } else if (gx && g.R == 3 && g.S == 3 && g.dh == 1 && g.dw == 1 && g.sh == 2 && g.sw == 2 && g.ph == 1 && g.pw == 1) {
+        // 3x3, stride 2, padding 1: one thread per 2 x 2 input block
+        const int HB = (g.H + 1) / 2, WB = (g.W + 1) / 2;
+        const size_t total = (size_t)g.N * g.C * HB * WB;
+        const unsigned blocks = (unsigned)((total + 255) / 256);
+        if (br == 0) dw_bwd_gx_s2_kernel<T, 0><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, HB, WB, (unsigned)total);
+        else if (br == 1) dw_bwd_gx_s2_kernel<T, 1><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, HB, WB, (unsigned)total);
+        else dw_bwd_gx_s2_kernel<T, 2><<<blocks, 256, 0, st>>>(g, alpha, beta, (const T*)gy, codes, (T*)gx, HB, WB, (unsigned)total);
+        g_launches += 1;
     } else if (gx) {
         const size_t total = (size_t)g.N * g.C * g.H * g.W;
         const unsigned blocks = (unsigned)((total + 255) / 256);

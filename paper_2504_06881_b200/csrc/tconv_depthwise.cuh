@@ -489,6 +489,78 @@ dw_fwd3_bf16_kernel(Geo g, const __nv_bfloat16* __restrict__ x, const __nv_bfloa
     }
 }
 
+// ---------------------------------------------------------------------------------- grad_x, 3x3 at stride 2
+// 3x3 window, stride 2, padding 1, dilation 1: the outputs that read an input element, and through
+// which tap, depend only on the parity of its row and column.  One thread owns the 2 x 2 input block
+// (2a, 2b) .. (2a + 1, 2b + 1) and the four outputs (a, b) .. (a + 1, b + 1) that reach it:
+//   (2a,   2b  ): (a, b) tap 4
+//   (2a,   2b+1): (a, b+1) tap 3, (a, b) tap 5
+//   (2a+1, 2b  ): (a+1, b) tap 1, (a, b) tap 7
+//   (2a+1, 2b+1): (a+1, b+1) tap 0, (a+1, b) tap 2, (a, b+1) tap 6, (a, b) tap 8
+// Every thread runs the same nine comparisons per branch, in ascending tap order per element.
+// BR: 0 both branches, 1 min branch only, 2 max branch only.
+template <typename T, int BR>
+__global__ void __launch_bounds__(256)
+dw_bwd_gx_s2_kernel(Geo g, const float* __restrict__ alpha, const float* __restrict__ beta,
+                    const T* __restrict__ gy, const uint8_t* __restrict__ codes, T* __restrict__ gx,
+                    int HB, int WB, unsigned total) {
+    const unsigned i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const unsigned t = i / (unsigned)WB;
+    const int b = (int)(i - t * (unsigned)WB);
+    const size_t nc = t / (unsigned)HB;
+    const int a = (int)(t - (unsigned)nc * (unsigned)HB);
+    const int c = (int)((unsigned)nc % (unsigned)g.C);
+    const float ca = (BR == 0 && alpha) ? alpha[c] : 1.0f, cb = (BR == 0 && beta) ? beta[c] : 1.0f;
+    const T* gp = gy + nc * (size_t)g.OH * g.OW;
+    const uint8_t* cp = codes + nc * (size_t)g.OH * g.OW;
+    // the four outputs; one outside the map gets a code no tap equals
+    unsigned code[2][2];
+    float gv[2][2];
+#pragma unroll
+    for (int da = 0; da < 2; ++da)
+#pragma unroll
+        for (int db = 0; db < 2; ++db) {
+            const int oh = a + da, ow = b + db;
+            const bool ok = oh < g.OH && ow < g.OW;
+            code[da][db] = ok ? (unsigned)__ldg(cp + (size_t)oh * g.OW + ow) : 0xffu;
+            gv[da][db] = ok ? to_f32(__ldg(gp + (size_t)oh * g.OW + ow)) : 0.0f;
+        }
+    auto take = [&](float acc, int da, int db, unsigned tap) {
+        const unsigned cd = code[da][db];
+        const float v = gv[da][db];
+        if ((BR == 0 || BR == 1) && (cd & 15u) == tap) acc = (BR == 0) ? __fmaf_rn(ca, v, acc) : acc + v;
+        if ((BR == 0 || BR == 2) && (cd >> 4) == tap) acc = (BR == 0) ? __fmaf_rn(cb, v, acc) : acc + v;
+        return acc;
+    };
+    const float e00 = take(0.0f, 0, 0, 4u);
+    const float e01 = take(take(0.0f, 0, 1, 3u), 0, 0, 5u);
+    const float e10 = take(take(0.0f, 1, 0, 1u), 0, 0, 7u);
+    const float e11 = take(take(take(take(0.0f, 1, 1, 0u), 1, 0, 2u), 0, 1, 6u), 0, 0, 8u);
+    const int ih = 2 * a, iw = 2 * b;
+    T* o = gx + (nc * g.H + ih) * (size_t)g.W + iw;
+    if ((g.W & 1) == 0) {
+        // even rows: the two columns of the block are one aligned pair
+        auto store2 = [](T* p, float v0, float v1) {
+            if constexpr (sizeof(T) == 4) {
+                *reinterpret_cast<float2*>(p) = make_float2(v0, v1);
+            } else {
+                *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(v0, v1);
+            }
+        };
+        store2(o, e00, e01);
+        if (ih + 1 < g.H) store2(o + g.W, e10, e11);
+        return;
+    }
+    const bool right = iw + 1 < g.W;
+    o[0] = from_f32<T>(e00);
+    if (right) o[1] = from_f32<T>(e01);
+    if (ih + 1 < g.H) {
+        o[g.W] = from_f32<T>(e10);
+        if (right) o[g.W + 1] = from_f32<T>(e11);
+    }
+}
+
 // ---------------------------------------------------------------------------------- grad_x
 // Gather form: one thread per input element visits, in ascending tap order, the outputs that read
 // it, and takes coef * grad_y from those whose winner is that tap.  No atomics, fixed order.
@@ -728,6 +800,7 @@ dw_bwd_params3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, c
                       float* __restrict__ partial, int nchunks, int need_ab, int QPR, int strips) {
     constexpr int RT = kDwRT;
     constexpr int L = 3 * SW + 3;
+    constexpr bool PACKED = sizeof(T) == 2 && SW == 1;
     extern __shared__ float col[];   // [kDwAcc][256]
     const int c = blockIdx.x, chunk = blockIdx.y, tid = threadIdx.x;
     for (int e = tid; e < kDwAcc * 256; e += 256) col[e] = 0.0f;
@@ -787,6 +860,36 @@ dw_bwd_params3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, c
                     if (ok) cq |= (unsigned)__ldg(cp + (size_t)oh * g.OW + j) << (8 * j);
                 }
             }
+            // bf16 at stride 1: the branch values of the four outputs on packed pairs, as in the forward
+            float bmn[4] = {0.0f, 0.0f, 0.0f, 0.0f}, bmx[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            if constexpr (PACKED) {
+                if (need_ab) {
+#pragma unroll
+                    for (int pr = 0; pr < 2; ++pr) {
+                        unsigned ta[9], tb[PAR ? 9 : 1];
+#pragma unroll
+                        for (int tap = 0; tap < 9; ++tap) {
+                            const T* row = win[(k + tap / 3) % 3];
+                            const int i = 2 * pr + tap % 3;
+                            const unsigned xv = (unsigned)__bfloat16_as_ushort(row[i]) |
+                                                ((unsigned)__bfloat16_as_ushort(row[i + 1]) << 16);
+                            ta[tap] = dw_hadd2(xv, 0x00010001u * (unsigned)__bfloat16_as_ushort(wa[tap]));
+                            if constexpr (PAR) tb[tap] = dw_hadd2(xv, 0x00010001u * (unsigned)__bfloat16_as_ushort(wb[tap]));
+                        }
+                        const unsigned* tm = PAR ? tb : ta;
+                        if (BR == 0 || BR == 1) {
+                            const unsigned m2 = dw_fold9_h2(ta, true);
+                            bmn[2 * pr] = __uint_as_float(m2 << 16);
+                            bmn[2 * pr + 1] = __uint_as_float(m2 & 0xffff0000u);
+                        }
+                        if (BR == 0 || BR == 2) {
+                            const unsigned m2 = dw_fold9_h2(tm, false);
+                            bmx[2 * pr] = __uint_as_float(m2 << 16);
+                            bmx[2 * pr + 1] = __uint_as_float(m2 & 0xffff0000u);
+                        }
+                    }
+                }
+            }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 if (!full && ow0 + j >= g.OW) continue;
@@ -796,16 +899,21 @@ dw_bwd_params3_kernel(Geo g, const T* __restrict__ x, const T* __restrict__ w, c
                 if (BR == 0 || BR == 1) mine[(code & 15u) * 256] += gv;
                 if (BR == 0 || BR == 2) mine[(16 + (code >> 4)) * 256] += gv;
                 if (need_ab) {
-                    float ta[9], tb[PAR ? 9 : 1];
+                    if constexpr (PACKED) {
+                        if (BR == 0 || BR == 1) sa = __fmaf_rn(gv, bmn[j], sa);
+                        if (BR == 0 || BR == 2) sb = __fmaf_rn(gv, bmx[j], sb);
+                    } else {
+                        float ta[9], tb[PAR ? 9 : 1];
 #pragma unroll
-                    for (int tap = 0; tap < 9; ++tap) {
-                        const T xv = win[(k * SW + tap / 3) % 3][j * SW + tap % 3];
-                        ta[tap] = tap_add(xv, wa[tap]);
-                        if constexpr (PAR) tb[tap] = tap_add(xv, wb[tap]);
+                        for (int tap = 0; tap < 9; ++tap) {
+                            const T xv = win[(k * SW + tap / 3) % 3][j * SW + tap % 3];
+                            ta[tap] = tap_add(xv, wa[tap]);
+                            if constexpr (PAR) tb[tap] = tap_add(xv, wb[tap]);
+                        }
+                        const float* tm = PAR ? tb : ta;
+                        if (BR == 0 || BR == 1) sa = __fmaf_rn(gv, dw_fold9(ta, true), sa);
+                        if (BR == 0 || BR == 2) sb = __fmaf_rn(gv, dw_fold9(tm, false), sb);
                     }
-                    const float* tm = PAR ? tb : ta;
-                    if (BR == 0 || BR == 1) sa = __fmaf_rn(gv, dw_fold9(ta, true), sa);
-                    if (BR == 0 || BR == 2) sb = __fmaf_rn(gv, dw_fold9(tm, false), sb);
                 }
             }
         }

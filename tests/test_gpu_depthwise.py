@@ -62,6 +62,8 @@ def test_depthwise_geometries(mode, dtype):
     mk = lambda N, C, H, W, R, S, **k: inputs.layer(N, C, H, W, C, R, S, mode=mode, dtype=dtype, **k)
     cases = [mk(2, 5, 9, 11, 3, 3, stride=1, pad=1),          # ragged width
              mk(3, 8, 16, 16, 3, 3, stride=2, pad=1),         # the stride-2 depthwise of an inverted residual
+             mk(2, 5, 7, 7, 3, 3, stride=2, pad=1),           # stride 2 on odd extents (7 -> 4)
+             mk(2, 3, 10, 13, 3, 3, stride=2, pad=1),         # stride 2, even height, odd width
              mk(2, 4, 12, 20, 3, 3, stride=1, pad=2, dil=2),
              mk(2, 3, 7, 7, 3, 3, stride=1, pad=0),           # no padding
              mk(1, 6, 10, 9, 1, 3, stride=1, pad=1),          # 1 x 3 window
