@@ -135,15 +135,21 @@ Plan1 plan_1d(const Geo3& g) {
     p.ks = (int)ks;
     p.part_floats = (size_t)p.ks * g.N * g.C * p.tiles * p.span;
     const int branches = two_branch(g.mode) ? 2 : 1;
+    // threads per block: 128, or fewer while the private columns of a block exceed 48 KB (two
+    // branches of a long window), so that several blocks stay resident per SM
     p.ptb = 128;
     for (;;) {
-        p.p_smem = ((size_t)branches * S * p.ptb + 2 * S + p.ptb) * sizeof(float);
-        if (p.p_smem <= kSmem1d || p.ptb == 32) break;
+        p.p_smem = ((size_t)branches * (S + 1) * p.ptb + 2 * S + p.ptb) * sizeof(float);
+        if (p.p_smem <= 48 * 1024 || p.ptb == 32) break;
         p.ptb /= 2;
     }
     if (p.p_smem > kSmem1d) return p;
+    // splits of the (n, position) range: as many blocks as are resident at once (one round), each
+    // split at least 2048 items long
     const long long kc = (long long)g.K * g.C, total = (long long)g.N * OL;
-    long long want = (4 * 148 + kc - 1) / kc;
+    long long per_sm = (long long)(200 * 1024 / (p.p_smem + 1024));
+    if (per_sm > 384 / p.ptb) per_sm = 384 / p.ptb;   // registers: the kernel's launch bounds
+    long long want = 148 * per_sm / kc;
     const long long most = (total + 2047) / 2048;
     if (want > most) want = most;
     if (want < 1) want = 1;

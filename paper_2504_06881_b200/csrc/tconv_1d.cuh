@@ -330,9 +330,10 @@ bwd1d_gx_finish_kernel(Geo3 g, int tiles, int ks, int span, int tile_x, const fl
 // column per thread and tap, col[tap][tb], then the branch weights and tb floats for the block
 // sums.  Outputs: part_min / part_max [split][k*C+c][tap] (sums of grad_y over the outputs a tap
 // won), part_ab [split][k*C+c][2] (sums of grad_y * branch value, two-branch layers) and, from the
-// blocks of channel 0, part_bias [split][k].
+// blocks of channel 0, part_bias [split][k].  (The launch bounds keep 384 threads resident per SM: the
+// host sizes the splits for one round of blocks.)
 template <typename T>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 3)
 bwd1d_params_kernel(Geo3 g, int nsplit, const T* __restrict__ x, const T* __restrict__ w,
                     const T* __restrict__ w2, const T* __restrict__ gy, const void* __restrict__ winners,
                     float* __restrict__ part_min, float* __restrict__ part_max,
@@ -343,58 +344,63 @@ bwd1d_params_kernel(Geo3 g, int nsplit, const T* __restrict__ x, const T* __rest
     const int kc = blockIdx.x, k = kc / g.C, c = kc % g.C, split = blockIdx.y;
     const bool twob = two_branch(g.mode);
     const bool use_min = g.mode != TCONV_MAX_PLUS, use_max = g.mode != TCONV_MIN_PLUS;
+    // S + 1 columns per present branch: column S takes the items that have no winner in the branch
     float* cmin = reinterpret_cast<float*>(smem_raw);
-    float* cmax = cmin + (use_min ? S * tb : 0);
-    float* wmin_s = cmax + (use_max ? S * tb : 0);
+    float* cmax = cmin + (use_min ? (S + 1) * tb : 0);
+    float* wmin_s = cmax + (use_max ? (S + 1) * tb : 0);
     float* wmax_s = wmin_s + S;
     float* red = wmax_s + S;
-    for (int i = tid; i < ((use_min ? 1 : 0) + (use_max ? 1 : 0)) * S * tb; i += tb) cmin[i] = 0.0f;
+    for (int i = tid; i < ((use_min ? 1 : 0) + (use_max ? 1 : 0)) * (S + 1) * tb; i += tb) cmin[i] = 0.0f;
     for (int s = tid; s < S; s += tb) {
         const size_t wi = ((size_t)k * g.C + c) * S + s;
         wmin_s[s] = to_f32(w[wi]);
         wmax_s[s] = to_f32(g.mode == TCONV_PARALLEL ? w2[wi] : w[wi]);
     }
     __syncthreads();
-    const long long total = (long long)g.N * OL;
-    const long long per = (total + nsplit - 1) / nsplit;
-    const long long j0 = split * per, j1 = min(total, j0 + per);
+    const int total = g.N * OL;   // (every tensor of the layer has fewer than 2^31 elements)
+    const int per = (total + nsplit - 1) / nsplit;
+    const int j0 = min(total, split * per), j1 = min(total, j0 + per);
     float sa = 0.0f, sb = 0.0f, sg = 0.0f;
     // Items (n, position) of this thread: j0 + tid, + tb, ...; eight at a time.  The winners and
     // gradients of the next eight are requested before the current eight are worked on; of the
     // current eight first the branch inputs are gathered, then the columns are updated in item order.
+    // An item past the end reads the first item of the row (a valid address) and counts as zero.
     const bool codes = g.chan == CH_SUM;
-    const size_t crow = (size_t)g.K * g.C * OL, cbase = ((size_t)k * g.C + c) * OL;  // uint16 [n][k][c][pos]
-    const size_t grow = (size_t)g.K * OL, gbase = (size_t)k * OL;                    // grad_y, int32 winners [n][k][pos]
-    const size_t xrow = (size_t)g.C * L, xbase = (size_t)c * L;
+    const int crow = g.K * g.C * OL, cbase = (k * g.C + c) * OL;  // uint16 codes [n][k][c][pos]
+    const int grow = g.K * OL, gbase = k * OL;                    // grad_y, int32 winners [n][k][pos]
+    const int xrow = g.C * L, xbase = c * L;
     const uint16_t* w16 = (const uint16_t*)winners;
     const int32_t* w32 = (const int32_t*)winners;
     struct Batch {
         unsigned raw[8];
         float gv[8];
-        int n[8], pos[8];
+        int xpl[8];   // offset of the item's input row, -1: no item
+        int li0[8];   // input index of the window's first tap
     };
-    long long j_cur = j0 + tid;
-    int n_cur = (int)(j_cur / OL), pos_cur = (int)(j_cur - (long long)n_cur * OL);
+    int j_cur = j0 + tid;
+    int n_cur = j_cur / OL, pos_cur = j_cur - n_cur * OL;
+    int cofs = n_cur * crow + cbase + pos_cur, gofs = n_cur * grow + gbase + pos_cur, xofs = n_cur * xrow + xbase;
     auto fetch = [&](Batch& bt) {
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            bt.n[u] = -1;
-            bt.pos[u] = 0;
-            bt.raw[u] = 0;
-            bt.gv[u] = 0.0f;
-            if (j_cur < j1) {
-                bt.n[u] = n_cur;
-                bt.pos[u] = pos_cur;
-                bt.raw[u] = codes ? (unsigned)w16[n_cur * crow + cbase + pos_cur]
-                                  : (unsigned)w32[n_cur * grow + gbase + pos_cur];
-                bt.gv[u] = to_f32(gy[n_cur * grow + gbase + pos_cur]);
-            }
+            const bool ok = j_cur < j1;
+            const int co = ok ? cofs : cbase, go = ok ? gofs : gbase;
+            bt.raw[u] = codes ? (unsigned)w16[co] : (unsigned)w32[go];
+            const float gv = to_f32(gy[go]);
+            bt.gv[u] = ok ? gv : 0.0f;
+            bt.xpl[u] = ok ? xofs : -1;
+            bt.li0[u] = pos_cur * g.sw - g.pw;
             j_cur += tb;
             pos_cur += tb;
+            cofs += tb;
+            gofs += tb;
             if (pos_cur >= OL) {
                 const int q = pos_cur / OL;
                 n_cur += q;
                 pos_cur -= q * OL;
+                cofs += q * (crow - OL);
+                gofs += q * (grow - OL);
+                xofs += q * xrow;
             }
         }
     };
@@ -403,44 +409,44 @@ bwd1d_params_kernel(Geo3 g, int nsplit, const T* __restrict__ x, const T* __rest
         float vmin[8], vmax[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
+            int tmn, tmx;
             if (codes) {
-                amn[u] = use_min ? (int)(bt.raw[u] & 0xFFu) : -1;
-                amx[u] = use_max ? (int)(bt.raw[u] >> 8) : -1;
+                tmn = (int)(bt.raw[u] & 0xFFu);
+                tmx = (int)(bt.raw[u] >> 8);
             } else {
                 const int v = (int)bt.raw[u] - c * S;
-                const int tap = (v >= 0 && v < S) ? v : -1;
-                amn[u] = use_min ? tap : -1;
-                amx[u] = use_min ? -1 : tap;
+                tmn = tmx = (v >= 0 && v < S) ? v : S;
             }
-            if (bt.n[u] < 0) amn[u] = amx[u] = -1;
+            const bool ok = bt.xpl[u] >= 0;
+            amn[u] = (ok && use_min) ? tmn : S;
+            amx[u] = (ok && use_max) ? tmx : S;
         }
         if (twob) {
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const T* xc = x + max(bt.n[u], 0) * xrow + xbase;
-                const int i0 = bt.pos[u] * g.sw - g.pw;
-                const int ia = i0 + max(amn[u], 0), ib = i0 + max(amx[u], 0);
+                const T* xc = x + max(bt.xpl[u], 0);
+                const int ta = min(amn[u], S - 1), tb2 = min(amx[u], S - 1);
+                const int ia = bt.li0[u] + ta, ib = bt.li0[u] + tb2;
                 const T xa = (ia >= 0 && ia < L) ? xc[ia] : zero_of<T>();
                 const T xb = (ib >= 0 && ib < L) ? xc[ib] : zero_of<T>();
-                vmin[u] = tap_add(xa, from_f32<T>(wmin_s[max(amn[u], 0)]));
-                vmax[u] = tap_add(xb, from_f32<T>(wmax_s[max(amx[u], 0)]));
+                vmin[u] = tap_add(xa, from_f32<T>(wmin_s[ta]));
+                vmax[u] = tap_add(xb, from_f32<T>(wmax_s[tb2]));
             }
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            sg += bt.gv[u];
-            if (amn[u] >= 0) {
-                cmin[amn[u] * tb + tid] += bt.gv[u];
-                if (twob) sa = __fmaf_rn(bt.gv[u], vmin[u], sa);
-            }
-            if (amx[u] >= 0) {
-                cmax[amx[u] * tb + tid] += bt.gv[u];
-                if (twob) sb = __fmaf_rn(bt.gv[u], vmax[u], sb);
+            const float gv = bt.gv[u];   // zero for an item past the end
+            sg += gv;
+            if (use_min) cmin[amn[u] * tb + tid] += gv;
+            if (use_max) cmax[amx[u] * tb + tid] += gv;
+            if (twob) {
+                sa = __fmaf_rn(gv, vmin[u], sa);
+                sb = __fmaf_rn(gv, vmax[u], sb);
             }
         }
     };
     {
-        const int batches = (int)((j1 - j0 + 8LL * tb - 1) / (8LL * tb));
+        const int batches = (j1 - j0 + 8 * tb - 1) / (8 * tb);
         Batch ba, bb;
         fetch(ba);
         for (int it = 0; it < batches; it += 2) {
