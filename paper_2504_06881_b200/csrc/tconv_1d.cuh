@@ -261,12 +261,13 @@ bwd1d_gx_kernel(Geo3 g, int pt, int ks, int span, const float* __restrict__ alph
     for (int k = slice * kper; k < kend; ++k) {
         float a = 1.0f, b = 1.0f;
         if (twob) {
-            if (alpha) a = alpha[(size_t)k * g.C + c];
-            if (beta) b = beta[(size_t)k * g.C + c];
+            if (alpha) a = alpha[k * g.C + c];
+            if (beta) b = beta[k * g.C + c];
         }
-        const T* grow = gy + ((size_t)n * g.K + k) * OL + p0;
-        const uint16_t* crow = (const uint16_t*)winners + (((size_t)n * g.K + k) * g.C + c) * OL + p0;
-        const int32_t* irow = (const int32_t*)winners + ((size_t)n * g.K + k) * OL + p0;
+        // (every tensor of the layer has fewer than 2^31 elements: 32-bit offsets)
+        const T* grow = gy + ((n * g.K + k) * OL + p0);
+        const uint16_t* crow = (const uint16_t*)winners + (((n * g.K + k) * g.C + c) * OL + p0);
+        const int32_t* irow = (const int32_t*)winners + ((n * g.K + k) * OL + p0);
         // eight positions at a time: their winners and gradients are requested together
         for (int i0 = 0; i0 < cnt; i0 += 8) {
             int amn[8], amx[8];
