@@ -251,12 +251,31 @@ int backward_t(const Geo& g, const void* x, const void* w, const void* w2, const
                     // the phases of this form are latency-bound: aim at three resident CTAs per SM
                     // (the tile shares the CTA's shared memory with the staging columns)
                     const size_t stage = (size_t)kIdxGxKB * 256 * 2 * sizeof(float);
+                    const size_t row = (size_t)g.C * g.W * sizeof(float);
+                    const int halo = (g.R - 1) * g.dh;
                     int thi2 = thi;
-                    while (((size_t)g.C * g.W * sizeof(float) * thi2 + stage > 73 * 1024 ||
-                            (size_t)g.C * g.W * sizeof(float) * thi2 + stage > kBwdSmemAttr) &&
-                           (thi2 + 1) / 2 >= 2 * (g.R - 1) * g.dh && thi2 > 4)
+                    while ((row * thi2 + stage > 73 * 1024 || row * thi2 + stage > kBwdSmemAttr) &&
+                           (thi2 + 1) / 2 >= 2 * halo && thi2 > 4)
                         thi2 = (thi2 + 1) / 2;
-                    if ((size_t)g.C * g.W * sizeof(float) * thi2 + stage > kBwdSmemAttr) thi2 = 0;
+                    if (row * thi2 + stage > kBwdSmemAttr) thi2 = 0;
+                    // among the band heights down to that one's half: the fewest rounds of resident
+                    // CTAs times the rows a CTA scans (a band that leaves a few CTAs for a last round
+                    // costs a whole round)
+                    if (thi2 > 0) {
+                        long best_cost = -1;
+                        int best = thi2;
+                        for (int t = thi2; t >= 4 && t >= 2 * halo && 2 * t >= thi2; --t) {
+                            const size_t sm = row * t + stage;
+                            long per_sm = (long)((227 * 1024) / (sm + 1024));
+                            if (per_sm > 8) per_sm = 8;
+                            if (per_sm < 1) continue;
+                            const long ctas = (long)g.N * ((g.H + t - 1) / t);
+                            const long rounds = (ctas + 148 * per_sm - 1) / (148 * per_sm);
+                            const long cost = rounds * (t + halo);
+                            if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = t; }
+                        }
+                        thi2 = best;
+                    }
                     auto kern = g.RS == 9 ? bwd_idx_gx2_kernel<T, 9> : bwd_idx_gx2_kernel<T, 0>;
                     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemAttr) != cudaSuccess)
                         return cuda_fail(cudaGetLastError());
