@@ -63,3 +63,25 @@ def test_runs_on_the_one_dimensional_kernels():
     tconv3d.backward(d, dev(t["x"]), dev(t["w"]), dev(t["g"]), None, dev(t["alpha"]), dev(t["beta"]), win)
     torch.cuda.synchronize()
     assert tconv3d.tconv3d_launch_count() - l0 == 7
+
+
+@pytest.mark.parametrize("seed", [1201, 1202, 1203])
+def test_seeded_random_one_dimensional_layers(seed):
+    """Twelve random layers per seed: window 4..256, stride 1, 2, 4 (the 1-D kernels) or 3 (any-shape
+    kernels), padding up to half the window, 1..6 input and 1..40 output channels, both dtypes, every
+    mode and channel combine."""
+    import numpy as np
+    rs = np.random.RandomState(seed)
+    done = 0
+    while done < 12:
+        mode, chan = MODES[rs.randint(len(MODES))]
+        S = int(rs.choice([4, 5, 7, 12, 16, 31, 64, 80, 100, 129, 256]))
+        st = int(rs.choice([1, 2, 4, 4, 3]))
+        L = int(rs.randint(S, 4 * S + 300))
+        d = layer1d(int(rs.randint(1, 4)), int(rs.randint(1, 7)), L, int(rs.randint(1, 41)), S, stride=st,
+                    pad=int(rs.randint(0, S // 2 + 1)), mode=mode, chan=chan, dtype=["f32", "bf16"][rs.randint(2)])
+        if min(inputs.output_dhw(d)) <= 0:
+            continue
+        done += 1
+        ties = rs.rand() < 0.3
+        check(d, seed * 100 + done, dists=dict(x=("ints", -2, 2), w=("ints", -1, 1)) if ties else None)

@@ -110,3 +110,66 @@ def test_outputs_and_workspace_stay_inside_their_buffers(seed):
             A.check(f"forward_noalloc {d}")
             assert torch.equal(y, y2)
         assert tconv.tconv_device_status() == 0
+
+
+@pytest.mark.parametrize("seed", [41, 42])
+def test_three_dimensional_entry_points_stay_inside_their_buffers(seed):
+    """The same guard bands around the outputs and the workspace of tconv3d_forward / tconv3d_backward,
+    on seeded random one-dimensional layers (long windows, the kernels with their own scratch layout)
+    and small volumes, stored and recomputed winners."""
+    from paper_2504_06881_b200 import tconv3d
+    rs = np.random.RandomState(seed)
+    done = 0
+    while done < 30:
+        mode, chan = ALL[rs.randint(len(ALL))]
+        dtype = ["f32", "bf16"][rs.randint(2)]
+        if rs.rand() < 0.7:          # one-dimensional
+            S = int(rs.choice([4, 5, 9, 16, 33, 80, 81, 200, 256]))
+            st = int(rs.choice([1, 2, 4, 3]))
+            L = int(rs.randint(S, 6 * S + 200))
+            d = inputs.layer3d(int(rs.randint(1, 5)), int(rs.randint(1, 6)), 1, 1, L, int(rs.randint(1, 40)),
+                               T=1, R=1, S=S, stride=(1, 1, st), pad=(0, 0, int(rs.randint(0, S // 2 + 1))),
+                               mode=mode, chan=chan, dtype=dtype)
+        else:
+            d = inputs.layer3d(int(rs.randint(1, 3)), int(rs.randint(1, 5)), int(rs.randint(3, 9)),
+                               int(rs.randint(3, 9)), int(rs.randint(3, 12)), int(rs.randint(1, 9)),
+                               T=int(rs.randint(1, 4)), R=int(rs.randint(1, 4)), S=int(rs.randint(1, 4)),
+                               stride=int(rs.randint(1, 3)), pad=int(rs.randint(0, 2)), mode=mode, chan=chan, dtype=dtype)
+        od = inputs.output_dhw(d)
+        if min(od) <= 0:
+            continue
+        done += 1
+        dt = tconv.TORCH_DTYPE[dtype]
+        two, par = mode in ("compound", "parallel"), mode == "parallel"
+        N, C, K = d["N"], d["C"], d["K"]
+        g = torch.Generator(device="cuda").manual_seed(int(rs.randint(1 << 30)))
+        xs, ws_ = (N, C, d["D"], d["H"], d["W"]), (K, C, d["T"], d["R"], d["S"])
+        x = torch.randn(xs, device="cuda", generator=g).to(dt)
+        w = (0.3 * torch.randn(ws_, device="cuda", generator=g)).to(dt)
+        w2 = (0.3 * torch.randn(ws_, device="cuda", generator=g)).to(dt) if par else None
+        al = torch.rand(K, C, device="cuda", generator=g) if two else None
+        be = torch.rand(K, C, device="cuda", generator=g) if two else None
+        bias = torch.rand(K, device="cuda", generator=g)
+        ys = (N, K) + tuple(od)
+        gy = torch.randn(ys, device="cuda", generator=g).to(dt)
+        es = 4 if dtype == "f32" else 2
+        ny, nx = int(np.prod(ys)) * es, int(np.prod(xs)) * es
+        nwin, nws = tconv3d.tconv3d_winner_bytes(d), tconv3d.tconv3d_workspace_bytes(d, True)
+        nw4 = int(np.prod(ws_)) * 4
+        arena = Arena(ny + nx + nwin + nws + 2 * nw4 + 3 * K * C * 4 + 16 * (GUARD + 256))
+        y = arena.take(ny, dt, ys)
+        win = arena.take(nwin)
+        wsb = arena.take(nws)
+        gx = arena.take(nx, dt, xs)
+        gw = arena.take(nw4, torch.float32, ws_)
+        gw2 = arena.take(nw4, torch.float32, ws_) if par else None
+        ga = arena.take(K * C * 4, torch.float32, (K, C)) if two else None
+        gb = arena.take(K * C * 4, torch.float32, (K, C)) if two else None
+        gbias = arena.take(K * 4, torch.float32, (K,))
+        assert tconv3d.tconv3d_forward(d, x, w, w2, al, be, bias, y, win) == 0
+        torch.cuda.synchronize()
+        arena.check(f"tconv3d_forward {d}")
+        for winners in (win, None):
+            assert tconv3d.tconv3d_backward(d, x, w, w2, al, be, gy, winners, gx, gw, gw2, ga, gb, gbias, wsb) == 0
+            torch.cuda.synchronize()
+            arena.check(f"tconv3d_backward (winners {'stored' if winners is not None else 'recomputed'}) {d}")
