@@ -35,10 +35,10 @@ WORKLOAD = "cfg2: one layer of each mode fwd+bwd fp32, N=128 C=K=64 32x32 3x3 s1
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch at the bench's full size
 # (N=128), from one-pass ncu captures of those two counters, summarised in
 # profiles/dram_traffic_cfg2_n128.md.  bwd_params is the grad_w kernel of the call.
-DRAM_BYTES_FULL = {("parallel", "fwd_winners"): 645.10e6, ("compound", "fwd_winners"): 647.08e6,
-                   ("compound", "bwd_params"): 758.47e6, ("parallel", "bwd_params"): 758.47e6,
-                   ("compound", "bwd_grad_x"): 601.28e6, ("parallel", "bwd_grad_x"): 601.28e6,
-                   ("max_plus", "bwd_grad_x"): 70.76e6, ("min_plus", "bwd_grad_x"): 70.76e6}
+DRAM_BYTES_FULL = {("parallel", "fwd_winners"): 645.95e6, ("compound", "fwd_winners"): 646.41e6,
+                   ("compound", "bwd_params"): 758.98e6, ("parallel", "bwd_params"): 758.98e6,
+                   ("compound", "bwd_grad_x"): 601.37e6, ("parallel", "bwd_grad_x"): 601.37e6,
+                   ("max_plus", "bwd_grad_x"): 70.50e6, ("min_plus", "bwd_grad_x"): 70.50e6}
 # probe variants whose best gives the add+max/min peak of a mode's instruction mix
 PROBES = {"max_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
           "min_plus": ("f32_add_max2", "f32_add_max3", "f32_add2_max3"),
