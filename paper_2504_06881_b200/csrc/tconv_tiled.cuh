@@ -76,7 +76,7 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-// mbarrier + TMA (single-CTA use; no multicast anywhere)
+// mbarrier + TMA (single-CTA use: every copy lands in the shared memory of the CTA that issued it)
 __device__ __forceinline__ void mbar_init(void* bar, unsigned count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
