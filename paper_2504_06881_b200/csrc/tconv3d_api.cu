@@ -176,15 +176,23 @@ int forward1d_t(const Geo3& g, const void* x, const void* w, const void* w2, con
     const int q4 = (((g.S + g.sw - 1) / g.sw) + 3) & ~3;
     const int br = g.mode == TCONV_MIN_PLUS ? 0 : (g.mode == TCONV_MAX_PLUS ? 1 : (g.mode == TCONV_COMPOUND ? 2 : 3));
     const int kb = 4 * f1_kt(br, winners != nullptr);
-    const size_t smem = ((size_t)g.sw * f1_xw(q4) + (size_t)q4 * g.sw * kb * (br == 3 ? 2 : 1)) * sizeof(T);
+    // signal segment, weights by tap, and with winners a second copy of the weights by channel
+    const size_t smem = ((size_t)g.sw * f1_xw(q4) + (size_t)q4 * g.sw * kb * (br == 3 ? 2 : 1) * (winners ? 2 : 1)) * sizeof(T);
     const dim3 grid((unsigned)((g.OW + kF1Pos - 1) / kF1Pos), (unsigned)((g.K + kb - 1) / kb), (unsigned)g.N);
+    // (long windows with winners in parallel mode stage up to 67 KB: above the default limit)
 #define TCONV1_LAUNCH(STV, BRV, WINV)                                                     \
-    fwd1d_kernel<T, STV, BRV, WINV><<<grid, kF1Threads, smem, st>>>(                       \
-        g, q4, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, bias, (T*)y, winners)
+    {                                                                                     \
+        if (smem > 48 * 1024 &&                                                           \
+            cudaFuncSetAttribute(fwd1d_kernel<T, STV, BRV, WINV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                 (int)kSmem1d) != cudaSuccess)                            \
+            return TCONV_ERR_CUDA;                                                        \
+        fwd1d_kernel<T, STV, BRV, WINV><<<grid, kF1Threads, smem, st>>>(                   \
+            g, q4, (const T*)x, (const T*)w, (const T*)w2, alpha, beta, bias, (T*)y, winners); \
+    }
 #define TCONV1_BY_WIN(STV, BRV)                                  \
     {                                                            \
-        if (winners) TCONV1_LAUNCH(STV, BRV, true);              \
-        else TCONV1_LAUNCH(STV, BRV, false);                     \
+        if (winners) TCONV1_LAUNCH(STV, BRV, true)               \
+        else TCONV1_LAUNCH(STV, BRV, false)                      \
     }
 #define TCONV1_BY_BR(STV)                                        \
     {                                                            \

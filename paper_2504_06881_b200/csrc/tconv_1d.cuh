@@ -55,8 +55,8 @@ __host__ __device__ constexpr int f1_xw(int q4) { return (kF1Pos + q4 + 4 + 7) &
 // signal segment of one input channel by phase, xs[ST][xw] with xs[p][i] = x[(P0 + i) * ST + p - pad]
 // (zero outside the signal), xw = 128 + q4 + 4 rounded up to a multiple of eight, and the weights of that channel for the block's
 // 4 * KT output channels, ws[s][4 * KT] for s < q4 * ST (NaN for s >= S), twice in parallel mode.
-// q4 = ceil(S / ST) rounded up to a multiple of four.  WIN: taps are visited in ascending order
-// with strict compares, so that the lowest tap wins a tie.
+// q4 = ceil(S / ST) rounded up to a multiple of four.  WIN: a second copy of the weights by
+// output channel follows, wst[4 * KT][q4 * ST] (twice in parallel mode).
 template <typename T, int ST, int BR, bool WIN>
 __global__ void __launch_bounds__(kF1Threads)
 fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
@@ -70,6 +70,9 @@ fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, c
     T* xs = reinterpret_cast<T*>(smem_raw);
     T* ws = xs + ST * xw;
     T* ws2 = ws + q4 * ST * KB;
+    // WIN: a second copy of the weights by output channel, wst[kk][s], for the second step
+    T* wst = ws2 + (BR == 3 ? q4 * ST * KB : 0);
+    T* wst2 = wst + q4 * ST * KB;
     const int tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
     const int P0 = blockIdx.x * kF1Pos, n = blockIdx.z;
     const int kb0 = blockIdx.y * KB, k0 = kb0 + wv * KT;
@@ -104,6 +107,10 @@ fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, c
                 }
                 ws[s * KB + kk] = a;
                 if (BR == 3) ws2[s * KB + kk] = b;
+                if constexpr (WIN) {
+                    wst[i] = a;
+                    if (BR == 3) wst2[i] = b;
+                }
             }
         }
         __syncthreads();
@@ -152,7 +159,18 @@ fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, c
                 }
             }
         } else {
+            // Winners in two steps.  First the windows are walked in blocks of BQ q (BQ * ST = 4 or
+            // 8 consecutive taps, blocks ascending): a block's extremum replaces the running one only
+            // when it is strictly better, and the block is remembered.  Then, per output and branch,
+            // the taps of the remembered block are formed again, highest first, and the lowest one
+            // that equals the extremum is the winner.
+            constexpr int BQ = ST == 4 ? 2 : 4;
             const T* xl = xs + 4 * lane;
+            int bmn[KT][4], bmx[KT][4];
+#pragma unroll
+            for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) bmn[kk][j] = bmx[kk][j] = 0;
             for (int q0 = 0; q0 < q4; q0 += 4) {
                 T r[ST][8];
 #pragma unroll
@@ -161,27 +179,91 @@ fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, c
                     *reinterpret_cast<Vec<T, 4>*>(r[p] + 4) =
                         *reinterpret_cast<const Vec<T, 4>*>(xl + p * xw + q0 + 4);
                 }
+                float cmn[KT][4], cmx[KT][4];
 #pragma unroll
-                for (int dq = 0; dq < 4; ++dq)
+                for (int dq = 0; dq < 4; dq += 2) {
+                    if (dq % BQ == 0) {
+#pragma unroll
+                        for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) { cmn[kk][j] = INFINITY; cmx[kk][j] = -INFINITY; }
+                    }
 #pragma unroll
                     for (int p = 0; p < ST; ++p) {
-                        const int s = (q0 + dq) * ST + p;
-                        const Vec<T, KT> wa = *reinterpret_cast<const Vec<T, KT>*>(ws + s * KB + wv * KT);
-                        Vec<T, KT> wb = wa;
-                        if constexpr (BR == 3) wb = *reinterpret_cast<const Vec<T, KT>*>(ws2 + s * KB + wv * KT);
+                        const int s0 = (q0 + dq) * ST + p, s1 = s0 + ST;
+                        const Vec<T, KT> wa0 = *reinterpret_cast<const Vec<T, KT>*>(ws + s0 * KB + wv * KT);
+                        const Vec<T, KT> wa1 = *reinterpret_cast<const Vec<T, KT>*>(ws + s1 * KB + wv * KT);
+                        Vec<T, KT> wb0 = wa0, wb1 = wa1;
+                        if constexpr (BR == 3) {
+                            wb0 = *reinterpret_cast<const Vec<T, KT>*>(ws2 + s0 * KB + wv * KT);
+                            wb1 = *reinterpret_cast<const Vec<T, KT>*>(ws2 + s1 * KB + wv * KT);
+                        }
 #pragma unroll
                         for (int kk = 0; kk < KT; ++kk)
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
-                                const float t = tap_add(r[p][dq + j], wa.v[kk]);
-                                const float u = (BR == 3) ? tap_add(r[p][dq + j], wb.v[kk]) : t;
-                                if constexpr (MIN)
-                                    if (t < mn[kk][j]) { mn[kk][j] = t; amn[kk][j] = s; }
-                                if constexpr (MAX)
-                                    if (u > mx[kk][j]) { mx[kk][j] = u; amx[kk][j] = s; }
+                                const float t0 = tap_add(r[p][dq + j], wa0.v[kk]);
+                                const float t1 = tap_add(r[p][dq + 1 + j], wa1.v[kk]);
+                                if constexpr (MIN) cmn[kk][j] = fmin3(cmn[kk][j], t0, t1);
+                                if constexpr (BR == 3) {
+                                    const float u0 = tap_add(r[p][dq + j], wb0.v[kk]);
+                                    const float u1 = tap_add(r[p][dq + 1 + j], wb1.v[kk]);
+                                    cmx[kk][j] = fmax3(cmx[kk][j], u0, u1);
+                                } else if constexpr (MAX) {
+                                    cmx[kk][j] = fmax3(cmx[kk][j], t0, t1);
+                                }
                             }
                     }
+                    if ((dq + 2) % BQ == 0) {   // the block that starts at q0 + dq + 2 - BQ is complete
+                        const int qb = q0 + dq + 2 - BQ;
+#pragma unroll
+                        for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                if constexpr (MIN)
+                                    if (cmn[kk][j] < mn[kk][j]) { mn[kk][j] = cmn[kk][j]; bmn[kk][j] = qb; }
+                                if constexpr (MAX)
+                                    if (cmx[kk][j] > mx[kk][j]) { mx[kk][j] = cmx[kk][j]; bmx[kk][j] = qb; }
+                            }
+                    }
+                }
             }
+            const int span = q4 * ST;
+            const T* wt = wst + wv * KT * span;
+            const T* wt2 = (BR == 3 ? wst2 : wst) + wv * KT * span;
+#pragma unroll
+            for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if constexpr (MIN) {
+                        const int qb = bmn[kk][j];
+                        const float m = mn[kk][j];
+                        int am = 0;
+#pragma unroll
+                        const T* wq = wt + kk * span + qb * ST;
+                        const T* xq = xl + j + qb;
+#pragma unroll
+                        for (int i = BQ * ST - 1; i >= 0; --i) {
+                            const float t = tap_add(xq[(i % ST) * xw + i / ST], wq[i]);
+                            if (t == m) am = qb * ST + i;
+                        }
+                        amn[kk][j] = am;
+                    }
+                    if constexpr (MAX) {
+                        const int qb = bmx[kk][j];
+                        const float m = mx[kk][j];
+                        int am = 0;
+#pragma unroll
+                        const T* wq = wt2 + kk * span + qb * ST;
+                        const T* xq = xl + j + qb;
+#pragma unroll
+                        for (int i = BQ * ST - 1; i >= 0; --i) {
+                            const float t = tap_add(xq[(i % ST) * xw + i / ST], wq[i]);
+                            if (t == m) am = qb * ST + i;
+                        }
+                        amx[kk][j] = am;
+                    }
+                }
         }
         // channel combine, channels ascending
 #pragma unroll
