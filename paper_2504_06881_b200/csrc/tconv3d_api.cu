@@ -177,7 +177,10 @@ int forward1d_t(const Geo3& g, const void* x, const void* w, const void* w2, con
     const int br = g.mode == TCONV_MIN_PLUS ? 0 : (g.mode == TCONV_MAX_PLUS ? 1 : (g.mode == TCONV_COMPOUND ? 2 : 3));
     const int kb = 4 * f1_kt(br, winners != nullptr);
     // signal segment, weights by tap, and with winners a second copy of the weights by channel
-    const size_t smem = ((size_t)g.sw * f1_xw(q4) + (size_t)q4 * g.sw * kb * (br == 3 ? 2 : 1) * (winners ? 2 : 1)) * sizeof(T);
+    // (a bf16 layer stages its weights by tap as 4-byte {w, w} pairs; with winners a second copy by
+    // channel follows in the layer's type)
+    const size_t wcopy = (size_t)q4 * g.sw * kb * (br == 3 ? 2 : 1);
+    const size_t smem = (size_t)g.sw * f1_xw(q4) * sizeof(T) + wcopy * 4 + (winners ? wcopy * sizeof(T) : 0);
     const dim3 grid((unsigned)((g.OW + kF1Pos - 1) / kF1Pos), (unsigned)((g.K + kb - 1) / kb), (unsigned)g.N);
     // (long windows with winners in parallel mode stage up to 67 KB: above the default limit)
 #define TCONV1_LAUNCH(STV, BRV, WINV)                                                     \

@@ -11,6 +11,8 @@
 // of even and odd index own one array each, a thread's positions cannot reach past its neighbour's),
 // the parameter gradients by private per-thread columns per tap; every sum has a fixed order.
 #pragma once
+#include <type_traits>
+
 #include "tconv_3d.cuh"
 
 namespace tconv {
@@ -34,6 +36,26 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
+
+// packed bf16 pairs (two adjacent output positions per register)
+__device__ __forceinline__ unsigned h1_add2(unsigned a, unsigned b) {
+    unsigned d;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ unsigned h1_min2(unsigned a, unsigned b) {
+    unsigned d;
+    asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ unsigned h1_max2(unsigned a, unsigned b) {
+    unsigned d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// {w, w} of a weight in the layer's type (bf16 only; the fp32 overload is never called)
+__device__ __forceinline__ unsigned h1_dup(__nv_bfloat16 v) { return 0x00010001u * (unsigned)__bfloat16_as_ushort(v); }
+__device__ __forceinline__ unsigned h1_dup(float) { return 0u; }
 
 template <typename T> __device__ __forceinline__ T nan_of();
 template <> __device__ __forceinline__ float nan_of<float>() { return __int_as_float(0x7fc00000); }
@@ -67,11 +89,16 @@ fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, c
     constexpr bool MIN = has_min(BR), MAX = has_max(BR);
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int xw = f1_xw(q4);
+    // bf16: two adjacent positions per register, the weights staged as {w, w} pairs
+    constexpr bool PK = sizeof(T) == 2;
+    using WT = typename std::conditional<PK, unsigned, T>::type;
     T* xs = reinterpret_cast<T*>(smem_raw);
-    T* ws = xs + ST * xw;
-    T* ws2 = ws + q4 * ST * KB;
+    WT* wsw = reinterpret_cast<WT*>(xs + ST * xw);
+    WT* wsw2 = wsw + q4 * ST * KB;
+    T* ws = reinterpret_cast<T*>(wsw);      // (the views used by the unpacked paths)
+    T* ws2 = reinterpret_cast<T*>(wsw2);
     // WIN: a second copy of the weights by output channel, wst[kk][s], for the second step
-    T* wst = ws2 + (BR == 3 ? q4 * ST * KB : 0);
+    T* wst = reinterpret_cast<T*>(wsw2 + (BR == 3 ? q4 * ST * KB : 0));
     T* wst2 = wst + q4 * ST * KB;
     const int tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
     const int P0 = blockIdx.x * kF1Pos, n = blockIdx.z;
@@ -105,8 +132,13 @@ fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, c
                     a = w[wi];
                     if (BR == 3) b = w2[wi];
                 }
-                ws[s * KB + kk] = a;
-                if (BR == 3) ws2[s * KB + kk] = b;
+                if constexpr (PK) {
+                    wsw[s * KB + kk] = h1_dup(a);
+                    if (BR == 3) wsw2[s * KB + kk] = h1_dup(b);
+                } else {
+                    ws[s * KB + kk] = a;
+                    if (BR == 3) ws2[s * KB + kk] = b;
+                }
                 if constexpr (WIN) {
                     wst[i] = a;
                     if (BR == 3) wst2[i] = b;
@@ -122,7 +154,60 @@ fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, c
             for (int j = 0; j < 4; ++j) {
                 mn[kk][j] = INFINITY; mx[kk][j] = -INFINITY; amn[kk][j] = 0; amx[kk][j] = 0;
             }
-        if constexpr (!WIN) {
+        if constexpr (PK && !WIN) {
+            // positions (0, 1) and (2, 3) of the lane as pairs; a tap at an odd offset into the window
+            // takes the pairs shifted by one element
+            unsigned mn2[KT][2], mx2[KT][2];
+#pragma unroll
+            for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                for (int pr = 0; pr < 2; ++pr) { mn2[kk][pr] = 0x7f807f80u; mx2[kk][pr] = 0xff80ff80u; }
+#pragma unroll
+            for (int p = 0; p < ST; ++p) {
+                const T* xp = xs + p * xw + 4 * lane;
+                for (int q0 = 0; q0 < q4; q0 += 4) {
+                    const uint2 lo = *reinterpret_cast<const uint2*>(xp + q0);
+                    const uint2 hi = *reinterpret_cast<const uint2*>(xp + q0 + 4);
+                    const unsigned ev[4] = {lo.x, lo.y, hi.x, hi.y};
+                    const unsigned od[3] = {__byte_perm(lo.x, lo.y, 0x5432), __byte_perm(lo.y, hi.x, 0x5432),
+                                            __byte_perm(hi.x, hi.y, 0x5432)};
+#pragma unroll
+                    for (int dq = 0; dq < 4; dq += 2) {
+                        const int s0 = (q0 + dq) * ST + p, s1 = s0 + ST;
+                        const Vec<unsigned, KT> wa0 = *reinterpret_cast<const Vec<unsigned, KT>*>(wsw + s0 * KB + wv * KT);
+                        const Vec<unsigned, KT> wa1 = *reinterpret_cast<const Vec<unsigned, KT>*>(wsw + s1 * KB + wv * KT);
+                        Vec<unsigned, KT> wb0 = wa0, wb1 = wa1;
+                        if constexpr (BR == 3) {
+                            wb0 = *reinterpret_cast<const Vec<unsigned, KT>*>(wsw2 + s0 * KB + wv * KT);
+                            wb1 = *reinterpret_cast<const Vec<unsigned, KT>*>(wsw2 + s1 * KB + wv * KT);
+                        }
+#pragma unroll
+                        for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                            for (int pr = 0; pr < 2; ++pr) {
+                                const unsigned x0 = ev[dq / 2 + pr], x1 = od[dq / 2 + pr];
+                                const unsigned t0 = h1_add2(x0, wa0.v[kk]), t1 = h1_add2(x1, wa1.v[kk]);
+                                if constexpr (MIN) mn2[kk][pr] = h1_min2(h1_min2(mn2[kk][pr], t0), t1);
+                                if constexpr (BR == 3) {
+                                    const unsigned u0 = h1_add2(x0, wb0.v[kk]), u1 = h1_add2(x1, wb1.v[kk]);
+                                    mx2[kk][pr] = h1_max2(h1_max2(mx2[kk][pr], u0), u1);
+                                } else if constexpr (MAX) {
+                                    mx2[kk][pr] = h1_max2(h1_max2(mx2[kk][pr], t0), t1);
+                                }
+                            }
+                    }
+                }
+            }
+#pragma unroll
+            for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                for (int pr = 0; pr < 2; ++pr) {
+                    mn[kk][2 * pr] = __uint_as_float(mn2[kk][pr] << 16);
+                    mn[kk][2 * pr + 1] = __uint_as_float(mn2[kk][pr] & 0xffff0000u);
+                    mx[kk][2 * pr] = __uint_as_float(mx2[kk][pr] << 16);
+                    mx[kk][2 * pr + 1] = __uint_as_float(mx2[kk][pr] & 0xffff0000u);
+                }
+        } else if constexpr (!WIN) {
 #pragma unroll
             for (int p = 0; p < ST; ++p) {
                 const T* xp = xs + p * xw + 4 * lane;
@@ -171,6 +256,97 @@ fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, c
             for (int kk = 0; kk < KT; ++kk)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) bmn[kk][j] = bmx[kk][j] = 0;
+            if constexpr (PK) {
+                // bf16: the first step on pairs of positions; per half a mask says where the block is
+                // strictly better, and takes the block's first q into that half of the block register
+                unsigned mn2[KT][2], mx2[KT][2], bmn2[KT][2], bmx2[KT][2];
+#pragma unroll
+                for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                    for (int pr = 0; pr < 2; ++pr) {
+                        mn2[kk][pr] = 0x7f807f80u; mx2[kk][pr] = 0xff80ff80u; bmn2[kk][pr] = bmx2[kk][pr] = 0u;
+                    }
+                for (int q0 = 0; q0 < q4; q0 += 4) {
+                    unsigned ev[ST][4], od[ST][3];
+#pragma unroll
+                    for (int p = 0; p < ST; ++p) {
+                        const uint2 lo = *reinterpret_cast<const uint2*>(xl + p * xw + q0);
+                        const uint2 hi = *reinterpret_cast<const uint2*>(xl + p * xw + q0 + 4);
+                        ev[p][0] = lo.x; ev[p][1] = lo.y; ev[p][2] = hi.x; ev[p][3] = hi.y;
+                        od[p][0] = __byte_perm(lo.x, lo.y, 0x5432);
+                        od[p][1] = __byte_perm(lo.y, hi.x, 0x5432);
+                        od[p][2] = __byte_perm(hi.x, hi.y, 0x5432);
+                    }
+                    unsigned cm2[KT][2], cx2[KT][2];
+#pragma unroll
+                    for (int dq = 0; dq < 4; dq += 2) {
+                        if (dq % BQ == 0) {
+#pragma unroll
+                            for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                                for (int pr = 0; pr < 2; ++pr) { cm2[kk][pr] = 0x7f807f80u; cx2[kk][pr] = 0xff80ff80u; }
+                        }
+#pragma unroll
+                        for (int p = 0; p < ST; ++p) {
+                            const int s0 = (q0 + dq) * ST + p, s1 = s0 + ST;
+                            const Vec<unsigned, KT> wa0 = *reinterpret_cast<const Vec<unsigned, KT>*>(wsw + s0 * KB + wv * KT);
+                            const Vec<unsigned, KT> wa1 = *reinterpret_cast<const Vec<unsigned, KT>*>(wsw + s1 * KB + wv * KT);
+                            Vec<unsigned, KT> wb0 = wa0, wb1 = wa1;
+                            if constexpr (BR == 3) {
+                                wb0 = *reinterpret_cast<const Vec<unsigned, KT>*>(wsw2 + s0 * KB + wv * KT);
+                                wb1 = *reinterpret_cast<const Vec<unsigned, KT>*>(wsw2 + s1 * KB + wv * KT);
+                            }
+#pragma unroll
+                            for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                                for (int pr = 0; pr < 2; ++pr) {
+                                    const unsigned x0 = ev[p][dq / 2 + pr], x1 = od[p][dq / 2 + pr];
+                                    const unsigned t0 = h1_add2(x0, wa0.v[kk]), t1 = h1_add2(x1, wa1.v[kk]);
+                                    if constexpr (MIN) cm2[kk][pr] = h1_min2(h1_min2(cm2[kk][pr], t0), t1);
+                                    if constexpr (BR == 3) {
+                                        const unsigned u0 = h1_add2(x0, wb0.v[kk]), u1 = h1_add2(x1, wb1.v[kk]);
+                                        cx2[kk][pr] = h1_max2(h1_max2(cx2[kk][pr], u0), u1);
+                                    } else if constexpr (MAX) {
+                                        cx2[kk][pr] = h1_max2(h1_max2(cx2[kk][pr], t0), t1);
+                                    }
+                                }
+                        }
+                        if ((dq + 2) % BQ == 0) {
+                            const unsigned qb2 = 0x00010001u * (unsigned)(q0 + dq + 2 - BQ);
+#pragma unroll
+                            for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                                for (int pr = 0; pr < 2; ++pr) {
+                                    if constexpr (MIN) {
+                                        const unsigned m = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&cm2[kk][pr]),
+                                                                       *reinterpret_cast<const __nv_bfloat162*>(&mn2[kk][pr]));
+                                        mn2[kk][pr] = h1_min2(mn2[kk][pr], cm2[kk][pr]);
+                                        bmn2[kk][pr] = (qb2 & m) | (bmn2[kk][pr] & ~m);
+                                    }
+                                    if constexpr (MAX) {
+                                        const unsigned m = __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&cx2[kk][pr]),
+                                                                       *reinterpret_cast<const __nv_bfloat162*>(&mx2[kk][pr]));
+                                        mx2[kk][pr] = h1_max2(mx2[kk][pr], cx2[kk][pr]);
+                                        bmx2[kk][pr] = (qb2 & m) | (bmx2[kk][pr] & ~m);
+                                    }
+                                }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int kk = 0; kk < KT; ++kk)
+#pragma unroll
+                    for (int pr = 0; pr < 2; ++pr) {
+                        mn[kk][2 * pr] = __uint_as_float(mn2[kk][pr] << 16);
+                        mn[kk][2 * pr + 1] = __uint_as_float(mn2[kk][pr] & 0xffff0000u);
+                        mx[kk][2 * pr] = __uint_as_float(mx2[kk][pr] << 16);
+                        mx[kk][2 * pr + 1] = __uint_as_float(mx2[kk][pr] & 0xffff0000u);
+                        bmn[kk][2 * pr] = (int)(bmn2[kk][pr] & 0xffffu);
+                        bmn[kk][2 * pr + 1] = (int)(bmn2[kk][pr] >> 16);
+                        bmx[kk][2 * pr] = (int)(bmx2[kk][pr] & 0xffffu);
+                        bmx[kk][2 * pr + 1] = (int)(bmx2[kk][pr] >> 16);
+                    }
+            } else
             for (int q0 = 0; q0 < q4; q0 += 4) {
                 T r[ST][8];
 #pragma unroll
