@@ -10,7 +10,7 @@ import ctypes
 
 import torch
 
-from .tconv import CHANS, DTYPES, MODES, TORCH_DTYPE, TconvError, _check, _lib, _p, _stream
+from .tconv import CHANS, DTYPES, MODES, TORCH_DTYPE, TconvError, _check, _lib, _on_stream, _p, _stream
 
 # every symbol include/tconv3d.h declares
 SYMBOLS = ("tconv3d_output_shape", "tconv3d_winner_bytes", "tconv3d_workspace_bytes", "tconv3d_forward",
@@ -110,6 +110,7 @@ def forward(d: dict, x, w, w2=None, alpha=None, beta=None, bias=None, want_winne
     _check(bias, (d["K"],), torch.float32, "bias")
     y = torch.empty(sy, dtype=dt, device=x.device)
     winners = winner_buffer(d, x.device) if want_winners else None
+    _on_stream(stream, y, winners)
     rc = tconv3d_forward(d, x, w, w2, alpha, beta, bias, y, winners, stream)
     if rc != 0:
         raise TconvError(rc, "tconv3d_forward")
@@ -133,6 +134,7 @@ def backward(d: dict, x, w, grad_y, w2=None, alpha=None, beta=None, winners=None
         out["grad_alpha"] = torch.empty((d["K"], d["C"]), dtype=f32, device=dev)
         out["grad_beta"] = torch.empty((d["K"], d["C"]), dtype=f32, device=dev)
     ws = torch.empty(tconv3d_workspace_bytes(d, True), dtype=torch.uint8, device=dev)
+    _on_stream(stream, ws, *out.values())
     rc = tconv3d_backward(d, x, w, w2, alpha, beta, grad_y, winners, out.get("grad_x"), out["grad_w"],
                           out.get("grad_w2"), out.get("grad_alpha"), out.get("grad_beta"), out["grad_bias"],
                           ws, stream)
