@@ -85,3 +85,11 @@ def test_seeded_random_one_dimensional_layers(seed):
         done += 1
         ties = rs.rand() < 0.3
         check(d, seed * 100 + done, dists=dict(x=("ints", -2, 2), w=("ints", -1, 1)) if ties else None)
+
+
+@pytest.mark.parametrize("mode,dtype,N", [("compound", "f32", 32), ("max_plus", "f32", 32), ("parallel", "bf16", 4)])
+def test_audio_opening_layer_at_the_benchmark_size(mode, dtype, N):
+    """The layer `bench.py --workload conv1d` times (32 signals of 16000 samples, 128 output channels,
+    window 80, stride 4), in full against the oracle: forward, winners and every gradient (the bf16
+    oracle is slower: four signals)."""
+    check(layer1d(N, 1, 16000, 128, 80, stride=4, mode=mode, dtype=dtype), 1300)
