@@ -92,3 +92,10 @@ def test_depthwise_descriptor_checks():
     d = inputs.layer(1, 4, 8, 8, 4, 3, 3, pad=1, mode="parallel")           # parallel needs w2
     y = torch.zeros(1, 4, 8, 8, device="cuda")
     assert tconv.tconv_dw_forward(d, x, w, None, None, None, None, y) == -1
+
+
+@pytest.mark.parametrize("dtype,N,stride", [("f32", 128, 1), ("bf16", 16, 1), ("f32", 32, 2), ("bf16", 8, 2)])
+def test_depthwise_at_the_benchmark_size(dtype, N, stride):
+    """The layer `bench.py --workload dw` times (144 channels, 56 x 56, 3 x 3, padding 1, compound) in
+    full against the oracle, and its stride-2 form (the bf16 oracle is slower: fewer images)."""
+    check(inputs.layer(N, 144, 56, 56, 144, 3, 3, stride=stride, pad=1, mode="compound", dtype=dtype), 3300 + N)
