@@ -75,10 +75,11 @@ __host__ __device__ constexpr int f1_xw(int q4) { return (kF1Pos + q4 + 4 + 7) &
 
 // Forward.  grid (ceil(OL / 128), ceil(K / (4 * KT)), N), 128 threads.  Shared memory: the block's
 // signal segment of one input channel by phase, xs[ST][xw] with xs[p][i] = x[(P0 + i) * ST + p - pad]
-// (zero outside the signal), xw = 128 + q4 + 4 rounded up to a multiple of eight, and the weights of that channel for the block's
-// 4 * KT output channels, ws[s][4 * KT] for s < q4 * ST (NaN for s >= S), twice in parallel mode.
-// q4 = ceil(S / ST) rounded up to a multiple of four.  WIN: a second copy of the weights by
-// output channel follows, wst[4 * KT][q4 * ST] (twice in parallel mode).
+// (zero outside the signal), xw = 128 + q4 + 4 rounded up to a multiple of eight, and the weights
+// of that channel for the block's 4 * KT output channels, ws[s][4 * KT] for s < q4 * ST (NaN for
+// s >= S; bf16 layers keep them as 4-byte {w, w} pairs), twice in parallel mode.  q4 = ceil(S / ST)
+// rounded up to a multiple of four.  WIN: a second copy of the weights by output channel follows,
+// wst[4 * KT][q4 * ST] in the layer's type (twice in parallel mode).
 template <typename T, int ST, int BR, bool WIN>
 __global__ void __launch_bounds__(kF1Threads)
 fwd1d_kernel(Geo3 g, int q4, const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2,
